@@ -1,0 +1,203 @@
+/*
+ * dybit.h -- C ABI of the DyBit quantize/pack + coded-operand GEMM library
+ * for NVIDIA B200 (sm_100a).
+ *
+ * DyBit ("DyBit: Dynamic Bit-Precision Numbers for Efficient Quantized
+ * Neural Network Inference", arXiv 2302.12510) is an N-bit number format
+ * with an optional sign bit, a unary (leading-ones) exponent field of
+ * variable length and the remaining bits as fraction (Section III-A, Eq. 1,
+ * Table I).  A tensor is stored as one per-tensor fp32 scale plus one code
+ * per element; real value = scale * value(code).
+ *
+ * Conventions for every entry point
+ *   - Pointers marked [dev] are device pointers, [host] host pointers.  The
+ *     caller owns every buffer, including workspace; the library allocates
+ *     no device memory.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *     Device work is enqueued on it and the call returns without waiting.
+ *   - Scales live in device memory as two floats: scale[0] = scale,
+ *     scale[1] = 1/scale as the encoder uses it.  No host sync is needed
+ *     between quantize and GEMM.
+ *   - Every function returns a dybit_status; argument errors are detected
+ *     before anything is launched.  Nothing aborts or throws.
+ *   - A code width `bits` is 2..8.  Signed formats spend the top bit on the
+ *     sign and have m = bits-1 magnitude bits; unsigned formats have
+ *     m = bits.  "Code 0" is the all-zero pattern and decodes to exactly 0.
+ */
+#ifndef DYBIT_H_
+#define DYBIT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    DYBIT_OK = 0,
+    DYBIT_ERR_INVALID_ARG = 1,    /* null pointer, negative size, bits outside 2..8 ...      */
+    DYBIT_ERR_UNSUPPORTED = 2,    /* valid but not implemented (e.g. K beyond int32 headroom) */
+    DYBIT_ERR_ALIGNMENT = 3,      /* a pointer or stride is not aligned as documented         */
+    DYBIT_ERR_WORKSPACE = 4,      /* workspace missing or smaller than the *_workspace_bytes  */
+    DYBIT_ERR_CUDA = 5,           /* a CUDA runtime / driver call failed                      */
+    DYBIT_ERR_DEVICE_TIMEOUT = 6  /* a bounded device-side wait expired (see dybit_last_device_status) */
+} dybit_status;
+
+/* One tensor's code format (Section III-A). */
+typedef struct {
+    int bits;       /* total code width, 2..8                                   */
+    int is_signed;  /* 1: MSB is the sign, bits-1 magnitude bits; 0: all magnitude */
+} dybit_fmt;
+
+/* Tensor-core input type the GEMM expands codes into: the narrowest type
+ * that holds every value of both operand formats exactly (Section III-B.3
+ * picks a multiplier mode per bitwidth pair; this is its analogue). */
+typedef enum {
+    DYBIT_CONTAINER_I8 = 0,    /* int8 x int8 -> int32, exact                */
+    DYBIT_CONTAINER_E4M3 = 1,  /* fp8 e4m3 x e4m3 -> fp32                    */
+    DYBIT_CONTAINER_BF16 = 2   /* bf16 x bf16 -> fp32                        */
+} dybit_container;
+
+/* Convolution geometry: X is [n][h][w][c] (NHWC), W is [k][r][s][c],
+ * Y is [n][oh][ow][k] with oh = (h + 2*pad - dilation*(r-1) - 1)/stride + 1
+ * (ow likewise).  Taps outside the image contribute 0. */
+typedef struct {
+    int n, h, w, c;
+    int k, r, s;
+    int stride, pad, dilation;
+} dybit_conv_desc;
+
+/* ---------------------------------------------------------------- host-only helpers */
+
+/* Static, NUL-terminated description of a status code. */
+const char *dybit_status_string(dybit_status st);
+
+/* Bytes of a packed 1-D tensor of n codes: ceil(n*bits/8) rounded up to 16.
+ * Returns 0 for invalid arguments. */
+size_t dybit_packed_bytes(int64_t n, int bits);
+
+/* Row stride, in bytes, of a packed matrix operand with k columns: k is
+ * padded up to a multiple of 128 codes, so the stride is a multiple of
+ * 16 bytes.  Returns 0 for invalid arguments. */
+size_t dybit_row_stride_bytes(int64_t k, int bits);
+
+/* Eq. 1 enumerated: table[c] = value of code c for c < 2^bits, 0 above.
+ * table: [host] 256 floats. */
+dybit_status dybit_decode_table(dybit_fmt fmt, float *table);
+
+/* Enumerates both formats' value tables and reports the container the GEMM
+ * will use for this pair, plus the power-of-two exponents by which each
+ * operand's values are multiplied before conversion (int8 container only:
+ * value * 2^exp is an integer; 0 for the floating containers).
+ * All three outputs: [host], each may be NULL. */
+dybit_status dybit_choose_container(dybit_fmt fa, dybit_fmt fb, dybit_container *container,
+                                    int *exp_a, int *exp_b);
+
+/* Workspace sizes (bytes) the caller must provide to dybit_gemm /
+ * dybit_conv2d.  0 is returned for invalid arguments; a valid problem never
+ * needs 0 bytes. */
+size_t dybit_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, dybit_fmt fa, dybit_fmt fb);
+size_t dybit_conv2d_workspace_bytes(const dybit_conv_desc *desc, dybit_fmt fx, dybit_fmt fw);
+
+/* Output spatial size of a convolution.  oh / ow: [host]. */
+dybit_status dybit_conv2d_out_hw(const dybit_conv_desc *desc, int *oh, int *ow);
+
+/* ---------------------------------------------------------------- device entry points */
+
+/* Per-tensor max-abs scale (Section I: the format adjusts its precision at
+ * the tensor level).  amax = largest finite |x|;
+ * scale_out[0] = amax / 2^(m-1), scale_out[1] = 2^(m-1) / amax (one fp32
+ * division).  amax == 0 (or n == 0) gives {1, 1}.
+ *   x         [dev]  n floats, 4-byte aligned (16-byte aligned runs fastest)
+ *   scale_out [dev]  2 floats, overwritten                                  */
+dybit_status dybit_absmax_scale(const float *x, int64_t n, dybit_fmt fmt, float *scale_out,
+                                void *stream);
+
+/* Quantize + pack a 1-D tensor (Section III-A format; encoder of
+ * Section III-B.2).  Per element: t = |x| * scale[1] in fp32; magnitude code
+ * = the code whose value is nearest to t (ties to the even code; t beyond
+ * the largest value saturates to all-ones; NaN -> code 0); the sign bit is
+ * the sign of x unless the magnitude code is 0; an unsigned format maps
+ * negative x to code 0.  Codes are written as a dense little-endian bit
+ * stream: code j occupies stream bits [j*bits, (j+1)*bits), stream bit b is
+ * bit b%8 of byte b/8.  Bits past the last code, up to
+ * dybit_packed_bytes(n, bits), are written as zero.
+ *   x         [dev]  n floats, 4-byte aligned
+ *   scale     [dev]  2 floats {scale, 1/scale}, or NULL: the max-abs scale
+ *                    is computed first and written to scale_out (which must
+ *                    then be non-NULL)
+ *   packed    [dev]  dybit_packed_bytes(n, bits) bytes, 16-byte aligned
+ *   scale_out [dev]  2 floats or NULL; receives the scale that was used     */
+dybit_status dybit_quantize_pack(const float *x, int64_t n, dybit_fmt fmt, const float *scale,
+                                 void *packed, float *scale_out, void *stream);
+
+/* Quantize + pack a matrix operand for dybit_gemm: rows x cols fp32, row r
+ * starting at x + r*ld, into rows of row_stride_bytes each; every row is
+ * its own bit stream and is zero-filled (code 0) from column `cols` to the
+ * end of the row.  With scale == NULL one max-abs scale over the whole
+ * matrix is computed first.
+ *   ld               in floats, >= cols
+ *   row_stride_bytes multiple of 16, >= dybit_row_stride_bytes(cols, bits) */
+dybit_status dybit_quantize_pack_2d(const float *x, int64_t rows, int64_t cols, int64_t ld,
+                                    dybit_fmt fmt, const float *scale, void *packed,
+                                    int64_t row_stride_bytes, float *scale_out, void *stream);
+
+/* Decode a packed 1-D tensor (decoder of Section III-B.2, as the
+ * enumerated table of Eq. 1): out[j] = scale[0] * value(code j), one fp32
+ * multiply.
+ *   packed [dev] dybit_packed_bytes(n, bits) bytes, 16-byte aligned
+ *   scale  [dev] 2 floats (only scale[0] is read), or NULL for scale 1
+ *   out    [dev] n floats                                                   */
+dybit_status dybit_decode(const void *packed, int64_t n, dybit_fmt fmt, const float *scale,
+                          float *out, void *stream);
+
+/* Matrix multiply on coded operands (the array of Section III-B.1 computes
+ * a layer as the sum of products of decoded values; Section III-B.3 picks
+ * the multiplier mode from the two bitwidths):
+ *     C[i][j] = sA * sB * sum_k value_A(A[i][k]) * value_B(B[j][k])
+ * Both operands are K-contiguous packed matrices (C = A * B^T), as written
+ * by dybit_quantize_pack_2d.
+ *   A        [dev] M rows of lda_bytes, B [dev] N rows of ldb_bytes; strides
+ *            multiples of 16 >= dybit_row_stride_bytes(K, bits); the row
+ *            tails past K must hold code 0
+ *   scale_a/b [dev] 2 floats each (only [0] is read)
+ *   C        [dev] M x N floats, row stride ldc floats (ldc >= N)
+ *   C_raw    [dev] optional (may be NULL) M x N int32, row stride ldc: the
+ *            exact integer sum of value*2^(m-1) products; only available
+ *            with the int8 container (DYBIT_ERR_UNSUPPORTED otherwise)
+ *   ws       [dev] dybit_gemm_workspace_bytes(...) bytes, 1024-byte aligned
+ * int8 container: C = (float)sum * alpha with
+ * alpha = (float)((double)sA*sB*2^-(expA+expB)), bit-exact.  Floating
+ * containers accumulate in fp32.  K above 2^19 is rejected for int8. */
+dybit_status dybit_gemm(int64_t M, int64_t N, int64_t K,
+                        const void *A, dybit_fmt fa, const float *scale_a, int64_t lda_bytes,
+                        const void *B, dybit_fmt fb, const float *scale_b, int64_t ldb_bytes,
+                        float *C, int64_t ldc, int32_t *C_raw,
+                        void *ws, size_t ws_bytes, void *stream);
+
+/* Convolution on coded operands as an implicit GEMM (Section III-C.4: conv
+ * and FC layers run on the GEMM dataflow), M = n*oh*ow, N = k, K = r*s*c:
+ *     Y[n][oh][ow][k] = sX*sW * sum_{r,s,c} value(X[n][ih][iw][c]) * value(W[k][r][s][c])
+ *   X     [dev] NHWC codes as ONE dense 1-D stream of n*h*w*c codes
+ *         (dybit_quantize_pack of the NHWC tensor), 16-byte aligned
+ *   W     [dev] k rows of r*s*c codes, row stride ldw_bytes
+ *         (dybit_quantize_pack_2d with rows = k, cols = r*s*c)
+ *   Y     [dev] n*oh*ow*k floats, dense;  Y_raw as C_raw above
+ *   ws    [dev] dybit_conv2d_workspace_bytes(...) bytes, 1024-byte aligned  */
+dybit_status dybit_conv2d(const dybit_conv_desc *desc,
+                          const void *X, dybit_fmt fx, const float *scale_x,
+                          const void *W, dybit_fmt fw, const float *scale_w, int64_t ldw_bytes,
+                          float *Y, int32_t *Y_raw,
+                          void *ws, size_t ws_bytes, void *stream);
+
+/* Reads and clears the device status word of the current device.  Blocks
+ * until `stream` has drained.  DYBIT_ERR_DEVICE_TIMEOUT means a kernel gave
+ * up on a bounded wait (results of that call are invalid); DYBIT_OK
+ * otherwise.  detail: [host] optional, receives the raw status word. */
+dybit_status dybit_last_device_status(void *stream, uint32_t *detail);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DYBIT_H_ */

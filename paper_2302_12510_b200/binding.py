@@ -1,0 +1,273 @@
+"""ctypes binding of libdybit.so: argument marshalling only.
+
+Function names follow include/dybit.h.  torch supplies device memory and the
+current stream; every computation happens inside the library's kernels.
+There is no fallback: if libdybit.so is absent the import fails.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import NamedTuple, Optional, Tuple
+
+import torch
+
+from . import _build
+
+__all__ = [
+    "Fmt", "ConvDesc", "DybitError", "lib", "CONTAINER_NAMES",
+    "dybit_status_string", "dybit_packed_bytes", "dybit_row_stride_bytes", "dybit_decode_table",
+    "dybit_choose_container", "dybit_gemm_workspace_bytes", "dybit_conv2d_workspace_bytes",
+    "dybit_conv2d_out_hw", "dybit_absmax_scale", "dybit_quantize_pack", "dybit_quantize_pack_2d",
+    "dybit_decode", "dybit_gemm", "dybit_conv2d", "dybit_last_device_status",
+]
+
+
+class Fmt(NamedTuple):
+    bits: int
+    is_signed: bool
+
+
+class _CFmt(C.Structure):
+    _fields_ = [("bits", C.c_int), ("is_signed", C.c_int)]
+
+
+class _CConvDesc(C.Structure):
+    _fields_ = [(n, C.c_int) for n in ("n", "h", "w", "c", "k", "r", "s", "stride", "pad", "dilation")]
+
+
+class ConvDesc(NamedTuple):
+    n: int
+    h: int
+    w: int
+    c: int
+    k: int
+    r: int
+    s: int
+    stride: int = 1
+    pad: int = 0
+    dilation: int = 1
+
+
+class DybitError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {dybit_status_string(status)} (status {status})")
+
+
+CONTAINER_NAMES = {0: "int8", 1: "e4m3", 2: "bf16"}
+
+
+def _load() -> C.CDLL:
+    path = _build.LIB_PATH
+    if not os.path.exists(path):
+        raise ImportError(
+            f"{path} is missing: build it with `python -m paper_2302_12510_b200._build` "
+            "(there is no CPU or PyTorch fallback)")
+    lib = C.CDLL(path)
+    i64, i32, sz, vp = C.c_int64, C.c_int, C.c_size_t, C.c_void_p
+    lib.dybit_status_string.restype = C.c_char_p
+    lib.dybit_status_string.argtypes = [i32]
+    lib.dybit_packed_bytes.restype = sz
+    lib.dybit_packed_bytes.argtypes = [i64, i32]
+    lib.dybit_row_stride_bytes.restype = sz
+    lib.dybit_row_stride_bytes.argtypes = [i64, i32]
+    lib.dybit_decode_table.argtypes = [_CFmt, C.POINTER(C.c_float)]
+    lib.dybit_choose_container.argtypes = [_CFmt, _CFmt, C.POINTER(i32), C.POINTER(i32), C.POINTER(i32)]
+    lib.dybit_gemm_workspace_bytes.restype = sz
+    lib.dybit_gemm_workspace_bytes.argtypes = [i64, i64, i64, _CFmt, _CFmt]
+    lib.dybit_conv2d_workspace_bytes.restype = sz
+    lib.dybit_conv2d_workspace_bytes.argtypes = [C.POINTER(_CConvDesc), _CFmt, _CFmt]
+    lib.dybit_conv2d_out_hw.argtypes = [C.POINTER(_CConvDesc), C.POINTER(i32), C.POINTER(i32)]
+    lib.dybit_absmax_scale.argtypes = [vp, i64, _CFmt, vp, vp]
+    lib.dybit_quantize_pack.argtypes = [vp, i64, _CFmt, vp, vp, vp, vp]
+    lib.dybit_quantize_pack_2d.argtypes = [vp, i64, i64, i64, _CFmt, vp, vp, i64, vp, vp]
+    lib.dybit_decode.argtypes = [vp, i64, _CFmt, vp, vp, vp]
+    lib.dybit_gemm.argtypes = [i64, i64, i64, vp, _CFmt, vp, i64, vp, _CFmt, vp, i64,
+                               vp, i64, vp, vp, sz, vp]
+    lib.dybit_conv2d.argtypes = [C.POINTER(_CConvDesc), vp, _CFmt, vp, vp, _CFmt, vp, i64,
+                                 vp, vp, vp, sz, vp]
+    lib.dybit_last_device_status.argtypes = [vp, C.POINTER(C.c_uint32)]
+    return lib
+
+
+lib = _load()
+
+
+def _fmt(f) -> _CFmt:
+    bits, sg = f
+    return _CFmt(int(bits), int(bool(sg)))
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> C.c_void_p:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream))
+
+
+def _check(status: int, where: str):
+    if status != 0:
+        raise DybitError(status, where)
+
+
+def _dev_f32(x: torch.Tensor, name: str) -> torch.Tensor:
+    if not (x.is_cuda and x.dtype == torch.float32 and x.is_contiguous()):
+        raise ValueError(f"{name} must be a contiguous float32 CUDA tensor")
+    return x
+
+
+# ---------------------------------------------------------------- host helpers
+
+def dybit_status_string(status: int) -> str:
+    return lib.dybit_status_string(int(status)).decode()
+
+
+def dybit_packed_bytes(n: int, bits: int) -> int:
+    return int(lib.dybit_packed_bytes(int(n), int(bits)))
+
+
+def dybit_row_stride_bytes(k: int, bits: int) -> int:
+    return int(lib.dybit_row_stride_bytes(int(k), int(bits)))
+
+
+def dybit_decode_table(fmt) -> list:
+    buf = (C.c_float * 256)()
+    _check(lib.dybit_decode_table(_fmt(fmt), buf), "dybit_decode_table")
+    return list(buf)
+
+
+def dybit_choose_container(fa, fb) -> Tuple[int, int, int]:
+    c, ea, eb = C.c_int(-1), C.c_int(0), C.c_int(0)
+    _check(lib.dybit_choose_container(_fmt(fa), _fmt(fb), C.byref(c), C.byref(ea), C.byref(eb)),
+           "dybit_choose_container")
+    return c.value, ea.value, eb.value
+
+
+def dybit_gemm_workspace_bytes(M: int, N: int, K: int, fa, fb) -> int:
+    return int(lib.dybit_gemm_workspace_bytes(int(M), int(N), int(K), _fmt(fa), _fmt(fb)))
+
+
+def _cdesc(d: ConvDesc) -> _CConvDesc:
+    return _CConvDesc(*[int(v) for v in d])
+
+
+def dybit_conv2d_workspace_bytes(desc: ConvDesc, fx, fw) -> int:
+    cd = _cdesc(desc)
+    return int(lib.dybit_conv2d_workspace_bytes(C.byref(cd), _fmt(fx), _fmt(fw)))
+
+
+def dybit_conv2d_out_hw(desc: ConvDesc) -> Tuple[int, int]:
+    cd = _cdesc(desc)
+    oh, ow = C.c_int(0), C.c_int(0)
+    _check(lib.dybit_conv2d_out_hw(C.byref(cd), C.byref(oh), C.byref(ow)), "dybit_conv2d_out_hw")
+    return oh.value, ow.value
+
+
+# ---------------------------------------------------------------- device entry points
+
+def dybit_absmax_scale(x: torch.Tensor, fmt, scale_out: Optional[torch.Tensor] = None, stream=None):
+    _dev_f32(x, "x")
+    if scale_out is None:
+        scale_out = torch.empty(2, dtype=torch.float32, device=x.device)
+    _check(lib.dybit_absmax_scale(_ptr(x), x.numel(), _fmt(fmt), _ptr(scale_out), _stream(stream)),
+           "dybit_absmax_scale")
+    return scale_out
+
+
+def dybit_quantize_pack(x: torch.Tensor, fmt, scale: Optional[torch.Tensor] = None,
+                        packed: Optional[torch.Tensor] = None,
+                        scale_out: Optional[torch.Tensor] = None, stream=None):
+    """Returns (packed uint8 tensor, scale tensor {scale, 1/scale})."""
+    _dev_f32(x, "x")
+    n = x.numel()
+    if packed is None:
+        packed = torch.empty(dybit_packed_bytes(n, fmt[0]), dtype=torch.uint8, device=x.device)
+    if scale is None and scale_out is None:
+        scale_out = torch.empty(2, dtype=torch.float32, device=x.device)
+    _check(lib.dybit_quantize_pack(_ptr(x), n, _fmt(fmt), _ptr(scale), _ptr(packed), _ptr(scale_out),
+                                   _stream(stream)), "dybit_quantize_pack")
+    return packed, (scale if scale is not None else scale_out)
+
+
+def dybit_quantize_pack_2d(x: torch.Tensor, fmt, scale: Optional[torch.Tensor] = None,
+                           packed: Optional[torch.Tensor] = None, row_stride_bytes: Optional[int] = None,
+                           scale_out: Optional[torch.Tensor] = None, ld: Optional[int] = None,
+                           cols: Optional[int] = None, stream=None):
+    """x: [rows][ld] float32 (cols <= ld used).  Returns (packed [rows][row_stride] uint8, scale)."""
+    if not (x.is_cuda and x.dtype == torch.float32 and x.dim() == 2 and x.stride(1) == 1):
+        raise ValueError("x must be a 2-D float32 CUDA tensor with unit inner stride")
+    rows = x.shape[0]
+    cols = x.shape[1] if cols is None else cols
+    ld = x.stride(0) if ld is None else ld
+    if row_stride_bytes is None:
+        row_stride_bytes = dybit_row_stride_bytes(cols, fmt[0])
+    if packed is None:
+        packed = torch.empty((rows, row_stride_bytes), dtype=torch.uint8, device=x.device)
+    if scale is None and scale_out is None:
+        scale_out = torch.empty(2, dtype=torch.float32, device=x.device)
+    _check(lib.dybit_quantize_pack_2d(_ptr(x), rows, cols, ld, _fmt(fmt), _ptr(scale), _ptr(packed),
+                                      row_stride_bytes, _ptr(scale_out), _stream(stream)),
+           "dybit_quantize_pack_2d")
+    return packed, (scale if scale is not None else scale_out)
+
+
+def dybit_decode(packed: torch.Tensor, n: int, fmt, scale: Optional[torch.Tensor] = None,
+                 out: Optional[torch.Tensor] = None, stream=None):
+    if out is None:
+        out = torch.empty(n, dtype=torch.float32, device=packed.device)
+    _check(lib.dybit_decode(_ptr(packed), int(n), _fmt(fmt), _ptr(scale), _ptr(out), _stream(stream)),
+           "dybit_decode")
+    return out
+
+
+def dybit_gemm(M: int, N: int, K: int, A: torch.Tensor, fa, scale_a: torch.Tensor,
+               B: torch.Tensor, fb, scale_b: torch.Tensor, C_out: Optional[torch.Tensor] = None,
+               want_raw: bool = False, C_raw: Optional[torch.Tensor] = None,
+               ws: Optional[torch.Tensor] = None, lda_bytes: Optional[int] = None,
+               ldb_bytes: Optional[int] = None, stream=None):
+    """C = sA*sB * value(A) @ value(B)^T.  Returns (C fp32 [M][N], C_raw int32 or None)."""
+    lda = A.stride(0) if lda_bytes is None else lda_bytes
+    ldb = B.stride(0) if ldb_bytes is None else ldb_bytes
+    if C_out is None:
+        C_out = torch.empty((M, N), dtype=torch.float32, device=A.device)
+    if want_raw and C_raw is None:
+        C_raw = torch.empty((M, N), dtype=torch.int32, device=A.device)
+    if ws is None:
+        ws = torch.empty(dybit_gemm_workspace_bytes(M, N, K, fa, fb) + 1024, dtype=torch.uint8, device=A.device)
+    off = (-ws.data_ptr()) % 1024
+    ws_ptr = C.c_void_p(ws.data_ptr() + off)
+    _check(lib.dybit_gemm(M, N, K, _ptr(A), _fmt(fa), _ptr(scale_a), lda, _ptr(B), _fmt(fb), _ptr(scale_b), ldb,
+                          _ptr(C_out), C_out.stride(0), _ptr(C_raw), ws_ptr, ws.numel() - off, _stream(stream)),
+           "dybit_gemm")
+    return C_out, C_raw
+
+
+def dybit_conv2d(desc: ConvDesc, X: torch.Tensor, fx, scale_x: torch.Tensor,
+                 W: torch.Tensor, fw, scale_w: torch.Tensor, Y: Optional[torch.Tensor] = None,
+                 want_raw: bool = False, Y_raw: Optional[torch.Tensor] = None,
+                 ws: Optional[torch.Tensor] = None, ldw_bytes: Optional[int] = None, stream=None):
+    """Returns (Y fp32 [n][oh][ow][k], Y_raw int32 or None)."""
+    oh, ow = dybit_conv2d_out_hw(desc)
+    ldw = W.stride(0) if ldw_bytes is None else ldw_bytes
+    if Y is None:
+        Y = torch.empty((desc.n, oh, ow, desc.k), dtype=torch.float32, device=X.device)
+    if want_raw and Y_raw is None:
+        Y_raw = torch.empty((desc.n, oh, ow, desc.k), dtype=torch.int32, device=X.device)
+    if ws is None:
+        ws = torch.empty(dybit_conv2d_workspace_bytes(desc, fx, fw) + 1024, dtype=torch.uint8, device=X.device)
+    off = (-ws.data_ptr()) % 1024
+    ws_ptr = C.c_void_p(ws.data_ptr() + off)
+    cd = _cdesc(desc)
+    _check(lib.dybit_conv2d(C.byref(cd), _ptr(X), _fmt(fx), _ptr(scale_x), _ptr(W), _fmt(fw), _ptr(scale_w), ldw,
+                            _ptr(Y), _ptr(Y_raw), ws_ptr, ws.numel() - off, _stream(stream)), "dybit_conv2d")
+    return Y, Y_raw
+
+
+def dybit_last_device_status(stream=None) -> Tuple[int, int]:
+    detail = C.c_uint32(0)
+    st = lib.dybit_last_device_status(_stream(stream), C.byref(detail))
+    return int(st), int(detail.value)

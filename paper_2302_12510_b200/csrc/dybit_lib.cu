@@ -1,0 +1,5 @@
+// libdybit: single translation unit (the device status word and the kernels
+// share one module, so no relocatable device code is needed).
+#include "dybit_host.cuh"
+#include "dybit_quantize.cuh"
+#include "dybit_gemm.cuh"

@@ -1,0 +1,475 @@
+// Streaming kernels: max-abs scale, quantize + pack, decode.  All HBM-bound.
+//
+// Work is cut into "chunks" of 1024 consecutive codes of one row (a 1-D tensor
+// is a single row).  One warp owns a chunk: eight coalesced 128-bit loads per
+// lane, encode in registers, a byte-wide transpose through shared memory so
+// that each lane holds 32 consecutive codes, a register bit-pack into `BITS`
+// 32-bit words, and coalesced 128-bit stores.  A chunk's output always starts
+// on a 16-byte boundary (1024 codes = 128 * BITS bytes).
+#pragma once
+
+#include "dybit_common.cuh"
+
+namespace dybit {
+
+constexpr int kChunkCodes = 1024;
+constexpr int kWarpsPerBlock = 8;
+constexpr int kStreamThreads = kWarpsPerBlock * 32;
+
+// ------------------------------------------------------------------ encode
+
+// Magnitude code of t = |x| / scale for M magnitude bits (inverse of Eq. 1).
+// Codes grow with the value they stand for, so the nearest code is found the
+// way a float is rounded: take the binade e of t (the sub-unit codes form one
+// linear region, e = -1), scale t so that one code step is 1.0, subtract the
+// binade's first code's offset and round to nearest-even; a carry out of the
+// fraction runs into the unary exponent field, which is exactly the first
+// code of the next binade (the encoder of Section III-B.2 places e+1 ones,
+// a zero and the leading fraction bits).  Every float operation below is
+// exact except the final round-to-integer.
+template <int M>
+__device__ __forceinline__ unsigned encode_magnitude(float t) {
+    constexpr unsigned kAllOnes = (1u << M) - 1u;
+    constexpr float kVmax = (float)(1u << (M - 1));
+    int e = (int)(__float_as_uint(t) >> 23) - 127;      // t >= 0: sign bit clear
+    e = max(e, -1);
+    e = min(e, M - 2);
+    const bool sub_unit = e < 0;
+    const int k = M - 2 - e;                            // fraction bits in binade e (e >= 0)
+    const int up = sub_unit ? (M - 1) : (k - e);        // t * 2^up: one code step == 1.0
+    const float offs = sub_unit ? 0.0f : (float)(1 << k);
+    const float p2 = __uint_as_float((unsigned)(127 + up) << 23);
+    const int r = __float2int_rn(__fmaf_rn(t, p2, -offs));
+    const unsigned base = (1u << M) - (1u << (M - 1 - e));   // e+1 ones, then zeros
+    unsigned mag = base + (unsigned)r;
+    mag = (t >= kVmax) ? kAllOnes : mag;
+    mag = (t != t) ? 0u : mag;
+    return mag;
+}
+
+template <int BITS, bool SIGNED>
+__device__ __forceinline__ unsigned encode_code(float x, float inv) {
+    constexpr int M = SIGNED ? BITS - 1 : BITS;
+    const float t = __fmul_rn(fabsf(x), inv);
+    unsigned mag = encode_magnitude<M>(t);
+    const unsigned neg = __float_as_uint(x) >> 31;
+    if (SIGNED) {
+        return mag | ((mag != 0u ? neg : 0u) << M);
+    } else {
+        return neg ? 0u : mag;
+    }
+}
+
+// ------------------------------------------------------------------ absmax
+
+__device__ __forceinline__ unsigned finite_abs_bits(float v) {
+    unsigned b = __float_as_uint(v) & 0x7fffffffu;
+    return b < 0x7f800000u ? b : 0u;
+}
+
+// Largest finite |x| as raw fp32 bits (non-negative floats order like their
+// bit patterns), max-reduced into *slot, which the host zeroes beforehand.
+// Handles rows x cols with leading dimension ld (ld == cols: one flat run).
+__global__ void __launch_bounds__(kStreamThreads)
+absmax_kernel(const float *__restrict__ x, int64_t rows, int64_t cols, int64_t ld,
+              unsigned *__restrict__ slot) {
+    unsigned best = 0;
+    const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t nthreads = (int64_t)gridDim.x * blockDim.x;
+    if (ld == cols) {
+        const int64_t n = rows * cols;
+        // scalar head up to the first 16-byte boundary, vector body, scalar tail
+        int64_t head = ((16 - (reinterpret_cast<uintptr_t>(x) & 15)) & 15) / 4;
+        if (head > n) head = n;
+        const int64_t nvec = (n - head) / 4;
+        const float4 *xv = reinterpret_cast<const float4 *>(x + head);
+        constexpr int kUnroll = 4;
+        int64_t i = tid;
+        for (; i + (kUnroll - 1) * nthreads < nvec; i += kUnroll * nthreads) {
+            float4 v[kUnroll];
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) v[u] = __ldcs(xv + i + u * nthreads);
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) {
+                best = max(best, max(max(finite_abs_bits(v[u].x), finite_abs_bits(v[u].y)),
+                                     max(finite_abs_bits(v[u].z), finite_abs_bits(v[u].w))));
+            }
+        }
+        for (; i < nvec; i += nthreads) {
+            float4 v = __ldcs(xv + i);
+            best = max(best, max(max(finite_abs_bits(v.x), finite_abs_bits(v.y)),
+                                 max(finite_abs_bits(v.z), finite_abs_bits(v.w))));
+        }
+        if (tid < head) best = max(best, finite_abs_bits(x[tid]));
+        const int64_t tail0 = head + nvec * 4;
+        if (tail0 + tid < n) best = max(best, finite_abs_bits(x[tail0 + tid]));   // tail < 4 elements
+    } else {
+        const int64_t total = rows * cols;
+        for (int64_t i = tid; i < total; i += nthreads) {
+            const int64_t r = i / cols, c = i - r * cols;
+            best = max(best, finite_abs_bits(x[r * ld + c]));
+        }
+    }
+    best = __reduce_max_sync(0xffffffffu, best);
+    __shared__ unsigned warp_best[kWarpsPerBlock];
+    if ((threadIdx.x & 31) == 0) warp_best[threadIdx.x >> 5] = best;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        unsigned b = threadIdx.x < kWarpsPerBlock ? warp_best[threadIdx.x] : 0u;
+        b = __reduce_max_sync(0xffffffffu, b);
+        if (threadIdx.x == 0 && b != 0u) atomicMax(slot, b);
+    }
+}
+
+// slot holds amax bits in scale[0] on entry; leaves {scale, 1/scale}.
+__global__ void finalize_scale_kernel(float *scale, int m) {
+    const float amax = scale[0];
+    if (amax == 0.0f) {
+        scale[0] = 1.0f;
+        scale[1] = 1.0f;
+    } else {
+        const float vmax = (float)(1u << (m - 1));
+        scale[0] = __fdiv_rn(amax, vmax);
+        scale[1] = __fdiv_rn(vmax, amax);
+    }
+}
+
+// ------------------------------------------------------------------ quantize + pack
+
+// Packs this lane's 32 consecutive codes (bytes, low to high) into BITS words.
+template <int BITS>
+__device__ __forceinline__ void pack32(const unsigned (&cw)[8], unsigned (&out)[BITS]) {
+    unsigned long long acc = 0;
+    int nb = 0, w = 0;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+        const unsigned code = (cw[i >> 2] >> ((i & 3) * 8)) & 0xffu;
+        acc |= (unsigned long long)code << nb;
+        nb += BITS;
+        if (nb >= 32) {
+            out[w++] = (unsigned)acc;
+            acc >>= 32;
+            nb -= 32;
+        }
+    }
+}
+
+template <int BITS, bool SIGNED>
+__global__ void __launch_bounds__(kStreamThreads)
+quantize_pack_kernel(const float *__restrict__ x, int64_t rows, int64_t cols, int64_t ld,
+                     const float *__restrict__ scale, uint8_t *__restrict__ out,
+                     int64_t row_stride_bytes, int64_t chunks_per_row) {
+    __shared__ __align__(16) unsigned s_codes[kWarpsPerBlock][kChunkCodes / 4];
+    __shared__ __align__(16) unsigned s_words[kWarpsPerBlock][32 * BITS];
+
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const float inv = __ldg(scale + 1);
+    const int64_t items = rows * chunks_per_row;
+    const int64_t warp0 = (int64_t)blockIdx.x * kWarpsPerBlock + warp;
+    const int64_t nwarps = (int64_t)gridDim.x * kWarpsPerBlock;
+    constexpr int kChunkBytes = kChunkCodes * BITS / 8;       // 128 * BITS
+    constexpr int kChunkVecs = kChunkBytes / 16;              // 8 * BITS
+
+    for (int64_t item = warp0; item < items; item += nwarps) {
+        const int64_t row = item / chunks_per_row;
+        const int64_t chunk = item - row * chunks_per_row;
+        const int64_t c0 = chunk * kChunkCodes;
+        const float *src = x + row * ld + c0;
+        const int64_t valid = min((int64_t)kChunkCodes, max((int64_t)0, cols - c0));
+        const int64_t bytes_left = row_stride_bytes - chunk * kChunkBytes;
+        const int nvec = (int)min((int64_t)kChunkVecs, bytes_left / 16);
+        const bool vec_ok = (reinterpret_cast<uintptr_t>(src) & 15) == 0;
+
+        float4 v[8];
+        if (valid == kChunkCodes && vec_ok) {
+            const float4 *s4 = reinterpret_cast<const float4 *>(src);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) v[j] = __ldcs(s4 + j * 32 + lane);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int64_t i0 = j * 128 + lane * 4;
+                v[j].x = (i0 + 0 < valid) ? src[i0 + 0] : 0.0f;
+                v[j].y = (i0 + 1 < valid) ? src[i0 + 1] : 0.0f;
+                v[j].z = (i0 + 2 < valid) ? src[i0 + 2] : 0.0f;
+                v[j].w = (i0 + 3 < valid) ? src[i0 + 3] : 0.0f;
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const unsigned c = encode_code<BITS, SIGNED>(v[j].x, inv) |
+                               (encode_code<BITS, SIGNED>(v[j].y, inv) << 8) |
+                               (encode_code<BITS, SIGNED>(v[j].z, inv) << 16) |
+                               (encode_code<BITS, SIGNED>(v[j].w, inv) << 24);
+            s_codes[warp][j * 32 + lane] = c;
+        }
+        __syncwarp();
+        // lane takes codes [32*lane, 32*lane + 32); the two 16-byte halves are
+        // read in lane-dependent order so that a quarter-warp spreads over all banks
+        unsigned cw[8];
+        {
+            const uint4 *s4 = reinterpret_cast<const uint4 *>(&s_codes[warp][lane * 8]);
+            const int first = (lane >> 2) & 1;
+            uint4 a = s4[first], b = s4[first ^ 1];
+            if (first) { uint4 t = a; a = b; b = t; }
+            cw[0] = a.x; cw[1] = a.y; cw[2] = a.z; cw[3] = a.w;
+            cw[4] = b.x; cw[5] = b.y; cw[6] = b.z; cw[7] = b.w;
+        }
+        unsigned w[BITS];
+        pack32<BITS>(cw, w);
+        uint8_t *dst = out + row * row_stride_bytes + chunk * kChunkBytes;
+        if constexpr (BITS == 4) {
+            if (lane < nvec) reinterpret_cast<uint4 *>(dst)[lane] = make_uint4(w[0], w[1], w[2], w[3]);
+        } else if constexpr (BITS == 8) {
+            if (2 * lane < nvec) reinterpret_cast<uint4 *>(dst)[2 * lane] = make_uint4(w[0], w[1], w[2], w[3]);
+            if (2 * lane + 1 < nvec) reinterpret_cast<uint4 *>(dst)[2 * lane + 1] = make_uint4(w[4], w[5], w[6], w[7]);
+        } else if constexpr (BITS == 2) {
+            if ((lane >> 1) < nvec) reinterpret_cast<uint2 *>(dst)[lane] = make_uint2(w[0], w[1]);
+        } else {
+#pragma unroll
+            for (int i = 0; i < BITS; ++i) s_words[warp][lane * BITS + i] = w[i];
+            __syncwarp();
+            const uint4 *s4 = reinterpret_cast<const uint4 *>(&s_words[warp][0]);
+            for (int i = lane; i < nvec; i += 32) reinterpret_cast<uint4 *>(dst)[i] = s4[i];
+        }
+        __syncwarp();
+    }
+}
+
+// ------------------------------------------------------------------ decode
+
+struct FloatTable { float v[256]; };
+
+// Inverse of pack32: BITS words -> this lane's 32 codes as bytes in 8 words.
+template <int BITS>
+__device__ __forceinline__ void unpack32(const unsigned (&in)[BITS], unsigned (&cw)[8]) {
+    unsigned long long acc = 0;
+    int nb = 0, w = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) cw[i] = 0;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+        if (nb < BITS) {
+            acc |= (unsigned long long)in[w++] << nb;
+            nb += 32;
+        }
+        const unsigned code = (unsigned)acc & ((1u << BITS) - 1u);
+        acc >>= BITS;
+        nb -= BITS;
+        cw[i >> 2] |= code << ((i & 3) * 8);
+    }
+}
+
+template <int BITS>
+__global__ void __launch_bounds__(kStreamThreads)
+decode_kernel(const uint8_t *__restrict__ packed, int64_t n, const float *__restrict__ scale,
+              const __grid_constant__ FloatTable table, float *__restrict__ out) {
+    __shared__ float s_lut[256];
+    __shared__ __align__(16) unsigned s_words[kWarpsPerBlock][32 * BITS];
+    __shared__ __align__(16) unsigned s_codes[kWarpsPerBlock][kChunkCodes / 4];
+    const float sc = scale ? __ldg(scale) : 1.0f;
+    for (int i = threadIdx.x; i < 256; i += blockDim.x) s_lut[i] = __fmul_rn(sc, table.v[i]);
+    __syncthreads();
+
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    constexpr int kChunkBytes = kChunkCodes * BITS / 8;
+    constexpr int kChunkVecs = kChunkBytes / 16;
+    const int64_t packed_bytes = ((n * BITS + 7) / 8 + 15) / 16 * 16;
+    const int64_t items = (n + kChunkCodes - 1) / kChunkCodes;
+    const int64_t warp0 = (int64_t)blockIdx.x * kWarpsPerBlock + warp;
+    const int64_t nwarps = (int64_t)gridDim.x * kWarpsPerBlock;
+    const bool out_vec_ok = (reinterpret_cast<uintptr_t>(out) & 15) == 0;
+
+    for (int64_t item = warp0; item < items; item += nwarps) {
+        const int64_t c0 = item * kChunkCodes;
+        const int64_t valid = min((int64_t)kChunkCodes, n - c0);
+        const int nvec = (int)min((int64_t)kChunkVecs, (packed_bytes - item * kChunkBytes) / 16);
+        const uint4 *src = reinterpret_cast<const uint4 *>(packed + item * kChunkBytes);
+        uint4 *s4 = reinterpret_cast<uint4 *>(&s_words[warp][0]);
+        for (int i = lane; i < kChunkVecs; i += 32) s4[i] = (i < nvec) ? __ldcs(src + i) : make_uint4(0, 0, 0, 0);
+        __syncwarp();
+        unsigned w[BITS], cw[8];
+#pragma unroll
+        for (int i = 0; i < BITS; ++i) w[i] = s_words[warp][lane * BITS + i];
+        unpack32<BITS>(w, cw);
+        {
+            uint4 *c4 = reinterpret_cast<uint4 *>(&s_codes[warp][lane * 8]);
+            c4[0] = make_uint4(cw[0], cw[1], cw[2], cw[3]);
+            c4[1] = make_uint4(cw[4], cw[5], cw[6], cw[7]);
+        }
+        __syncwarp();
+        float *dst = out + c0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const unsigned c = s_codes[warp][j * 32 + lane];
+            float4 r;
+            r.x = s_lut[c & 0xffu];
+            r.y = s_lut[(c >> 8) & 0xffu];
+            r.z = s_lut[(c >> 16) & 0xffu];
+            r.w = s_lut[c >> 24];
+            const int64_t i0 = j * 128 + lane * 4;
+            if (out_vec_ok && i0 + 3 < valid) {
+                __stcs(reinterpret_cast<float4 *>(dst + i0), r);
+            } else {
+                if (i0 + 0 < valid) dst[i0 + 0] = r.x;
+                if (i0 + 1 < valid) dst[i0 + 1] = r.y;
+                if (i0 + 2 < valid) dst[i0 + 2] = r.z;
+                if (i0 + 3 < valid) dst[i0 + 3] = r.w;
+            }
+        }
+        __syncwarp();
+    }
+}
+
+// ------------------------------------------------------------------ host launchers
+
+static int stream_grid(int64_t items_per_warp_unit) {
+    // persistent-style grid: a few blocks per SM, never more than the work
+    int64_t blocks = (items_per_warp_unit + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    int64_t cap = (int64_t)sm_count() * 8;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    return (int)blocks;
+}
+
+static dybit_status launch_absmax(const float *x, int64_t rows, int64_t cols, int64_t ld, dybit_fmt fmt,
+                                  float *scale_out, cudaStream_t s) {
+    DYBIT_CUDA_TRY(cudaMemsetAsync(scale_out, 0, 2 * sizeof(float), s));
+    const int64_t n = rows * cols;
+    if (n > 0) {
+        int64_t blocks = (n / 4 + kStreamThreads * 4 - 1) / (kStreamThreads * 4);
+        int64_t cap = (int64_t)sm_count() * 8;
+        if (blocks > cap) blocks = cap;
+        if (blocks < 1) blocks = 1;
+        absmax_kernel<<<(int)blocks, kStreamThreads, 0, s>>>(x, rows, cols, ld,
+                                                             reinterpret_cast<unsigned *>(scale_out));
+        if (launch_status() != DYBIT_OK) return DYBIT_ERR_CUDA;
+    }
+    finalize_scale_kernel<<<1, 1, 0, s>>>(scale_out, mag_bits(fmt));
+    return launch_status();
+}
+
+template <int BITS>
+static dybit_status launch_quantize_bits(const float *x, int64_t rows, int64_t cols, int64_t ld, bool is_signed,
+                                         const float *scale, uint8_t *out, int64_t row_stride_bytes,
+                                         cudaStream_t s) {
+    constexpr int kChunkBytes = kChunkCodes * BITS / 8;
+    const int64_t chunks_per_row = (row_stride_bytes + kChunkBytes - 1) / kChunkBytes;
+    const int64_t items = rows * chunks_per_row;
+    if (items == 0) return DYBIT_OK;
+    const int grid = stream_grid(items);
+    if (is_signed)
+        quantize_pack_kernel<BITS, true><<<grid, kStreamThreads, 0, s>>>(x, rows, cols, ld, scale, out,
+                                                                        row_stride_bytes, chunks_per_row);
+    else
+        quantize_pack_kernel<BITS, false><<<grid, kStreamThreads, 0, s>>>(x, rows, cols, ld, scale, out,
+                                                                         row_stride_bytes, chunks_per_row);
+    return launch_status();
+}
+
+static dybit_status launch_quantize(const float *x, int64_t rows, int64_t cols, int64_t ld, dybit_fmt fmt,
+                                    const float *scale, uint8_t *out, int64_t row_stride_bytes,
+                                    cudaStream_t s) {
+    const bool sg = fmt.is_signed != 0;
+    switch (fmt.bits) {
+        case 2: return launch_quantize_bits<2>(x, rows, cols, ld, sg, scale, out, row_stride_bytes, s);
+        case 3: return launch_quantize_bits<3>(x, rows, cols, ld, sg, scale, out, row_stride_bytes, s);
+        case 4: return launch_quantize_bits<4>(x, rows, cols, ld, sg, scale, out, row_stride_bytes, s);
+        case 5: return launch_quantize_bits<5>(x, rows, cols, ld, sg, scale, out, row_stride_bytes, s);
+        case 6: return launch_quantize_bits<6>(x, rows, cols, ld, sg, scale, out, row_stride_bytes, s);
+        case 7: return launch_quantize_bits<7>(x, rows, cols, ld, sg, scale, out, row_stride_bytes, s);
+        case 8: return launch_quantize_bits<8>(x, rows, cols, ld, sg, scale, out, row_stride_bytes, s);
+    }
+    return DYBIT_ERR_INVALID_ARG;
+}
+
+template <int BITS>
+static dybit_status launch_decode_bits(const uint8_t *packed, int64_t n, const float *scale,
+                                       const FloatTable &table, float *out, cudaStream_t s) {
+    const int64_t items = (n + kChunkCodes - 1) / kChunkCodes;
+    if (items == 0) return DYBIT_OK;
+    decode_kernel<BITS><<<stream_grid(items), kStreamThreads, 0, s>>>(packed, n, scale, table, out);
+    return launch_status();
+}
+
+}  // namespace dybit
+
+extern "C" {
+
+dybit_status dybit_absmax_scale(const float *x, int64_t n, dybit_fmt fmt, float *scale_out, void *stream) {
+    using namespace dybit;
+    if (!fmt_ok(fmt) || n < 0 || scale_out == nullptr || (n > 0 && x == nullptr)) return DYBIT_ERR_INVALID_ARG;
+    if (!aligned(x, 4) || !aligned(scale_out, 4)) return DYBIT_ERR_ALIGNMENT;
+    return launch_absmax(x, 1, n, n, fmt, scale_out, static_cast<cudaStream_t>(stream));
+}
+
+dybit_status dybit_quantize_pack(const float *x, int64_t n, dybit_fmt fmt, const float *scale, void *packed,
+                                 float *scale_out, void *stream) {
+    using namespace dybit;
+    if (!fmt_ok(fmt) || n < 0) return DYBIT_ERR_INVALID_ARG;
+    if (n > 0 && (x == nullptr || packed == nullptr)) return DYBIT_ERR_INVALID_ARG;
+    if (scale == nullptr && scale_out == nullptr) return DYBIT_ERR_INVALID_ARG;
+    if (!aligned(x, 4) || !aligned(packed, 16) || !aligned(scale, 4) || !aligned(scale_out, 4))
+        return DYBIT_ERR_ALIGNMENT;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (scale == nullptr) {
+        dybit_status st = launch_absmax(x, 1, n, n, fmt, scale_out, s);
+        if (st != DYBIT_OK) return st;
+        scale = scale_out;
+    } else if (scale_out != nullptr && scale_out != scale) {
+        DYBIT_CUDA_TRY(cudaMemcpyAsync(scale_out, scale, 2 * sizeof(float), cudaMemcpyDeviceToDevice, s));
+    }
+    if (n == 0) return DYBIT_OK;
+    return launch_quantize(x, 1, n, n, fmt, scale, static_cast<uint8_t *>(packed),
+                           (int64_t)dybit_packed_bytes(n, fmt.bits), s);
+}
+
+dybit_status dybit_quantize_pack_2d(const float *x, int64_t rows, int64_t cols, int64_t ld, dybit_fmt fmt,
+                                    const float *scale, void *packed, int64_t row_stride_bytes,
+                                    float *scale_out, void *stream) {
+    using namespace dybit;
+    if (!fmt_ok(fmt) || rows < 0 || cols <= 0 || ld < cols) return DYBIT_ERR_INVALID_ARG;
+    if (rows > 0 && (x == nullptr || packed == nullptr)) return DYBIT_ERR_INVALID_ARG;
+    if (scale == nullptr && scale_out == nullptr) return DYBIT_ERR_INVALID_ARG;
+    if (row_stride_bytes < (int64_t)dybit_row_stride_bytes(cols, fmt.bits)) return DYBIT_ERR_INVALID_ARG;
+    if (row_stride_bytes % 16 != 0 || !aligned(x, 4) || !aligned(packed, 16) || !aligned(scale, 4) ||
+        !aligned(scale_out, 4))
+        return DYBIT_ERR_ALIGNMENT;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (scale == nullptr) {
+        dybit_status st = launch_absmax(x, rows, cols, ld, fmt, scale_out, s);
+        if (st != DYBIT_OK) return st;
+        scale = scale_out;
+    } else if (scale_out != nullptr && scale_out != scale) {
+        DYBIT_CUDA_TRY(cudaMemcpyAsync(scale_out, scale, 2 * sizeof(float), cudaMemcpyDeviceToDevice, s));
+    }
+    if (rows == 0) return DYBIT_OK;
+    return launch_quantize(x, rows, cols, ld, fmt, scale, static_cast<uint8_t *>(packed), row_stride_bytes, s);
+}
+
+dybit_status dybit_decode(const void *packed, int64_t n, dybit_fmt fmt, const float *scale, float *out,
+                          void *stream) {
+    using namespace dybit;
+    if (!fmt_ok(fmt) || n < 0) return DYBIT_ERR_INVALID_ARG;
+    if (n > 0 && (packed == nullptr || out == nullptr)) return DYBIT_ERR_INVALID_ARG;
+    if (!aligned(packed, 16) || !aligned(out, 4) || !aligned(scale, 4)) return DYBIT_ERR_ALIGNMENT;
+    if (n == 0) return DYBIT_OK;
+    FloatTable table;
+    fill_table(fmt, table.v);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const uint8_t *p = static_cast<const uint8_t *>(packed);
+    switch (fmt.bits) {
+        case 2: return launch_decode_bits<2>(p, n, scale, table, out, s);
+        case 3: return launch_decode_bits<3>(p, n, scale, table, out, s);
+        case 4: return launch_decode_bits<4>(p, n, scale, table, out, s);
+        case 5: return launch_decode_bits<5>(p, n, scale, table, out, s);
+        case 6: return launch_decode_bits<6>(p, n, scale, table, out, s);
+        case 7: return launch_decode_bits<7>(p, n, scale, table, out, s);
+        case 8: return launch_decode_bits<8>(p, n, scale, table, out, s);
+    }
+    return DYBIT_ERR_INVALID_ARG;
+}
+
+}  // extern "C"
