@@ -152,7 +152,10 @@ unsigned orc_encode_one(float x, float inv, int bits, int is_signed)
     unsigned best = 0;
     if (isnan(t)) {
         best = 0;
-    } else if (isinf(t)) {
+    } else if (isinf(t) || (double)t >= orc_decode_mag(m, ncodes - 1u)) {
+        /* at or beyond the largest value: the nearest value is the largest one.
+         * (Taken explicitly because for huge t the distances below would all
+         * round to the same double.) */
         best = ncodes - 1u;
     } else {
         double bestd = INFINITY;

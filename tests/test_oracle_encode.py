@@ -150,6 +150,8 @@ def test_special_values_and_saturation(bits, signed):
     assert orc.encode_one(np.inf, 1.0, bits, signed) == ones
     assert orc.encode_one(3e38, 1e30, bits, signed) == ones      # product overflows to inf
     assert orc.encode_one(2.0 ** (m - 1) * 1.5, 1.0, bits, signed) == ones
+    assert orc.encode_one(3e38, 1.0, bits, signed) == ones            # finite, far beyond double's exact range of distances
+    assert orc.encode_one(1e20, 1.0, bits, signed) == ones
     assert orc.encode_one(0.0, 1.0, bits, signed) == 0
     assert orc.encode_one(-0.0, 1.0, bits, signed) == 0
     assert orc.encode_one(-1e-30, 1.0, bits, signed) == 0
