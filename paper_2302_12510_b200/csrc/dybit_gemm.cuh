@@ -1,13 +1,726 @@
-// placeholder until the tcgen05 GEMM lands
+// GEMM / implicit-GEMM convolution on DyBit-coded operands.
+//
+// Two steps per call:
+//   1. expand: packed codes -> the container type (int8 / e4m3 / bf16) through
+//      the enumerated value table, written once into caller workspace
+//      (O(MK + NK) work, HBM-bound);
+//   2. a persistent, warp-specialised tcgen05 GEMM on the expanded operands:
+//      TMA (128-byte swizzle) -> shared-memory ring -> tcgen05.mma with the
+//      accumulator in tensor memory -> epilogue warps read TMEM, apply alpha
+//      and store fp32 (and the raw int32 sum when asked).
+// The convolution is the same kernel with the A tile gathered straight from the
+// expanded NHWC activation (im2col addressing, zero fill for padding taps).
 #pragma once
+
 #include "dybit_common.cuh"
-extern "C" {
-size_t dybit_gemm_workspace_bytes(int64_t, int64_t, int64_t, dybit_fmt, dybit_fmt) { return 0; }
-size_t dybit_conv2d_workspace_bytes(const dybit_conv_desc *, dybit_fmt, dybit_fmt) { return 0; }
-dybit_status dybit_gemm(int64_t, int64_t, int64_t, const void *, dybit_fmt, const float *, int64_t,
-                        const void *, dybit_fmt, const float *, int64_t, float *, int64_t, int32_t *,
-                        void *, size_t, void *) { return DYBIT_ERR_UNSUPPORTED; }
-dybit_status dybit_conv2d(const dybit_conv_desc *, const void *, dybit_fmt, const float *,
-                          const void *, dybit_fmt, const float *, int64_t, float *, int32_t *,
-                          void *, size_t, void *) { return DYBIT_ERR_UNSUPPORTED; }
+#include "dybit_host.cuh"
+#include "dybit_quantize.cuh"
+#include "dybit_sm100.cuh"
+
+namespace dybit {
+
+using namespace sm100;
+
+// ------------------------------------------------------------------ expand kernels
+
+struct ElemTable {
+    uint16_t v[256];   // container bit pattern of each code's value (low byte used for 1-byte containers)
+};
+
+// bf16 / e4m3 / int8 bit patterns of a value that is known to be exactly representable.
+static uint16_t to_bf16_bits(float v) {
+    uint32_t u;
+    memcpy(&u, &v, 4);
+    return (uint16_t)(u >> 16);
 }
+
+static uint8_t to_e4m3_bits(float v) {
+    if (v == 0.0f) return 0;
+    uint8_t sign = v < 0 ? 0x80 : 0;
+    float a = fabsf(v);
+    int e;
+    float fr = frexpf(a, &e);            // a = fr * 2^e, fr in [0.5,1)  ->  1.f * 2^(e-1)
+    int exp = e - 1;
+    if (exp >= -6) {
+        int mant = (int)lrintf(ldexpf(fr, 4)) - 8;          // 3 fraction bits
+        return sign | (uint8_t)(((exp + 7) << 3) | mant);
+    }
+    int mant = (int)lrintf(ldexpf(a, 9));                   // subnormal: multiples of 2^-9
+    return sign | (uint8_t)mant;
+}
+
+static ElemTable make_elem_table(dybit_fmt f, dybit_container cont, int int_exp) {
+    float tab[256];
+    fill_table(f, tab);
+    ElemTable t;
+    for (int c = 0; c < 256; ++c) {
+        switch (cont) {
+            case DYBIT_CONTAINER_I8: t.v[c] = (uint16_t)(uint8_t)(int8_t)lrintf(ldexpf(tab[c], int_exp)); break;
+            case DYBIT_CONTAINER_E4M3: t.v[c] = to_e4m3_bits(tab[c]); break;
+            default: t.v[c] = to_bf16_bits(tab[c]); break;
+        }
+    }
+    return t;
+}
+
+// Rows of packed codes -> rows of container elements.  A warp expands 1024 codes at a time.
+template <int BITS, int ELEM>
+__global__ void __launch_bounds__(kStreamThreads)
+expand_rows_kernel(const uint8_t *__restrict__ packed, int64_t rows, int64_t in_stride, int64_t cols,
+                   uint8_t *__restrict__ out, int64_t out_stride, const __grid_constant__ ElemTable table) {
+    __shared__ uint16_t s_lut[256];
+    __shared__ __align__(16) unsigned s_words[kWarpsPerBlock][32 * BITS];
+    for (int i = threadIdx.x; i < 256; i += blockDim.x) s_lut[i] = table.v[i];
+    __syncthreads();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    constexpr int kChunkBytes = kChunkCodes * BITS / 8;
+    constexpr int kChunkVecs = kChunkBytes / 16;
+    const int64_t chunks_per_row = (cols + kChunkCodes - 1) / kChunkCodes;
+    const int64_t items = rows * chunks_per_row;
+    const int64_t in_row_bytes = ((cols * BITS + 7) / 8 + 15) / 16 * 16;
+    for (int64_t item = (int64_t)blockIdx.x * kWarpsPerBlock + warp; item < items;
+         item += (int64_t)gridDim.x * kWarpsPerBlock) {
+        const int64_t row = item / chunks_per_row, chunk = item - row * chunks_per_row;
+        const int64_t c0 = chunk * kChunkCodes;
+        const int valid = (int)min((int64_t)kChunkCodes, cols - c0);
+        const int nvec = (int)min((int64_t)kChunkVecs, (in_row_bytes - chunk * kChunkBytes) / 16);
+        const uint4 *src = reinterpret_cast<const uint4 *>(packed + row * in_stride + chunk * kChunkBytes);
+        uint4 *s4 = reinterpret_cast<uint4 *>(&s_words[warp][0]);
+        for (int i = lane; i < kChunkVecs; i += 32) s4[i] = (i < nvec) ? __ldg(src + i) : make_uint4(0, 0, 0, 0);
+        __syncwarp();
+        unsigned w[BITS], cw[8];
+#pragma unroll
+        for (int i = 0; i < BITS; ++i) w[i] = s_words[warp][lane * BITS + i];
+        unpack32<BITS>(w, cw);
+        uint8_t *dst = out + row * out_stride + (c0 + lane * 32) * ELEM;
+        if constexpr (ELEM == 1) {
+            unsigned o[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                o[i] = (unsigned)(s_lut[cw[i] & 0xffu] & 0xffu) | ((unsigned)(s_lut[(cw[i] >> 8) & 0xffu] & 0xffu) << 8) |
+                       ((unsigned)(s_lut[(cw[i] >> 16) & 0xffu] & 0xffu) << 16) |
+                       ((unsigned)(s_lut[cw[i] >> 24] & 0xffu) << 24);
+            }
+            if (lane * 32 < valid) reinterpret_cast<uint4 *>(dst)[0] = make_uint4(o[0], o[1], o[2], o[3]);
+            if (lane * 32 + 16 < valid) reinterpret_cast<uint4 *>(dst)[1] = make_uint4(o[4], o[5], o[6], o[7]);
+        } else {
+            unsigned o[16];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                o[2 * i] = (unsigned)s_lut[cw[i] & 0xffu] | ((unsigned)s_lut[(cw[i] >> 8) & 0xffu] << 16);
+                o[2 * i + 1] = (unsigned)s_lut[(cw[i] >> 16) & 0xffu] | ((unsigned)s_lut[cw[i] >> 24] << 16);
+            }
+#pragma unroll
+            for (int v = 0; v < 4; ++v)
+                if (lane * 32 + v * 8 < valid)
+                    reinterpret_cast<uint4 *>(dst)[v] = make_uint4(o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
+        }
+        __syncwarp();
+    }
+}
+
+// Generic (slow) expand with channel padding: output row = taps x cp elements, where tap t
+// takes codes [t*c, t*c + c) of the input row's bit stream and pads channels c..cp-1 with 0.
+// One thread writes one 16-byte output chunk.
+__global__ void expand_pad_kernel(const uint8_t *__restrict__ packed, int bits, int64_t rows, int64_t in_stride,
+                                  int64_t taps, int c, int cp, int elem, uint8_t *__restrict__ out,
+                                  int64_t out_stride, const __grid_constant__ ElemTable table) {
+    const int per_chunk = 16 / elem;
+    const int64_t chunks_per_tap = cp / per_chunk;
+    const int64_t total = rows * taps * chunks_per_tap;
+    for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+         idx += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t g = idx % chunks_per_tap;
+        const int64_t t = (idx / chunks_per_tap) % taps;
+        const int64_t row = idx / (chunks_per_tap * taps);
+        const uint8_t *src = packed + row * in_stride;
+        unsigned o[4] = {0, 0, 0, 0};
+        for (int e = 0; e < per_chunk; ++e) {
+            const int ch = (int)g * per_chunk + e;
+            unsigned code = 0;
+            if (ch < c) {
+                const int64_t bit = (t * c + ch) * bits;
+                const int sh = (int)(bit & 7);
+                unsigned two = src[bit >> 3];
+                if (sh + bits > 8) two |= (unsigned)src[(bit >> 3) + 1] << 8;
+                code = (two >> sh) & ((1u << bits) - 1u);
+            }
+            const unsigned v = table.v[code];
+            if (elem == 1) o[e >> 2] |= (v & 0xffu) << ((e & 3) * 8);
+            else o[e >> 1] |= v << ((e & 1) * 16);
+        }
+        uint8_t *dst = out + row * out_stride + (t * cp + g * per_chunk) * elem;
+        *reinterpret_cast<uint4 *>(dst) = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+}
+
+template <int ELEM>
+static dybit_status launch_expand_rows(const uint8_t *packed, int bits, int64_t rows, int64_t in_stride, int64_t cols,
+                                       uint8_t *out, int64_t out_stride, const ElemTable &t, cudaStream_t s) {
+    const int64_t items = rows * ((cols + kChunkCodes - 1) / kChunkCodes);
+    if (items == 0) return DYBIT_OK;
+    const int grid = stream_grid(items);
+    switch (bits) {
+        case 2: expand_rows_kernel<2, ELEM><<<grid, kStreamThreads, 0, s>>>(packed, rows, in_stride, cols, out, out_stride, t); break;
+        case 3: expand_rows_kernel<3, ELEM><<<grid, kStreamThreads, 0, s>>>(packed, rows, in_stride, cols, out, out_stride, t); break;
+        case 4: expand_rows_kernel<4, ELEM><<<grid, kStreamThreads, 0, s>>>(packed, rows, in_stride, cols, out, out_stride, t); break;
+        case 5: expand_rows_kernel<5, ELEM><<<grid, kStreamThreads, 0, s>>>(packed, rows, in_stride, cols, out, out_stride, t); break;
+        case 6: expand_rows_kernel<6, ELEM><<<grid, kStreamThreads, 0, s>>>(packed, rows, in_stride, cols, out, out_stride, t); break;
+        case 7: expand_rows_kernel<7, ELEM><<<grid, kStreamThreads, 0, s>>>(packed, rows, in_stride, cols, out, out_stride, t); break;
+        case 8: expand_rows_kernel<8, ELEM><<<grid, kStreamThreads, 0, s>>>(packed, rows, in_stride, cols, out, out_stride, t); break;
+        default: return DYBIT_ERR_INVALID_ARG;
+    }
+    return launch_status();
+}
+
+static dybit_status launch_expand(const uint8_t *packed, int bits, int64_t rows, int64_t in_stride, int64_t cols,
+                                  int elem, uint8_t *out, int64_t out_stride, const ElemTable &t, cudaStream_t s) {
+    return elem == 1 ? launch_expand_rows<1>(packed, bits, rows, in_stride, cols, out, out_stride, t, s)
+                     : launch_expand_rows<2>(packed, bits, rows, in_stride, cols, out, out_stride, t, s);
+}
+
+// ------------------------------------------------------------------ the tcgen05 GEMM
+
+constexpr int kBM = 128;            // tile rows (UMMA M)
+constexpr int kBKBytes = 128;       // one swizzle row of K per pipeline stage
+constexpr int kUmmaKBytes = 32;     // K bytes consumed by one tcgen05.mma
+constexpr int kStageBytesTotal = 192 * 1024;
+constexpr unsigned long long kWaitLimitNs = 4000000000ull;
+
+struct GemmParams {
+    int M, N;                 // output extent
+    int k_blocks;             // 128-byte K blocks per row
+    int m_tiles, n_tiles;
+    float *C;
+    int32_t *C_raw;
+    int64_t ldc;
+    const float *scale_a, *scale_b;
+    double pow2;              // alpha = (float)(scale_a * scale_b * pow2)
+    // implicit-GEMM gather of A (convolution only)
+    const uint8_t *xe;        // expanded activation, [n*h*w][cpb] bytes
+    int H, W, OH, OW, R, S, stride, pad, dil;
+    int cpb;                  // bytes per pixel in xe (padded channels * element size)
+};
+
+// Waits for the phase with the given parity; gives up after kWaitLimitNs, records
+// the site in the device status word and raises the CTA-wide abort flag.
+__device__ __forceinline__ bool wait_bounded(uint64_t *bar, uint32_t parity, volatile uint32_t *abort_flag,
+                                             unsigned site) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_timer_ns();
+    unsigned spins = 0;
+    for (;;) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((++spins & 63u) == 0u) {
+            if (*abort_flag) return false;
+            if (global_timer_ns() - t0 > kWaitLimitNs) {
+                atomicOr(&g_device_status, (site << 8) | 1u);
+                *abort_flag = 1u;
+                return false;
+            }
+        }
+    }
+}
+
+template <int BN>
+struct GemmSmem {
+    static constexpr int kAStage = kBM * kBKBytes;
+    static constexpr int kBStage = BN * kBKBytes;
+    static constexpr int kStages = kStageBytesTotal / (kAStage + kBStage);
+    static constexpr int kBarrierBytes = 256;
+    static constexpr int kBytes = kStages * (kAStage + kBStage) + kBarrierBytes + 1024;   // + alignment slack
+};
+
+__device__ __forceinline__ void tile_coords(int tile, int m_tiles, int n_tiles, int &m_blk, int &n_blk) {
+    // groups of 8 tile-rows sweep all tile-columns, so one wave of CTAs shares few A and B tiles
+    constexpr int kGroup = 8;
+    const int per_group = kGroup * n_tiles;
+    const int group = tile / per_group;
+    const int first_m = group * kGroup;
+    const int gsz = min(kGroup, m_tiles - first_m);
+    const int in_group = tile - group * per_group;
+    m_blk = first_m + in_group % gsz;
+    n_blk = in_group / gsz;
+}
+
+template <Kind KIND, int BN, bool CONV>
+__global__ void __launch_bounds__(CONV ? 320 : 192, 1)
+dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                  const GemmParams p) {
+    using L = GemmSmem<BN>;
+    constexpr int kStages = L::kStages;
+    constexpr int kGatherThreads = 128;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t *a_stages = smem;
+    uint8_t *b_stages = smem + kStages * L::kAStage;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + kStages * (L::kAStage + L::kBStage));
+    uint64_t *full = bars;
+    uint64_t *empty = bars + kStages;
+    uint64_t *acc_full = bars + 2 * kStages;
+    uint64_t *acc_empty = acc_full + 2;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_empty + 2);
+    volatile uint32_t *abort_flag = tmem_slot + 1;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int total_tiles = p.m_tiles * p.n_tiles;
+    constexpr uint32_t kTmemCols = 2 * BN;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&full[s], CONV ? 1 + kGatherThreads : 1);
+            mbar_init(&empty[s], 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(&acc_full[a], 1);
+            mbar_init(&acc_empty[a], 4);
+        }
+        *abort_flag = 0;
+        fence_mbar_init();
+        if (!CONV) prefetch_tensormap(&tmap_a);
+        prefetch_tensormap(&tmap_b);
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+                int m_blk, n_blk;
+                tile_coords(tile, p.m_tiles, p.n_tiles, m_blk, n_blk);
+                for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+                    const int s = it % kStages;
+                    const uint32_t ph = (it / kStages) & 1u;
+                    if (!wait_bounded(&empty[s], ph ^ 1u, abort_flag, 1)) { ok = false; break; }
+                    mbar_arrive_expect_tx(&full[s], CONV ? L::kBStage : L::kAStage + L::kBStage);
+                    if (!CONV) tma_load_2d(a_stages + s * L::kAStage, &tmap_a, kb * kBKBytes, m_blk * kBM, &full[s]);
+                    tma_load_2d(b_stages + s * L::kBStage, &tmap_b, kb * kBKBytes, n_blk * BN, &full[s]);
+                }
+            }
+            if (!ok) {
+                // give copies already in flight a bounded time to land before the CTA retires
+                for (int i = 0; i < 64; ++i) __nanosleep(2000);
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t kCFormat = (KIND == Kind::I8) ? 2u : 1u;           // s32 : f32
+            constexpr uint32_t kABFormat = (KIND == Kind::F8F6F4) ? 0u : 1u;      // e4m3 : (s8 | bf16)
+            constexpr uint32_t idesc = umma_idesc(kCFormat, kABFormat, kBM, BN);
+            uint32_t it = 0, lt = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++lt) {
+                const uint32_t as = lt & 1u, aph = (lt >> 1) & 1u;
+                if (!wait_bounded(&acc_empty[as], aph ^ 1u, abort_flag, 2)) { ok = false; break; }
+                tc_fence_after_sync();
+                const uint32_t d = tmem_base + as * BN;
+                for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+                    const int s = it % kStages;
+                    const uint32_t ph = (it / kStages) & 1u;
+                    if (!wait_bounded(&full[s], ph, abort_flag, 3)) { ok = false; break; }
+                    tc_fence_after_sync();
+                    const uint64_t adesc = umma_desc_sw128(smem_u32(a_stages + s * L::kAStage));
+                    const uint64_t bdesc = umma_desc_sw128(smem_u32(b_stages + s * L::kBStage));
+#pragma unroll
+                    for (int k = 0; k < kBKBytes / kUmmaKBytes; ++k) {
+                        umma<KIND>(d, adesc + (uint64_t)(k * (kUmmaKBytes >> 4)), bdesc + (uint64_t)(k * (kUmmaKBytes >> 4)),
+                                   idesc, (uint32_t)((kb | k) != 0));
+                    }
+                    umma_commit(&empty[s]);
+                }
+                if (ok) umma_commit(&acc_full[as]);
+            }
+        }
+    } else if (warp < 6) {
+        // ------------------------------------------------ epilogue: TMEM -> registers -> global
+        const int q = warp & 3;                       // TMEM lane quarter this warp may read
+        const float alpha = (float)((double)__ldg(p.scale_a) * (double)__ldg(p.scale_b) * p.pow2);
+        const bool vec_ok = ((reinterpret_cast<uintptr_t>(p.C) & 15) == 0) && (p.ldc % 4 == 0) &&
+                            (p.C_raw == nullptr || (reinterpret_cast<uintptr_t>(p.C_raw) & 15) == 0);
+        uint32_t lt = 0;
+        for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++lt) {
+            int m_blk, n_blk;
+            tile_coords(tile, p.m_tiles, p.n_tiles, m_blk, n_blk);
+            const uint32_t as = lt & 1u, aph = (lt >> 1) & 1u;
+            bool ok = wait_bounded(&acc_full[as], aph, abort_flag, 4);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after_sync();
+            const int row = m_blk * kBM + q * 32 + lane;
+            const uint32_t taddr = tmem_base + as * BN + ((uint32_t)(q * 32) << 16);
+#pragma unroll 1
+            for (int cc = 0; cc < BN / 32; ++cc) {
+                uint32_t r[32];
+                tmem_ld_32x32(taddr + cc * 32, r);
+                tmem_ld_wait();
+                const int col0 = n_blk * BN + cc * 32;
+                if (row < p.M && col0 < p.N) {
+                    float *crow = p.C + (int64_t)row * p.ldc + col0;
+                    int32_t *rrow = p.C_raw ? p.C_raw + (int64_t)row * p.ldc + col0 : nullptr;
+                    float f[32];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const float acc = (KIND == Kind::I8) ? __int2float_rn((int)r[j]) : __uint_as_float(r[j]);
+                        f[j] = __fmul_rn(acc, alpha);
+                    }
+                    if (vec_ok && col0 + 32 <= p.N) {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+                            __stcs(reinterpret_cast<float4 *>(crow) + j, make_float4(f[4 * j], f[4 * j + 1], f[4 * j + 2], f[4 * j + 3]));
+                        if (KIND == Kind::I8 && rrow) {
+#pragma unroll
+                            for (int j = 0; j < 8; ++j)
+                                __stcs(reinterpret_cast<int4 *>(rrow) + j, make_int4((int)r[4 * j], (int)r[4 * j + 1], (int)r[4 * j + 2], (int)r[4 * j + 3]));
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            if (col0 + j < p.N) {
+                                crow[j] = f[j];
+                                if (KIND == Kind::I8 && rrow) rrow[j] = (int)r[j];
+                            }
+                        }
+                    }
+                }
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_empty[as]);
+        }
+    } else if (CONV) {
+        // ------------------------------------------------ im2col gather of the A tile (4 warps, one row per thread)
+        const int t = threadIdx.x - 192;              // tile row 0..127
+        const int sw = t & 7;
+        constexpr int kAhead = 2;                     // stages issued but not yet published
+        uint32_t it = 0, issued = 0, published = 0;
+        const int taps = p.R * p.S;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+            int m_blk, n_blk;
+            tile_coords(tile, p.m_tiles, p.n_tiles, m_blk, n_blk);
+            const int m = m_blk * kBM + t;
+            const bool row_ok = m < p.M;
+            const int img = row_ok ? m / (p.OH * p.OW) : 0;
+            const int rem = row_ok ? m - img * (p.OH * p.OW) : 0;
+            const int oh = rem / p.OW, ow = rem - oh * p.OW;
+            const int ih0 = oh * p.stride - p.pad, iw0 = ow * p.stride - p.pad;
+            const uint8_t *img_base = p.xe + (int64_t)img * p.H * p.W * p.cpb;
+            for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+                const int s = it % kStages;
+                const uint32_t ph = (it / kStages) & 1u;
+                if (!wait_bounded(&empty[s], ph ^ 1u, abort_flag, 5)) { ok = false; break; }
+                const uint32_t dst_row = smem_u32(a_stages + s * L::kAStage) + (uint32_t)t * kBKBytes;
+                const int kbyte0 = kb * kBKBytes;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const int kbyte = kbyte0 + j * 16;
+                    const int tap = kbyte / p.cpb;
+                    const int cb = kbyte - tap * p.cpb;
+                    const int fr = tap / p.S, fs = tap - fr * p.S;
+                    const int ih = ih0 + fr * p.dil, iw = iw0 + fs * p.dil;
+                    const bool in = row_ok && tap < taps && ih >= 0 && ih < p.H && iw >= 0 && iw < p.W;
+                    const uint8_t *src = in ? img_base + ((int64_t)ih * p.W + iw) * p.cpb + cb : p.xe;
+                    cp_async_16(dst_row + (uint32_t)((j ^ sw) << 4), src, in ? 16u : 0u);
+                }
+                cp_async_commit();
+                ++issued;
+                if (issued - published > kAhead) {
+                    cp_async_wait_group<kAhead>();
+                    fence_proxy_async_smem();
+                    mbar_arrive(&full[published % kStages]);
+                    ++published;
+                }
+            }
+        }
+        cp_async_wait_group<0>();
+        fence_proxy_async_smem();
+        while (ok && published < issued) {
+            mbar_arrive(&full[published % kStages]);
+            ++published;
+        }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+// ------------------------------------------------------------------ host side
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (fn == nullptr) {
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+        else
+            (void)cudaGetLastError();
+    }
+    return fn;
+}
+
+// Byte matrix [rows][row_bytes] with row stride `stride`; box = 128 bytes x box_rows, 128-byte swizzle.
+static dybit_status make_operand_map(CUtensorMap *map, const void *base, int64_t rows, int64_t row_bytes, int64_t stride,
+                                     int box_rows) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (fn == nullptr) return DYBIT_ERR_CUDA;
+    cuuint64_t dims[2] = {(cuuint64_t)row_bytes, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)stride};
+    cuuint32_t box[2] = {(cuuint32_t)kBKBytes, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? DYBIT_OK : DYBIT_ERR_CUDA;
+}
+
+template <Kind KIND, int BN, bool CONV>
+static dybit_status launch_gemm_inst(const CUtensorMap &ta, const CUtensorMap &tb, const GemmParams &p, cudaStream_t s) {
+    using L = GemmSmem<BN>;
+    auto kern = dybit_gemm_kernel<KIND, BN, CONV>;
+    static bool configured[64] = {};
+    int dev = 0;
+    DYBIT_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return DYBIT_ERR_CUDA;
+    if (!configured[dev]) {
+        DYBIT_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kBytes));
+        configured[dev] = true;
+    }
+    const int tiles = p.m_tiles * p.n_tiles;
+    const int grid = tiles < sm_count() ? tiles : sm_count();
+    kern<<<grid, CONV ? 320 : 192, L::kBytes, s>>>(ta, tb, p);
+    return launch_status();
+}
+
+template <Kind KIND, bool CONV>
+static dybit_status launch_gemm_bn(int bn, const CUtensorMap &ta, const CUtensorMap &tb, const GemmParams &p,
+                                   cudaStream_t s) {
+    switch (bn) {
+        case 64: return launch_gemm_inst<KIND, 64, CONV>(ta, tb, p, s);
+        case 128: return launch_gemm_inst<KIND, 128, CONV>(ta, tb, p, s);
+        default: return launch_gemm_inst<KIND, 256, CONV>(ta, tb, p, s);
+    }
+}
+
+template <bool CONV>
+static dybit_status launch_gemm_kind(dybit_container cont, int bn, const CUtensorMap &ta, const CUtensorMap &tb,
+                                     const GemmParams &p, cudaStream_t s) {
+    switch (cont) {
+        case DYBIT_CONTAINER_I8: return launch_gemm_bn<Kind::I8, CONV>(bn, ta, tb, p, s);
+        case DYBIT_CONTAINER_E4M3: return launch_gemm_bn<Kind::F8F6F4, CONV>(bn, ta, tb, p, s);
+        default: return launch_gemm_bn<Kind::F16, CONV>(bn, ta, tb, p, s);
+    }
+}
+
+// Tile width along N: the narrowest of 64/128/256 that covers N, but never so wide that
+// the grid leaves most SMs idle.
+static int choose_bn(int64_t M, int64_t N) {
+    int bn = N <= 64 ? 64 : (N <= 128 ? 128 : 256);
+    const int64_t m_tiles = (M + kBM - 1) / kBM;
+    while (bn > 64 && m_tiles * ((N + bn - 1) / bn) < sm_count()) bn >>= 1;
+    return bn;
+}
+
+static int pad_grid(int64_t chunks) {
+    int64_t b = (chunks + 255) / 256, cap = (int64_t)sm_count() * 16;
+    if (b > cap) b = cap;
+    return b < 1 ? 1 : (int)b;
+}
+
+struct GemmLayout {
+    dybit_container cont;
+    int elem;
+    int exp_a, exp_b;
+    int64_t kp;             // K padded to 128 elements... in elements
+    int64_t a_bytes, b_bytes, a_off, b_off, total;
+};
+
+static inline int64_t k_row_bytes(int64_t k_elems, int elem) { return round_up(k_elems * elem, kBKBytes); }
+
+}  // namespace dybit
+
+extern "C" {
+
+size_t dybit_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, dybit_fmt fa, dybit_fmt fb) {
+    using namespace dybit;
+    ContainerPlan plan;
+    if (M <= 0 || N <= 0 || K <= 0 || plan_container(fa, fb, &plan) != DYBIT_OK) return 0;
+    const int elem = container_elem_bytes(plan.container);
+    const int64_t rb = k_row_bytes(round_up(K, 128), elem);
+    return (size_t)(round_up(M * rb, 1024) + round_up(N * rb, 1024) + 1024);
+}
+
+size_t dybit_conv2d_workspace_bytes(const dybit_conv_desc *d, dybit_fmt fx, dybit_fmt fw) {
+    using namespace dybit;
+    ContainerPlan plan;
+    int oh, ow;
+    if (dybit_conv2d_out_hw(d, &oh, &ow) != DYBIT_OK || plan_container(fx, fw, &plan) != DYBIT_OK) return 0;
+    const int elem = container_elem_bytes(plan.container);
+    const int64_t cp = round_up(d->c, 16);
+    const int64_t x_bytes = round_up((int64_t)d->n * d->h * d->w * cp * elem, 1024);
+    const int64_t w_bytes = round_up((int64_t)d->k * k_row_bytes((int64_t)d->r * d->s * cp, elem), 1024);
+    return (size_t)(x_bytes + w_bytes + 2048);
+}
+
+dybit_status dybit_gemm(int64_t M, int64_t N, int64_t K, const void *A, dybit_fmt fa, const float *scale_a,
+                        int64_t lda_bytes, const void *B, dybit_fmt fb, const float *scale_b, int64_t ldb_bytes,
+                        float *C, int64_t ldc, int32_t *C_raw, void *ws, size_t ws_bytes, void *stream) {
+    using namespace dybit;
+    if (M <= 0 || N <= 0 || K <= 0 || !fmt_ok(fa) || !fmt_ok(fb)) return DYBIT_ERR_INVALID_ARG;
+    if (!A || !B || !C || !scale_a || !scale_b || ldc < N) return DYBIT_ERR_INVALID_ARG;
+    if (M > INT32_MAX - 256 || N > INT32_MAX - 256 || K > (1 << 24)) return DYBIT_ERR_UNSUPPORTED;
+    if (lda_bytes < (int64_t)dybit_row_stride_bytes(K, fa.bits) || ldb_bytes < (int64_t)dybit_row_stride_bytes(K, fb.bits))
+        return DYBIT_ERR_INVALID_ARG;
+    if (lda_bytes % 16 || ldb_bytes % 16 || !aligned(A, 16) || !aligned(B, 16) || !aligned(C, 4) || !aligned(C_raw, 4) ||
+        !aligned(scale_a, 4) || !aligned(scale_b, 4))
+        return DYBIT_ERR_ALIGNMENT;
+    ContainerPlan plan;
+    dybit_status st = plan_container(fa, fb, &plan);
+    if (st != DYBIT_OK) return st;
+    if (C_raw && plan.container != DYBIT_CONTAINER_I8) return DYBIT_ERR_UNSUPPORTED;
+    if (plan.container == DYBIT_CONTAINER_I8 && (K > (1 << 19) || K * plan.max_product > (int64_t)INT32_MAX))
+        return DYBIT_ERR_UNSUPPORTED;
+    const size_t need = dybit_gemm_workspace_bytes(M, N, K, fa, fb);
+    if (!ws || ws_bytes < need) return DYBIT_ERR_WORKSPACE;
+    if (!aligned(ws, 1024)) return DYBIT_ERR_ALIGNMENT;
+
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int elem = container_elem_bytes(plan.container);
+    const int64_t kp = round_up(K, 128);
+    const int64_t rb = k_row_bytes(kp, elem);
+    uint8_t *ae = static_cast<uint8_t *>(ws);
+    uint8_t *be = ae + round_up(M * rb, 1024);
+    const ElemTable ta = make_elem_table(fa, plan.container, plan.exp_a);
+    const ElemTable tb = make_elem_table(fb, plan.container, plan.exp_b);
+    st = launch_expand(static_cast<const uint8_t *>(A), fa.bits, M, lda_bytes, kp, elem, ae, rb, ta, s);
+    if (st != DYBIT_OK) return st;
+    st = launch_expand(static_cast<const uint8_t *>(B), fb.bits, N, ldb_bytes, kp, elem, be, rb, tb, s);
+    if (st != DYBIT_OK) return st;
+
+    const int bn = choose_bn(M, N);
+    CUtensorMap map_a, map_b;
+    st = make_operand_map(&map_a, ae, M, rb, rb, kBM);
+    if (st != DYBIT_OK) return st;
+    st = make_operand_map(&map_b, be, N, rb, rb, bn);
+    if (st != DYBIT_OK) return st;
+    GemmParams p = {};
+    p.M = (int)M;
+    p.N = (int)N;
+    p.k_blocks = (int)(rb / kBKBytes);
+    p.m_tiles = (int)((M + kBM - 1) / kBM);
+    p.n_tiles = (int)((N + bn - 1) / bn);
+    p.C = C;
+    p.C_raw = C_raw;
+    p.ldc = ldc;
+    p.scale_a = scale_a;
+    p.scale_b = scale_b;
+    p.pow2 = ldexp(1.0, -(plan.exp_a + plan.exp_b));
+    return launch_gemm_kind<false>(plan.container, bn, map_a, map_b, p, s);
+}
+
+dybit_status dybit_conv2d(const dybit_conv_desc *d, const void *X, dybit_fmt fx, const float *scale_x, const void *W,
+                          dybit_fmt fw, const float *scale_w, int64_t ldw_bytes, float *Y, int32_t *Y_raw, void *ws,
+                          size_t ws_bytes, void *stream) {
+    using namespace dybit;
+    int oh, ow;
+    dybit_status st = dybit_conv2d_out_hw(d, &oh, &ow);
+    if (st != DYBIT_OK) return st;
+    if (!fmt_ok(fx) || !fmt_ok(fw) || !X || !W || !Y || !scale_x || !scale_w) return DYBIT_ERR_INVALID_ARG;
+    const int64_t K = (int64_t)d->r * d->s * d->c;
+    const int64_t M = (int64_t)d->n * oh * ow;
+    const int64_t N = d->k;
+    if (M > INT32_MAX - 256 || K > (1 << 24)) return DYBIT_ERR_UNSUPPORTED;
+    if (ldw_bytes < (int64_t)dybit_row_stride_bytes(K, fw.bits)) return DYBIT_ERR_INVALID_ARG;
+    if (ldw_bytes % 16 || !aligned(X, 16) || !aligned(W, 16) || !aligned(Y, 4) || !aligned(Y_raw, 4) ||
+        !aligned(scale_x, 4) || !aligned(scale_w, 4))
+        return DYBIT_ERR_ALIGNMENT;
+    ContainerPlan plan;
+    st = plan_container(fx, fw, &plan);
+    if (st != DYBIT_OK) return st;
+    if (Y_raw && plan.container != DYBIT_CONTAINER_I8) return DYBIT_ERR_UNSUPPORTED;
+    if (plan.container == DYBIT_CONTAINER_I8 && (K > (1 << 19) || K * plan.max_product > (int64_t)INT32_MAX))
+        return DYBIT_ERR_UNSUPPORTED;
+    const size_t need = dybit_conv2d_workspace_bytes(d, fx, fw);
+    if (!ws || ws_bytes < need) return DYBIT_ERR_WORKSPACE;
+    if (!aligned(ws, 1024)) return DYBIT_ERR_ALIGNMENT;
+
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int elem = container_elem_bytes(plan.container);
+    const int64_t cp = round_up(d->c, 16);
+    const int64_t pixels = (int64_t)d->n * d->h * d->w;
+    const int64_t x_bytes = round_up(pixels * cp * elem, 1024);
+    const int64_t wrb = k_row_bytes((int64_t)d->r * d->s * cp, elem);
+    uint8_t *xe = static_cast<uint8_t *>(ws);
+    uint8_t *we = xe + x_bytes;
+    const ElemTable tx = make_elem_table(fx, plan.container, plan.exp_a);
+    const ElemTable tw = make_elem_table(fw, plan.container, plan.exp_b);
+    if (cp == d->c) {
+        // channels already a multiple of 16: X is one flat run, W rows expand with their zero tail
+        st = launch_expand(static_cast<const uint8_t *>(X), fx.bits, 1, 0, pixels * cp, elem, xe, 0, tx, s);
+        if (st != DYBIT_OK) return st;
+        st = launch_expand(static_cast<const uint8_t *>(W), fw.bits, N, ldw_bytes, wrb / elem, elem, we, wrb, tw, s);
+        if (st != DYBIT_OK) return st;
+    } else {
+        const int64_t taps = (int64_t)d->r * d->s;
+        DYBIT_CUDA_TRY(cudaMemsetAsync(we, 0, (size_t)(N * wrb), s));
+        int64_t chunks = pixels * (cp * elem / 16);
+        expand_pad_kernel<<<pad_grid(chunks), 256, 0, s>>>(
+            static_cast<const uint8_t *>(X), fx.bits, 1, 0, pixels, d->c, (int)cp, elem, xe, 0, tx);
+        if (launch_status() != DYBIT_OK) return DYBIT_ERR_CUDA;
+        chunks = N * taps * (cp * elem / 16);
+        expand_pad_kernel<<<pad_grid(chunks), 256, 0, s>>>(
+            static_cast<const uint8_t *>(W), fw.bits, N, ldw_bytes, taps, d->c, (int)cp, elem, we, wrb, tw);
+        if (launch_status() != DYBIT_OK) return DYBIT_ERR_CUDA;
+    }
+
+    const int bn = choose_bn(M, N);
+    CUtensorMap map_b;
+    st = make_operand_map(&map_b, we, N, wrb, wrb, bn);
+    if (st != DYBIT_OK) return st;
+    GemmParams p = {};
+    p.M = (int)M;
+    p.N = (int)N;
+    p.k_blocks = (int)(wrb / kBKBytes);
+    p.m_tiles = (int)((M + kBM - 1) / kBM);
+    p.n_tiles = (int)((N + bn - 1) / bn);
+    p.C = Y;
+    p.C_raw = Y_raw;
+    p.ldc = N;
+    p.scale_a = scale_x;
+    p.scale_b = scale_w;
+    p.pow2 = ldexp(1.0, -(plan.exp_a + plan.exp_b));
+    p.xe = xe;
+    p.H = d->h;
+    p.W = d->w;
+    p.OH = oh;
+    p.OW = ow;
+    p.R = d->r;
+    p.S = d->s;
+    p.stride = d->stride;
+    p.pad = d->pad;
+    p.dil = d->dilation;
+    p.cpb = (int)(cp * elem);
+    return launch_gemm_kind<true>(plan.container, bn, map_b, map_b, p, s);
+}
+
+}  // extern "C"
