@@ -197,6 +197,19 @@ dybit_status dybit_conv2d(const dybit_conv_desc *desc,
  * otherwise.  detail: [host] optional, receives the raw status word. */
 dybit_status dybit_last_device_status(void *stream, uint32_t *detail);
 
+/* ---------------------------------------------------------------- measurement hooks
+ * (no counterpart in the paper: they exist so that a benchmark can attribute
+ * time to the tensor-core kernel alone and count the library's launches) */
+
+/* Number of kernels this library has launched in the calling process so far. */
+uint64_t dybit_launch_count(void);
+
+/* Arms the calling thread: the next dybit_gemm / dybit_conv2d records
+ * ev_start on its stream immediately before its tensor-core kernel and
+ * ev_stop immediately after it (the expand kernels stay outside the pair),
+ * then disarms.  Both are cudaEvent_t passed as void*; NULL, NULL disarms. */
+dybit_status dybit_profile_next_gemm(void *ev_start, void *ev_stop);
+
 #ifdef __cplusplus
 }
 #endif

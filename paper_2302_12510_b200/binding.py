@@ -20,6 +20,7 @@ __all__ = [
     "dybit_choose_container", "dybit_gemm_workspace_bytes", "dybit_conv2d_workspace_bytes",
     "dybit_conv2d_out_hw", "dybit_absmax_scale", "dybit_quantize_pack", "dybit_quantize_pack_2d",
     "dybit_decode", "dybit_gemm", "dybit_conv2d", "dybit_last_device_status",
+    "dybit_launch_count", "dybit_profile_next_gemm",
 ]
 
 
@@ -88,6 +89,9 @@ def _load() -> C.CDLL:
     lib.dybit_conv2d.argtypes = [C.POINTER(_CConvDesc), vp, _CFmt, vp, vp, _CFmt, vp, i64,
                                  vp, vp, vp, sz, vp]
     lib.dybit_last_device_status.argtypes = [vp, C.POINTER(C.c_uint32)]
+    lib.dybit_launch_count.restype = C.c_uint64
+    lib.dybit_launch_count.argtypes = []
+    lib.dybit_profile_next_gemm.argtypes = [vp, vp]
     return lib
 
 
@@ -271,3 +275,19 @@ def dybit_last_device_status(stream=None) -> Tuple[int, int]:
     detail = C.c_uint32(0)
     st = lib.dybit_last_device_status(_stream(stream), C.byref(detail))
     return int(st), int(detail.value)
+
+
+def dybit_launch_count() -> int:
+    return int(lib.dybit_launch_count())
+
+
+def dybit_profile_next_gemm(ev_start: Optional[torch.cuda.Event], ev_stop: Optional[torch.cuda.Event]):
+    """Arms event recording around the next GEMM/conv tensor-core kernel (events need enable_timing=True)."""
+    if ev_start is None:
+        _check(lib.dybit_profile_next_gemm(None, None), "dybit_profile_next_gemm")
+        return
+    for ev in (ev_start, ev_stop):
+        if not ev.cuda_event:           # torch creates the handle lazily on first record
+            ev.record()
+    _check(lib.dybit_profile_next_gemm(C.c_void_p(ev_start.cuda_event), C.c_void_p(ev_stop.cuda_event)),
+           "dybit_profile_next_gemm")

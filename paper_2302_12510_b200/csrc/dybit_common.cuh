@@ -28,8 +28,24 @@ inline int64_t round_up(int64_t v, int64_t a) { return (v + a - 1) / a * a; }
         }                                            \
     } while (0)
 
+// Every kernel launch of the library is followed by launch_status(), which
+// also counts it.
+inline unsigned long long &launch_counter() {
+    static unsigned long long n = 0;
+    return n;
+}
+
 inline dybit_status launch_status() {
+    ++launch_counter();
     return cudaGetLastError() == cudaSuccess ? DYBIT_OK : DYBIT_ERR_CUDA;
+}
+
+struct ProfileEvents {
+    cudaEvent_t start = nullptr, stop = nullptr;
+};
+inline ProfileEvents &profile_events() {
+    static thread_local ProfileEvents ev;
+    return ev;
 }
 
 // Device status word: 0 = fine; otherwise (site << 8) | 1 of the first bounded

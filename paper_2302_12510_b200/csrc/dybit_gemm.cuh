@@ -508,8 +508,13 @@ static dybit_status launch_gemm_inst(const CUtensorMap &ta, const CUtensorMap &t
     }
     const int tiles = p.m_tiles * p.n_tiles;
     const int grid = tiles < sm_count() ? tiles : sm_count();
+    ProfileEvents ev = profile_events();
+    profile_events() = ProfileEvents();
+    if (ev.start) DYBIT_CUDA_TRY(cudaEventRecord(ev.start, s));
     kern<<<grid, CONV ? 320 : 192, L::kBytes, s>>>(ta, tb, p);
-    return launch_status();
+    const dybit_status st = launch_status();
+    if (ev.stop) DYBIT_CUDA_TRY(cudaEventRecord(ev.stop, s));
+    return st;
 }
 
 template <Kind KIND, bool CONV>

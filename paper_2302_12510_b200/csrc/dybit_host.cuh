@@ -183,6 +183,15 @@ dybit_status dybit_conv2d_out_hw(const dybit_conv_desc *d, int *oh, int *ow) {
     return DYBIT_OK;
 }
 
+uint64_t dybit_launch_count(void) { return dybit::launch_counter(); }
+
+dybit_status dybit_profile_next_gemm(void *ev_start, void *ev_stop) {
+    if ((ev_start == nullptr) != (ev_stop == nullptr)) return DYBIT_ERR_INVALID_ARG;
+    dybit::profile_events().start = static_cast<cudaEvent_t>(ev_start);
+    dybit::profile_events().stop = static_cast<cudaEvent_t>(ev_stop);
+    return DYBIT_OK;
+}
+
 dybit_status dybit_last_device_status(void *stream, uint32_t *detail) {
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     unsigned int word = 0, zero = 0;

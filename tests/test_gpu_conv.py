@@ -1,0 +1,79 @@
+"""GPU parity: dybit_conv2d (implicit GEMM) against the oracle's direct convolution."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2302_12510_b200 as dy
+from paper_2302_12510_b200 import workloads as wl
+from oracle import dybit_oracle as orc
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def run_conv(layer, fx, fw, seed=0):
+    """Quantize synthetic NHWC activations / KRSC weights on the GPU, convolve, compare with the oracle."""
+    x = wl.half_normal((layer.n, layer.h, layer.w, layer.c), seed=seed)
+    if fx[1]:
+        x = x - 0.5
+    w = wl.kaiming_normal(layer.k, layer.r, layer.s, layer.c, seed=seed + 1)
+    px, sx = dy.dybit_quantize_pack(x.to(DEV), fx)
+    pw, sw = dy.dybit_quantize_pack_2d(w.reshape(layer.k, -1).to(DEV), fw)
+    spx = orc.absmax_scale(x.numpy(), fx[0], bool(fx[1]))
+    spw = orc.absmax_scale(w.numpy(), fw[0], bool(fw[1]))
+    cx = orc.quantize(x.numpy(), fx[0], bool(fx[1]), spx[1])
+    cw = orc.quantize(w.numpy(), fw[0], bool(fw[1]), spw[1])
+    assert np.array_equal(px.cpu().numpy(), orc.pack(cx, fx[0]))
+    assert np.array_equal(pw.cpu().numpy(), orc.pack_rows(cw.reshape(layer.k, -1), fw[0]))
+    desc = dy.ConvDesc(layer.n, layer.h, layer.w, layer.c, layer.k, layer.r, layer.s, layer.stride, layer.pad, 1)
+    cont, _, _ = dy.dybit_choose_container(fx, fw)
+    Y, Y_raw = dy.dybit_conv2d(desc, px, fx, sx, pw, fw, sw, want_raw=(cont == 0))
+    torch.cuda.synchronize()
+    assert dy.dybit_last_device_status() == (0, 0)
+    S, Y_ref = orc.conv2d(cx, fx, spx[0], cw, fw, spw[0], stride=layer.stride, pad=layer.pad)
+    assert tuple(Y.shape) == Y_ref.shape
+    if cont == 0:
+        assert np.array_equal(Y_raw.cpu().numpy().astype(np.int64), S)
+        assert np.array_equal(Y.cpu().numpy(), Y_ref)
+    else:
+        amax = float(spx[0]) * float(np.abs(orc.decode_table(fx[0], bool(fx[1]))).max())
+        bmax = float(spw[0]) * float(np.abs(orc.decode_table(fw[0], bool(fw[1]))).max())
+        tol = 1e-5 * layer.gemm_k * amax * bmax
+        err = np.abs(Y.cpu().numpy().astype(np.float64) - Y_ref.astype(np.float64)).max()
+        assert err <= tol, (err, tol)
+    return cont
+
+
+def _distinct_shapes(layers):
+    seen, out = set(), []
+    for L in layers:
+        key = (L.h, L.w, L.c, L.k, L.r, L.s, L.stride, L.pad)
+        if key not in seen:
+            seen.add(key)
+            out.append(L)
+    return out
+
+
+@pytest.mark.parametrize("layer", _distinct_shapes(wl.resnet18_layers(2)), ids=lambda L: L.name)
+def test_resnet18_shapes_batch2_uniform_4bit(layer):
+    # every distinct ResNet-18 layer shape, weights signed 4-bit, activations unsigned 4-bit
+    assert run_conv(layer, (4, 0), (4, 1), seed=hash(layer.name) % 1000) == 0
+
+
+@pytest.mark.parametrize("fx,fw", [((2, 0), (2, 1)), ((3, 0), (5, 1)), ((5, 0), (4, 1)), ((6, 0), (3, 1)),
+                                   ((8, 0), (8, 1)), ((4, 1), (6, 1))])
+def test_mixed_bitwidths_small_conv(fx, fw):
+    L = wl.ConvLayer("t", 2, 14, 14, 64, 96, 3, 3, 1, 1)
+    run_conv(L, fx, fw, seed=fx[0] * 10 + fw[0])
+
+
+@pytest.mark.parametrize("shape", [
+    wl.ConvLayer("stride2_3x3_ragged", 3, 15, 13, 32, 40, 3, 3, 2, 1),
+    wl.ConvLayer("pointwise_stride2", 2, 9, 9, 48, 130, 1, 1, 2, 0),
+    wl.ConvLayer("c3_7x7", 1, 32, 32, 3, 64, 7, 7, 2, 3),
+    wl.ConvLayer("c20_pad_channels", 2, 8, 8, 20, 24, 3, 3, 1, 1),
+    wl.ConvLayer("fc_like", 5, 1, 1, 512, 1000, 1, 1, 1, 0),
+    wl.ConvLayer("one_pixel", 1, 1, 1, 16, 1, 1, 1, 1, 0),
+], ids=lambda L: L.name)
+def test_edge_geometries(shape):
+    assert run_conv(shape, (4, 0), (4, 1), seed=3) == 0

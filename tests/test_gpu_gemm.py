@@ -114,7 +114,7 @@ def test_gemm_argument_errors():
     one = torch.tensor([1.0, 1.0], device=DEV)
     ws = torch.zeros(16, dtype=torch.uint8, device=DEV)
     with pytest.raises(dy.DybitError) as e:
-        dy.dybit_gemm(4, 4, 128, pa, fa, one, pa, fb, one, ws=torch.zeros(4096, dtype=torch.uint8, device=DEV))
+        dy.dybit_gemm(4, 4, 128, pa, fa, one, pa, fb, one, ws=torch.zeros(2048, dtype=torch.uint8, device=DEV))
     assert e.value.status == 4           # workspace too small
     with pytest.raises(dy.DybitError) as e:
         dy.dybit_gemm(4, 4, 256, pa, fa, one, pa, fb, one)
