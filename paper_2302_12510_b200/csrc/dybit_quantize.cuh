@@ -18,45 +18,66 @@ constexpr int kStreamThreads = kWarpsPerBlock * 32;
 
 // ------------------------------------------------------------------ encode
 
-// Magnitude code of t = |x| / scale for M magnitude bits (inverse of Eq. 1).
-// Codes grow with the value they stand for, so the nearest code is found the
-// way a float is rounded: take the binade e of t (the sub-unit codes form one
-// linear region, e = -1), scale t so that one code step is 1.0, subtract the
-// binade's first code's offset and round to nearest-even; a carry out of the
-// fraction runs into the unary exponent field, which is exactly the first
-// code of the next binade (the encoder of Section III-B.2 places e+1 ones,
-// a zero and the leading fraction bits).  Every float operation below is
-// exact except the final round-to-integer.
+// Magnitude code of a = |x| (a >= 0, never NaN) for M magnitude bits: the
+// inverse of Eq. 1 with round-to-nearest, ties to the even code.  The result
+// is returned with a bias: its low byte is the code.
+//
+// Codes grow with the value they stand for.  Below 1 they are linear, so the
+// code is round(t * 2^(M-1)).  In binade e (t in [2^e, 2^(e+1)): e+1 leading
+// ones, a zero, k = M-2-e fraction bits -- the encoder of Section III-B.2) the
+// code is first_code(e) + round(t * 2^(k-e) - 2^k); a carry out of the
+// fraction lands on the next binade's first code by itself.  Along the code
+// axis the sub-unit line lies above every binade's line for t >= 1 and below
+// the e = 0 line for t < 1, so taking the smaller of the two candidates picks
+// the right one without a branch.  Each product is a power-of-two scaling
+// (exact); adding 1.5 * 2^23 (minus 2^k) inside the same FMA rounds the exact
+// sum to an integer, ties to even, and leaves that integer -- negative ones
+// too -- as an offset in the low mantissa bits.
 template <int M>
-__device__ __forceinline__ unsigned encode_magnitude(float t) {
-    constexpr unsigned kAllOnes = (1u << M) - 1u;
-    constexpr float kVmax = (float)(1u << (M - 1));
-    int e = (int)(__float_as_uint(t) >> 23) - 127;      // t >= 0: sign bit clear
-    e = max(e, -1);
-    e = min(e, M - 2);
-    const bool sub_unit = e < 0;
-    const int k = M - 2 - e;                            // fraction bits in binade e (e >= 0)
-    const int up = sub_unit ? (M - 1) : (k - e);        // t * 2^up: one code step == 1.0
-    const float offs = sub_unit ? 0.0f : (float)(1 << k);
-    const float p2 = __uint_as_float((unsigned)(127 + up) << 23);
-    const int r = __float2int_rn(__fmaf_rn(t, p2, -offs));
-    const unsigned base = (1u << M) - (1u << (M - 1 - e));   // e+1 ones, then zeros
-    unsigned mag = base + (unsigned)r;
-    mag = (t >= kVmax) ? kAllOnes : mag;
-    mag = (t != t) ? 0u : mag;
-    return mag;
+__device__ __forceinline__ unsigned magnitude_code_biased(float a, float inv) {
+    constexpr unsigned kMagicBits = 0x4B400000u;                           // 1.5 * 2^23: ulp 1 on both sides
+    // largest float below the top value 2^(M-1): everything from 1.5 * 2^(M-2) up rounds to all-ones anyway
+    const float below_top = __uint_as_float(((unsigned)(127 + M - 1) << 23) - 1u);
+    const float t = fminf(__fmul_rn(a, inv), below_top);
+    const unsigned sub = __float_as_uint(__fmaf_rn(t, (float)(1u << (M - 1)), __uint_as_float(kMagicBits)));
+    if constexpr (M == 1) {
+        return sub;
+    } else {
+        const unsigned E = max(__float_as_uint(t) >> 23, 127u);           // biased exponent, sub-unit folded onto e = 0
+        const float scale_e = __uint_as_float(((unsigned)(381 + M - 2) << 23) - (E << 24));   // 2^(k-e)
+        const unsigned k = (unsigned)(127 + M - 2) - E;
+        const unsigned one_k = 1u << k;
+        const unsigned sup = __float_as_uint(__fmaf_rn(t, scale_e, __uint_as_float(kMagicBits - one_k)));
+        const unsigned cand = sup + (1u << M) - 2u * one_k;                // + first_code(e) = 2^M - 2^(k+1)
+        return min(sub, cand);
+    }
 }
 
+// Four elements -> four codes, one per byte of the result.
 template <int BITS, bool SIGNED>
-__device__ __forceinline__ unsigned encode_code(float x, float inv) {
+__device__ __forceinline__ unsigned encode4(const float4 v, const float inv) {
     constexpr int M = SIGNED ? BITS - 1 : BITS;
-    const float t = __fmul_rn(fabsf(x), inv);
-    unsigned mag = encode_magnitude<M>(t);
-    const unsigned neg = __float_as_uint(x) >> 31;
-    if (SIGNED) {
-        return mag | ((mag != 0u ? neg : 0u) << M);
+    if constexpr (SIGNED) {
+        // fmaxf(|x|, 0) maps NaN to 0
+        const unsigned m0 = magnitude_code_biased<M>(fmaxf(fabsf(v.x), 0.0f), inv);
+        const unsigned m1 = magnitude_code_biased<M>(fmaxf(fabsf(v.y), 0.0f), inv);
+        const unsigned m2 = magnitude_code_biased<M>(fmaxf(fabsf(v.z), 0.0f), inv);
+        const unsigned m3 = magnitude_code_biased<M>(fmaxf(fabsf(v.w), 0.0f), inv);
+        const unsigned mags = __byte_perm(__byte_perm(m0, m1, 0x0040), __byte_perm(m2, m3, 0x0040), 0x5410);
+        // top byte of each float carries its sign in bit 7
+        const unsigned tops = __byte_perm(__byte_perm(__float_as_uint(v.x), __float_as_uint(v.y), 0x0073),
+                                          __byte_perm(__float_as_uint(v.z), __float_as_uint(v.w), 0x0073), 0x5410);
+        // bit 7 of each byte set where the magnitude code is non-zero (codes are < 128)
+        const unsigned nonzero = (mags + 0x7f7f7f7fu) | mags;
+        const unsigned sign = ((tops & nonzero & 0x80808080u) >> (7 - M));
+        return mags | sign;
     } else {
-        return neg ? 0u : mag;
+        // no sign bit: negative inputs (and NaN) take the nearest value the format has, 0
+        const unsigned m0 = magnitude_code_biased<M>(fmaxf(v.x, 0.0f), inv);
+        const unsigned m1 = magnitude_code_biased<M>(fmaxf(v.y, 0.0f), inv);
+        const unsigned m2 = magnitude_code_biased<M>(fmaxf(v.z, 0.0f), inv);
+        const unsigned m3 = magnitude_code_biased<M>(fmaxf(v.w, 0.0f), inv);
+        return __byte_perm(__byte_perm(m0, m1, 0x0040), __byte_perm(m2, m3, 0x0040), 0x5410);
     }
 }
 
@@ -139,6 +160,29 @@ __global__ void finalize_scale_kernel(float *scale, int m) {
 // Packs this lane's 32 consecutive codes (bytes, low to high) into BITS words.
 template <int BITS>
 __device__ __forceinline__ void pack32(const unsigned (&cw)[8], unsigned (&out)[BITS]) {
+    if constexpr (BITS == 8) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) out[i] = cw[i];
+        return;
+    } else if constexpr (BITS == 4) {
+        // bytes {a,b,c,d} -> (a | b<<4) in byte 0 and (c | d<<4) in byte 2, then gather the even bytes
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const unsigned lo = cw[2 * i] | (cw[2 * i] >> 4), hi = cw[2 * i + 1] | (cw[2 * i + 1] >> 4);
+            out[i] = __byte_perm(lo, hi, 0x6420);
+        }
+        return;
+    } else if constexpr (BITS == 2) {
+        unsigned b[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const unsigned t = cw[i] | (cw[i] >> 6);       // byte 0: a | b<<2, byte 2: c | d<<2
+            b[i] = t | (t >> 12);                           // byte 0: a | b<<2 | c<<4 | d<<6
+        }
+        out[0] = __byte_perm(__byte_perm(b[0], b[1], 0x0040), __byte_perm(b[2], b[3], 0x0040), 0x5410);
+        out[1] = __byte_perm(__byte_perm(b[4], b[5], 0x0040), __byte_perm(b[6], b[7], 0x0040), 0x5410);
+        return;
+    }
     unsigned long long acc = 0;
     int nb = 0, w = 0;
 #pragma unroll
@@ -198,11 +242,7 @@ quantize_pack_kernel(const float *__restrict__ x, int64_t rows, int64_t cols, in
         }
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
-            const unsigned c = encode_code<BITS, SIGNED>(v[j].x, inv) |
-                               (encode_code<BITS, SIGNED>(v[j].y, inv) << 8) |
-                               (encode_code<BITS, SIGNED>(v[j].z, inv) << 16) |
-                               (encode_code<BITS, SIGNED>(v[j].w, inv) << 24);
-            s_codes[warp][j * 32 + lane] = c;
+            s_codes[warp][j * 32 + lane] = encode4<BITS, SIGNED>(v[j], inv);
         }
         __syncwarp();
         // lane takes codes [32*lane, 32*lane + 32); the two 16-byte halves are
