@@ -191,6 +191,35 @@ dybit_status dybit_conv2d(const dybit_conv_desc *desc,
                           float *Y, int32_t *Y_raw,
                           void *ws, size_t ws_bytes, void *stream);
 
+/* (No counterpart in the paper.)  dybit_gemm for callers that cannot call
+ * cudaMalloc -- or any allocator built on it -- at the point where they need
+ * a GEMM: code running under a fixed memory budget that was handed out at
+ * start-up, plug-ins of a host application that owns all device memory, code
+ * on a path where an allocation's implicit synchronisation or possible failure
+ * is not acceptable.  Same arguments and same result, bit for bit, as
+ * dybit_gemm, minus the workspace: the expanded operands go to a scratch array
+ * of DYBIT_STATIC_WS_BYTES that is part of this library's device image.  Every
+ * GPU on which the process uses the library holds that array from module load
+ * until the process exits.
+ *   - Problems with dybit_gemm_workspace_bytes(M, N, K, fa, fb) above
+ *     DYBIT_STATIC_WS_BYTES are refused with DYBIT_ERR_WORKSPACE and nothing
+ *     is launched (e.g. int8-container operands up to (M + N) * roundup(K,128)
+ *     of about 16 Mi elements fit).
+ *   - The call itself allocates nothing and frees nothing.  The first call on
+ *     each device looks up the array's device address (cudaGetSymbolAddress,
+ *     with that device current) and remembers it; make that first call outside
+ *     any stream capture.
+ *   - All calls on a device share the one array.  Nothing in it has to be
+ *     zero beforehand and nothing is kept between calls: each call rewrites
+ *     every byte it later reads.  Two calls whose device work overlaps (two
+ *     streams, or two host threads) would overwrite each other's operands:
+ *     keep calls to this entry point ordered on one stream per device. */
+#define DYBIT_STATIC_WS_BYTES (16u * 1024u * 1024u)
+dybit_status dybit_gemm_static_ws(int64_t M, int64_t N, int64_t K,
+                                  const void *A, dybit_fmt fa, const float *scale_a, int64_t lda_bytes,
+                                  const void *B, dybit_fmt fb, const float *scale_b, int64_t ldb_bytes,
+                                  float *C, int64_t ldc, int32_t *C_raw, void *stream);
+
 /* Reads and clears the device status word of the current device.  Blocks
  * until `stream` has drained.  DYBIT_ERR_DEVICE_TIMEOUT means a kernel gave
  * up on a bounded wait (results of that call are invalid); DYBIT_OK

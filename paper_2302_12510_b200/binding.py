@@ -20,7 +20,7 @@ __all__ = [
     "dybit_choose_container", "dybit_gemm_workspace_bytes", "dybit_conv2d_workspace_bytes",
     "dybit_conv2d_out_hw", "dybit_absmax_scale", "dybit_quantize_pack", "dybit_quantize_pack_2d",
     "dybit_decode", "dybit_gemm", "dybit_conv2d", "dybit_last_device_status",
-    "dybit_launch_count", "dybit_profile_next_gemm",
+    "dybit_launch_count", "dybit_profile_next_gemm", "dybit_gemm_static_ws", "STATIC_WS_BYTES",
 ]
 
 
@@ -92,6 +92,7 @@ def _load() -> C.CDLL:
     lib.dybit_launch_count.restype = C.c_uint64
     lib.dybit_launch_count.argtypes = []
     lib.dybit_profile_next_gemm.argtypes = [vp, vp]
+    lib.dybit_gemm_static_ws.argtypes = [i64, i64, i64, vp, _CFmt, vp, i64, vp, _CFmt, vp, i64, vp, i64, vp, vp]
     return lib
 
 
@@ -291,3 +292,25 @@ def dybit_profile_next_gemm(ev_start: Optional[torch.cuda.Event], ev_stop: Optio
             ev.record()
     _check(lib.dybit_profile_next_gemm(C.c_void_p(ev_start.cuda_event), C.c_void_p(ev_stop.cuda_event)),
            "dybit_profile_next_gemm")
+
+
+STATIC_WS_BYTES = 16 * 1024 * 1024   # DYBIT_STATIC_WS_BYTES in include/dybit.h
+
+
+def dybit_gemm_static_ws(M: int, N: int, K: int, A: torch.Tensor, fa, scale_a: torch.Tensor,
+                         B: torch.Tensor, fb, scale_b: torch.Tensor, C_out: torch.Tensor,
+                         C_raw: Optional[torch.Tensor] = None, lda_bytes: Optional[int] = None,
+                         ldb_bytes: Optional[int] = None, stream=None):
+    """dybit_gemm without a workspace argument, for callers that cannot allocate device memory.
+
+    The caller passes every input and output buffer (C_out too: this wrapper creates no tensor);
+    the library's built-in scratch array holds the expanded operands.  Problems that need more
+    than STATIC_WS_BYTES raise DybitError (status 4).  Calls share the scratch: keep them on one
+    stream per device.
+    """
+    lda = A.stride(0) if lda_bytes is None else lda_bytes
+    ldb = B.stride(0) if ldb_bytes is None else ldb_bytes
+    _check(lib.dybit_gemm_static_ws(M, N, K, _ptr(A), _fmt(fa), _ptr(scale_a), lda, _ptr(B), _fmt(fb),
+                                    _ptr(scale_b), ldb, _ptr(C_out), C_out.stride(0), _ptr(C_raw),
+                                    _stream(stream)), "dybit_gemm_static_ws")
+    return C_out, C_raw

@@ -3,3 +3,4 @@
 #include "dybit_host.cuh"
 #include "dybit_quantize.cuh"
 #include "dybit_gemm.cuh"
+#include "dybit_static_ws.cuh"
