@@ -182,7 +182,7 @@ static dybit_status launch_expand(const uint8_t *packed, int bits, int64_t rows,
 // ------------------------------------------------------------------ the tcgen05 GEMM
 
 constexpr int kBM = 128;            // tile rows (UMMA M)
-constexpr int kBKBytes = 128;       // one swizzle row of K per pipeline stage
+constexpr int kBKBytes = 128;       // one 128-byte swizzle row of K per pipeline stage (64 in the SWB = 64 variant)
 constexpr int kUmmaKBytes = 32;     // K bytes consumed by one tcgen05.mma
 constexpr int kStageBytesTotal = 192 * 1024;
 constexpr unsigned long long kWaitLimitNs = 4000000000ull;
@@ -196,10 +196,11 @@ struct GemmParams {
     int64_t ldc;
     const float *scale_a, *scale_b;
     double pow2;              // alpha = (float)(scale_a * scale_b * pow2)
-    // implicit-GEMM gather of A (convolution only)
+    // implicit-GEMM addressing of A (convolution only)
     const uint8_t *xe;        // expanded activation, [n*h*w][cpb] bytes
     int H, W, OH, OW, R, S, stride, pad, dil;
     int cpb;                  // bytes per pixel in xe (padded channels * element size)
+    int kb_per_tap;           // im2col mode: SWB-byte blocks per filter tap (cpb / SWB)
 };
 
 // Waits for the phase with the given parity; gives up after kWaitLimitNs, records
@@ -222,12 +223,18 @@ __device__ __forceinline__ bool wait_bounded(uint64_t *bar, uint32_t parity, vol
     }
 }
 
-template <int BN>
+// How the A tile reaches shared memory.
+enum AMode { kATiled = 0,    // GEMM: 2-D tiled TMA
+             kAGather = 1,   // conv: four warps gather 16-byte chunks with cp.async (any channel count)
+             kAIm2col = 2 }; // conv: one im2col TMA per stage (pixel = a whole number of SWB-byte blocks)
+
+template <int BN, int SWB>
 struct GemmSmem {
-    static constexpr int kAStage = kBM * kBKBytes;
-    static constexpr int kBStage = BN * kBKBytes;
-    static constexpr int kStages = kStageBytesTotal / (kAStage + kBStage);
-    static constexpr int kBarrierBytes = 256;
+    static constexpr int kAStage = kBM * SWB;
+    static constexpr int kBStage = BN * SWB;
+    static constexpr int kFit = kStageBytesTotal / (kAStage + kBStage);
+    static constexpr int kStages = kFit > 12 ? 12 : kFit;
+    static constexpr int kBarrierBytes = 512;
     static constexpr int kBytes = kStages * (kAStage + kBStage) + kBarrierBytes + 1024;   // + alignment slack
 };
 
@@ -243,11 +250,13 @@ __device__ __forceinline__ void tile_coords(int tile, int m_tiles, int n_tiles, 
     n_blk = in_group / gsz;
 }
 
-template <Kind KIND, int BN, bool CONV>
-__global__ void __launch_bounds__(CONV ? 320 : 192, 1)
+template <Kind KIND, int BN, int AMODE, int SWB>
+__global__ void __launch_bounds__(AMODE == kAGather ? 320 : 192, 1)
 dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                   const GemmParams p) {
-    using L = GemmSmem<BN>;
+    static_assert(AMODE != kAGather || SWB == 128, "the cp.async gather writes 128-byte rows");
+    constexpr bool CONV = AMODE == kAGather;          // extra gather warps present
+    using L = GemmSmem<BN, SWB>;
     constexpr int kStages = L::kStages;
     constexpr int kGatherThreads = 128;
     extern __shared__ uint8_t smem_raw[];
@@ -278,7 +287,7 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         }
         *abort_flag = 0;
         fence_mbar_init();
-        if (!CONV) prefetch_tensormap(&tmap_a);
+        if (AMODE != kAGather) prefetch_tensormap(&tmap_a);
         prefetch_tensormap(&tmap_b);
     }
     if (warp == 1) {
@@ -298,13 +307,32 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
                 int m_blk, n_blk;
                 tile_coords(tile, p.m_tiles, p.n_tiles, m_blk, n_blk);
+                // im2col mode: window origin of the tile's first output pixel, and the running filter tap
+                int iw = 0, ih = 0, img = 0, fr = 0, fs = 0, cb = 0;
+                if (AMODE == kAIm2col) {
+                    const int m0 = m_blk * kBM;
+                    img = m0 / (p.OH * p.OW);
+                    const int rem = m0 - img * (p.OH * p.OW);
+                    const int oh = rem / p.OW;
+                    ih = oh * p.stride - p.pad;
+                    iw = (rem - oh * p.OW) * p.stride - p.pad;
+                }
                 for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
                     const int s = it % kStages;
                     const uint32_t ph = (it / kStages) & 1u;
                     if (!wait_bounded(&empty[s], ph ^ 1u, abort_flag, 1)) { ok = false; break; }
                     mbar_arrive_expect_tx(&full[s], CONV ? L::kBStage : L::kAStage + L::kBStage);
-                    if (!CONV) tma_load_2d(a_stages + s * L::kAStage, &tmap_a, kb * kBKBytes, m_blk * kBM, &full[s]);
-                    tma_load_2d(b_stages + s * L::kBStage, &tmap_b, kb * kBKBytes, n_blk * BN, &full[s]);
+                    if (AMODE == kATiled) {
+                        tma_load_2d(a_stages + s * L::kAStage, &tmap_a, kb * SWB, m_blk * kBM, &full[s]);
+                    } else if (AMODE == kAIm2col) {
+                        tma_load_im2col_4d(a_stages + s * L::kAStage, &tmap_a, cb * SWB, iw, ih, img, &full[s],
+                                           (uint16_t)(fs * p.dil), (uint16_t)(fr * p.dil));
+                        if (++cb == p.kb_per_tap) {
+                            cb = 0;
+                            if (++fs == p.S) { fs = 0; ++fr; }
+                        }
+                    }
+                    tma_load_2d(b_stages + s * L::kBStage, &tmap_b, kb * SWB, n_blk * BN, &full[s]);
                 }
             }
             if (!ok) {
@@ -330,10 +358,10 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     const uint32_t ph = (it / kStages) & 1u;
                     if (!wait_bounded(&full[s], ph, abort_flag, 3)) { ok = false; break; }
                     tc_fence_after_sync();
-                    const uint64_t adesc = umma_desc_sw128(smem_u32(a_stages + s * L::kAStage));
-                    const uint64_t bdesc = umma_desc_sw128(smem_u32(b_stages + s * L::kBStage));
+                    const uint64_t adesc = umma_desc_kmajor<SWB>(smem_u32(a_stages + s * L::kAStage));
+                    const uint64_t bdesc = umma_desc_kmajor<SWB>(smem_u32(b_stages + s * L::kBStage));
 #pragma unroll
-                    for (int k = 0; k < kBKBytes / kUmmaKBytes; ++k) {
+                    for (int k = 0; k < SWB / kUmmaKBytes; ++k) {
                         umma<KIND>(d, adesc + (uint64_t)(k * (kUmmaKBytes >> 4)), bdesc + (uint64_t)(k * (kUmmaKBytes >> 4)),
                                    idesc, (uint32_t)((kb | k) != 0));
                     }
@@ -404,7 +432,6 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         const int sw = t & 7;
         constexpr int kAhead = 2;                     // stages issued but not yet published
         uint32_t it = 0, issued = 0, published = 0;
-        const int taps = p.R * p.S;
         bool ok = true;
         for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
             int m_blk, n_blk;
@@ -416,22 +443,39 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             const int oh = rem / p.OW, ow = rem - oh * p.OW;
             const int ih0 = oh * p.stride - p.pad, iw0 = ow * p.stride - p.pad;
             const uint8_t *img_base = p.xe + (int64_t)img * p.H * p.W * p.cpb;
+            // filter tap (fr, fs) and byte offset inside the pixel, advanced chunk by chunk: K runs (r, s, c)
+            int fr = 0, fs = 0, cb = 0;
             for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
                 const int s = it % kStages;
                 const uint32_t ph = (it / kStages) & 1u;
                 if (!wait_bounded(&empty[s], ph ^ 1u, abort_flag, 5)) { ok = false; break; }
                 const uint32_t dst_row = smem_u32(a_stages + s * L::kAStage) + (uint32_t)t * kBKBytes;
-                const int kbyte0 = kb * kBKBytes;
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const int kbyte = kbyte0 + j * 16;
-                    const int tap = kbyte / p.cpb;
-                    const int cb = kbyte - tap * p.cpb;
-                    const int fr = tap / p.S, fs = tap - fr * p.S;
+                if (p.cpb % kBKBytes == 0) {
+                    // a pixel holds whole 128-byte blocks: the eight chunks share one tap and are contiguous
                     const int ih = ih0 + fr * p.dil, iw = iw0 + fs * p.dil;
-                    const bool in = row_ok && tap < taps && ih >= 0 && ih < p.H && iw >= 0 && iw < p.W;
+                    const bool in = row_ok && fr < p.R && (unsigned)ih < (unsigned)p.H && (unsigned)iw < (unsigned)p.W;
                     const uint8_t *src = in ? img_base + ((int64_t)ih * p.W + iw) * p.cpb + cb : p.xe;
-                    cp_async_16(dst_row + (uint32_t)((j ^ sw) << 4), src, in ? 16u : 0u);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        cp_async_16(dst_row + (uint32_t)((j ^ sw) << 4), in ? src + j * 16 : src, in ? 16u : 0u);
+                    cb += kBKBytes;
+                    if (cb == p.cpb) {
+                        cb = 0;
+                        if (++fs == p.S) { fs = 0; ++fr; }
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const int ih = ih0 + fr * p.dil, iw = iw0 + fs * p.dil;
+                        const bool in = row_ok && fr < p.R && (unsigned)ih < (unsigned)p.H && (unsigned)iw < (unsigned)p.W;
+                        const uint8_t *src = in ? img_base + ((int64_t)ih * p.W + iw) * p.cpb + cb : p.xe;
+                        cp_async_16(dst_row + (uint32_t)((j ^ sw) << 4), src, in ? 16u : 0u);
+                        cb += 16;
+                        if (cb == p.cpb) {
+                            cb = 0;
+                            if (++fs == p.S) { fs = 0; ++fr; }
+                        }
+                    }
                 }
                 cp_async_commit();
                 ++issued;
@@ -479,25 +523,63 @@ static EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
-// Byte matrix [rows][row_bytes] with row stride `stride`; box = 128 bytes x box_rows, 128-byte swizzle.
+// Byte matrix [rows][row_bytes] with row stride `stride`; box = swb bytes x box_rows, swb-byte swizzle.
 static dybit_status make_operand_map(CUtensorMap *map, const void *base, int64_t rows, int64_t row_bytes, int64_t stride,
-                                     int box_rows) {
+                                     int box_rows, int swb = 128) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (fn == nullptr) return DYBIT_ERR_CUDA;
     cuuint64_t dims[2] = {(cuuint64_t)row_bytes, (cuuint64_t)rows};
     cuuint64_t strides[1] = {(cuuint64_t)stride};
-    cuuint32_t box[2] = {(cuuint32_t)kBKBytes, (cuuint32_t)box_rows};
+    cuuint32_t box[2] = {(cuuint32_t)swb, (cuuint32_t)box_rows};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(base), dims, strides, box, estr,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, swb == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? DYBIT_OK : DYBIT_ERR_CUDA;
 }
 
-template <Kind KIND, int BN, bool CONV>
+typedef CUresult (*EncodeIm2colFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                   const cuuint64_t *, const int *, const int *, cuuint32_t, cuuint32_t,
+                                   const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeIm2colFn encode_im2col_fn() {
+    static EncodeIm2colFn fn = nullptr;
+    if (fn == nullptr) {
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeIm2colFn>(ptr);
+        else
+            (void)cudaGetLastError();
+    }
+    return fn;
+}
+
+// Expanded activation [n][h][w][cpb bytes] as an im2col map: one load brings 128 consecutive output
+// pixels x swb bytes of one filter tap, walking w, then h, then n with the convolution's stride and
+// zero-filling taps outside the image.  The pixel box runs from -pad to pad - (filter - 1) * dilation.
+static dybit_status make_im2col_map(CUtensorMap *map, const void *xe, const dybit_conv_desc *d, int64_t cpb, int swb) {
+    EncodeIm2colFn fn = encode_im2col_fn();
+    if (fn == nullptr) return DYBIT_ERR_CUDA;
+    cuuint64_t dims[4] = {(cuuint64_t)cpb, (cuuint64_t)d->w, (cuuint64_t)d->h, (cuuint64_t)d->n};
+    cuuint64_t strides[3] = {(cuuint64_t)cpb, (cuuint64_t)cpb * d->w, (cuuint64_t)cpb * d->w * d->h};
+    int lower[2] = {-d->pad, -d->pad};
+    int upper[2] = {d->pad - (d->s - 1) * d->dilation, d->pad - (d->r - 1) * d->dilation};
+    cuuint32_t estr[4] = {1, (cuuint32_t)d->stride, (cuuint32_t)d->stride, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void *>(xe), dims, strides, lower, upper,
+                    (cuuint32_t)swb, (cuuint32_t)kBM, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    swb == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? DYBIT_OK : DYBIT_ERR_CUDA;
+}
+
+template <Kind KIND, int BN, int AMODE, int SWB>
 static dybit_status launch_gemm_inst(const CUtensorMap &ta, const CUtensorMap &tb, const GemmParams &p, cudaStream_t s) {
-    using L = GemmSmem<BN>;
-    auto kern = dybit_gemm_kernel<KIND, BN, CONV>;
+    using L = GemmSmem<BN, SWB>;
+    auto kern = dybit_gemm_kernel<KIND, BN, AMODE, SWB>;
+    constexpr bool CONV = AMODE == kAGather;
     static bool configured[64] = {};
     int dev = 0;
     DYBIT_CUDA_TRY(cudaGetDevice(&dev));
@@ -517,23 +599,23 @@ static dybit_status launch_gemm_inst(const CUtensorMap &ta, const CUtensorMap &t
     return st;
 }
 
-template <Kind KIND, bool CONV>
+template <Kind KIND, int AMODE, int SWB>
 static dybit_status launch_gemm_bn(int bn, const CUtensorMap &ta, const CUtensorMap &tb, const GemmParams &p,
                                    cudaStream_t s) {
     switch (bn) {
-        case 64: return launch_gemm_inst<KIND, 64, CONV>(ta, tb, p, s);
-        case 128: return launch_gemm_inst<KIND, 128, CONV>(ta, tb, p, s);
-        default: return launch_gemm_inst<KIND, 256, CONV>(ta, tb, p, s);
+        case 64: return launch_gemm_inst<KIND, 64, AMODE, SWB>(ta, tb, p, s);
+        case 128: return launch_gemm_inst<KIND, 128, AMODE, SWB>(ta, tb, p, s);
+        default: return launch_gemm_inst<KIND, 256, AMODE, SWB>(ta, tb, p, s);
     }
 }
 
-template <bool CONV>
+template <int AMODE, int SWB>
 static dybit_status launch_gemm_kind(dybit_container cont, int bn, const CUtensorMap &ta, const CUtensorMap &tb,
                                      const GemmParams &p, cudaStream_t s) {
     switch (cont) {
-        case DYBIT_CONTAINER_I8: return launch_gemm_bn<Kind::I8, CONV>(bn, ta, tb, p, s);
-        case DYBIT_CONTAINER_E4M3: return launch_gemm_bn<Kind::F8F6F4, CONV>(bn, ta, tb, p, s);
-        default: return launch_gemm_bn<Kind::F16, CONV>(bn, ta, tb, p, s);
+        case DYBIT_CONTAINER_I8: return launch_gemm_bn<Kind::I8, AMODE, SWB>(bn, ta, tb, p, s);
+        case DYBIT_CONTAINER_E4M3: return launch_gemm_bn<Kind::F8F6F4, AMODE, SWB>(bn, ta, tb, p, s);
+        default: return launch_gemm_bn<Kind::F16, AMODE, SWB>(bn, ta, tb, p, s);
     }
 }
 
@@ -640,7 +722,7 @@ dybit_status dybit_gemm(int64_t M, int64_t N, int64_t K, const void *A, dybit_fm
     p.scale_a = scale_a;
     p.scale_b = scale_b;
     p.pow2 = ldexp(1.0, -(plan.exp_a + plan.exp_b));
-    return launch_gemm_kind<false>(plan.container, bn, map_a, map_b, p, s);
+    return launch_gemm_kind<kATiled, 128>(plan.container, bn, map_a, map_b, p, s);
 }
 
 dybit_status dybit_conv2d(const dybit_conv_desc *d, const void *X, dybit_fmt fx, const float *scale_x, const void *W,
@@ -699,13 +781,10 @@ dybit_status dybit_conv2d(const dybit_conv_desc *d, const void *X, dybit_fmt fx,
     }
 
     const int bn = choose_bn(M, N);
-    CUtensorMap map_b;
-    st = make_operand_map(&map_b, we, N, wrb, wrb, bn);
-    if (st != DYBIT_OK) return st;
+    const int64_t cpb = cp * elem;
     GemmParams p = {};
     p.M = (int)M;
     p.N = (int)N;
-    p.k_blocks = (int)(wrb / kBKBytes);
     p.m_tiles = (int)((M + kBM - 1) / kBM);
     p.n_tiles = (int)((N + bn - 1) / bn);
     p.C = Y;
@@ -724,8 +803,39 @@ dybit_status dybit_conv2d(const dybit_conv_desc *d, const void *X, dybit_fmt fx,
     p.stride = d->stride;
     p.pad = d->pad;
     p.dil = d->dilation;
-    p.cpb = (int)(cp * elem);
-    return launch_gemm_kind<true>(plan.container, bn, map_b, map_b, p, s);
+    p.cpb = (int)cpb;
+
+    CUtensorMap map_a, map_b;
+    const bool pointwise = d->r == 1 && d->s == 1 && d->stride == 1 && d->pad == 0;
+    if (pointwise) {
+        // a 1x1 stride-1 convolution is the GEMM [pixels][cpb] x [k][cpb]^T on the expanded activation
+        st = make_operand_map(&map_a, xe, M, cpb, cpb, kBM);
+        if (st != DYBIT_OK) return st;
+        st = make_operand_map(&map_b, we, N, wrb, wrb, bn);
+        if (st != DYBIT_OK) return st;
+        p.k_blocks = (int)(wrb / kBKBytes);
+        return launch_gemm_kind<kATiled, 128>(plan.container, bn, map_a, map_b, p, s);
+    }
+    // im2col TMA: a pixel must be a whole number of swizzle-span blocks, corners and tap offsets must
+    // fit the descriptor's 8-bit fields, and the tensor must not be tiny (tiny ones take the gather path)
+    const int swb = (cpb % 128 == 0) ? 128 : (cpb == 64 ? 64 : 0);
+    const int up_w = d->pad - (d->s - 1) * d->dilation, up_h = d->pad - (d->r - 1) * d->dilation;
+    const bool im2col_ok = swb != 0 && pixels * cpb >= 131072 && d->pad <= 127 && up_w >= -128 && up_h >= -128 &&
+                           (d->s - 1) * d->dilation <= 255 && (d->r - 1) * d->dilation <= 255 && d->stride <= 8;
+    if (im2col_ok) {
+        st = make_im2col_map(&map_a, xe, d, cpb, swb);
+        if (st != DYBIT_OK) return st;
+        st = make_operand_map(&map_b, we, N, wrb, wrb, bn, swb);
+        if (st != DYBIT_OK) return st;
+        p.kb_per_tap = (int)(cpb / swb);
+        p.k_blocks = (int)((int64_t)d->r * d->s * p.kb_per_tap);
+        return swb == 128 ? launch_gemm_kind<kAIm2col, 128>(plan.container, bn, map_a, map_b, p, s)
+                          : launch_gemm_kind<kAIm2col, 64>(plan.container, bn, map_a, map_b, p, s);
+    }
+    st = make_operand_map(&map_b, we, N, wrb, wrb, bn);
+    if (st != DYBIT_OK) return st;
+    p.k_blocks = (int)(wrb / kBKBytes);
+    return launch_gemm_kind<kAGather, 128>(plan.container, bn, map_b, map_b, p, s);
 }
 
 }  // extern "C"

@@ -80,6 +80,18 @@ __device__ __forceinline__ void tma_load_2d(void *smem_dst, const CUtensorMap *m
         : "memory");
 }
 
+// 4-D im2col load (tensor [N][H][W][C], coordinates c, w, h, n of the first pixel's window origin,
+// filter-tap offsets along w and h): gathers `pixelsPerColumn` consecutive output pixels x the
+// map's channel box, zero-filling taps that fall outside the image.
+__device__ __forceinline__ void tma_load_im2col_4d(void *smem_dst, const CUtensorMap *map, int c, int w, int h, int n,
+                                                   uint64_t *bar, uint16_t off_w, uint16_t off_h) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%2, %3, %4, %5}], [%6], {%7, %8};" ::"r"(smem_u32(smem_dst)),
+        "l"(reinterpret_cast<uint64_t>(map)), "r"(c), "r"(w), "r"(h), "r"(n), "r"(smem_u32(bar)), "h"(off_w), "h"(off_h)
+        : "memory");
+}
+
 // ---------------------------------------------------------------- cp.async (16-byte, zero-fill)
 
 __device__ __forceinline__ void cp_async_16(uint32_t smem_dst, const void *gsrc, uint32_t src_bytes) {
@@ -132,14 +144,16 @@ __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.
 enum class Kind { I8, F8F6F4, F16 };
 
 // Shared-memory matrix descriptor for a K-major operand tile whose rows are
-// 128 bytes and use the 128-byte swizzle: 8-row groups are 1024 bytes apart.
-__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr) {
+// SWB (128 or 64) bytes and use the SWB-byte swizzle: 8-row groups are 8*SWB bytes apart.
+template <int SWB>
+__device__ __forceinline__ uint64_t umma_desc_kmajor(uint32_t smem_addr) {
+    static_assert(SWB == 128 || SWB == 64, "swizzle span");
     uint64_t d = 0;
     d |= (uint64_t)((smem_addr & 0x3ffffu) >> 4);      // start address, 16-byte units
     d |= (uint64_t)1 << 16;                            // leading byte offset (unused with swizzle)
-    d |= (uint64_t)(1024 >> 4) << 32;                  // stride byte offset between 8-row groups
+    d |= (uint64_t)((8 * SWB) >> 4) << 32;             // stride byte offset between 8-row groups
     d |= (uint64_t)1 << 46;                            // descriptor version for sm_100
-    d |= (uint64_t)2 << 61;                            // 128-byte swizzle
+    d |= (uint64_t)(SWB == 128 ? 2 : 4) << 61;         // 128-byte / 64-byte swizzle
     return d;
 }
 

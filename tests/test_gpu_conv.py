@@ -77,3 +77,32 @@ def test_mixed_bitwidths_small_conv(fx, fw):
 ], ids=lambda L: L.name)
 def test_edge_geometries(shape):
     assert run_conv(shape, (4, 0), (4, 1), seed=3) == 0
+
+
+# Large enough activations that the TMA im2col path is taken (>= 128 KiB expanded), for both swizzle
+# spans (64-byte pixels and multiples of 128 bytes), strides, dilation, ragged last tile.
+@pytest.mark.parametrize("shape,fx,fw", [
+    (wl.ConvLayer("c64_3x3_s1", 8, 28, 28, 64, 64, 3, 3, 1, 1), (4, 0), (4, 1)),
+    (wl.ConvLayer("c64_3x3_s2_ragged", 5, 29, 27, 64, 72, 3, 3, 2, 1), (4, 0), (4, 1)),
+    (wl.ConvLayer("c64_1x1_s2", 6, 28, 28, 64, 128, 1, 1, 2, 0), (4, 0), (4, 1)),
+    (wl.ConvLayer("c128_3x3_s1", 6, 20, 20, 128, 96, 3, 3, 1, 1), (4, 0), (4, 1)),
+    (wl.ConvLayer("c256_3x3_s2", 8, 14, 14, 256, 256, 3, 3, 2, 1), (4, 0), (4, 1)),
+    (wl.ConvLayer("c512_3x3_s1", 8, 7, 7, 512, 512, 3, 3, 1, 1), (4, 0), (4, 1)),
+    (wl.ConvLayer("c256_1x1_s2", 8, 14, 14, 256, 512, 1, 1, 2, 0), (3, 0), (2, 1)),
+    (wl.ConvLayer("c128_5x5_pad2", 4, 18, 18, 128, 40, 5, 5, 1, 2), (4, 1), (4, 1)),
+    (wl.ConvLayer("c64_bf16", 6, 20, 20, 64, 96, 3, 3, 1, 1), (8, 0), (8, 1)),
+    (wl.ConvLayer("c128_e4m3", 6, 20, 20, 128, 96, 3, 3, 2, 1), (5, 0), (4, 1)),
+    (wl.ConvLayer("c32_bf16_64B_pixels", 8, 24, 24, 32, 48, 3, 3, 1, 1), (6, 0), (8, 1)),
+], ids=lambda v: v.name if hasattr(v, "name") else str(v))
+def test_im2col_tma_path(shape, fx, fw):
+    run_conv(shape, fx, fw, seed=11)
+
+
+@pytest.mark.parametrize("shape", [
+    wl.ConvLayer("pw_c64", 4, 28, 28, 64, 256, 1, 1, 1, 0),
+    wl.ConvLayer("pw_c256_ragged", 3, 13, 11, 256, 100, 1, 1, 1, 0),
+    wl.ConvLayer("pw_c48", 2, 9, 9, 48, 64, 1, 1, 1, 0),
+], ids=lambda L: L.name)
+def test_pointwise_conv_runs_as_plain_gemm(shape):
+    run_conv(shape, (4, 0), (4, 1), seed=5)
+    run_conv(shape, (8, 0), (6, 1), seed=6)
