@@ -346,6 +346,11 @@ def main():
     ap.add_argument("--batch", type=int, default=32, help="images per step (32 = the quoted configuration)")
     ap.add_argument("--no-targets", action="store_true", help="skip the single-kernel target measurements")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--targets-only", action="store_true",
+                    help="run only the single-kernel target measurements (small cases for profiler captures)")
+    ap.add_argument("--gemm-size", type=int, default=8192, help="M=N=K of the square 4-bit GEMM target")
+    ap.add_argument("--quant-log2n", type=int, default=28, help="log2 of the element count of the quantize target")
+    ap.add_argument("--quant-bits", type=int, default=4)
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
@@ -368,6 +373,14 @@ def main():
     from paper_2302_12510_b200 import workloads as wl
     peaks = load_peaks()
     warmup = max(3, args.warmup)
+    if args.targets_only:
+        out = {}
+        if args.gemm_size > 0:
+            out["gemm_w4a4"] = target_gemm(dy, wl, device, peaks, size=args.gemm_size)
+        if args.quant_log2n > 0:
+            out["quantize_pack"] = target_quantize(dy, wl, device, peaks, log2n=args.quant_log2n, bits=args.quant_bits)
+        print(json.dumps({"targets": out}))
+        return
 
     work = Resnet18Step(dy, wl, device, batch=args.batch)
     for _ in range(warmup):
@@ -461,8 +474,8 @@ def main():
 
     if rank == 0 and not args.no_targets:
         result["targets"] = {
-            "gemm_w4a4": target_gemm(dy, wl, device, peaks),
-            "quantize_pack": target_quantize(dy, wl, device, peaks),
+            "gemm_w4a4": target_gemm(dy, wl, device, peaks, size=args.gemm_size),
+            "quantize_pack": target_quantize(dy, wl, device, peaks, log2n=args.quant_log2n, bits=args.quant_bits),
         }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         result["cpu_baseline"] = cpu_baseline(wl)
