@@ -369,3 +369,48 @@ void orc_conv2d(int n, int h, int w, int c, int k, int r, int s,
         }
     }
 }
+
+/* The same convolution for chosen outputs only, starting from the fp32
+ * activation: each needed element is encoded on the spot with
+ * orc_encode_one (t = |x| * inv_x), so a test can check sampled outputs of a
+ * layer too large to quantise and convolve in full.  idx[e] is the flat index
+ * into Y[n][oh][ow][k]. */
+void orc_conv2d_sampled(int n, int h, int w, int c, int k, int r, int s,
+                        int stride, int pad, int dilation,
+                        const float *X, int bits_x, int signed_x, float scale_x, float inv_x,
+                        const uint8_t *W, int bits_w, int signed_w, float scale_w,
+                        const int64_t *idx, int64_t n_samples, int64_t *S, float *Y)
+{
+    int oh = (h + 2 * pad - dilation * (r - 1) - 1) / stride + 1;
+    int ow = (w + 2 * pad - dilation * (s - 1) - 1) / stride + 1;
+    (void)n;
+    float alpha = orc_alpha(scale_x, bits_x, signed_x, scale_w, bits_w, signed_w);
+    int64_t tx[256], tw[256];
+    int_table(bits_x, signed_x, tx);
+    int_table(bits_w, signed_w, tw);
+#pragma omp parallel for schedule(dynamic, 4)
+    for (int64_t e = 0; e < n_samples; ++e) {
+        int64_t o = idx[e];
+        int ko = (int)(o % k); o /= k;
+        int jo = (int)(o % ow); o /= ow;
+        int io = (int)(o % oh); o /= oh;
+        int in = (int)o;
+        int64_t acc = 0;
+        for (int ir = 0; ir < r; ++ir) {
+            int ih = io * stride - pad + ir * dilation;
+            if (ih < 0 || ih >= h) continue;
+            for (int is = 0; is < s; ++is) {
+                int iw = jo * stride - pad + is * dilation;
+                if (iw < 0 || iw >= w) continue;
+                for (int ic = 0; ic < c; ++ic) {
+                    float xv = X[(((int64_t)in * h + ih) * w + iw) * c + ic];
+                    unsigned cx = orc_encode_one(xv, inv_x, bits_x, signed_x);
+                    unsigned cw = W[(((int64_t)ko * r + ir) * s + is) * c + ic];
+                    acc += tx[cx] * tw[cw];
+                }
+            }
+        }
+        if (S) S[e] = acc;
+        if (Y) Y[e] = (float)acc * alpha;
+    }
+}

@@ -62,6 +62,7 @@ def _load():
         lib.orc_gemm_sampled.argtypes = [i64, i64, vp, i32, i32, f32, vp, i32, i32, f32,
                                          vp, vp, i64, vp, vp]
         lib.orc_conv2d.argtypes = [i32] * 10 + [vp, i32, i32, f32, vp, i32, i32, f32, vp, vp]
+        lib.orc_conv2d_sampled.argtypes = [i32] * 10 + [vp, i32, i32, f32, f32, vp, i32, i32, f32, vp, i64, vp, vp]
         _lib = lib
     return _lib
 
@@ -222,4 +223,25 @@ def conv2d(codes_x, fmt_x, scale_x, codes_w, fmt_w, scale_w, stride=1, pad=0, di
                        _p(x), fmt_x[0], int(fmt_x[1]), float(np.float32(scale_x)),
                        _p(wt), fmt_w[0], int(fmt_w[1]), float(np.float32(scale_w)),
                        _p(acc), _p(y))
+    return acc, y
+
+
+def conv2d_sampled(x_fp32, fmt_x, scale_pair_x, codes_w, fmt_w, scale_w, flat_idx, stride=1, pad=0, dilation=1):
+    """Chosen outputs of the convolution, quantising the needed fp32 activations on the spot.
+
+    x_fp32: [n][h][w][c] float32; scale_pair_x: (scale, inv); flat_idx: indices into Y[n][oh][ow][k].
+    Returns (S int64, Y fp32), one entry per index."""
+    x, wt = _f32(x_fp32), _u8(codes_w)
+    n, h, w, c = x.shape
+    k, r, s, c2 = wt.shape
+    assert c == c2
+    idx = np.ascontiguousarray(flat_idx, dtype=np.int64)
+    oh, ow = conv_out_hw(h, w, r, s, stride, pad, dilation)
+    assert idx.size == 0 or (idx.min() >= 0 and idx.max() < n * oh * ow * k)
+    acc = np.zeros(idx.size, dtype=np.int64)
+    y = np.zeros(idx.size, dtype=np.float32)
+    _load().orc_conv2d_sampled(n, h, w, c, k, r, s, stride, pad, dilation, _p(x), fmt_x[0], int(fmt_x[1]),
+                               float(np.float32(scale_pair_x[0])), float(np.float32(scale_pair_x[1])),
+                               _p(wt), fmt_w[0], int(fmt_w[1]), float(np.float32(scale_w)),
+                               _p(idx), idx.size, _p(acc), _p(y))
     return acc, y

@@ -1,0 +1,179 @@
+"""GPU parity at the sizes and launch configurations bench.py times.
+
+Outputs too large for the oracle to recompute in full are checked on sampled
+entries the oracle computes one by one, plus properties that hold at any size
+(exact column/row checksums of the integer GEMM, the scale's closed form).
+"""
+import numpy as np
+import pytest
+import torch
+
+import paper_2302_12510_b200 as dy
+from paper_2302_12510_b200 import workloads as wl
+from oracle import dybit_oracle as orc
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _check_packed_samples(x_dev, packed, fmt, scale, rng, n_chunks=48, chunk=8192):
+    """Sampled 8192-code windows (aligned so that they start on a byte) + the tail, against the oracle."""
+    n = x_dev.numel()
+    bits = fmt[0]
+    xs = x_dev.reshape(-1)
+    # closed form of the scale from the full tensor
+    amax = float(xs.abs().max().item())
+    m = bits - 1 if fmt[1] else bits
+    sp = (np.float32(amax) / np.float32(2.0 ** (m - 1)), np.float32(2.0 ** (m - 1)) / np.float32(amax))
+    assert np.array_equal(scale.cpu().numpy(), np.array(sp, dtype=np.float32))
+    starts = [int(s) * 8 for s in rng.integers(0, max(1, (n - chunk) // 8), n_chunks)] + [max(0, (n - chunk) // 8 * 8), 0]
+    for s0 in starts:
+        cnt = min(chunk, n - s0)
+        xh = xs[s0:s0 + cnt].cpu().numpy()
+        want = orc.pack(orc.quantize(xh, bits, bool(fmt[1]), sp[1]), bits)
+        nbytes = (cnt * bits + 7) // 8
+        got = packed[s0 * bits // 8: s0 * bits // 8 + nbytes].cpu().numpy()
+        if (cnt * bits) % 8 == 0:
+            assert np.array_equal(got, want[:nbytes]), (fmt, s0)
+        else:
+            assert np.array_equal(got[:-1], want[:nbytes - 1]), (fmt, s0)
+
+
+@pytest.mark.parametrize("dist,fmt,log2n", [
+    ("normal", (4, 1), 28), ("laplace", (2, 1), 26), ("half_normal", (3, 0), 26), ("normal", (6, 1), 26),
+    ("laplace", (8, 1), 26), ("half_normal", (8, 0), 24), ("normal", (4, 1), 30),
+])
+def test_quantize_sweep_sizes_sampled(dist, fmt, log2n):
+    n = 1 << log2n
+    x = wl.DISTRIBUTIONS[dist]((n,), seed=log2n + fmt[0], device=DEV)
+    packed, scale = dy.dybit_quantize_pack(x, fmt)
+    assert packed.numel() == dy.dybit_packed_bytes(n, fmt[0])
+    _check_packed_samples(x, packed, fmt, scale, np.random.default_rng(log2n))
+    # decode(quantize(x)) is within half a code step of x wherever x is inside the range (spot check of the whole tensor)
+    back = dy.dybit_decode(packed, n, fmt, scale)
+    err = (back - x).abs().max().item()
+    top = scale[0].item() * 2.0 ** ((fmt[0] - 1 if fmt[1] else fmt[0]) - 1)
+    assert err <= top / 2 + 1e-6
+    del x, packed, back
+    torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("fmt", [(2, 1), (3, 1), (4, 1), (6, 1), (8, 1)])
+@pytest.mark.parametrize("dist", ["normal", "laplace", "half_normal"])
+def test_quantize_sweep_2p20_full_parity(fmt, dist):
+    n = 1 << 20
+    f = fmt if dist != "half_normal" else (fmt[0], 0)
+    x = wl.DISTRIBUTIONS[dist]((n,), seed=fmt[0])
+    packed, scale = dy.dybit_quantize_pack(x.to(DEV), f)
+    sp = orc.absmax_scale(x.numpy(), f[0], bool(f[1]))
+    assert np.array_equal(scale.cpu().numpy(), np.array(sp, dtype=np.float32))
+    assert np.array_equal(packed.cpu().numpy(), orc.pack(orc.quantize(x.numpy(), f[0], bool(f[1]), sp[1]), f[0]))
+
+
+def _square_gemm(size, fmt, rng, n_rows, n_cols, n_points):
+    a = wl.normal((size, size), seed=size + fmt[0], device=DEV)
+    b = wl.normal((size, size), seed=size + fmt[0] + 1, device=DEV)
+    pa, sa = dy.dybit_quantize_pack_2d(a, fmt)
+    pb, sb = dy.dybit_quantize_pack_2d(b, fmt)
+    cont, _, _ = dy.dybit_choose_container(fmt, fmt)
+    C, C_raw = dy.dybit_gemm(size, size, size, pa, fmt, sa, pb, fmt, sb, want_raw=(cont == 0))
+    torch.cuda.synchronize()
+    assert dy.dybit_last_device_status() == (0, 0)
+    # oracle codes of both operands (full), from the same fp32 buffers
+    ah, bh = a.cpu().numpy(), b.cpu().numpy()
+    del a, b
+    spa = orc.absmax_scale(ah, fmt[0], bool(fmt[1]))
+    spb = orc.absmax_scale(bh, fmt[0], bool(fmt[1]))
+    ca = orc.quantize(ah, fmt[0], bool(fmt[1]), spa[1])
+    cb = orc.quantize(bh, fmt[0], bool(fmt[1]), spb[1])
+    assert np.array_equal(pa.cpu().numpy(), orc.pack_rows(ca, fmt[0]))
+    rows = rng.choice(size, n_rows, replace=False)
+    cols = rng.choice(size, n_cols, replace=False)
+    ri = np.concatenate([np.repeat(rows, size), np.tile(np.arange(size), n_cols), rng.integers(0, size, n_points)])
+    ci = np.concatenate([np.tile(np.arange(size), n_rows), np.repeat(cols, size), rng.integers(0, size, n_points)])
+    S, Cref = orc.gemm_sampled(ca, fmt, spa[0], cb, fmt, spb[0], ri, ci)
+    got = C[torch.from_numpy(ri).to(DEV), torch.from_numpy(ci).to(DEV)].cpu().numpy()
+    if cont == 0:
+        got_raw = C_raw[torch.from_numpy(ri).to(DEV), torch.from_numpy(ci).to(DEV)].cpu().numpy()
+        assert np.array_equal(got_raw.astype(np.int64), S)
+        assert np.array_equal(got, Cref)
+        # exact checksums over the whole output: column sums and row sums of the integer GEMM
+        m = fmt[0] - 1 if fmt[1] else fmt[0]
+        tab = np.round(orc.decode_table(fmt[0], bool(fmt[1])) * 2.0 ** (m - 1)).astype(np.int64)
+        IA, IB = tab[ca], tab[cb]
+        raw = C_raw.cpu().numpy().astype(np.int64)
+        assert np.array_equal(raw.sum(axis=0), IA.sum(axis=0) @ IB.T)
+        assert np.array_equal(raw.sum(axis=1), IA @ IB.sum(axis=0))
+    else:
+        amax = float(spa[0]) * float(np.abs(orc.decode_table(fmt[0], bool(fmt[1]))).max())
+        bmax = float(spb[0]) * float(np.abs(orc.decode_table(fmt[0], bool(fmt[1]))).max())
+        assert np.abs(got.astype(np.float64) - Cref.astype(np.float64)).max() <= 1e-5 * size * amax * bmax
+    torch.cuda.empty_cache()
+
+
+def test_square_gemm_8192_4bit_bench_configuration():
+    _square_gemm(8192, (4, 1), np.random.default_rng(1), n_rows=16, n_cols=16, n_points=20000)
+
+
+@pytest.mark.parametrize("size,fmt", [(1024, (4, 1)), (2048, (4, 1)), (4096, (4, 1)), (1024, (8, 1)), (4096, (8, 1)),
+                                      (8192, (8, 1))])
+def test_square_gemm_sweep(size, fmt):
+    _square_gemm(size, fmt, np.random.default_rng(size), n_rows=8, n_cols=8, n_points=5000)
+
+
+def _conv_layer_sampled(L, fx, fw, seed, n_samples=1500):
+    x = wl.half_normal((L.n, L.h, L.w, L.c), seed=seed, device=DEV)
+    w = wl.kaiming_normal(L.k, L.r, L.s, L.c, seed=seed + 1)
+    px, sx = dy.dybit_quantize_pack(x, fx)
+    pw, sw = dy.dybit_quantize_pack_2d(w.reshape(L.k, -1).to(DEV), fw)
+    desc = dy.ConvDesc(L.n, L.h, L.w, L.c, L.k, L.r, L.s, L.stride, L.pad, 1)
+    cont, _, _ = dy.dybit_choose_container(fx, fw)
+    Y, Y_raw = dy.dybit_conv2d(desc, px, fx, sx, pw, fw, sw, want_raw=(cont == 0))
+    torch.cuda.synchronize()
+    assert dy.dybit_last_device_status() == (0, 0)
+    xh = x.cpu().numpy()
+    spx = orc.absmax_scale(xh, fx[0], bool(fx[1]))
+    spw = orc.absmax_scale(w.numpy(), fw[0], bool(fw[1]))
+    assert np.array_equal(sx.cpu().numpy(), np.array(spx, dtype=np.float32))
+    cw = orc.quantize(w.numpy(), fw[0], bool(fw[1]), spw[1])
+    rng = np.random.default_rng(seed)
+    total = Y.numel()
+    idx = np.unique(np.concatenate([rng.integers(0, total, n_samples), [0, total - 1],
+                                    np.arange(total - L.k, total)]))          # incl. the last output pixel
+    S, Yref = orc.conv2d_sampled(xh, fx, spx, cw, fw, spw[0], idx, stride=L.stride, pad=L.pad)
+    got = Y.reshape(-1)[torch.from_numpy(idx).to(DEV)].cpu().numpy()
+    if cont == 0:
+        got_raw = Y_raw.reshape(-1)[torch.from_numpy(idx).to(DEV)].cpu().numpy()
+        assert np.array_equal(got_raw.astype(np.int64), S), L.name
+        assert np.array_equal(got, Yref), L.name
+    else:
+        amax = float(spx[0]) * float(np.abs(orc.decode_table(fx[0], bool(fx[1]))).max())
+        bmax = float(spw[0]) * float(np.abs(orc.decode_table(fw[0], bool(fw[1]))).max())
+        assert np.abs(got.astype(np.float64) - Yref.astype(np.float64)).max() <= 1e-5 * L.gemm_k * amax * bmax, L.name
+    return cont
+
+
+def _distinct(layers):
+    seen, out = set(), []
+    for i, L in enumerate(layers):
+        key = (L.h, L.w, L.c, L.k, L.r, L.s, L.stride, L.pad)
+        if key not in seen:
+            seen.add(key)
+            out.append((i, L))
+    return out
+
+
+@pytest.mark.parametrize("i,L", _distinct(wl.resnet18_layers(32)), ids=lambda v: getattr(v, "name", str(v)))
+def test_resnet18_batch32_uniform_4bit_sampled(i, L):
+    assert _conv_layer_sampled(L, (4, 0), (4, 1), seed=1000 + i) == 0
+
+
+_R50 = wl.resnet50_layers(64)
+_R50_BITS = wl.mixed_bitwidths(len(_R50), seed=0)
+
+
+@pytest.mark.parametrize("i,L", _distinct(_R50), ids=lambda v: getattr(v, "name", str(v)))
+def test_resnet50_batch64_mixed_bitwidths_sampled(i, L):
+    wbits, abits = _R50_BITS[i]
+    _conv_layer_sampled(L, (abits, 0), (wbits, 1), seed=3000 + i, n_samples=800)
+    torch.cuda.empty_cache()

@@ -200,3 +200,16 @@ def test_conv_equals_gemm_on_explicit_patches():
             row += 1
     Sg, _ = orc.gemm(patches, fx, 1.0, W.reshape(k, -1), fw, 1.0)
     assert np.array_equal(S.reshape(-1, k), Sg)
+
+
+def test_sampled_conv_is_the_full_conv_on_quantised_input():
+    fx, fw = (4, False), (3, True)
+    rng = np.random.default_rng(12)
+    n, h, w, c, k, r, stride, pad = 2, 9, 8, 6, 5, 3, 2, 1
+    x = np.abs(rng.normal(size=(n, h, w, c))).astype(np.float32)
+    W = rng.integers(0, 8, (k, r, r, c), dtype=np.uint8)
+    sp = orc.absmax_scale(x, *fx)
+    S, Y = orc.conv2d(orc.quantize(x, fx[0], fx[1], sp[1]), fx, sp[0], W, fw, 0.3, stride=stride, pad=pad)
+    idx = rng.permutation(S.size)[:97]
+    Ss, Ys = orc.conv2d_sampled(x, fx, sp, W, fw, 0.3, idx, stride=stride, pad=pad)
+    assert np.array_equal(Ss, S.ravel()[idx]) and np.array_equal(Ys, Y.ravel()[idx])
