@@ -187,12 +187,21 @@ def timed_region(fn, steps, dist, device):
     torch.cuda.synchronize(device)
     if dist is not None:
         dist.barrier()
-    ms = e0.elapsed_time(e1)
-    if dist is not None:
-        t = torch.tensor([ms], dtype=torch.float64, device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    return ms
+    return max_over_ranks(e0.elapsed_time(e1), dist, device)
+
+
+def max_over_ranks(ms, dist, device):
+    """The slowest rank's time: every multi-GPU number is reported against it."""
+    if dist is None:
+        return float(ms)
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tops(macs_per_rank, world, ms_step):
+    """Replicas: every rank runs the same step on its own GPU, so the job's work is world x one rank's."""
+    return world * 2.0 * macs_per_rank / (ms_step * 1e-3) / 1e12
 
 
 # --------------------------------------------------------------------------- single-kernel targets
@@ -314,7 +323,7 @@ def run_reference(args):
     from oracle import dybit_oracle as orc
     t1, _ = oracle_step(orc, wl, 1)
     per_step_budget = 120.0 / max(1, args.steps + args.warmup)
-    batch = max(1, min(32, int(per_step_budget / max(t1, 1e-3))))
+    batch = max(1, min(args.batch, int(per_step_budget / max(t1, 1e-3))))
     for _ in range(args.warmup):
         oracle_step(orc, wl, batch)
     total_t, total_macs = 0.0, 0
@@ -412,7 +421,7 @@ def main():
     ms_total = timed_region(graph.replay, args.steps, dist, device)
     launches = launches_per_step * args.steps
     ms_step = ms_total / args.steps
-    value = world * 2.0 * work.macs / (ms_step * 1e-3) / 1e12
+    value = whole_job_tops(work.macs, world, ms_step)
 
     # ---- the same K steps launched directly, with events around each layer's tensor-core kernel
     events = [[] for _ in work.layers]
@@ -440,7 +449,7 @@ def main():
         "peak_how": (f"2 x sustained bf16 ({peaks['source']})" if tensor_bound else f"copy bandwidth ({peaks['source']})"),
         "how": "CUDA events recorded by the library around this kernel alone, same K steps launched directly "
                "(not as a graph) right after the timed region",
-        "ms_per_step_in_kernel": mma_total_ms, "share_of_step": mma_total_ms / ms_step,
+        "ms_per_step_in_kernel": mma_total_ms, "share_of_step": mma_total_ms / ms_eager,
         "ms_per_step_direct_launch": ms_eager,
         "layers_us": {L.name: [round(t * 1e3, 1), round(b[2] * 1e6, 1)] for L, t, b in zip(work.layers, mma_ms, bounds)},
         "frac_of_layerwise_bound": ideal_s / (mma_total_ms * 1e-3),
@@ -453,7 +462,7 @@ def main():
         work.step_e2e()
     e2e_steps = max(2, min(args.steps, 5))
     ms_e2e = timed_region(work.step_e2e, e2e_steps, dist, device) / e2e_steps
-    e2e = {"value": world * 2.0 * work.macs / (ms_e2e * 1e-3) / 1e12, "unit": "TOPS",
+    e2e = {"value": whole_job_tops(work.macs, world, ms_e2e), "unit": "TOPS",
            "ms_per_step": ms_e2e, "h2d_bytes_per_step": work.h2d_bytes, "d2h_bytes_per_step": work.d2h_bytes}
 
     result = {

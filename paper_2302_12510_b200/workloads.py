@@ -122,7 +122,8 @@ def half_normal(shape, seed: int, device="cpu") -> torch.Tensor:
 def laplace(shape, seed: int, device="cpu") -> torch.Tensor:
     """Laplace(0,1) by inverse CDF of a uniform draw."""
     u = torch.rand(shape, generator=_gen(seed, device), device=device, dtype=torch.float32) - 0.5
-    return -torch.sign(u) * torch.log1p(-2.0 * u.abs())
+    mag = u.abs().clamp_(max=0.5 - 2.0 ** -25)          # rand() may return exactly 0: keep the log finite
+    return -torch.sign(u) * torch.log1p(-2.0 * mag)
 
 
 def kaiming_normal(k: int, r: int, s: int, c: int, seed: int, device="cpu") -> torch.Tensor:
