@@ -29,26 +29,28 @@ constexpr int kStreamThreads = kWarpsPerBlock * 32;
 // fraction lands on the next binade's first code by itself.  Along the code
 // axis the sub-unit line lies above every binade's line for t >= 1 and below
 // the e = 0 line for t < 1, so taking the smaller of the two candidates picks
-// the right one without a branch.  Each product is a power-of-two scaling
-// (exact); adding 1.5 * 2^23 (minus 2^k) inside the same FMA rounds the exact
-// sum to an integer, ties to even, and leaves that integer -- negative ones
-// too -- as an offset in the low mantissa bits.
+// the right one without a branch.  Each candidate is ONE FMA: the product is
+// a power-of-two scaling (exact), and the addend is 1.5 * 2^23 plus the
+// integer constant of the line (first_code(e) - 2^k = 2^M - 3 * 2^k), so the
+// FMA's single rounding is round-to-nearest-even on the final code itself and
+// leaves 0x4B400000 + code in the result's bit pattern.  The binade's
+// constants come straight from the exponent field of t.
 template <int M>
 __device__ __forceinline__ unsigned magnitude_code_biased(float a, float inv) {
-    constexpr unsigned kMagicBits = 0x4B400000u;                           // 1.5 * 2^23: ulp 1 on both sides
+    constexpr float kMagic = 12582912.0f;                                  // 1.5 * 2^23: ulp 1 on both sides
     // largest float below the top value 2^(M-1): everything from 1.5 * 2^(M-2) up rounds to all-ones anyway
     const float below_top = __uint_as_float(((unsigned)(127 + M - 1) << 23) - 1u);
     const float t = fminf(__fmul_rn(a, inv), below_top);
-    const unsigned sub = __float_as_uint(__fmaf_rn(t, (float)(1u << (M - 1)), __uint_as_float(kMagicBits)));
+    const unsigned sub = __float_as_uint(__fmaf_rn(t, (float)(1u << (M - 1)), kMagic));
     if constexpr (M == 1) {
         return sub;
     } else {
-        const unsigned E = max(__float_as_uint(t) >> 23, 127u);           // biased exponent, sub-unit folded onto e = 0
-        const float scale_e = __uint_as_float(((unsigned)(381 + M - 2) << 23) - (E << 24));   // 2^(k-e)
-        const unsigned k = (unsigned)(127 + M - 2) - E;
-        const unsigned one_k = 1u << k;
-        const unsigned sup = __float_as_uint(__fmaf_rn(t, scale_e, __uint_as_float(kMagicBits - one_k)));
-        const unsigned cand = sup + (1u << M) - 2u * one_k;                // + first_code(e) = 2^M - 2^(k+1)
+        // exponent field of max(t, 1): the sub-unit range is folded onto binade 0
+        const unsigned eb = __float_as_uint(fmaxf(t, 1.0f)) & 0x7f800000u;
+        const float scale_e = __uint_as_float(((unsigned)(379 + M) << 23) - 2u * eb);                 // 2^(k-e)
+        const float three_2k = __uint_as_float((((unsigned)(253 + M) << 23) | 0x400000u) - eb);       // 3 * 2^k
+        const float addend = (kMagic + (float)(1u << M)) - three_2k;                                   // exact integer
+        const unsigned cand = __float_as_uint(__fmaf_rn(t, scale_e, addend));
         return min(sub, cand);
     }
 }
@@ -69,8 +71,7 @@ __device__ __forceinline__ unsigned encode4(const float4 v, const float inv) {
                                           __byte_perm(__float_as_uint(v.z), __float_as_uint(v.w), 0x0073), 0x5410);
         // bit 7 of each byte set where the magnitude code is non-zero (codes are < 128)
         const unsigned nonzero = (mags + 0x7f7f7f7fu) | mags;
-        const unsigned sign = ((tops & nonzero & 0x80808080u) >> (7 - M));
-        return mags | sign;
+        return mags | (((tops & nonzero) >> (7 - M)) & (0x01010101u << M));
     } else {
         // no sign bit: negative inputs (and NaN) take the nearest value the format has, 0
         const unsigned m0 = magnitude_code_biased<M>(fmaxf(v.x, 0.0f), inv);
@@ -199,7 +200,7 @@ __device__ __forceinline__ void pack32(const unsigned (&cw)[8], unsigned (&out)[
 }
 
 template <int BITS, bool SIGNED>
-__global__ void __launch_bounds__(kStreamThreads)
+__global__ void __launch_bounds__(kStreamThreads, 3)
 quantize_pack_kernel(const float *__restrict__ x, int64_t rows, int64_t cols, int64_t ld,
                      const float *__restrict__ scale, uint8_t *__restrict__ out,
                      int64_t row_stride_bytes, int64_t chunks_per_row) {
