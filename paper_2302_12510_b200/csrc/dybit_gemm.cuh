@@ -119,6 +119,59 @@ expand_rows_kernel(const uint8_t *__restrict__ packed, int64_t rows, int64_t in_
     }
 }
 
+// 4-bit codes -> 1-byte container elements without shared memory.  A 32-bit word holds eight codes; the
+// byte-permute unit looks four of them up at once in a 16-entry table kept in four registers.  A selector
+// nibble with its top bit set makes prmt replicate the selected byte's sign bit, which is 0x00 for the
+// non-negative bytes stored here, so "lookup in the low half with the raw nibbles" and "lookup in the high
+// half with the top bits flipped" each yield 0 for the codes that belong to the other half.
+//   neg_high = false: the table's entries are used as they are (all 16 values non-negative): result = lo | hi
+//   neg_high = true : entries 8..15 hold MAGNITUDES of negative values: result = lo - hi, byte-wise
+// Two independent operands (jobs) can share one launch.
+struct Expand4Job {
+    const uint8_t *packed;
+    uint8_t *out;
+    int64_t rows, in_stride, out_stride;
+    int64_t vecs_per_row;      // 16-byte input vectors (32 codes) per row
+    unsigned tab[4];           // 16 table bytes
+    int neg_high;
+};
+
+// prmt in its generic form: selector nibble bits 0-2 pick one of the eight source bytes, bit 3 asks
+// for that byte's sign bit replicated instead of the byte (the __byte_perm intrinsic drops bit 3).
+__device__ __forceinline__ unsigned prmt_generic(unsigned a, unsigned b, unsigned sel) {
+    unsigned d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+
+__device__ __forceinline__ unsigned expand4_lookup(unsigned sel, const unsigned (&t)[4], bool neg_high) {
+    const unsigned lo = prmt_generic(t[0], t[1], sel);
+    const unsigned hi = prmt_generic(t[2], t[3], sel ^ 0x8888u);
+    // byte-wise lo - hi: never both non-zero; the 0x80 guard bits stop borrows between bytes
+    return neg_high ? (((lo | 0x80808080u) - hi) ^ 0x80808080u) : (lo | hi);
+}
+
+__global__ void __launch_bounds__(256) expand4_kernel(const Expand4Job j0, const Expand4Job j1, int64_t vecs0) {
+    const int64_t total = vecs0 + j1.rows * j1.vecs_per_row;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const bool first = i < vecs0;
+        const Expand4Job &j = first ? j0 : j1;
+        const int64_t v = first ? i : i - vecs0;
+        const int64_t row = v / j.vecs_per_row, col = v - row * j.vecs_per_row;
+        const uint4 w = __ldg(reinterpret_cast<const uint4 *>(j.packed + row * j.in_stride) + col);
+        const unsigned t[4] = {j.tab[0], j.tab[1], j.tab[2], j.tab[3]};
+        const bool ng = j.neg_high != 0;
+        uint4 o0, o1;
+        o0.x = expand4_lookup(w.x, t, ng); o0.y = expand4_lookup(w.x >> 16, t, ng);
+        o0.z = expand4_lookup(w.y, t, ng); o0.w = expand4_lookup(w.y >> 16, t, ng);
+        o1.x = expand4_lookup(w.z, t, ng); o1.y = expand4_lookup(w.z >> 16, t, ng);
+        o1.z = expand4_lookup(w.w, t, ng); o1.w = expand4_lookup(w.w >> 16, t, ng);
+        uint4 *dst = reinterpret_cast<uint4 *>(j.out + row * j.out_stride + col * 32);
+        dst[0] = o0;
+        dst[1] = o1;
+    }
+}
+
 // Generic (slow) expand with channel padding: output row = taps x cp elements, where tap t
 // takes codes [t*c, t*c + c) of the input row's bit stream and pads channels c..cp-1 with 0.
 // One thread writes one 16-byte output chunk.
@@ -154,6 +207,49 @@ __global__ void expand_pad_kernel(const uint8_t *__restrict__ packed, int bits, 
     }
 }
 
+// One operand's expand job: rows of `cols` codes -> rows of container elements.
+struct ExpandOperand {
+    const uint8_t *packed;
+    int bits;
+    int64_t rows, in_stride, cols;
+    uint8_t *out;
+    int64_t out_stride;
+    const ElemTable *table;
+};
+
+// True when the 4-bit register-table kernel applies: 1-byte container, whole 32-code vectors, and a table
+// whose low half is non-negative and whose high half is either non-negative or the negated low-half style.
+static bool expand4_job(const ExpandOperand &op, int elem, bool int8_container, Expand4Job *job) {
+    if (op.bits != 4 || elem != 1 || op.cols % 32 != 0 || op.rows <= 0) return false;
+    if (op.rows > 1 && (op.in_stride % 16 != 0 || op.out_stride % 16 != 0)) return false;
+    int8_t v[16];
+    for (int c = 0; c < 16; ++c) v[c] = (int8_t)(op.table->v[c] & 0xff);
+    bool low_ok = true, high_pos = true, high_neg = true;
+    for (int c = 0; c < 8; ++c) low_ok = low_ok && v[c] >= 0;
+    for (int c = 8; c < 16; ++c) {
+        high_pos = high_pos && v[c] >= 0;
+        high_neg = high_neg && int8_container && v[c] <= 0 && v[c] > -128;   // two's complement only
+    }
+    if (!low_ok || !(high_pos || high_neg)) return false;
+    job->packed = op.packed;
+    job->out = op.out;
+    job->rows = op.rows;
+    job->in_stride = op.in_stride;
+    job->out_stride = op.out_stride;
+    job->vecs_per_row = op.cols / 32;
+    job->neg_high = high_pos ? 0 : 1;
+    for (int w = 0; w < 4; ++w) {
+        unsigned word = 0;
+        for (int b = 0; b < 4; ++b) {
+            const int c = w * 4 + b;
+            const int mag = (c >= 8 && !high_pos) ? -v[c] : v[c];
+            word |= (unsigned)(mag & 0xff) << (8 * b);
+        }
+        job->tab[w] = word;
+    }
+    return true;
+}
+
 template <int ELEM>
 static dybit_status launch_expand_rows(const uint8_t *packed, int bits, int64_t rows, int64_t in_stride, int64_t cols,
                                        uint8_t *out, int64_t out_stride, const ElemTable &t, cudaStream_t s) {
@@ -177,6 +273,33 @@ static dybit_status launch_expand(const uint8_t *packed, int bits, int64_t rows,
                                   int elem, uint8_t *out, int64_t out_stride, const ElemTable &t, cudaStream_t s) {
     return elem == 1 ? launch_expand_rows<1>(packed, bits, rows, in_stride, cols, out, out_stride, t, s)
                      : launch_expand_rows<2>(packed, bits, rows, in_stride, cols, out, out_stride, t, s);
+}
+
+// Expands both operands of a GEMM: one launch when both take the 4-bit register-table kernel.
+static dybit_status launch_expand_pair(const ExpandOperand &a, const ExpandOperand &b, int elem, bool int8_container,
+                                       cudaStream_t s) {
+    Expand4Job ja, jb;
+    const bool fa = expand4_job(a, elem, int8_container, &ja), fb = expand4_job(b, elem, int8_container, &jb);
+    if (fa || fb) {
+        Expand4Job none = {};
+        const Expand4Job &j0 = fa ? ja : jb;
+        const Expand4Job &j1 = (fa && fb) ? jb : none;
+        const int64_t vecs0 = j0.rows * j0.vecs_per_row;
+        const int64_t total = vecs0 + j1.rows * j1.vecs_per_row;
+        int64_t blocks = (total + 255) / 256, cap = (int64_t)sm_count() * 16;
+        if (blocks > cap) blocks = cap;
+        expand4_kernel<<<(int)blocks, 256, 0, s>>>(j0, j1, vecs0);
+        if (launch_status() != DYBIT_OK) return DYBIT_ERR_CUDA;
+    }
+    if (!fa) {
+        dybit_status st = launch_expand(a.packed, a.bits, a.rows, a.in_stride, a.cols, elem, a.out, a.out_stride, *a.table, s);
+        if (st != DYBIT_OK) return st;
+    }
+    if (!fb) {
+        dybit_status st = launch_expand(b.packed, b.bits, b.rows, b.in_stride, b.cols, elem, b.out, b.out_stride, *b.table, s);
+        if (st != DYBIT_OK) return st;
+    }
+    return DYBIT_OK;
 }
 
 // ------------------------------------------------------------------ the tcgen05 GEMM
@@ -699,9 +822,9 @@ dybit_status dybit_gemm(int64_t M, int64_t N, int64_t K, const void *A, dybit_fm
     uint8_t *be = ae + round_up(M * rb, 1024);
     const ElemTable ta = make_elem_table(fa, plan.container, plan.exp_a);
     const ElemTable tb = make_elem_table(fb, plan.container, plan.exp_b);
-    st = launch_expand(static_cast<const uint8_t *>(A), fa.bits, M, lda_bytes, kp, elem, ae, rb, ta, s);
-    if (st != DYBIT_OK) return st;
-    st = launch_expand(static_cast<const uint8_t *>(B), fb.bits, N, ldb_bytes, kp, elem, be, rb, tb, s);
+    const ExpandOperand opa = {static_cast<const uint8_t *>(A), fa.bits, M, lda_bytes, kp, ae, rb, &ta};
+    const ExpandOperand opb = {static_cast<const uint8_t *>(B), fb.bits, N, ldb_bytes, kp, be, rb, &tb};
+    st = launch_expand_pair(opa, opb, elem, plan.container == DYBIT_CONTAINER_I8, s);
     if (st != DYBIT_OK) return st;
 
     const int bn = choose_bn(M, N);
@@ -763,9 +886,9 @@ dybit_status dybit_conv2d(const dybit_conv_desc *d, const void *X, dybit_fmt fx,
     const ElemTable tw = make_elem_table(fw, plan.container, plan.exp_b);
     if (cp == d->c) {
         // channels already a multiple of 16: X is one flat run, W rows expand with their zero tail
-        st = launch_expand(static_cast<const uint8_t *>(X), fx.bits, 1, 0, pixels * cp, elem, xe, 0, tx, s);
-        if (st != DYBIT_OK) return st;
-        st = launch_expand(static_cast<const uint8_t *>(W), fw.bits, N, ldw_bytes, wrb / elem, elem, we, wrb, tw, s);
+        const ExpandOperand opx = {static_cast<const uint8_t *>(X), fx.bits, 1, 0, pixels * cp, xe, 0, &tx};
+        const ExpandOperand opw = {static_cast<const uint8_t *>(W), fw.bits, N, ldw_bytes, wrb / elem, we, wrb, &tw};
+        st = launch_expand_pair(opx, opw, elem, plan.container == DYBIT_CONTAINER_I8, s);
         if (st != DYBIT_OK) return st;
     } else {
         const int64_t taps = (int64_t)d->r * d->s;

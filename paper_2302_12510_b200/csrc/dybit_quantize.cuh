@@ -90,11 +90,14 @@ __device__ __forceinline__ unsigned finite_abs_bits(float v) {
 }
 
 // Largest finite |x| as raw fp32 bits (non-negative floats order like their
-// bit patterns), max-reduced into *slot, which the host zeroes beforehand.
+// bit patterns), max-reduced into slot[0]; slot[1] counts finished blocks.  The
+// host zeroes both words beforehand.  The block that finishes last turns the
+// pair into {scale, 1/scale} for m magnitude bits: amax / 2^(m-1) and one IEEE
+// division 2^(m-1) / amax ({1, 1} for an all-zero tensor).
 // Handles rows x cols with leading dimension ld (ld == cols: one flat run).
 __global__ void __launch_bounds__(kStreamThreads)
 absmax_kernel(const float *__restrict__ x, int64_t rows, int64_t cols, int64_t ld,
-              unsigned *__restrict__ slot) {
+              unsigned *__restrict__ slot, int m) {
     unsigned best = 0;
     const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int64_t nthreads = (int64_t)gridDim.x * blockDim.x;
@@ -139,21 +142,31 @@ absmax_kernel(const float *__restrict__ x, int64_t rows, int64_t cols, int64_t l
     if (threadIdx.x < 32) {
         unsigned b = threadIdx.x < kWarpsPerBlock ? warp_best[threadIdx.x] : 0u;
         b = __reduce_max_sync(0xffffffffu, b);
-        if (threadIdx.x == 0 && b != 0u) atomicMax(slot, b);
+        if (threadIdx.x == 0) {
+            if (b != 0u) atomicMax(slot, b);
+            __threadfence();
+            const unsigned ticket = atomicAdd(slot + 1, 1u);
+            if (ticket == gridDim.x - 1) {
+                __threadfence();
+                const float amax = __uint_as_float(atomicMax(slot, 0u));     // the final maximum
+                float *scale = reinterpret_cast<float *>(slot);
+                if (amax == 0.0f) {
+                    scale[0] = 1.0f;
+                    scale[1] = 1.0f;
+                } else {
+                    const float vmax = (float)(1u << (m - 1));
+                    scale[0] = __fdiv_rn(amax, vmax);
+                    scale[1] = __fdiv_rn(vmax, amax);
+                }
+            }
+        }
     }
 }
 
-// slot holds amax bits in scale[0] on entry; leaves {scale, 1/scale}.
-__global__ void finalize_scale_kernel(float *scale, int m) {
-    const float amax = scale[0];
-    if (amax == 0.0f) {
-        scale[0] = 1.0f;
-        scale[1] = 1.0f;
-    } else {
-        const float vmax = (float)(1u << (m - 1));
-        scale[0] = __fdiv_rn(amax, vmax);
-        scale[1] = __fdiv_rn(vmax, amax);
-    }
+// Empty tensor: no reduction runs, the scale is {1, 1}.
+__global__ void unit_scale_kernel(float *scale) {
+    scale[0] = 1.0f;
+    scale[1] = 1.0f;
 }
 
 // ------------------------------------------------------------------ quantize + pack
@@ -385,10 +398,10 @@ static dybit_status launch_absmax(const float *x, int64_t rows, int64_t cols, in
         if (blocks > cap) blocks = cap;
         if (blocks < 1) blocks = 1;
         absmax_kernel<<<(int)blocks, kStreamThreads, 0, s>>>(x, rows, cols, ld,
-                                                             reinterpret_cast<unsigned *>(scale_out));
-        if (launch_status() != DYBIT_OK) return DYBIT_ERR_CUDA;
+                                                             reinterpret_cast<unsigned *>(scale_out), mag_bits(fmt));
+        return launch_status();
     }
-    finalize_scale_kernel<<<1, 1, 0, s>>>(scale_out, mag_bits(fmt));
+    unit_scale_kernel<<<1, 1, 0, s>>>(scale_out);
     return launch_status();
 }
 
