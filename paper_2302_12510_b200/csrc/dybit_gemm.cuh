@@ -250,6 +250,66 @@ static bool expand4_job(const ExpandOperand &op, int elem, bool int8_container, 
     return true;
 }
 
+// Patch matrix for convolutions with few channels (pixel = neither 64 nor a multiple of 128 container
+// bytes, e.g. the 3-channel stem): row m = output pixel, columns = the R*S*C taps in (r, s, c) order,
+// decoded straight from the packed activation stream, zero where a tap falls outside the image, rows
+// padded with zeros to krow bytes.  One thread assembles one row in shared memory (for a fixed r the
+// S*C codes of the window are contiguous in NHWC); the block then writes its rows out coalesced.
+struct PatchParams {
+    const uint8_t *packed;     // dense NHWC code stream
+    uint8_t *out;              // [M][krow] container bytes
+    int bits, elem;
+    int H, W, C, R, S, OH, OW, stride, pad, dil;
+    int M, krow, row_pitch;    // row_pitch = krow + 4: odd word count, so threads hit distinct banks
+};
+
+__global__ void __launch_bounds__(128)
+patch_expand_kernel(const PatchParams p, const __grid_constant__ ElemTable table) {
+    extern __shared__ __align__(16) uint8_t s_rows[];
+    __shared__ uint16_t s_lut[256];
+    for (int i = threadIdx.x; i < 256; i += blockDim.x) s_lut[i] = table.v[i];
+    // zero everything first: padding taps and the row tail stay zero
+    for (int i = threadIdx.x; i < (128 * p.row_pitch) / 4; i += blockDim.x) reinterpret_cast<unsigned *>(s_rows)[i] = 0u;
+    __syncthreads();
+    const int m = blockIdx.x * 128 + threadIdx.x;
+    if (m < p.M) {
+        const int img = m / (p.OH * p.OW);
+        const int rem = m - img * (p.OH * p.OW);
+        const int oh = rem / p.OW, ow = rem - oh * p.OW;
+        const int ih0 = oh * p.stride - p.pad, iw0 = ow * p.stride - p.pad;
+        const unsigned mask = (1u << p.bits) - 1u;
+        uint8_t *row = s_rows + threadIdx.x * p.row_pitch;
+        for (int fr = 0; fr < p.R; ++fr) {
+            const int ih = ih0 + fr * p.dil;
+            if ((unsigned)ih >= (unsigned)p.H) continue;
+            for (int fs = 0; fs < p.S; ++fs) {
+                const int iw = iw0 + fs * p.dil;
+                if ((unsigned)iw >= (unsigned)p.W) continue;
+                int64_t bit = ((((int64_t)img * p.H + ih) * p.W + iw) * p.C) * p.bits;
+                uint8_t *dst = row + ((fr * p.S + fs) * p.C) * p.elem;
+                for (int c = 0; c < p.C; ++c, bit += p.bits) {
+                    const int sh = (int)(bit & 7);
+                    unsigned two = __ldg(p.packed + (bit >> 3));
+                    if (sh + p.bits > 8) two |= (unsigned)__ldg(p.packed + (bit >> 3) + 1) << 8;
+                    const unsigned v = s_lut[(two >> sh) & mask];
+                    if (p.elem == 1) dst[c] = (uint8_t)v;
+                    else reinterpret_cast<uint16_t *>(dst)[c] = (uint16_t)v;
+                }
+            }
+        }
+    }
+    __syncthreads();
+    // rows [blockIdx*128, +128) x krow bytes, 16 bytes per thread per step
+    const int vec_per_row = p.krow / 16;
+    const int rows_here = min(128, p.M - blockIdx.x * 128);
+    for (int i = threadIdx.x; i < rows_here * vec_per_row; i += blockDim.x) {
+        const int r = i / vec_per_row, v = i - r * vec_per_row;
+        const unsigned *src = reinterpret_cast<const unsigned *>(s_rows + r * p.row_pitch + v * 16);
+        const uint4 val = make_uint4(src[0], src[1], src[2], src[3]);
+        *reinterpret_cast<uint4 *>(p.out + ((int64_t)blockIdx.x * 128 + r) * p.krow + v * 16) = val;
+    }
+}
+
 template <int ELEM>
 static dybit_status launch_expand_rows(const uint8_t *packed, int bits, int64_t rows, int64_t in_stride, int64_t cols,
                                        uint8_t *out, int64_t out_stride, const ElemTable &t, cudaStream_t s) {
@@ -767,6 +827,51 @@ struct GemmLayout {
 
 static inline int64_t k_row_bytes(int64_t k_elems, int elem) { return round_up(k_elems * elem, kBKBytes); }
 
+// How a convolution is lowered, and what it needs in the workspace.
+enum ConvMode { kConvPointwise, kConvIm2col, kConvPatch, kConvGather };
+struct ConvPlan {
+    ConvMode mode;
+    int elem, swb;
+    int64_t cp, cpb, pixels;       // padded channels, bytes per pixel of the expanded activation
+    int64_t a_bytes;               // first workspace region: expanded activation or patch matrix
+    int64_t krow;                  // patch mode: bytes per patch row
+    int64_t wrb;                   // bytes per expanded weight row
+    bool pad_channels;             // expanded activation / weights carry zero channels c..cp-1
+};
+
+static ConvPlan plan_conv(const dybit_conv_desc *d, int oh, int ow, int elem) {
+    ConvPlan c = {};
+    c.elem = elem;
+    c.cp = round_up(d->c, 16);
+    c.cpb = c.cp * elem;
+    c.pixels = (int64_t)d->n * d->h * d->w;
+    const int64_t M = (int64_t)d->n * oh * ow;
+    const int64_t taps = (int64_t)d->r * d->s;
+    const bool pointwise = d->r == 1 && d->s == 1 && d->stride == 1 && d->pad == 0;
+    // im2col TMA: a pixel must be a whole number of swizzle-span blocks, corners and tap offsets must fit the
+    // descriptor's 8-bit fields, and the tensor must not be tiny
+    c.swb = (c.cpb % 128 == 0) ? 128 : (c.cpb == 64 ? 64 : 0);
+    const int up_w = d->pad - (d->s - 1) * d->dilation, up_h = d->pad - (d->r - 1) * d->dilation;
+    const bool im2col_ok = c.swb != 0 && c.pixels * c.cpb >= 131072 && d->pad <= 127 && up_w >= -128 && up_h >= -128 &&
+                           (d->s - 1) * d->dilation <= 255 && (d->r - 1) * d->dilation <= 255 && d->stride <= 8;
+    const int64_t krow = round_up(taps * d->c * elem, 16);
+    if (pointwise) c.mode = kConvPointwise;
+    else if (im2col_ok) c.mode = kConvIm2col;
+    else if (krow <= 1024 && M * krow <= ((int64_t)1 << 32)) c.mode = kConvPatch;
+    else c.mode = kConvGather;
+    if (c.mode == kConvPatch) {
+        c.krow = krow;
+        c.a_bytes = round_up(M * krow, 1024);
+        c.wrb = k_row_bytes(taps * d->c, elem);
+        c.pad_channels = false;
+    } else {
+        c.a_bytes = round_up(c.pixels * c.cpb, 1024);
+        c.wrb = k_row_bytes(taps * c.cp, elem);
+        c.pad_channels = c.cp != d->c;
+    }
+    return c;
+}
+
 }  // namespace dybit
 
 extern "C" {
@@ -785,11 +890,8 @@ size_t dybit_conv2d_workspace_bytes(const dybit_conv_desc *d, dybit_fmt fx, dybi
     ContainerPlan plan;
     int oh, ow;
     if (dybit_conv2d_out_hw(d, &oh, &ow) != DYBIT_OK || plan_container(fx, fw, &plan) != DYBIT_OK) return 0;
-    const int elem = container_elem_bytes(plan.container);
-    const int64_t cp = round_up(d->c, 16);
-    const int64_t x_bytes = round_up((int64_t)d->n * d->h * d->w * cp * elem, 1024);
-    const int64_t w_bytes = round_up((int64_t)d->k * k_row_bytes((int64_t)d->r * d->s * cp, elem), 1024);
-    return (size_t)(x_bytes + w_bytes + 2048);
+    const ConvPlan c = plan_conv(d, oh, ow, container_elem_bytes(plan.container));
+    return (size_t)(c.a_bytes + round_up((int64_t)d->k * c.wrb, 1024) + 2048);
 }
 
 dybit_status dybit_gemm(int64_t M, int64_t N, int64_t K, const void *A, dybit_fmt fa, const float *scale_a,
@@ -876,19 +978,43 @@ dybit_status dybit_conv2d(const dybit_conv_desc *d, const void *X, dybit_fmt fx,
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const int elem = container_elem_bytes(plan.container);
-    const int64_t cp = round_up(d->c, 16);
-    const int64_t pixels = (int64_t)d->n * d->h * d->w;
-    const int64_t x_bytes = round_up(pixels * cp * elem, 1024);
-    const int64_t wrb = k_row_bytes((int64_t)d->r * d->s * cp, elem);
+    const ConvPlan cv = plan_conv(d, oh, ow, elem);
+    const int64_t cp = cv.cp, pixels = cv.pixels, wrb = cv.wrb;
     uint8_t *xe = static_cast<uint8_t *>(ws);
-    uint8_t *we = xe + x_bytes;
+    uint8_t *we = xe + cv.a_bytes;
     const ElemTable tx = make_elem_table(fx, plan.container, plan.exp_a);
     const ElemTable tw = make_elem_table(fw, plan.container, plan.exp_b);
-    if (cp == d->c) {
+    const bool i8 = plan.container == DYBIT_CONTAINER_I8;
+    if (cv.mode == kConvPatch) {
+        // patch matrix from the packed activation in one kernel; weights expand as plain rows (K order r, s, c)
+        PatchParams pp = {};
+        pp.packed = static_cast<const uint8_t *>(X);
+        pp.out = xe;
+        pp.bits = fx.bits;
+        pp.elem = elem;
+        pp.H = d->h; pp.W = d->w; pp.C = d->c; pp.R = d->r; pp.S = d->s;
+        pp.OH = oh; pp.OW = ow; pp.stride = d->stride; pp.pad = d->pad; pp.dil = d->dilation;
+        pp.M = (int)M;
+        pp.krow = (int)cv.krow;
+        pp.row_pitch = (int)cv.krow + 4;
+        const size_t smem = (size_t)128 * pp.row_pitch;
+        static bool patch_configured[64] = {};
+        int dev = 0;
+        DYBIT_CUDA_TRY(cudaGetDevice(&dev));
+        if (dev >= 0 && dev < 64 && !patch_configured[dev]) {
+            DYBIT_CUDA_TRY(cudaFuncSetAttribute(patch_expand_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                128 * (1024 + 4)));
+            patch_configured[dev] = true;
+        }
+        patch_expand_kernel<<<(int)((M + 127) / 128), 128, smem, s>>>(pp, tx);
+        if (launch_status() != DYBIT_OK) return DYBIT_ERR_CUDA;
+        st = launch_expand(static_cast<const uint8_t *>(W), fw.bits, N, ldw_bytes, wrb / elem, elem, we, wrb, tw, s);
+        if (st != DYBIT_OK) return st;
+    } else if (!cv.pad_channels) {
         // channels already a multiple of 16: X is one flat run, W rows expand with their zero tail
         const ExpandOperand opx = {static_cast<const uint8_t *>(X), fx.bits, 1, 0, pixels * cp, xe, 0, &tx};
         const ExpandOperand opw = {static_cast<const uint8_t *>(W), fw.bits, N, ldw_bytes, wrb / elem, we, wrb, &tw};
-        st = launch_expand_pair(opx, opw, elem, plan.container == DYBIT_CONTAINER_I8, s);
+        st = launch_expand_pair(opx, opw, elem, i8, s);
         if (st != DYBIT_OK) return st;
     } else {
         const int64_t taps = (int64_t)d->r * d->s;
@@ -929,23 +1055,18 @@ dybit_status dybit_conv2d(const dybit_conv_desc *d, const void *X, dybit_fmt fx,
     p.cpb = (int)cpb;
 
     CUtensorMap map_a, map_b;
-    const bool pointwise = d->r == 1 && d->s == 1 && d->stride == 1 && d->pad == 0;
-    if (pointwise) {
-        // a 1x1 stride-1 convolution is the GEMM [pixels][cpb] x [k][cpb]^T on the expanded activation
-        st = make_operand_map(&map_a, xe, M, cpb, cpb, kBM);
+    if (cv.mode == kConvPointwise || cv.mode == kConvPatch) {
+        // a GEMM on a row-major A: the expanded activation itself (1x1, stride 1) or the patch matrix
+        const int64_t arow = cv.mode == kConvPatch ? cv.krow : cpb;
+        st = make_operand_map(&map_a, xe, M, arow, arow, kBM);
         if (st != DYBIT_OK) return st;
         st = make_operand_map(&map_b, we, N, wrb, wrb, bn);
         if (st != DYBIT_OK) return st;
         p.k_blocks = (int)(wrb / kBKBytes);
         return launch_gemm_kind<kATiled, 128>(plan.container, bn, map_a, map_b, p, s);
     }
-    // im2col TMA: a pixel must be a whole number of swizzle-span blocks, corners and tap offsets must
-    // fit the descriptor's 8-bit fields, and the tensor must not be tiny (tiny ones take the gather path)
-    const int swb = (cpb % 128 == 0) ? 128 : (cpb == 64 ? 64 : 0);
-    const int up_w = d->pad - (d->s - 1) * d->dilation, up_h = d->pad - (d->r - 1) * d->dilation;
-    const bool im2col_ok = swb != 0 && pixels * cpb >= 131072 && d->pad <= 127 && up_w >= -128 && up_h >= -128 &&
-                           (d->s - 1) * d->dilation <= 255 && (d->r - 1) * d->dilation <= 255 && d->stride <= 8;
-    if (im2col_ok) {
+    if (cv.mode == kConvIm2col) {
+        const int swb = cv.swb;
         st = make_im2col_map(&map_a, xe, d, cpb, swb);
         if (st != DYBIT_OK) return st;
         st = make_operand_map(&map_b, we, N, wrb, wrb, bn, swb);
