@@ -257,6 +257,7 @@ static bool expand4_job(const ExpandOperand &op, int elem, bool int8_container, 
 // S*C codes of the window are contiguous in NHWC); the block then writes its rows out coalesced.
 struct PatchParams {
     const uint8_t *packed;     // dense NHWC code stream
+    int64_t packed_words;      // its length in 32-bit words
     uint8_t *out;              // [M][krow] container bytes
     int bits, elem;
     int H, W, C, R, S, OH, OW, stride, pad, dil;
@@ -279,9 +280,39 @@ patch_expand_kernel(const PatchParams p, const __grid_constant__ ElemTable table
         const int ih0 = oh * p.stride - p.pad, iw0 = ow * p.stride - p.pad;
         const unsigned mask = (1u << p.bits) - 1u;
         uint8_t *row = s_rows + threadIdx.x * p.row_pitch;
+        const unsigned *w32 = reinterpret_cast<const unsigned *>(p.packed);
         for (int fr = 0; fr < p.R; ++fr) {
             const int ih = ih0 + fr * p.dil;
             if ((unsigned)ih >= (unsigned)p.H) continue;
+            if (p.dil == 1) {
+                // the taps of one filter row that fall inside the image are one contiguous run of codes
+                const int s_lo = max(0, -iw0), s_hi = min(p.S, p.W - iw0);
+                if (s_lo >= s_hi) continue;
+                const int64_t bit = ((((int64_t)img * p.H + ih) * p.W + (iw0 + s_lo)) * p.C) * p.bits;
+                uint8_t *dst = row + ((fr * p.S + s_lo) * p.C) * p.elem;
+                const int count = (s_hi - s_lo) * p.C;
+                // 64-bit window over the stream, refilled one word at a time
+                int64_t wi = bit >> 5;
+                const int sh = (int)(bit & 31);
+                unsigned long long buf = __ldg(w32 + wi);
+                if (wi + 1 < p.packed_words) buf |= (unsigned long long)__ldg(w32 + wi + 1) << 32;
+                buf >>= sh;
+                int avail = 64 - sh;
+                wi += 2;
+                for (int c = 0; c < count; ++c) {
+                    if (avail < p.bits) {
+                        if (wi < p.packed_words) buf |= (unsigned long long)__ldg(w32 + wi) << avail;
+                        ++wi;
+                        avail += 32;
+                    }
+                    const unsigned v = s_lut[(unsigned)buf & mask];
+                    buf >>= p.bits;
+                    avail -= p.bits;
+                    if (p.elem == 1) dst[c] = (uint8_t)v;
+                    else reinterpret_cast<uint16_t *>(dst)[c] = (uint16_t)v;
+                }
+                continue;
+            }
             for (int fs = 0; fs < p.S; ++fs) {
                 const int iw = iw0 + fs * p.dil;
                 if ((unsigned)iw >= (unsigned)p.W) continue;
@@ -989,6 +1020,7 @@ dybit_status dybit_conv2d(const dybit_conv_desc *d, const void *X, dybit_fmt fx,
         // patch matrix from the packed activation in one kernel; weights expand as plain rows (K order r, s, c)
         PatchParams pp = {};
         pp.packed = static_cast<const uint8_t *>(X);
+        pp.packed_words = (int64_t)dybit_packed_bytes(pixels * d->c, fx.bits) / 4;
         pp.out = xe;
         pp.bits = fx.bits;
         pp.elem = elem;

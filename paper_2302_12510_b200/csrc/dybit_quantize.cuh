@@ -95,6 +95,7 @@ __device__ __forceinline__ unsigned finite_abs_bits(float v) {
 // pair into {scale, 1/scale} for m magnitude bits: amax / 2^(m-1) and one IEEE
 // division 2^(m-1) / amax ({1, 1} for an all-zero tensor).
 // Handles rows x cols with leading dimension ld (ld == cols: one flat run).
+template <bool STREAM>   // STREAM: evict-first loads (tensor larger than L2); otherwise leave it in L2 for the next pass
 __global__ void __launch_bounds__(kStreamThreads)
 absmax_kernel(const float *__restrict__ x, int64_t rows, int64_t cols, int64_t ld,
               unsigned *__restrict__ slot, int m) {
@@ -113,7 +114,7 @@ absmax_kernel(const float *__restrict__ x, int64_t rows, int64_t cols, int64_t l
         for (; i + (kUnroll - 1) * nthreads < nvec; i += kUnroll * nthreads) {
             float4 v[kUnroll];
 #pragma unroll
-            for (int u = 0; u < kUnroll; ++u) v[u] = __ldcs(xv + i + u * nthreads);
+            for (int u = 0; u < kUnroll; ++u) v[u] = STREAM ? __ldcs(xv + i + u * nthreads) : __ldg(xv + i + u * nthreads);
 #pragma unroll
             for (int u = 0; u < kUnroll; ++u) {
                 best = max(best, max(max(finite_abs_bits(v[u].x), finite_abs_bits(v[u].y)),
@@ -121,7 +122,7 @@ absmax_kernel(const float *__restrict__ x, int64_t rows, int64_t cols, int64_t l
             }
         }
         for (; i < nvec; i += nthreads) {
-            float4 v = __ldcs(xv + i);
+            float4 v = STREAM ? __ldcs(xv + i) : __ldg(xv + i);
             best = max(best, max(max(finite_abs_bits(v.x), finite_abs_bits(v.y)),
                                  max(finite_abs_bits(v.z), finite_abs_bits(v.w))));
         }
@@ -143,7 +144,7 @@ absmax_kernel(const float *__restrict__ x, int64_t rows, int64_t cols, int64_t l
         unsigned b = threadIdx.x < kWarpsPerBlock ? warp_best[threadIdx.x] : 0u;
         b = __reduce_max_sync(0xffffffffu, b);
         if (threadIdx.x == 0) {
-            if (b != 0u) atomicMax(slot, b);
+            if (b > *reinterpret_cast<volatile unsigned *>(slot)) atomicMax(slot, b);   // the slot only ever grows
             __threadfence();
             const unsigned ticket = atomicAdd(slot + 1, 1u);
             if (ticket == gridDim.x - 1) {
@@ -393,12 +394,17 @@ static dybit_status launch_absmax(const float *x, int64_t rows, int64_t cols, in
     DYBIT_CUDA_TRY(cudaMemsetAsync(scale_out, 0, 2 * sizeof(float), s));
     const int64_t n = rows * cols;
     if (n > 0) {
-        int64_t blocks = (n / 4 + kStreamThreads * 4 - 1) / (kStreamThreads * 4);
-        int64_t cap = (int64_t)sm_count() * 8;
+        // few, fat blocks: every block ends with two atomics on the same words
+        int64_t blocks = (n / 4 + kStreamThreads * 8 - 1) / (kStreamThreads * 8);
+        int64_t cap = (int64_t)sm_count() * 4;
         if (blocks > cap) blocks = cap;
         if (blocks < 1) blocks = 1;
-        absmax_kernel<<<(int)blocks, kStreamThreads, 0, s>>>(x, rows, cols, ld,
-                                                             reinterpret_cast<unsigned *>(scale_out), mag_bits(fmt));
+        if (n * 4 > ((int64_t)64 << 20))
+            absmax_kernel<true><<<(int)blocks, kStreamThreads, 0, s>>>(x, rows, cols, ld,
+                                                                       reinterpret_cast<unsigned *>(scale_out), mag_bits(fmt));
+        else
+            absmax_kernel<false><<<(int)blocks, kStreamThreads, 0, s>>>(x, rows, cols, ld,
+                                                                        reinterpret_cast<unsigned *>(scale_out), mag_bits(fmt));
         return launch_status();
     }
     unit_scale_kernel<<<1, 1, 0, s>>>(scale_out);
