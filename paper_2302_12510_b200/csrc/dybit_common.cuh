@@ -40,6 +40,31 @@ inline dybit_status launch_status() {
     return cudaGetLastError() == cudaSuccess ? DYBIT_OK : DYBIT_ERR_CUDA;
 }
 
+// Every kernel of the library is launched with programmatic stream serialization: a kernel may be
+// scheduled while its predecessor in the stream is still draining, runs its prologue, and then blocks in
+// pdl_enter() until the predecessor has completed and its writes are visible.  pdl_enter() also releases
+// the kernel's own successor, so at most one successor is ever waiting.  Chains of short dependent kernels
+// (absmax -> quantize -> expand -> GEMM) overlap their launch and ramp-up this way.
+template <typename... KArgs, typename... Args>
+inline void launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args &&...args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    (void)cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
+__device__ __forceinline__ void pdl_enter() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 struct ProfileEvents {
     cudaEvent_t start = nullptr, stop = nullptr;
 };

@@ -73,6 +73,7 @@ expand_rows_kernel(const uint8_t *__restrict__ packed, int64_t rows, int64_t in_
     for (int i = threadIdx.x; i < 256; i += blockDim.x) s_lut[i] = table.v[i];
     __syncthreads();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    pdl_enter();
     constexpr int kChunkBytes = kChunkCodes * BITS / 8;
     constexpr int kChunkVecs = kChunkBytes / 16;
     const int64_t chunks_per_row = (cols + kChunkCodes - 1) / kChunkCodes;
@@ -152,6 +153,7 @@ __device__ __forceinline__ unsigned expand4_lookup(unsigned sel, const unsigned 
 }
 
 __global__ void __launch_bounds__(256) expand4_kernel(const Expand4Job j0, const Expand4Job j1, int64_t vecs0) {
+    pdl_enter();
     const int64_t total = vecs0 + j1.rows * j1.vecs_per_row;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
         const bool first = i < vecs0;
@@ -180,6 +182,7 @@ __global__ void expand_pad_kernel(const uint8_t *__restrict__ packed, int bits, 
                                   int64_t out_stride, const __grid_constant__ ElemTable table) {
     const int per_chunk = 16 / elem;
     const int64_t chunks_per_tap = cp / per_chunk;
+    pdl_enter();
     const int64_t total = rows * taps * chunks_per_tap;
     for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
          idx += (int64_t)gridDim.x * blockDim.x) {
@@ -272,6 +275,7 @@ patch_expand_kernel(const PatchParams p, const __grid_constant__ ElemTable table
     // zero everything first: padding taps and the row tail stay zero
     for (int i = threadIdx.x; i < (128 * p.row_pitch) / 4; i += blockDim.x) reinterpret_cast<unsigned *>(s_rows)[i] = 0u;
     __syncthreads();
+    pdl_enter();
     const int m = blockIdx.x * 128 + threadIdx.x;
     if (m < p.M) {
         const int img = m / (p.OH * p.OW);
@@ -348,13 +352,13 @@ static dybit_status launch_expand_rows(const uint8_t *packed, int bits, int64_t 
     if (items == 0) return DYBIT_OK;
     const int grid = stream_grid(items);
     switch (bits) {
-        case 2: expand_rows_kernel<2, ELEM><<<grid, kStreamThreads, 0, s>>>(packed, rows, in_stride, cols, out, out_stride, t); break;
-        case 3: expand_rows_kernel<3, ELEM><<<grid, kStreamThreads, 0, s>>>(packed, rows, in_stride, cols, out, out_stride, t); break;
-        case 4: expand_rows_kernel<4, ELEM><<<grid, kStreamThreads, 0, s>>>(packed, rows, in_stride, cols, out, out_stride, t); break;
-        case 5: expand_rows_kernel<5, ELEM><<<grid, kStreamThreads, 0, s>>>(packed, rows, in_stride, cols, out, out_stride, t); break;
-        case 6: expand_rows_kernel<6, ELEM><<<grid, kStreamThreads, 0, s>>>(packed, rows, in_stride, cols, out, out_stride, t); break;
-        case 7: expand_rows_kernel<7, ELEM><<<grid, kStreamThreads, 0, s>>>(packed, rows, in_stride, cols, out, out_stride, t); break;
-        case 8: expand_rows_kernel<8, ELEM><<<grid, kStreamThreads, 0, s>>>(packed, rows, in_stride, cols, out, out_stride, t); break;
+        case 2: launch_k(expand_rows_kernel<2, ELEM>, dim3((unsigned)(grid)), dim3((unsigned)(kStreamThreads)), (size_t)(0), s, packed, rows, in_stride, cols, out, out_stride, t); break;
+        case 3: launch_k(expand_rows_kernel<3, ELEM>, dim3((unsigned)(grid)), dim3((unsigned)(kStreamThreads)), (size_t)(0), s, packed, rows, in_stride, cols, out, out_stride, t); break;
+        case 4: launch_k(expand_rows_kernel<4, ELEM>, dim3((unsigned)(grid)), dim3((unsigned)(kStreamThreads)), (size_t)(0), s, packed, rows, in_stride, cols, out, out_stride, t); break;
+        case 5: launch_k(expand_rows_kernel<5, ELEM>, dim3((unsigned)(grid)), dim3((unsigned)(kStreamThreads)), (size_t)(0), s, packed, rows, in_stride, cols, out, out_stride, t); break;
+        case 6: launch_k(expand_rows_kernel<6, ELEM>, dim3((unsigned)(grid)), dim3((unsigned)(kStreamThreads)), (size_t)(0), s, packed, rows, in_stride, cols, out, out_stride, t); break;
+        case 7: launch_k(expand_rows_kernel<7, ELEM>, dim3((unsigned)(grid)), dim3((unsigned)(kStreamThreads)), (size_t)(0), s, packed, rows, in_stride, cols, out, out_stride, t); break;
+        case 8: launch_k(expand_rows_kernel<8, ELEM>, dim3((unsigned)(grid)), dim3((unsigned)(kStreamThreads)), (size_t)(0), s, packed, rows, in_stride, cols, out, out_stride, t); break;
         default: return DYBIT_ERR_INVALID_ARG;
     }
     return launch_status();
@@ -379,7 +383,7 @@ static dybit_status launch_expand_pair(const ExpandOperand &a, const ExpandOpera
         const int64_t total = vecs0 + j1.rows * j1.vecs_per_row;
         int64_t blocks = (total + 255) / 256, cap = (int64_t)sm_count() * 16;
         if (blocks > cap) blocks = cap;
-        expand4_kernel<<<(int)blocks, 256, 0, s>>>(j0, j1, vecs0);
+        launch_k(expand4_kernel, dim3((unsigned)((int)blocks)), dim3((unsigned)(256)), (size_t)(0), s, j0, j1, vecs0);
         if (launch_status() != DYBIT_OK) return DYBIT_ERR_CUDA;
     }
     if (!fa) {
@@ -512,6 +516,8 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    // everything above touched only this CTA's own resources; operands, scales and outputs come next
+    pdl_enter();
 
     if (warp == 0) {
         // ------------------------------------------------ TMA producer
@@ -807,7 +813,7 @@ static dybit_status launch_gemm_inst(const CUtensorMap &ta, const CUtensorMap &t
     ProfileEvents ev = profile_events();
     profile_events() = ProfileEvents();
     if (ev.start) DYBIT_CUDA_TRY(cudaEventRecord(ev.start, s));
-    kern<<<grid, CONV ? 320 : 192, L::kBytes, s>>>(ta, tb, p);
+    launch_k(kern, dim3((unsigned)(grid)), dim3((unsigned)(CONV ? 320 : 192)), (size_t)(L::kBytes), s, ta, tb, p);
     const dybit_status st = launch_status();
     if (ev.stop) DYBIT_CUDA_TRY(cudaEventRecord(ev.stop, s));
     return st;
@@ -1038,7 +1044,7 @@ dybit_status dybit_conv2d(const dybit_conv_desc *d, const void *X, dybit_fmt fx,
                                                 128 * (1024 + 4)));
             patch_configured[dev] = true;
         }
-        patch_expand_kernel<<<(int)((M + 127) / 128), 128, smem, s>>>(pp, tx);
+        launch_k(patch_expand_kernel, dim3((unsigned)((int)((M + 127) / 128))), dim3((unsigned)(128)), (size_t)(smem), s, pp, tx);
         if (launch_status() != DYBIT_OK) return DYBIT_ERR_CUDA;
         st = launch_expand(static_cast<const uint8_t *>(W), fw.bits, N, ldw_bytes, wrb / elem, elem, we, wrb, tw, s);
         if (st != DYBIT_OK) return st;
@@ -1052,11 +1058,11 @@ dybit_status dybit_conv2d(const dybit_conv_desc *d, const void *X, dybit_fmt fx,
         const int64_t taps = (int64_t)d->r * d->s;
         DYBIT_CUDA_TRY(cudaMemsetAsync(we, 0, (size_t)(N * wrb), s));
         int64_t chunks = pixels * (cp * elem / 16);
-        expand_pad_kernel<<<pad_grid(chunks), 256, 0, s>>>(
+        launch_k(expand_pad_kernel, dim3((unsigned)(pad_grid(chunks))), dim3((unsigned)(256)), (size_t)(0), s, 
             static_cast<const uint8_t *>(X), fx.bits, 1, 0, pixels, d->c, (int)cp, elem, xe, 0, tx);
         if (launch_status() != DYBIT_OK) return DYBIT_ERR_CUDA;
         chunks = N * taps * (cp * elem / 16);
-        expand_pad_kernel<<<pad_grid(chunks), 256, 0, s>>>(
+        launch_k(expand_pad_kernel, dim3((unsigned)(pad_grid(chunks))), dim3((unsigned)(256)), (size_t)(0), s, 
             static_cast<const uint8_t *>(W), fw.bits, N, ldw_bytes, taps, d->c, (int)cp, elem, we, wrb, tw);
         if (launch_status() != DYBIT_OK) return DYBIT_ERR_CUDA;
     }

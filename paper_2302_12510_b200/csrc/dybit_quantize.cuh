@@ -100,6 +100,7 @@ __global__ void __launch_bounds__(kStreamThreads)
 absmax_kernel(const float *__restrict__ x, int64_t rows, int64_t cols, int64_t ld,
               unsigned *__restrict__ slot, int m) {
     unsigned best = 0;
+    pdl_enter();
     const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int64_t nthreads = (int64_t)gridDim.x * blockDim.x;
     if (ld == cols) {
@@ -166,6 +167,7 @@ absmax_kernel(const float *__restrict__ x, int64_t rows, int64_t cols, int64_t l
 
 // Empty tensor: no reduction runs, the scale is {1, 1}.
 __global__ void unit_scale_kernel(float *scale) {
+    pdl_enter();
     scale[0] = 1.0f;
     scale[1] = 1.0f;
 }
@@ -221,6 +223,7 @@ quantize_pack_kernel(const float *__restrict__ x, int64_t rows, int64_t cols, in
     __shared__ __align__(16) unsigned s_codes[kWarpsPerBlock][kChunkCodes / 4];
     __shared__ __align__(16) unsigned s_words[kWarpsPerBlock][32 * BITS];
 
+    pdl_enter();
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     const float inv = __ldg(scale + 1);
@@ -323,6 +326,7 @@ decode_kernel(const uint8_t *__restrict__ packed, int64_t n, const float *__rest
     __shared__ float s_lut[256];
     __shared__ __align__(16) unsigned s_words[kWarpsPerBlock][32 * BITS];
     __shared__ __align__(16) unsigned s_codes[kWarpsPerBlock][kChunkCodes / 4];
+    pdl_enter();
     const float sc = scale ? __ldg(scale) : 1.0f;
     for (int i = threadIdx.x; i < 256; i += blockDim.x) s_lut[i] = __fmul_rn(sc, table.v[i]);
     __syncthreads();
@@ -400,14 +404,14 @@ static dybit_status launch_absmax(const float *x, int64_t rows, int64_t cols, in
         if (blocks > cap) blocks = cap;
         if (blocks < 1) blocks = 1;
         if (n * 4 > ((int64_t)64 << 20))
-            absmax_kernel<true><<<(int)blocks, kStreamThreads, 0, s>>>(x, rows, cols, ld,
+            launch_k(absmax_kernel<true>, dim3((unsigned)((int)blocks)), dim3((unsigned)(kStreamThreads)), (size_t)(0), s, x, rows, cols, ld,
                                                                        reinterpret_cast<unsigned *>(scale_out), mag_bits(fmt));
         else
-            absmax_kernel<false><<<(int)blocks, kStreamThreads, 0, s>>>(x, rows, cols, ld,
+            launch_k(absmax_kernel<false>, dim3((unsigned)((int)blocks)), dim3((unsigned)(kStreamThreads)), (size_t)(0), s, x, rows, cols, ld,
                                                                         reinterpret_cast<unsigned *>(scale_out), mag_bits(fmt));
         return launch_status();
     }
-    unit_scale_kernel<<<1, 1, 0, s>>>(scale_out);
+    launch_k(unit_scale_kernel, dim3((unsigned)(1)), dim3((unsigned)(1)), (size_t)(0), s, scale_out);
     return launch_status();
 }
 
@@ -421,10 +425,10 @@ static dybit_status launch_quantize_bits(const float *x, int64_t rows, int64_t c
     if (items == 0) return DYBIT_OK;
     const int grid = stream_grid(items);
     if (is_signed)
-        quantize_pack_kernel<BITS, true><<<grid, kStreamThreads, 0, s>>>(x, rows, cols, ld, scale, out,
+        launch_k(quantize_pack_kernel<BITS, true>, dim3((unsigned)(grid)), dim3((unsigned)(kStreamThreads)), (size_t)(0), s, x, rows, cols, ld, scale, out,
                                                                         row_stride_bytes, chunks_per_row);
     else
-        quantize_pack_kernel<BITS, false><<<grid, kStreamThreads, 0, s>>>(x, rows, cols, ld, scale, out,
+        launch_k(quantize_pack_kernel<BITS, false>, dim3((unsigned)(grid)), dim3((unsigned)(kStreamThreads)), (size_t)(0), s, x, rows, cols, ld, scale, out,
                                                                          row_stride_bytes, chunks_per_row);
     return launch_status();
 }
@@ -450,7 +454,7 @@ static dybit_status launch_decode_bits(const uint8_t *packed, int64_t n, const f
                                        const FloatTable &table, float *out, cudaStream_t s) {
     const int64_t items = (n + kChunkCodes - 1) / kChunkCodes;
     if (items == 0) return DYBIT_OK;
-    decode_kernel<BITS><<<stream_grid(items), kStreamThreads, 0, s>>>(packed, n, scale, table, out);
+    launch_k(decode_kernel<BITS>, dim3((unsigned)(stream_grid(items))), dim3((unsigned)(kStreamThreads)), (size_t)(0), s, packed, n, scale, table, out);
     return launch_status();
 }
 
