@@ -419,6 +419,7 @@ struct GemmParams {
     int H, W, OH, OW, R, S, stride, pad, dil;
     int cpb;                  // bytes per pixel in xe (padded channels * element size)
     int kb_per_tap;           // im2col mode: SWB-byte blocks per filter tap (cpb / SWB)
+    int tma_store;            // 1: C leaves through shared memory and TMA stores (needs 16-byte aligned C rows)
 };
 
 // Waits for the phase with the given parity; gives up after kWaitLimitNs, records
@@ -453,7 +454,8 @@ struct GemmSmem {
     static constexpr int kFit = kStageBytesTotal / (kAStage + kBStage);
     static constexpr int kStages = kFit > 12 ? 12 : kFit;
     static constexpr int kBarrierBytes = 512;
-    static constexpr int kBytes = kStages * (kAStage + kBStage) + kBarrierBytes + 1024;   // + alignment slack
+    static constexpr int kCStage = kBM * 128;                  // 128 rows x 32 fp32 columns of the output tile
+    static constexpr int kBytes = kStages * (kAStage + kBStage) + 2 * kCStage + kBarrierBytes + 1024;   // + alignment slack
 };
 
 __device__ __forceinline__ void tile_coords(int tile, int m_tiles, int n_tiles, int &m_blk, int &n_blk) {
@@ -471,7 +473,7 @@ __device__ __forceinline__ void tile_coords(int tile, int m_tiles, int n_tiles, 
 template <Kind KIND, int BN, int AMODE, int SWB>
 __global__ void __launch_bounds__(AMODE == kAGather ? 320 : 192, 1)
 dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-                  const GemmParams p) {
+                  const __grid_constant__ CUtensorMap tmap_c, const GemmParams p) {
     static_assert(AMODE != kAGather || SWB == 128, "the cp.async gather writes 128-byte rows");
     constexpr bool CONV = AMODE == kAGather;          // extra gather warps present
     using L = GemmSmem<BN, SWB>;
@@ -481,7 +483,8 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t *a_stages = smem;
     uint8_t *b_stages = smem + kStages * L::kAStage;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + kStages * (L::kAStage + L::kBStage));
+    uint8_t *c_stages = smem + kStages * (L::kAStage + L::kBStage);       // two output staging buffers
+    uint64_t *bars = reinterpret_cast<uint64_t *>(c_stages + 2 * L::kCStage);
     uint64_t *full = bars;
     uint64_t *empty = bars + kStages;
     uint64_t *acc_full = bars + 2 * kStages;
@@ -507,6 +510,7 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         fence_mbar_init();
         if (AMODE != kAGather) prefetch_tensormap(&tmap_a);
         prefetch_tensormap(&tmap_b);
+        if (p.tma_store) prefetch_tensormap(&tmap_c);
     }
     if (warp == 1) {
         tmem_alloc(tmem_slot, kTmemCols);
@@ -591,12 +595,14 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             }
         }
     } else if (warp < 6) {
-        // ------------------------------------------------ epilogue: TMEM -> registers -> global
+        // ------------------------------------------------ epilogue: TMEM -> registers -> (shared -> TMA store | global)
         const int q = warp & 3;                       // TMEM lane quarter this warp may read
+        const int row_in_tile = q * 32 + lane;
+        const bool issuer = threadIdx.x == 64;        // issues and tracks the TMA stores
         const float alpha = (float)((double)__ldg(p.scale_a) * (double)__ldg(p.scale_b) * p.pow2);
         const bool vec_ok = ((reinterpret_cast<uintptr_t>(p.C) & 15) == 0) && (p.ldc % 4 == 0) &&
                             (p.C_raw == nullptr || (reinterpret_cast<uintptr_t>(p.C_raw) & 15) == 0);
-        uint32_t lt = 0;
+        uint32_t lt = 0, chunk_no = 0;
         for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++lt) {
             int m_blk, n_blk;
             tile_coords(tile, p.m_tiles, p.n_tiles, m_blk, n_blk);
@@ -605,27 +611,49 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after_sync();
-            const int row = m_blk * kBM + q * 32 + lane;
+            const int row = m_blk * kBM + row_in_tile;
             const uint32_t taddr = tmem_base + as * BN + ((uint32_t)(q * 32) << 16);
 #pragma unroll 1
             for (int cc = 0; cc < BN / 32; ++cc) {
+                const int col0 = n_blk * BN + cc * 32;
+                if (col0 >= p.N) break;                // uniform over the CTA: the rest of the tile lies outside C
                 uint32_t r[32];
                 tmem_ld_32x32(taddr + cc * 32, r);
                 tmem_ld_wait();
-                const int col0 = n_blk * BN + cc * 32;
-                if (row < p.M && col0 < p.N) {
+                float f[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    const float acc = (KIND == Kind::I8) ? __int2float_rn((int)r[j]) : __uint_as_float(r[j]);
+                    f[j] = __fmul_rn(acc, alpha);
+                }
+                if (p.tma_store) {
+                    // stage 128 rows x 128 bytes in the TMA's 128-byte swizzle, then one thread stores the box;
+                    // rows / columns beyond C are clipped by the tensor map
+                    uint8_t *stage = c_stages + (chunk_no & 1u) * L::kCStage;
+                    if (issuer) bulk_wait_group_read<1>();        // the store that last read this buffer is done with it
+                    named_barrier(1, 128);
+                    uint8_t *srow = stage + row_in_tile * 128;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        *reinterpret_cast<float4 *>(srow + ((j ^ (row_in_tile & 7)) << 4)) =
+                            make_float4(f[4 * j], f[4 * j + 1], f[4 * j + 2], f[4 * j + 3]);
+                    fence_proxy_async_smem();
+                    named_barrier(1, 128);
+                    if (issuer) {
+                        tma_store_2d(&tmap_c, stage, col0, m_blk * kBM);
+                        bulk_commit_group();
+                    }
+                    ++chunk_no;
+                }
+                if (row < p.M) {
                     float *crow = p.C + (int64_t)row * p.ldc + col0;
                     int32_t *rrow = p.C_raw ? p.C_raw + (int64_t)row * p.ldc + col0 : nullptr;
-                    float f[32];
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const float acc = (KIND == Kind::I8) ? __int2float_rn((int)r[j]) : __uint_as_float(r[j]);
-                        f[j] = __fmul_rn(acc, alpha);
-                    }
                     if (vec_ok && col0 + 32 <= p.N) {
+                        if (!p.tma_store) {
 #pragma unroll
-                        for (int j = 0; j < 8; ++j)
-                            __stcs(reinterpret_cast<float4 *>(crow) + j, make_float4(f[4 * j], f[4 * j + 1], f[4 * j + 2], f[4 * j + 3]));
+                            for (int j = 0; j < 8; ++j)
+                                __stcs(reinterpret_cast<float4 *>(crow) + j, make_float4(f[4 * j], f[4 * j + 1], f[4 * j + 2], f[4 * j + 3]));
+                        }
                         if (KIND == Kind::I8 && rrow) {
 #pragma unroll
                             for (int j = 0; j < 8; ++j)
@@ -635,7 +663,7 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
 #pragma unroll
                         for (int j = 0; j < 32; ++j) {
                             if (col0 + j < p.N) {
-                                crow[j] = f[j];
+                                if (!p.tma_store) crow[j] = f[j];
                                 if (KIND == Kind::I8 && rrow) rrow[j] = (int)r[j];
                             }
                         }
@@ -646,6 +674,7 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             __syncwarp();
             if (lane == 0) mbar_arrive(&acc_empty[as]);
         }
+        if (issuer) bulk_wait_group_read<0>();             // shared memory must outlive the last store's read
     } else if (CONV) {
         // ------------------------------------------------ im2col gather of the A tile (4 warps, one row per thread)
         const int t = threadIdx.x - 192;              // tile row 0..127
@@ -795,8 +824,25 @@ static dybit_status make_im2col_map(CUtensorMap *map, const void *xe, const dybi
     return r == CUDA_SUCCESS ? DYBIT_OK : DYBIT_ERR_CUDA;
 }
 
+// fp32 output [M][ldc] as a map whose box is 32 columns x 128 rows, 128-byte swizzle (the staging layout).
+static bool make_output_map(CUtensorMap *map, float *C, int64_t M, int64_t N, int64_t ldc) {
+    if ((reinterpret_cast<uintptr_t>(C) & 15) != 0 || (ldc * 4) % 16 != 0) return false;
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (fn == nullptr) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)M};
+    cuuint64_t strides[1] = {(cuuint64_t)ldc * 4};
+    cuuint32_t box[2] = {32, (cuuint32_t)kBM};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, C, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <Kind KIND, int BN, int AMODE, int SWB>
-static dybit_status launch_gemm_inst(const CUtensorMap &ta, const CUtensorMap &tb, const GemmParams &p, cudaStream_t s) {
+static dybit_status launch_gemm_inst(const CUtensorMap &ta, const CUtensorMap &tb, const GemmParams &p_in, cudaStream_t s) {
+    GemmParams p = p_in;
+    CUtensorMap tc;
+    memset(&tc, 0, sizeof(tc));
+    p.tma_store = make_output_map(&tc, p.C, p.M, p.N, p.ldc) ? 1 : 0;
     using L = GemmSmem<BN, SWB>;
     auto kern = dybit_gemm_kernel<KIND, BN, AMODE, SWB>;
     constexpr bool CONV = AMODE == kAGather;
@@ -813,7 +859,7 @@ static dybit_status launch_gemm_inst(const CUtensorMap &ta, const CUtensorMap &t
     ProfileEvents ev = profile_events();
     profile_events() = ProfileEvents();
     if (ev.start) DYBIT_CUDA_TRY(cudaEventRecord(ev.start, s));
-    launch_k(kern, dim3((unsigned)(grid)), dim3((unsigned)(CONV ? 320 : 192)), (size_t)(L::kBytes), s, ta, tb, p);
+    launch_k(kern, dim3((unsigned)(grid)), dim3((unsigned)(CONV ? 320 : 192)), (size_t)(L::kBytes), s, ta, tb, tc, p);
     const dybit_status st = launch_status();
     if (ev.stop) DYBIT_CUDA_TRY(cudaEventRecord(ev.stop, s));
     return st;
