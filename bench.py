@@ -111,37 +111,42 @@ class ClockSampler:
 
 # --------------------------------------------------------------------------- workload
 
-class Resnet18Step:
-    """Device buffers and the per-step call sequence for the ResNet-18-shaped workload."""
+class LayerwiseStep:
+    """Device buffers and the per-step call sequence for a list of independent conv/FC layers.
 
-    def __init__(self, dy, wl, device, batch=32, pinned_host=True):
+    bits[i] = (weight bits, activation bits) of layer i; weights are signed, activations unsigned."""
+
+    def __init__(self, dy, wl, device, layers, bits, host_copies=True):
         self.dy, self.device = dy, device
-        self.layers = wl.resnet18_layers(batch)
+        self.layers = layers
+        self.fw = [(wb, 1) for wb, _ in bits]
+        self.fa = [(ab, 0) for _, ab in bits]
         self.x_host, self.x_dev, self.pw, self.sw, self.px, self.sx, self.y, self.y_host = [], [], [], [], [], [], [], []
         self.desc = []
         ws_bytes = 0
         for i, L in enumerate(self.layers):
-            xh = wl.half_normal((L.n, L.h, L.w, L.c), seed=1000 + i)
-            if pinned_host:
-                xh = xh.pin_memory()
-            self.x_host.append(xh)
-            self.x_dev.append(xh.to(device))
+            if host_copies:
+                xh = wl.half_normal((L.n, L.h, L.w, L.c), seed=1000 + i).pin_memory()
+                self.x_host.append(xh)
+                self.x_dev.append(xh.to(device))
+            else:
+                self.x_dev.append(wl.half_normal((L.n, L.h, L.w, L.c), seed=1000 + i, device=device))
             w = wl.kaiming_normal(L.k, L.r, L.s, L.c, seed=2000 + i).reshape(L.k, -1).to(device)
-            pw, sw = dy.dybit_quantize_pack_2d(w, FMT_W)
+            pw, sw = dy.dybit_quantize_pack_2d(w, self.fw[i])
             self.pw.append(pw)
             self.sw.append(sw)
-            n = xh.numel()
-            self.px.append(torch.empty(dy.dybit_packed_bytes(n, FMT_A[0]), dtype=torch.uint8, device=device))
+            n = self.x_dev[i].numel()
+            self.px.append(torch.empty(dy.dybit_packed_bytes(n, self.fa[i][0]), dtype=torch.uint8, device=device))
             self.sx.append(torch.empty(2, dtype=torch.float32, device=device))
             self.y.append(torch.empty((L.n, L.oh, L.ow, L.k), dtype=torch.float32, device=device))
             d = dy.ConvDesc(L.n, L.h, L.w, L.c, L.k, L.r, L.s, L.stride, L.pad, 1)
             self.desc.append(d)
-            ws_bytes = max(ws_bytes, dy.dybit_conv2d_workspace_bytes(d, FMT_A, FMT_W))
+            ws_bytes = max(ws_bytes, dy.dybit_conv2d_workspace_bytes(d, self.fa[i], self.fw[i]))
         self.ws = torch.empty(ws_bytes + 1024, dtype=torch.uint8, device=device)
         self.macs = sum(L.macs for L in self.layers)
-        self.h2d_bytes = sum(x.numel() * 4 for x in self.x_host)
+        self.h2d_bytes = sum(x.numel() * 4 for x in self.x_dev)
         self.d2h_bytes = sum(y.numel() * 4 for y in self.y)
-        self.quant_elems = sum(x.numel() for x in self.x_host)
+        self.quant_elems = sum(x.numel() for x in self.x_dev)
 
     def alloc_host_outputs(self):
         self.y_host = [torch.empty(y.shape, dtype=torch.float32).pin_memory() for y in self.y]
@@ -149,12 +154,12 @@ class Resnet18Step:
     def step(self, events=None):
         dy = self.dy
         for i in range(len(self.layers)):
-            dy.dybit_quantize_pack(self.x_dev[i], FMT_A, packed=self.px[i], scale_out=self.sx[i])
+            dy.dybit_quantize_pack(self.x_dev[i], self.fa[i], packed=self.px[i], scale_out=self.sx[i])
             if events is not None:
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 dy.dybit_profile_next_gemm(e0, e1)
                 events[i].append((e0, e1))
-            dy.dybit_conv2d(self.desc[i], self.px[i], FMT_A, self.sx[i], self.pw[i], FMT_W, self.sw[i],
+            dy.dybit_conv2d(self.desc[i], self.px[i], self.fa[i], self.sx[i], self.pw[i], self.fw[i], self.sw[i],
                             Y=self.y[i], ws=self.ws)
 
     def step_e2e(self):
@@ -167,9 +172,9 @@ class Resnet18Step:
     def layer_bounds(self, tensor_tops, hbm_gbs):
         """Per layer: (flops, algorithmic bytes of the conv, ideal seconds = max of the two bounds)."""
         out = []
-        for L in self.layers:
+        for L, fa, fw in zip(self.layers, self.fa, self.fw):
             flops = 2.0 * L.macs
-            byts = (L.n * L.h * L.w * L.c * FMT_A[0] / 8 + L.k * L.gemm_k * FMT_W[0] / 8 + 4.0 * L.gemm_m * L.k)
+            byts = (L.n * L.h * L.w * L.c * fa[0] / 8 + L.k * L.gemm_k * fw[0] / 8 + 4.0 * L.gemm_m * L.k)
             out.append((flops, byts, max(flops / (tensor_tops * 1e12), byts / (hbm_gbs * 1e9))))
         return out
 
@@ -204,6 +209,18 @@ def whole_job_tops(macs_per_rank, world, ms_step):
     return world * 2.0 * macs_per_rank / (ms_step * 1e-3) / 1e12
 
 
+def capture_step(work, device):
+    """One step captured as a CUDA graph (the library's calls are plain stream work, so they capture)."""
+    graph = torch.cuda.CUDAGraph()
+    cap_stream = torch.cuda.Stream(device)
+    cap_stream.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(cap_stream):
+        with torch.cuda.graph(graph, stream=cap_stream):
+            work.step()
+    torch.cuda.current_stream().wait_stream(cap_stream)
+    return graph
+
+
 # --------------------------------------------------------------------------- single-kernel targets
 
 def time_calls(fn, iters, warmup=3):
@@ -219,17 +236,18 @@ def time_calls(fn, iters, warmup=3):
     return e0.elapsed_time(e1) / iters
 
 
-def target_gemm(dy, wl, device, peaks, size=8192):
-    """Square 4-bit DyBit GEMM (both operands N(0,1), signed 4-bit -> int8 container)."""
+def target_gemm(dy, wl, device, peaks, size=8192, fmt=(4, 1)):
+    """Square DyBit GEMM, both operands N(0,1) in the same signed format (4-bit -> int8, 8-bit -> bf16 container)."""
     a = wl.normal((size, size), seed=11, device=device)
     b = wl.normal((size, size), seed=12, device=device)
-    pa, sa = dy.dybit_quantize_pack_2d(a, (4, 1))
-    pb, sb = dy.dybit_quantize_pack_2d(b, (4, 1))
+    pa, sa = dy.dybit_quantize_pack_2d(a, fmt)
+    pb, sb = dy.dybit_quantize_pack_2d(b, fmt)
     del a, b
+    cont = CONTAINERS[dy.dybit_choose_container(fmt, fmt)[0]]
     c = torch.empty((size, size), dtype=torch.float32, device=device)
-    ws = torch.empty(dy.dybit_gemm_workspace_bytes(size, size, size, (4, 1), (4, 1)) + 1024, dtype=torch.uint8,
+    ws = torch.empty(dy.dybit_gemm_workspace_bytes(size, size, size, fmt, fmt) + 1024, dtype=torch.uint8,
                      device=device)
-    call = lambda: dy.dybit_gemm(size, size, size, pa, (4, 1), sa, pb, (4, 1), sb, C_out=c, ws=ws)  # noqa: E731
+    call = lambda: dy.dybit_gemm(size, size, size, pa, fmt, sa, pb, fmt, sb, C_out=c, ws=ws)  # noqa: E731
     ms_call = time_calls(call, 10)
     # tensor-core kernel alone
     evs = []
@@ -241,23 +259,29 @@ def target_gemm(dy, wl, device, peaks, size=8192):
     torch.cuda.synchronize()
     ms_kernel = sorted(e0.elapsed_time(e1) for e0, e1 in evs)[len(evs) // 2]
     ops = 2.0 * size ** 3
-    peak_burst = 2.0 * peaks["bf16_tflops"]
-    out = {"M=N=K": size, "formats": "s4 x s4 -> int8 container",
+    ratio = 1.0 if cont == "bf16" else 2.0                   # nominal int8 (fp8) : bf16 tensor throughput
+    peak_burst = ratio * peaks["bf16_tflops"]
+    out = {"M=N=K": size, "formats": f"s{fmt[0]} x s{fmt[0]} -> {cont} container", "container": cont,
            "ms_call": ms_call, "ms_mma_kernel": ms_kernel,
            "tops_call": ops / ms_call / 1e9, "tops_mma_kernel": ops / ms_kernel / 1e9,
            "peak_tops": peak_burst,
-           "peak_how": f"2 x bf16 burst ({peaks['source']}) : nominal int8/bf16 ratio",
+           "peak_how": f"{ratio:g} x bf16 burst ({peaks['source']}); int8/fp8 : bf16 = 2 : 1 nominal",
            "frac_call": ops / ms_call / 1e9 / peak_burst, "frac_mma_kernel": ops / ms_kernel / 1e9 / peak_burst,
            "nominal_int8_tops": NOMINAL["int8_tops"]}
-    # context: a plain library int8 matmul of the same shape on this machine
+    # context: a plain library matmul of the container type and the same shape on this machine
     try:
-        x = torch.randint(-8, 8, (size, size), dtype=torch.int8, device=device)
-        y = torch.randint(-8, 8, (size, size), dtype=torch.int8, device=device)
-        ms_lib = time_calls(lambda: torch._int_mm(x, y), 10)
-        out["library_int8_matmul_tops"] = ops / ms_lib / 1e9
+        if cont == "int8":
+            x = torch.randint(-8, 8, (size, size), dtype=torch.int8, device=device)
+            y = torch.randint(-8, 8, (size, size), dtype=torch.int8, device=device)
+            ms_lib = time_calls(lambda: torch._int_mm(x, y), 10)
+        else:
+            x = torch.randn((size, size), dtype=torch.bfloat16, device=device)
+            y = torch.randn((size, size), dtype=torch.bfloat16, device=device)
+            ms_lib = time_calls(lambda: torch.matmul(x, y), 10)
+        out["library_matmul_tops"] = ops / ms_lib / 1e9
     except Exception as exc:  # pragma: no cover
-        out["library_int8_matmul_tops"] = None
-        out["library_int8_matmul_note"] = str(exc)[:80]
+        out["library_matmul_tops"] = None
+        out["library_matmul_note"] = str(exc)[:80]
     return out
 
 
@@ -279,6 +303,74 @@ def target_quantize(dy, wl, device, peaks, log2n=28, bits=4):
                              "frac": bytes_maxabs / ms_maxabs / 1e6 / peaks["hbm_gbs"]},
             "peak_gbs": peaks["hbm_gbs"], "peak_how": f"copy bandwidth ({peaks['source']})",
             "nominal_gbs": NOMINAL["hbm_gbs"]}
+
+
+# --------------------------------------------------------------------------- the other configurations
+
+def time_calls_flushed(fn, iters, flush):
+    """Per-call CUDA-event time with L2 overwritten before every call (inputs smaller than L2)."""
+    fn()
+    torch.cuda.synchronize()
+    ms = []
+    for _ in range(iters):
+        flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        torch.cuda.synchronize()
+        ms.append(e0.elapsed_time(e1))
+    ms.sort()
+    return ms[len(ms) // 2]
+
+
+def run_sweeps(dy, wl, device, peaks):
+    """Configs 3-5 of the workload list: quantize/pack sweep, square GEMM sweep, ResNet-50 mixed bitwidths."""
+    out = {"peaks": peaks}
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+    rows = []
+    for log2n in (20, 22, 24, 26, 28, 30):
+        n = 1 << log2n
+        for dist in ("normal", "laplace", "half_normal"):
+            x = wl.DISTRIBUTIONS[dist]((n,), seed=log2n, device=device)
+            for bits in (2, 3, 4, 6, 8):
+                fmt = (bits, 0 if dist == "half_normal" else 1)
+                packed = torch.empty(dy.dybit_packed_bytes(n, bits), dtype=torch.uint8, device=device)
+                scale = dy.dybit_absmax_scale(x, fmt)
+                so = torch.empty(2, dtype=torch.float32, device=device)
+                ms_g = time_calls_flushed(lambda: dy.dybit_quantize_pack(x, fmt, scale=scale, packed=packed), 7, flush)
+                ms_m = time_calls_flushed(lambda: dy.dybit_quantize_pack(x, fmt, packed=packed, scale_out=so), 7, flush)
+                rows.append({"log2n": log2n, "dist": dist, "bits": bits,
+                             "gbs_scale_given": n * (4 + bits / 8) / ms_g / 1e6,
+                             "gbs_with_max_abs": n * (8 + bits / 8) / ms_m / 1e6})
+            del x
+            torch.cuda.empty_cache()
+    out["quantize_sweep"] = rows
+    out["gemm_sweep"] = []
+    for fmt in ((4, 1), (8, 1)):
+        for size in (1024, 2048, 4096, 8192):
+            r = target_gemm(dy, wl, device, peaks, size=size, fmt=fmt)
+            out["gemm_sweep"].append({"size": size, "bits": fmt[0], "container": r["container"],
+                                      "tops_call": r["tops_call"], "tops_mma_kernel": r["tops_mma_kernel"],
+                                      "library_matmul_tops": r.get("library_matmul_tops")})
+    layers = wl.resnet50_layers(64)
+    bits = wl.mixed_bitwidths(len(layers), seed=0)
+    work = LayerwiseStep(dy, wl, device, layers, bits, host_copies=False)
+    for _ in range(3):
+        work.step()
+    graph = capture_step(work, device)
+    for _ in range(3):
+        graph.replay()
+    ms = timed_region(graph.replay, 10, None, device) / 10
+    conts = [CONTAINERS[dy.dybit_choose_container(fa, fw)[0]] for fa, fw in zip(work.fa, work.fw)]
+    out["resnet50_b64_mixed"] = {"ms_per_step": ms, "tops": 2.0 * work.macs / (ms * 1e-3) / 1e12,
+                                 "layers": len(layers), "seed": 0,
+                                 "containers": {c: conts.count(c) for c in sorted(set(conts))},
+                                 "bits_w_a": bits}
+    return out
+
+
+CONTAINERS = {0: "int8", 1: "e4m3", 2: "bf16"}
 
 
 # --------------------------------------------------------------------------- CPU oracle legs
@@ -360,6 +452,9 @@ def main():
     ap.add_argument("--gemm-size", type=int, default=8192, help="M=N=K of the square 4-bit GEMM target")
     ap.add_argument("--quant-log2n", type=int, default=28, help="log2 of the element count of the quantize target")
     ap.add_argument("--quant-bits", type=int, default=4)
+    ap.add_argument("--sweeps", action="store_true",
+                    help="measure the other configurations instead (quantize sweep, square GEMM sweep, "
+                         "ResNet-50 batch 64 with mixed bitwidths) and print them as one JSON object")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
@@ -382,6 +477,9 @@ def main():
     from paper_2302_12510_b200 import workloads as wl
     peaks = load_peaks()
     warmup = max(3, args.warmup)
+    if args.sweeps:
+        print(json.dumps({"sweeps": run_sweeps(dy, wl, device, peaks)}))
+        return
     if args.targets_only:
         out = {}
         if args.gemm_size > 0:
@@ -391,7 +489,8 @@ def main():
         print(json.dumps({"targets": out}))
         return
 
-    work = Resnet18Step(dy, wl, device, batch=args.batch)
+    layers = wl.resnet18_layers(args.batch)
+    work = LayerwiseStep(dy, wl, device, layers, [(FMT_W[0], FMT_A[0])] * len(layers))
     for _ in range(warmup):
         work.step()
     torch.cuda.synchronize()
@@ -401,13 +500,7 @@ def main():
 
     # ---- one step captured as a CUDA graph (the library's calls are plain stream work, so they capture)
     launches0 = dy.dybit_launch_count()
-    graph = torch.cuda.CUDAGraph()
-    cap_stream = torch.cuda.Stream(device)
-    cap_stream.wait_stream(torch.cuda.current_stream())
-    with torch.cuda.stream(cap_stream):
-        with torch.cuda.graph(graph, stream=cap_stream):
-            work.step()
-    torch.cuda.current_stream().wait_stream(cap_stream)
+    graph = capture_step(work, device)
     launches_per_step = dy.dybit_launch_count() - launches0
     for _ in range(warmup):
         graph.replay()

@@ -49,7 +49,7 @@ static uint8_t to_e4m3_bits(float v) {
     return sign | (uint8_t)mant;
 }
 
-static ElemTable make_elem_table(dybit_fmt f, dybit_container cont, int int_exp) {
+static ElemTable make_elem_table_uncached(dybit_fmt f, dybit_container cont, int int_exp) {
     float tab[256];
     fill_table(f, tab);
     ElemTable t;
@@ -61,6 +61,28 @@ static ElemTable make_elem_table(dybit_fmt f, dybit_container cont, int int_exp)
         }
     }
     return t;
+}
+
+// One table per (format, container); the int8 rescale exponent is a function of the format alone.
+static const ElemTable &make_elem_table(dybit_fmt f, dybit_container cont, int int_exp) {
+    struct Entry {
+        std::atomic<int> state{0};
+        ElemTable table;
+    };
+    static Entry cache[14][3];
+    static thread_local ElemTable scratch;
+    Entry &e = cache[fmt_index(f)][(int)cont];
+    if (e.state.load(std::memory_order_acquire) != 2) {
+        int expected = 0;
+        if (e.state.compare_exchange_strong(expected, 1)) {
+            e.table = make_elem_table_uncached(f, cont, int_exp);
+            e.state.store(2, std::memory_order_release);
+        } else {
+            scratch = make_elem_table_uncached(f, cont, int_exp);
+            return scratch;
+        }
+    }
+    return e.table;
 }
 
 // Rows of packed codes -> rows of container elements.  A warp expands 1024 codes at a time.
@@ -1005,8 +1027,8 @@ dybit_status dybit_gemm(int64_t M, int64_t N, int64_t K, const void *A, dybit_fm
     const int64_t rb = k_row_bytes(kp, elem);
     uint8_t *ae = static_cast<uint8_t *>(ws);
     uint8_t *be = ae + round_up(M * rb, 1024);
-    const ElemTable ta = make_elem_table(fa, plan.container, plan.exp_a);
-    const ElemTable tb = make_elem_table(fb, plan.container, plan.exp_b);
+    const ElemTable &ta = make_elem_table(fa, plan.container, plan.exp_a);
+    const ElemTable &tb = make_elem_table(fb, plan.container, plan.exp_b);
     const ExpandOperand opa = {static_cast<const uint8_t *>(A), fa.bits, M, lda_bytes, kp, ae, rb, &ta};
     const ExpandOperand opb = {static_cast<const uint8_t *>(B), fb.bits, N, ldb_bytes, kp, be, rb, &tb};
     st = launch_expand_pair(opa, opb, elem, plan.container == DYBIT_CONTAINER_I8, s);
@@ -1065,8 +1087,8 @@ dybit_status dybit_conv2d(const dybit_conv_desc *d, const void *X, dybit_fmt fx,
     const int64_t cp = cv.cp, pixels = cv.pixels, wrb = cv.wrb;
     uint8_t *xe = static_cast<uint8_t *>(ws);
     uint8_t *we = xe + cv.a_bytes;
-    const ElemTable tx = make_elem_table(fx, plan.container, plan.exp_a);
-    const ElemTable tw = make_elem_table(fw, plan.container, plan.exp_b);
+    const ElemTable &tx = make_elem_table(fx, plan.container, plan.exp_a);
+    const ElemTable &tw = make_elem_table(fw, plan.container, plan.exp_b);
     const bool i8 = plan.container == DYBIT_CONTAINER_I8;
     if (cv.mode == kConvPatch) {
         // patch matrix from the packed activation in one kernel; weights expand as plain rows (K order r, s, c)

@@ -4,6 +4,8 @@
 #include <math.h>
 #include <string.h>
 
+#include <atomic>
+
 #include "dybit_common.cuh"
 
 namespace dybit {
@@ -103,7 +105,7 @@ struct ContainerPlan {
     int64_t max_product;    // int8: max |ia * ib|
 };
 
-static dybit_status plan_container(dybit_fmt fa, dybit_fmt fb, ContainerPlan *plan) {
+static dybit_status plan_container_uncached(dybit_fmt fa, dybit_fmt fb, ContainerPlan *plan) {
     if (!fmt_ok(fa) || !fmt_ok(fb)) return DYBIT_ERR_INVALID_ARG;
     TableFacts a = enumerate_facts(fa), b = enumerate_facts(fb);
     plan->exp_a = plan->exp_b = 0;
@@ -121,6 +123,33 @@ static dybit_status plan_container(dybit_fmt fa, dybit_fmt fb, ContainerPlan *pl
         return DYBIT_ERR_UNSUPPORTED;
     }
     return DYBIT_OK;
+}
+
+// There are only 14 formats: every pair is enumerated once per process (the enumeration walks up to 256
+// codes with several libm calls each, far too slow to repeat on every GEMM call).
+static int fmt_index(dybit_fmt f) { return (f.bits - 2) * 2 + (f.is_signed ? 1 : 0); }
+
+static dybit_status plan_container(dybit_fmt fa, dybit_fmt fb, ContainerPlan *plan) {
+    if (!fmt_ok(fa) || !fmt_ok(fb)) return DYBIT_ERR_INVALID_ARG;
+    struct Entry {
+        std::atomic<int> state{0};      // 0 empty, 1 being filled, 2 ready
+        ContainerPlan plan;
+        dybit_status status;
+    };
+    static Entry cache[14][14];
+    Entry &e = cache[fmt_index(fa)][fmt_index(fb)];
+    if (e.state.load(std::memory_order_acquire) != 2) {
+        int expected = 0;
+        if (e.state.compare_exchange_strong(expected, 1)) {
+            e.status = plan_container_uncached(fa, fb, &e.plan);
+            e.state.store(2, std::memory_order_release);
+        } else {
+            // another thread is filling the entry: compute privately rather than wait
+            return plan_container_uncached(fa, fb, plan);
+        }
+    }
+    *plan = e.plan;
+    return e.status;
 }
 
 static inline int container_elem_bytes(dybit_container c) { return c == DYBIT_CONTAINER_BF16 ? 2 : 1; }
