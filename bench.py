@@ -36,6 +36,7 @@ import torch  # noqa: E402
 FMT_W = (4, 1)      # weights: signed 4-bit
 FMT_A = (4, 0)      # post-ReLU activations: unsigned 4-bit
 NOMINAL = {"hbm_gbs": 7700.0, "bf16_tflops": 2250.0, "int8_tops": 4500.0, "fp8_tflops": 4500.0}
+GEMM_KERNEL_DRAM_BYTES_PER_LAUNCH = 8.53e6   # ncu capture of the current dybit_gemm_kernel, see profiles/
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -537,7 +538,10 @@ def main():
     roofline = {
         "kernel": "dybit_gemm_kernel<I8, conv> (21 launches per step, one per layer)",
         "bound": "tensor" if tensor_bound else "hbm", "achieved": achieved, "peak": peak, "unit": unit,
-        "frac": achieved / peak, "traffic": None,
+        "frac": achieved / peak,
+        # dram__bytes_read.sum + dram__bytes_write.sum per launch, averaged over the 21 launches of one step
+        # (profiles/dybit_gemm_kernel_conv_resnet18_b32_dram_traffic.txt); only valid for the batch-32 workload
+        "traffic": GEMM_KERNEL_DRAM_BYTES_PER_LAUNCH if args.batch == 32 else None,
         "peak_how": (f"2 x sustained bf16 ({peaks['source']})" if tensor_bound else f"copy bandwidth ({peaks['source']})"),
         "how": "CUDA events recorded by the library around this kernel alone, same K steps launched directly "
                "(not as a graph) right after the timed region",
