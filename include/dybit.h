@@ -191,6 +191,33 @@ dybit_status dybit_conv2d(const dybit_conv_desc *desc,
                           float *Y, int32_t *Y_raw,
                           void *ws, size_t ws_bytes, void *stream);
 
+/* GEMM / convolution with the re-quantizing epilogue of Section III-B.1 ("the FP intermediate results will be
+ * quantized to DyBit format before being written back"): instead of fp32, the result leaves the kernel as packed
+ * DyBit codes of format fq, ready to be the next layer's activation.  Per output element
+ *     y = fmul_rn((float)sum, alpha)            exactly as dybit_gemm / dybit_conv2d compute it
+ *     y = max(y, 0)                             if relu != 0
+ *     code = encode(y, scale_q[1])              the encoder of dybit_quantize_pack (nearest value, ties to even code)
+ * and row m of the output (N codes; N = desc->k for the convolution) is written as a dense little-endian bit
+ * stream starting at Q + m * ldq_bytes.
+ *   scale_q [dev] {scale, 1/scale} of the OUTPUT tensor, given by the caller (e.g. a calibrated or trained scale;
+ *           the maximum of the result is not known before it is computed)
+ *   Q       [dev] M rows of ldq_bytes; ldq_bytes >= N*fq.bits/8 and N*fq.bits a multiple of 8 (rows that start on
+ *           4-byte boundaries are written with word stores, others byte by byte).  Only the first N*fq.bits/8 bytes of each row are written: a caller that wants padded
+ *           rows (ldq_bytes = dybit_row_stride_bytes(N, fq.bits), to feed dybit_gemm) zero-fills the buffer once.
+ *           dybit_conv2d_requant writes the dense NHWK stream (ldq_bytes = k*fq.bits/8), which is exactly the X
+ *           argument of the next dybit_conv2d.
+ * Everything else as in dybit_gemm / dybit_conv2d (same workspace sizes).  int8-container results are bit-exact. */
+dybit_status dybit_gemm_requant(int64_t M, int64_t N, int64_t K,
+                                const void *A, dybit_fmt fa, const float *scale_a, int64_t lda_bytes,
+                                const void *B, dybit_fmt fb, const float *scale_b, int64_t ldb_bytes,
+                                dybit_fmt fq, const float *scale_q, int relu, void *Q, int64_t ldq_bytes,
+                                void *ws, size_t ws_bytes, void *stream);
+dybit_status dybit_conv2d_requant(const dybit_conv_desc *desc,
+                                  const void *X, dybit_fmt fx, const float *scale_x,
+                                  const void *W, dybit_fmt fw, const float *scale_w, int64_t ldw_bytes,
+                                  dybit_fmt fq, const float *scale_q, int relu, void *Q,
+                                  void *ws, size_t ws_bytes, void *stream);
+
 /* (No counterpart in the paper.)  dybit_gemm for callers that cannot call
  * cudaMalloc -- or any allocator built on it -- at the point where they need
  * a GEMM: code running under a fixed memory budget that was handed out at

@@ -21,6 +21,7 @@ __all__ = [
     "dybit_conv2d_out_hw", "dybit_absmax_scale", "dybit_quantize_pack", "dybit_quantize_pack_2d",
     "dybit_decode", "dybit_gemm", "dybit_conv2d", "dybit_last_device_status",
     "dybit_launch_count", "dybit_profile_next_gemm", "dybit_gemm_static_ws", "STATIC_WS_BYTES",
+    "dybit_gemm_requant", "dybit_conv2d_requant",
 ]
 
 
@@ -92,6 +93,10 @@ def _load() -> C.CDLL:
     lib.dybit_launch_count.restype = C.c_uint64
     lib.dybit_launch_count.argtypes = []
     lib.dybit_profile_next_gemm.argtypes = [vp, vp]
+    lib.dybit_gemm_requant.argtypes = [i64, i64, i64, vp, _CFmt, vp, i64, vp, _CFmt, vp, i64,
+                                       _CFmt, vp, i32, vp, i64, vp, sz, vp]
+    lib.dybit_conv2d_requant.argtypes = [C.POINTER(_CConvDesc), vp, _CFmt, vp, vp, _CFmt, vp, i64,
+                                         _CFmt, vp, i32, vp, vp, sz, vp]
     lib.dybit_gemm_static_ws.argtypes = [i64, i64, i64, vp, _CFmt, vp, i64, vp, _CFmt, vp, i64, vp, i64, vp, vp]
     return lib
 
@@ -314,3 +319,43 @@ def dybit_gemm_static_ws(M: int, N: int, K: int, A: torch.Tensor, fa, scale_a: t
                                     _ptr(scale_b), ldb, _ptr(C_out), C_out.stride(0), _ptr(C_raw),
                                     _stream(stream)), "dybit_gemm_static_ws")
     return C_out, C_raw
+
+
+def _ws_ptr(ws: torch.Tensor):
+    off = (-ws.data_ptr()) % 1024
+    return C.c_void_p(ws.data_ptr() + off), ws.numel() - off
+
+
+def dybit_gemm_requant(M: int, N: int, K: int, A: torch.Tensor, fa, scale_a: torch.Tensor,
+                       B: torch.Tensor, fb, scale_b: torch.Tensor, fq, scale_q: torch.Tensor, relu: bool = False,
+                       Q: Optional[torch.Tensor] = None, ldq_bytes: Optional[int] = None,
+                       ws: Optional[torch.Tensor] = None, stream=None):
+    """GEMM whose result is written as packed DyBit codes of format fq (scale given).  Returns Q [M][ldq] uint8."""
+    if ldq_bytes is None:
+        ldq_bytes = N * fq[0] // 8
+    if Q is None:
+        Q = torch.zeros((M, ldq_bytes), dtype=torch.uint8, device=A.device)
+    if ws is None:
+        ws = torch.empty(dybit_gemm_workspace_bytes(M, N, K, fa, fb) + 1024, dtype=torch.uint8, device=A.device)
+    wp, wn = _ws_ptr(ws)
+    _check(lib.dybit_gemm_requant(M, N, K, _ptr(A), _fmt(fa), _ptr(scale_a), A.stride(0), _ptr(B), _fmt(fb),
+                                  _ptr(scale_b), B.stride(0), _fmt(fq), _ptr(scale_q), int(bool(relu)), _ptr(Q),
+                                  ldq_bytes, wp, wn, _stream(stream)), "dybit_gemm_requant")
+    return Q
+
+
+def dybit_conv2d_requant(desc: ConvDesc, X: torch.Tensor, fx, scale_x: torch.Tensor, W: torch.Tensor, fw,
+                         scale_w: torch.Tensor, fq, scale_q: torch.Tensor, relu: bool = False,
+                         Q: Optional[torch.Tensor] = None, ws: Optional[torch.Tensor] = None, stream=None):
+    """Convolution whose result is the dense NHWK stream of packed codes (the next layer's X).  Returns Q (1-D uint8)."""
+    oh, ow = dybit_conv2d_out_hw(desc)
+    if Q is None:
+        Q = torch.zeros(dybit_packed_bytes(desc.n * oh * ow * desc.k, fq[0]), dtype=torch.uint8, device=X.device)
+    if ws is None:
+        ws = torch.empty(dybit_conv2d_workspace_bytes(desc, fx, fw) + 1024, dtype=torch.uint8, device=X.device)
+    wp, wn = _ws_ptr(ws)
+    cd = _cdesc(desc)
+    _check(lib.dybit_conv2d_requant(C.byref(cd), _ptr(X), _fmt(fx), _ptr(scale_x), _ptr(W), _fmt(fw), _ptr(scale_w),
+                                    W.stride(0), _fmt(fq), _ptr(scale_q), int(bool(relu)), _ptr(Q), wp, wn,
+                                    _stream(stream)), "dybit_conv2d_requant")
+    return Q

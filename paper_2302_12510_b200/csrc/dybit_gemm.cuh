@@ -442,6 +442,11 @@ struct GemmParams {
     int cpb;                  // bytes per pixel in xe (padded channels * element size)
     int kb_per_tap;           // im2col mode: SWB-byte blocks per filter tap (cpb / SWB)
     int tma_store;            // 1: C leaves through shared memory and TMA stores (needs 16-byte aligned C rows)
+    // re-quantizing epilogue: when Q is set the result is encoded and packed instead of stored as fp32
+    uint8_t *Q;               // row m starts at Q + m * ldq; N codes of q_bits each
+    int64_t ldq;
+    const float *scale_q;     // {scale, 1/scale} of the output tensor
+    int q_bits, q_signed, relu;
 };
 
 // Waits for the phase with the given parity; gives up after kWaitLimitNs, records
@@ -468,6 +473,47 @@ __device__ __forceinline__ bool wait_bounded(uint64_t *bar, uint32_t parity, vol
 enum AMode { kATiled = 0,    // GEMM: 2-D tiled TMA
              kAGather = 1,   // conv: four warps gather 16-byte chunks with cp.async (any channel count)
              kAIm2col = 2 }; // conv: one im2col TMA per stage (pixel = a whole number of SWB-byte blocks)
+
+// Re-quantizing epilogue (Section III-B.1: results are quantized to DyBit before they are written back):
+// 32 consecutive outputs of one row -> 32 codes of the output format -> 4*BITS bytes at dst.
+// `valid` < 32 only in the last column chunk; then only whole bytes of valid codes are written.
+template <int BITS, bool SIGNED>
+__device__ __noinline__ void requant_store32(const float *f, float inv, uint8_t *dst, int valid) {
+    unsigned cw[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+        cw[j] = encode4<BITS, SIGNED>(make_float4(f[4 * j], f[4 * j + 1], f[4 * j + 2], f[4 * j + 3]), inv);
+    unsigned w[BITS];
+    pack32<BITS>(cw, w);
+    if (valid >= 32 && (reinterpret_cast<uintptr_t>(dst) & 3) == 0) {
+#pragma unroll
+        for (int i = 0; i < BITS; ++i) reinterpret_cast<unsigned *>(dst)[i] = w[i];
+    } else {
+        const int bytes = (valid < 32 ? valid : 32) * BITS / 8;
+        for (int b = 0; b < bytes; ++b) dst[b] = (uint8_t)(w[b >> 2] >> ((b & 3) * 8));
+    }
+}
+
+__device__ __forceinline__ void requant_dispatch(int bits, int is_signed, const float *f, float inv, uint8_t *dst,
+                                                 int valid) {
+    switch (bits * 2 + is_signed) {
+        case 4: requant_store32<2, false>(f, inv, dst, valid); break;
+        case 5: requant_store32<2, true>(f, inv, dst, valid); break;
+        case 6: requant_store32<3, false>(f, inv, dst, valid); break;
+        case 7: requant_store32<3, true>(f, inv, dst, valid); break;
+        case 8: requant_store32<4, false>(f, inv, dst, valid); break;
+        case 9: requant_store32<4, true>(f, inv, dst, valid); break;
+        case 10: requant_store32<5, false>(f, inv, dst, valid); break;
+        case 11: requant_store32<5, true>(f, inv, dst, valid); break;
+        case 12: requant_store32<6, false>(f, inv, dst, valid); break;
+        case 13: requant_store32<6, true>(f, inv, dst, valid); break;
+        case 14: requant_store32<7, false>(f, inv, dst, valid); break;
+        case 15: requant_store32<7, true>(f, inv, dst, valid); break;
+        case 16: requant_store32<8, false>(f, inv, dst, valid); break;
+        case 17: requant_store32<8, true>(f, inv, dst, valid); break;
+        default: break;
+    }
+}
 
 template <int BN, int SWB>
 struct GemmSmem {
@@ -622,6 +668,7 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         const int row_in_tile = q * 32 + lane;
         const bool issuer = threadIdx.x == 64;        // issues and tracks the TMA stores
         const float alpha = (float)((double)__ldg(p.scale_a) * (double)__ldg(p.scale_b) * p.pow2);
+        const float inv_q = p.Q ? __ldg(p.scale_q + 1) : 1.0f;
         const bool vec_ok = ((reinterpret_cast<uintptr_t>(p.C) & 15) == 0) && (p.ldc % 4 == 0) &&
                             (p.C_raw == nullptr || (reinterpret_cast<uintptr_t>(p.C_raw) & 15) == 0);
         uint32_t lt = 0, chunk_no = 0;
@@ -647,6 +694,17 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 for (int j = 0; j < 32; ++j) {
                     const float acc = (KIND == Kind::I8) ? __int2float_rn((int)r[j]) : __uint_as_float(r[j]);
                     f[j] = __fmul_rn(acc, alpha);
+                }
+                if (p.Q) {
+                    if (row < p.M) {
+                        if (p.relu) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) f[j] = fmaxf(f[j], 0.0f);
+                        }
+                        requant_dispatch(p.q_bits, p.q_signed, f, inv_q,
+                                         p.Q + (int64_t)row * p.ldq + (int64_t)col0 * p.q_bits / 8, p.N - col0);
+                    }
+                    continue;
                 }
                 if (p.tma_store) {
                     // stage 128 rows x 128 bytes in the TMA's 128-byte swizzle, then one thread stores the box;
@@ -864,7 +922,7 @@ static dybit_status launch_gemm_inst(const CUtensorMap &ta, const CUtensorMap &t
     GemmParams p = p_in;
     CUtensorMap tc;
     memset(&tc, 0, sizeof(tc));
-    p.tma_store = make_output_map(&tc, p.C, p.M, p.N, p.ldc) ? 1 : 0;
+    p.tma_store = (p.Q == nullptr && make_output_map(&tc, p.C, p.M, p.N, p.ldc)) ? 1 : 0;
     using L = GemmSmem<BN, SWB>;
     auto kern = dybit_gemm_kernel<KIND, BN, AMODE, SWB>;
     constexpr bool CONV = AMODE == kAGather;
@@ -931,6 +989,33 @@ struct GemmLayout {
 };
 
 static inline int64_t k_row_bytes(int64_t k_elems, int elem) { return round_up(k_elems * elem, kBKBytes); }
+
+// Output of the re-quantizing entry points.
+struct RequantSpec {
+    dybit_fmt fq;
+    const float *scale_q;
+    int relu;
+    void *Q;
+    int64_t ldq;
+};
+
+static dybit_status check_requant(const RequantSpec *rq, int64_t N) {
+    if (rq == nullptr) return DYBIT_OK;
+    if (!fmt_ok(rq->fq) || rq->Q == nullptr || rq->scale_q == nullptr) return DYBIT_ERR_INVALID_ARG;
+    if ((N * rq->fq.bits) % 8 != 0 || rq->ldq < N * rq->fq.bits / 8) return DYBIT_ERR_INVALID_ARG;
+    if (!aligned(rq->scale_q, 4)) return DYBIT_ERR_ALIGNMENT;
+    return DYBIT_OK;
+}
+
+static void apply_requant(GemmParams &p, const RequantSpec *rq) {
+    if (rq == nullptr) return;
+    p.Q = static_cast<uint8_t *>(rq->Q);
+    p.ldq = rq->ldq;
+    p.scale_q = rq->scale_q;
+    p.q_bits = rq->fq.bits;
+    p.q_signed = rq->fq.is_signed;
+    p.relu = rq->relu;
+}
 
 // How a convolution is lowered, and what it needs in the workspace.
 enum ConvMode { kConvPointwise, kConvIm2col, kConvPatch, kConvGather };
@@ -999,12 +1084,21 @@ size_t dybit_conv2d_workspace_bytes(const dybit_conv_desc *d, dybit_fmt fx, dybi
     return (size_t)(c.a_bytes + round_up((int64_t)d->k * c.wrb, 1024) + 2048);
 }
 
-dybit_status dybit_gemm(int64_t M, int64_t N, int64_t K, const void *A, dybit_fmt fa, const float *scale_a,
-                        int64_t lda_bytes, const void *B, dybit_fmt fb, const float *scale_b, int64_t ldb_bytes,
-                        float *C, int64_t ldc, int32_t *C_raw, void *ws, size_t ws_bytes, void *stream) {
-    using namespace dybit;
+}  // extern "C"
+
+namespace dybit {
+
+static dybit_status gemm_impl(int64_t M, int64_t N, int64_t K, const void *A, dybit_fmt fa, const float *scale_a,
+                              int64_t lda_bytes, const void *B, dybit_fmt fb, const float *scale_b, int64_t ldb_bytes,
+                              float *C, int64_t ldc, int32_t *C_raw, const RequantSpec *rq, void *ws, size_t ws_bytes,
+                              void *stream) {
     if (M <= 0 || N <= 0 || K <= 0 || !fmt_ok(fa) || !fmt_ok(fb)) return DYBIT_ERR_INVALID_ARG;
-    if (!A || !B || !C || !scale_a || !scale_b || ldc < N) return DYBIT_ERR_INVALID_ARG;
+    if (!A || !B || !scale_a || !scale_b) return DYBIT_ERR_INVALID_ARG;
+    if (rq == nullptr && (!C || ldc < N)) return DYBIT_ERR_INVALID_ARG;
+    {
+        const dybit_status rs = check_requant(rq, N);
+        if (rs != DYBIT_OK) return rs;
+    }
     if (M > INT32_MAX - 256 || N > INT32_MAX - 256 || K > (1 << 24)) return DYBIT_ERR_UNSUPPORTED;
     if (lda_bytes < (int64_t)dybit_row_stride_bytes(K, fa.bits) || ldb_bytes < (int64_t)dybit_row_stride_bytes(K, fb.bits))
         return DYBIT_ERR_INVALID_ARG;
@@ -1052,17 +1146,22 @@ dybit_status dybit_gemm(int64_t M, int64_t N, int64_t K, const void *A, dybit_fm
     p.scale_a = scale_a;
     p.scale_b = scale_b;
     p.pow2 = ldexp(1.0, -(plan.exp_a + plan.exp_b));
+    apply_requant(p, rq);
     return launch_gemm_kind<kATiled, 128>(plan.container, bn, map_a, map_b, p, s);
 }
 
-dybit_status dybit_conv2d(const dybit_conv_desc *d, const void *X, dybit_fmt fx, const float *scale_x, const void *W,
-                          dybit_fmt fw, const float *scale_w, int64_t ldw_bytes, float *Y, int32_t *Y_raw, void *ws,
-                          size_t ws_bytes, void *stream) {
-    using namespace dybit;
+static dybit_status conv_impl(const dybit_conv_desc *d, const void *X, dybit_fmt fx, const float *scale_x, const void *W,
+                              dybit_fmt fw, const float *scale_w, int64_t ldw_bytes, float *Y, int32_t *Y_raw,
+                              const RequantSpec *rq, void *ws, size_t ws_bytes, void *stream) {
     int oh, ow;
     dybit_status st = dybit_conv2d_out_hw(d, &oh, &ow);
     if (st != DYBIT_OK) return st;
-    if (!fmt_ok(fx) || !fmt_ok(fw) || !X || !W || !Y || !scale_x || !scale_w) return DYBIT_ERR_INVALID_ARG;
+    if (!fmt_ok(fx) || !fmt_ok(fw) || !X || !W || !scale_x || !scale_w) return DYBIT_ERR_INVALID_ARG;
+    if (rq == nullptr && !Y) return DYBIT_ERR_INVALID_ARG;
+    {
+        const dybit_status rs = check_requant(rq, d->k);
+        if (rs != DYBIT_OK) return rs;
+    }
     const int64_t K = (int64_t)d->r * d->s * d->c;
     const int64_t M = (int64_t)d->n * oh * ow;
     const int64_t N = d->k;
@@ -1159,6 +1258,7 @@ dybit_status dybit_conv2d(const dybit_conv_desc *d, const void *X, dybit_fmt fx,
     p.pad = d->pad;
     p.dil = d->dilation;
     p.cpb = (int)cpb;
+    apply_requant(p, rq);
 
     CUtensorMap map_a, map_b;
     if (cv.mode == kConvPointwise || cv.mode == kConvPatch) {
@@ -1186,6 +1286,40 @@ dybit_status dybit_conv2d(const dybit_conv_desc *d, const void *X, dybit_fmt fx,
     if (st != DYBIT_OK) return st;
     p.k_blocks = (int)(wrb / kBKBytes);
     return launch_gemm_kind<kAGather, 128>(plan.container, bn, map_b, map_b, p, s);
+}
+
+}  // namespace dybit
+
+extern "C" {
+
+dybit_status dybit_gemm(int64_t M, int64_t N, int64_t K, const void *A, dybit_fmt fa, const float *scale_a,
+                        int64_t lda_bytes, const void *B, dybit_fmt fb, const float *scale_b, int64_t ldb_bytes,
+                        float *C, int64_t ldc, int32_t *C_raw, void *ws, size_t ws_bytes, void *stream) {
+    return dybit::gemm_impl(M, N, K, A, fa, scale_a, lda_bytes, B, fb, scale_b, ldb_bytes, C, ldc, C_raw, nullptr, ws,
+                            ws_bytes, stream);
+}
+
+dybit_status dybit_conv2d(const dybit_conv_desc *d, const void *X, dybit_fmt fx, const float *scale_x, const void *W,
+                          dybit_fmt fw, const float *scale_w, int64_t ldw_bytes, float *Y, int32_t *Y_raw, void *ws,
+                          size_t ws_bytes, void *stream) {
+    return dybit::conv_impl(d, X, fx, scale_x, W, fw, scale_w, ldw_bytes, Y, Y_raw, nullptr, ws, ws_bytes, stream);
+}
+
+dybit_status dybit_gemm_requant(int64_t M, int64_t N, int64_t K, const void *A, dybit_fmt fa, const float *scale_a,
+                                int64_t lda_bytes, const void *B, dybit_fmt fb, const float *scale_b,
+                                int64_t ldb_bytes, dybit_fmt fq, const float *scale_q, int relu, void *Q,
+                                int64_t ldq_bytes, void *ws, size_t ws_bytes, void *stream) {
+    const dybit::RequantSpec rq = {fq, scale_q, relu ? 1 : 0, Q, ldq_bytes};
+    return dybit::gemm_impl(M, N, K, A, fa, scale_a, lda_bytes, B, fb, scale_b, ldb_bytes, nullptr, 0, nullptr, &rq, ws,
+                            ws_bytes, stream);
+}
+
+dybit_status dybit_conv2d_requant(const dybit_conv_desc *d, const void *X, dybit_fmt fx, const float *scale_x,
+                                  const void *W, dybit_fmt fw, const float *scale_w, int64_t ldw_bytes, dybit_fmt fq,
+                                  const float *scale_q, int relu, void *Q, void *ws, size_t ws_bytes, void *stream) {
+    if (d == nullptr) return DYBIT_ERR_INVALID_ARG;
+    const dybit::RequantSpec rq = {fq, scale_q, relu ? 1 : 0, Q, (int64_t)d->k * fq.bits / 8};
+    return dybit::conv_impl(d, X, fx, scale_x, W, fw, scale_w, ldw_bytes, nullptr, nullptr, &rq, ws, ws_bytes, stream);
 }
 
 }  // extern "C"

@@ -177,3 +177,33 @@ def test_resnet50_batch64_mixed_bitwidths_sampled(i, L):
     wbits, abits = _R50_BITS[i]
     _conv_layer_sampled(L, (abits, 0), (wbits, 1), seed=3000 + i, n_samples=800)
     torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("i,L", _distinct(wl.resnet18_layers(32)), ids=lambda v: getattr(v, "name", str(v)))
+def test_resnet18_batch32_requant_epilogue_sampled(i, L):
+    """Bench-size layers through the re-quantizing epilogue: sampled output codes against the oracle
+    (sampled conv -> ReLU -> encode with the given output scale)."""
+    fx, fw, fq = (4, 0), (4, 1), (4, 0)
+    x = wl.half_normal((L.n, L.h, L.w, L.c), seed=1000 + i, device=DEV)
+    w = wl.kaiming_normal(L.k, L.r, L.s, L.c, seed=2000 + i)
+    px, sx = dy.dybit_quantize_pack(x, fx)
+    pw, sw = dy.dybit_quantize_pack_2d(w.reshape(L.k, -1).to(DEV), fw)
+    xh = x.cpu().numpy()
+    spx = orc.absmax_scale(xh, 4, False)
+    spw = orc.absmax_scale(w.numpy(), 4, True)
+    cw = orc.quantize(w.numpy(), 4, True, spw[1])
+    total = L.gemm_m * L.k
+    rng = np.random.default_rng(i)
+    idx = np.unique(np.concatenate([rng.integers(0, total, 1200), [0, total - 1]]))
+    _, yref = orc.conv2d_sampled(xh, fx, spx, cw, fw, spw[0], idx, stride=L.stride, pad=L.pad)
+    # output scale from the sampled activations (a stand-in for a calibrated scale); some samples saturate
+    sq = orc.absmax_scale(np.maximum(yref, 0) * 0.8, 4, False)
+    scale_q = torch.tensor([float(sq[0]), float(sq[1])], dtype=torch.float32, device=DEV)
+    desc = dy.ConvDesc(L.n, L.h, L.w, L.c, L.k, L.r, L.s, L.stride, L.pad, 1)
+    Q = dy.dybit_conv2d_requant(desc, px, fx, sx, pw, fw, sw, fq, scale_q, relu=True)
+    torch.cuda.synchronize()
+    assert dy.dybit_last_device_status() == (0, 0)
+    qb = Q.cpu().numpy()
+    got = (qb[idx // 2] >> ((idx % 2) * 4)) & 0xF                    # 4-bit codes: two per byte, low nibble first
+    want = orc.quantize(np.maximum(yref, 0), 4, False, sq[1])
+    assert np.array_equal(got, want), L.name

@@ -1,0 +1,136 @@
+"""GPU parity of the re-quantizing epilogue (results written back as DyBit codes, Section III-B.1).
+
+Oracle = the oracle's own GEMM / conv, then (ReLU), then the oracle's quantize with the given output scale, then
+its pack: no new arithmetic.  int8-container layers must match bit for bit.  For the floating containers the fp32
+value carries an accumulation tolerance, so the codes are checked against the oracle's encoder applied to the
+GPU's own fp32 output (which the GEMM tests pin separately)."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2302_12510_b200 as dy
+from paper_2302_12510_b200 import workloads as wl
+from oracle import dybit_oracle as orc
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _quant(x, fmt):
+    packed, scale = dy.dybit_quantize_pack_2d(x.to(DEV), fmt)
+    sp = orc.absmax_scale(x.numpy(), fmt[0], bool(fmt[1]))
+    return packed, scale, orc.quantize(x.numpy(), fmt[0], bool(fmt[1]), sp[1]), sp
+
+
+def _expect(y_ref, fq, inv_q, relu):
+    y = np.maximum(y_ref, 0) if relu else y_ref
+    codes = orc.quantize(y.astype(np.float32), fq[0], bool(fq[1]), inv_q)
+    return np.stack([orc.pack(r, fq[0])[: y.shape[1] * fq[0] // 8] for r in codes])
+
+
+@pytest.mark.parametrize("M,N,K", [(128, 256, 128), (300, 520, 400), (777, 64, 1153), (64, 1000, 512), (5, 8, 77)])
+@pytest.mark.parametrize("fq,relu", [((4, 0), True), ((4, 1), False), ((8, 1), False), ((2, 0), True), ((3, 1), False),
+                                     ((6, 0), True)])
+def test_gemm_requant_int8_container_bit_exact(M, N, K, fq, relu):
+    fa, fb = (4, 0), (4, 1)
+    a = wl.half_normal((M, K), seed=M + K)
+    b = wl.normal((N, K), seed=N + K, std=0.05)
+    pa, sa, ca, spa = _quant(a, fa)
+    pb, sb, cb, spb = _quant(b, fb)
+    _, y_ref = orc.gemm(ca, fa, spa[0], cb, fb, spb[0])
+    # a "calibrated" output scale: slightly below the observed maximum, so that saturation is exercised too
+    sq = orc.absmax_scale(y_ref * 0.9, fq[0], bool(fq[1]))
+    scale_q = torch.tensor([float(sq[0]), float(sq[1])], dtype=torch.float32, device=DEV)
+    Q = dy.dybit_gemm_requant(M, N, K, pa, fa, sa, pb, fb, sb, fq, scale_q, relu=relu)
+    torch.cuda.synchronize()
+    assert dy.dybit_last_device_status() == (0, 0)
+    assert np.array_equal(Q.cpu().numpy(), _expect(y_ref, fq, sq[1], relu))
+
+
+def test_gemm_requant_padded_rows_feed_the_next_gemm():
+    # layer 1 writes codes with GEMM-operand row padding; layer 2 consumes them directly
+    fa, fb, fq = (4, 0), (4, 1), (4, 0)
+    M, N1, K1, N2 = 200, 256, 300, 96
+    a = wl.half_normal((M, K1), seed=1)
+    w1 = wl.normal((N1, K1), seed=2, std=0.05)
+    w2 = wl.normal((N2, N1), seed=3, std=0.05)
+    pa, sa, ca, spa = _quant(a, fa)
+    p1, s1, c1, sp1 = _quant(w1, fb)
+    p2, s2, c2, sp2 = _quant(w2, fb)
+    _, y1 = orc.gemm(ca, fa, spa[0], c1, fb, sp1[0])
+    sq = orc.absmax_scale(np.maximum(y1, 0), fq[0], False)
+    scale_q = torch.tensor([float(sq[0]), float(sq[1])], dtype=torch.float32, device=DEV)
+    ldq = dy.dybit_row_stride_bytes(N1, fq[0])
+    Q = dy.dybit_gemm_requant(M, N1, K1, pa, fa, sa, p1, fb, s1, fq, scale_q, relu=True, ldq_bytes=ldq)
+    C2, C2_raw = dy.dybit_gemm(M, N2, N1, Q, fq, scale_q, p2, fb, s2, want_raw=True)
+    q_codes = orc.quantize(np.maximum(y1, 0), fq[0], False, sq[1])
+    assert np.array_equal(Q.cpu().numpy(), orc.pack_rows(q_codes, fq[0]))
+    S2, y2 = orc.gemm(q_codes, fq, sq[0], c2, fb, sp2[0])
+    assert np.array_equal(C2_raw.cpu().numpy().astype(np.int64), S2)
+    assert np.array_equal(C2.cpu().numpy(), y2)
+
+
+@pytest.mark.parametrize("fa,fb", [((8, 0), (8, 1)), ((5, 0), (4, 1))])
+def test_gemm_requant_float_containers_encode_their_own_output(fa, fb):
+    M, N, K, fq = 260, 320, 500, (4, 0)
+    a = wl.half_normal((M, K), seed=4)
+    b = wl.normal((N, K), seed=5, std=0.05)
+    pa, sa, _, _ = _quant(a, fa)
+    pb, sb, _, _ = _quant(b, fb)
+    C, _ = dy.dybit_gemm(M, N, K, pa, fa, sa, pb, fb, sb)
+    y_gpu = C.cpu().numpy()
+    sq = orc.absmax_scale(np.maximum(y_gpu, 0), fq[0], False)
+    scale_q = torch.tensor([float(sq[0]), float(sq[1])], dtype=torch.float32, device=DEV)
+    Q = dy.dybit_gemm_requant(M, N, K, pa, fa, sa, pb, fb, sb, fq, scale_q, relu=True)
+    assert np.array_equal(Q.cpu().numpy(), _expect(y_gpu, fq, sq[1], True))
+
+
+@pytest.mark.parametrize("layer", [
+    wl.ConvLayer("c64_3x3", 4, 28, 28, 64, 64, 3, 3, 1, 1),
+    wl.ConvLayer("c128_3x3_s2", 4, 20, 20, 128, 96, 3, 3, 2, 1),
+    wl.ConvLayer("stem_c3_7x7", 2, 32, 32, 3, 64, 7, 7, 2, 3),
+    wl.ConvLayer("pointwise", 3, 14, 14, 256, 128, 1, 1, 1, 0),
+    wl.ConvLayer("small_gather", 2, 8, 8, 64, 40, 3, 3, 1, 1),
+], ids=lambda L: L.name)
+def test_conv_requant_chains_into_the_next_conv(layer):
+    fx, fw, fq = (4, 0), (4, 1), (4, 0)
+    L = layer
+    x = wl.half_normal((L.n, L.h, L.w, L.c), seed=7)
+    w = wl.kaiming_normal(L.k, L.r, L.s, L.c, seed=8)
+    px, sx = dy.dybit_quantize_pack(x.to(DEV), fx)
+    pw, sw = dy.dybit_quantize_pack_2d(w.reshape(L.k, -1).to(DEV), fw)
+    spx = orc.absmax_scale(x.numpy(), 4, False)
+    spw = orc.absmax_scale(w.numpy(), 4, True)
+    cx = orc.quantize(x.numpy(), 4, False, spx[1])
+    cw = orc.quantize(w.numpy(), 4, True, spw[1])
+    _, y = orc.conv2d(cx, fx, spx[0], cw, fw, spw[0], stride=L.stride, pad=L.pad)
+    sq = orc.absmax_scale(np.maximum(y, 0) * 0.95, 4, False)
+    scale_q = torch.tensor([float(sq[0]), float(sq[1])], dtype=torch.float32, device=DEV)
+    desc = dy.ConvDesc(L.n, L.h, L.w, L.c, L.k, L.r, L.s, L.stride, L.pad, 1)
+    Q = dy.dybit_conv2d_requant(desc, px, fx, sx, pw, fw, sw, fq, scale_q, relu=True)
+    torch.cuda.synchronize()
+    assert dy.dybit_last_device_status() == (0, 0)
+    q_codes = orc.quantize(np.maximum(y, 0), 4, False, sq[1])
+    assert np.array_equal(Q.cpu().numpy(), orc.pack(q_codes, 4))
+    # the stream is the next layer's X: a 1x1 conv on it must match the oracle on the oracle's codes
+    k2 = 32
+    w2 = wl.kaiming_normal(k2, 1, 1, L.k, seed=9)
+    pw2, sw2 = dy.dybit_quantize_pack_2d(w2.reshape(k2, -1).to(DEV), fw)
+    spw2 = orc.absmax_scale(w2.numpy(), 4, True)
+    cw2 = orc.quantize(w2.numpy(), 4, True, spw2[1])
+    d2 = dy.ConvDesc(L.n, L.oh, L.ow, L.k, k2, 1, 1, 1, 0, 1)
+    Y2, Y2_raw = dy.dybit_conv2d(d2, Q, fq, scale_q, pw2, fw, sw2, want_raw=True)
+    S2, y2 = orc.conv2d(q_codes, fq, sq[0], cw2, fw, spw2[0])
+    assert np.array_equal(Y2_raw.cpu().numpy().astype(np.int64), S2)
+    assert np.array_equal(Y2.cpu().numpy(), y2)
+
+
+def test_requant_argument_errors():
+    one = torch.tensor([1.0, 1.0], device=DEV)
+    pa = torch.zeros((4, 64), dtype=torch.uint8, device=DEV)
+    with pytest.raises(dy.DybitError) as e:       # N * bits not a whole number of bytes
+        dy.dybit_gemm_requant(4, 3, 128, pa, (4, 1), one, pa, (4, 1), one, (3, 0), one, Q=torch.zeros((4, 4), dtype=torch.uint8, device=DEV), ldq_bytes=4)
+    assert e.value.status == 1
+    with pytest.raises(dy.DybitError) as e:       # rows shorter than N codes
+        dy.dybit_gemm_requant(4, 4, 128, pa, (4, 1), one, pa, (4, 1), one, (8, 0), one, Q=torch.zeros((4, 4), dtype=torch.uint8, device=DEV), ldq_bytes=0)
+    assert e.value.status == 1
