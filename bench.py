@@ -163,6 +163,25 @@ class LayerwiseStep:
             dy.dybit_conv2d(self.desc[i], self.px[i], self.fa[i], self.sx[i], self.pw[i], self.fw[i], self.sw[i],
                             Y=self.y[i], ws=self.ws)
 
+    def prepare_requant(self, fq=(4, 0)):
+        """Output scales for the re-quantizing epilogue: max-abs of each layer's fp32 output from one normal step
+        (a stand-in for calibrated scales); packed output buffers."""
+        dy = self.dy
+        self.fq = fq
+        self.step()
+        self.sq = [dy.dybit_absmax_scale(y.reshape(-1).clamp_min(0), fq) for y in self.y]
+        self.q = [torch.zeros(dy.dybit_packed_bytes(y.numel(), fq[0]), dtype=torch.uint8, device=self.device)
+                  for y in self.y]
+        self.q_bytes = sum(q.numel() for q in self.q)
+
+    def step_requant(self):
+        """The same step with results written back as packed DyBit codes (ReLU + encode in the epilogue)."""
+        dy = self.dy
+        for i in range(len(self.layers)):
+            dy.dybit_quantize_pack(self.x_dev[i], self.fa[i], packed=self.px[i], scale_out=self.sx[i])
+            dy.dybit_conv2d_requant(self.desc[i], self.px[i], self.fa[i], self.sx[i], self.pw[i], self.fw[i], self.sw[i],
+                                    self.fq, self.sq[i], relu=True, Q=self.q[i], ws=self.ws)
+
     def step_e2e(self):
         for i in range(len(self.layers)):
             self.x_dev[i].copy_(self.x_host[i], non_blocking=True)
@@ -210,14 +229,14 @@ def whole_job_tops(macs_per_rank, world, ms_step):
     return world * 2.0 * macs_per_rank / (ms_step * 1e-3) / 1e12
 
 
-def capture_step(work, device):
+def capture_step(work, device, fn=None):
     """One step captured as a CUDA graph (the library's calls are plain stream work, so they capture)."""
     graph = torch.cuda.CUDAGraph()
     cap_stream = torch.cuda.Stream(device)
     cap_stream.wait_stream(torch.cuda.current_stream())
     with torch.cuda.stream(cap_stream):
         with torch.cuda.graph(graph, stream=cap_stream):
-            work.step()
+            (fn or work.step)()
     torch.cuda.current_stream().wait_stream(cap_stream)
     return graph
 
@@ -575,6 +594,19 @@ def main():
         "gpu_launches": launches, "clocks": clocks, "e2e": e2e, "roofline": roofline,
         "quantize_elems_per_step": work.quant_elems,
     }
+    # ---- the same step with the re-quantizing epilogue (results leave as 4-bit codes instead of fp32)
+    work.prepare_requant()
+    for _ in range(3):
+        work.step_requant()
+    graph_q = capture_step(work, device, work.step_requant)
+    for _ in range(3):
+        graph_q.replay()
+    ms_q = timed_region(graph_q.replay, args.steps, dist, device) / args.steps
+    result["requant_epilogue"] = {
+        "what": "same 21 layers, results written back as unsigned 4-bit DyBit codes (ReLU + encode in the GEMM epilogue, "
+                "given output scales) instead of fp32",
+        "ms_per_step": ms_q, "value": whole_job_tops(work.macs, world, ms_q), "unit": "TOPS",
+        "output_bytes_per_step": work.q_bytes, "fp32_output_bytes_per_step": work.d2h_bytes}
     del work
     torch.cuda.empty_cache()
 

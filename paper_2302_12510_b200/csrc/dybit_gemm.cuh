@@ -425,6 +425,7 @@ constexpr int kBM = 128;            // tile rows (UMMA M)
 constexpr int kBKBytes = 128;       // one 128-byte swizzle row of K per pipeline stage (64 in the SWB = 64 variant)
 constexpr int kUmmaKBytes = 32;     // K bytes consumed by one tcgen05.mma
 constexpr int kStageBytesTotal = 192 * 1024;
+constexpr int kEpilogueWarps = 8;     // two groups of four (one warp per TMEM lane quarter in each)
 constexpr unsigned long long kWaitLimitNs = 4000000000ull;
 
 struct GemmParams {
@@ -494,23 +495,53 @@ __device__ __noinline__ void requant_store32(const float *f, float inv, uint8_t 
     }
 }
 
-__device__ __forceinline__ void requant_dispatch(int bits, int is_signed, const float *f, float inv, uint8_t *dst,
+// The same, fully inlined and fed from registers: used for the output widths the search space of
+// Section III-C.3 selects (2, 4 and 8 bits); the other widths go through the out-of-line version.
+template <int BITS, bool SIGNED>
+__device__ __forceinline__ void requant_store32_inline(const float (&f)[32], float inv, uint8_t *dst, int valid) {
+    unsigned cw[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+        cw[j] = encode4<BITS, SIGNED>(make_float4(f[4 * j], f[4 * j + 1], f[4 * j + 2], f[4 * j + 3]), inv);
+    unsigned w[BITS];
+    pack32<BITS>(cw, w);
+    if (valid >= 32 && (reinterpret_cast<uintptr_t>(dst) & (BITS == 2 ? 7 : 15)) == 0) {
+        if constexpr (BITS == 2) *reinterpret_cast<uint2 *>(dst) = make_uint2(w[0], w[1]);
+        else if constexpr (BITS == 4) *reinterpret_cast<uint4 *>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+        else {
+            reinterpret_cast<uint4 *>(dst)[0] = make_uint4(w[0], w[1], w[2], w[3]);
+            reinterpret_cast<uint4 *>(dst)[1] = make_uint4(w[4 % BITS], w[5 % BITS], w[6 % BITS], w[7 % BITS]);
+        }
+    } else {
+        const int bytes = (valid < 32 ? valid : 32) * BITS / 8;
+        for (int b = 0; b < bytes; ++b) dst[b] = (uint8_t)(w[b >> 2] >> ((b & 3) * 8));
+    }
+}
+
+__device__ __forceinline__ void requant_dispatch(int bits, int is_signed, const float (&f)[32], float inv, uint8_t *dst,
                                                  int valid) {
     switch (bits * 2 + is_signed) {
-        case 4: requant_store32<2, false>(f, inv, dst, valid); break;
-        case 5: requant_store32<2, true>(f, inv, dst, valid); break;
-        case 6: requant_store32<3, false>(f, inv, dst, valid); break;
-        case 7: requant_store32<3, true>(f, inv, dst, valid); break;
-        case 8: requant_store32<4, false>(f, inv, dst, valid); break;
-        case 9: requant_store32<4, true>(f, inv, dst, valid); break;
-        case 10: requant_store32<5, false>(f, inv, dst, valid); break;
-        case 11: requant_store32<5, true>(f, inv, dst, valid); break;
-        case 12: requant_store32<6, false>(f, inv, dst, valid); break;
-        case 13: requant_store32<6, true>(f, inv, dst, valid); break;
-        case 14: requant_store32<7, false>(f, inv, dst, valid); break;
-        case 15: requant_store32<7, true>(f, inv, dst, valid); break;
-        case 16: requant_store32<8, false>(f, inv, dst, valid); break;
-        case 17: requant_store32<8, true>(f, inv, dst, valid); break;
+        case 4: requant_store32_inline<2, false>(f, inv, dst, valid); return;
+        case 5: requant_store32_inline<2, true>(f, inv, dst, valid); return;
+        case 8: requant_store32_inline<4, false>(f, inv, dst, valid); return;
+        case 9: requant_store32_inline<4, true>(f, inv, dst, valid); return;
+        case 16: requant_store32_inline<8, false>(f, inv, dst, valid); return;
+        case 17: requant_store32_inline<8, true>(f, inv, dst, valid); return;
+        default: break;
+    }
+    // the other widths run out of line on a copy, so that f itself can stay in registers
+    float tmp[32];
+#pragma unroll
+    for (int j = 0; j < 32; ++j) tmp[j] = f[j];
+    switch (bits * 2 + is_signed) {
+        case 6: requant_store32<3, false>(tmp, inv, dst, valid); break;
+        case 7: requant_store32<3, true>(tmp, inv, dst, valid); break;
+        case 10: requant_store32<5, false>(tmp, inv, dst, valid); break;
+        case 11: requant_store32<5, true>(tmp, inv, dst, valid); break;
+        case 12: requant_store32<6, false>(tmp, inv, dst, valid); break;
+        case 13: requant_store32<6, true>(tmp, inv, dst, valid); break;
+        case 14: requant_store32<7, false>(tmp, inv, dst, valid); break;
+        case 15: requant_store32<7, true>(tmp, inv, dst, valid); break;
         default: break;
     }
 }
@@ -539,7 +570,7 @@ __device__ __forceinline__ void tile_coords(int tile, int m_tiles, int n_tiles, 
 }
 
 template <Kind KIND, int BN, int AMODE, int SWB>
-__global__ void __launch_bounds__(AMODE == kAGather ? 320 : 192, 1)
+__global__ void __launch_bounds__(AMODE == kAGather ? 448 : 320, 1)
 dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                   const __grid_constant__ CUtensorMap tmap_c, const GemmParams p) {
     static_assert(AMODE != kAGather || SWB == 128, "the cp.async gather writes 128-byte rows");
@@ -572,7 +603,7 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(&acc_full[a], 1);
-            mbar_init(&acc_empty[a], 4);
+            mbar_init(&acc_empty[a], kEpilogueWarps);
         }
         *abort_flag = 0;
         fence_mbar_init();
@@ -662,16 +693,18 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 if (ok) umma_commit(&acc_full[as]);
             }
         }
-    } else if (warp < 6) {
+    } else if (warp < 2 + kEpilogueWarps) {
         // ------------------------------------------------ epilogue: TMEM -> registers -> (shared -> TMA store | global)
         const int q = warp & 3;                       // TMEM lane quarter this warp may read
         const int row_in_tile = q * 32 + lane;
-        const bool issuer = threadIdx.x == 64;        // issues and tracks the TMA stores
+        // two groups of four warps; group g takes the 32-column chunks cc = g, g + 2, ... and owns staging buffer g
+        const int group = (warp - 2) >> 2;
+        const bool issuer = (threadIdx.x & 127) == 64; // first lane of each group: issues and tracks its TMA stores
         const float alpha = (float)((double)__ldg(p.scale_a) * (double)__ldg(p.scale_b) * p.pow2);
         const float inv_q = p.Q ? __ldg(p.scale_q + 1) : 1.0f;
         const bool vec_ok = ((reinterpret_cast<uintptr_t>(p.C) & 15) == 0) && (p.ldc % 4 == 0) &&
                             (p.C_raw == nullptr || (reinterpret_cast<uintptr_t>(p.C_raw) & 15) == 0);
-        uint32_t lt = 0, chunk_no = 0;
+        uint32_t lt = 0;
         for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++lt) {
             int m_blk, n_blk;
             tile_coords(tile, p.m_tiles, p.n_tiles, m_blk, n_blk);
@@ -683,9 +716,9 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             const int row = m_blk * kBM + row_in_tile;
             const uint32_t taddr = tmem_base + as * BN + ((uint32_t)(q * 32) << 16);
 #pragma unroll 1
-            for (int cc = 0; cc < BN / 32; ++cc) {
+            for (int cc = group; cc < BN / 32; cc += kEpilogueWarps / 4) {
                 const int col0 = n_blk * BN + cc * 32;
-                if (col0 >= p.N) break;                // uniform over the CTA: the rest of the tile lies outside C
+                if (col0 >= p.N) break;                // uniform over the group: the rest of the tile lies outside C
                 uint32_t r[32];
                 tmem_ld_32x32(taddr + cc * 32, r);
                 tmem_ld_wait();
@@ -709,21 +742,20 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 if (p.tma_store) {
                     // stage 128 rows x 128 bytes in the TMA's 128-byte swizzle, then one thread stores the box;
                     // rows / columns beyond C are clipped by the tensor map
-                    uint8_t *stage = c_stages + (chunk_no & 1u) * L::kCStage;
-                    if (issuer) bulk_wait_group_read<1>();        // the store that last read this buffer is done with it
-                    named_barrier(1, 128);
+                    uint8_t *stage = c_stages + group * L::kCStage;
+                    if (issuer) bulk_wait_group_read<0>();        // the store that last read this buffer is done with it
+                    named_barrier(1 + group, 128);
                     uint8_t *srow = stage + row_in_tile * 128;
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
                         *reinterpret_cast<float4 *>(srow + ((j ^ (row_in_tile & 7)) << 4)) =
                             make_float4(f[4 * j], f[4 * j + 1], f[4 * j + 2], f[4 * j + 3]);
                     fence_proxy_async_smem();
-                    named_barrier(1, 128);
+                    named_barrier(1 + group, 128);
                     if (issuer) {
                         tma_store_2d(&tmap_c, stage, col0, m_blk * kBM);
                         bulk_commit_group();
                     }
-                    ++chunk_no;
                 }
                 if (row < p.M) {
                     float *crow = p.C + (int64_t)row * p.ldc + col0;
@@ -757,7 +789,7 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         if (issuer) bulk_wait_group_read<0>();             // shared memory must outlive the last store's read
     } else if (CONV) {
         // ------------------------------------------------ im2col gather of the A tile (4 warps, one row per thread)
-        const int t = threadIdx.x - 192;              // tile row 0..127
+        const int t = threadIdx.x - 32 * (2 + kEpilogueWarps);   // tile row 0..127
         const int sw = t & 7;
         constexpr int kAhead = 2;                     // stages issued but not yet published
         uint32_t it = 0, issued = 0, published = 0;
@@ -939,7 +971,7 @@ static dybit_status launch_gemm_inst(const CUtensorMap &ta, const CUtensorMap &t
     ProfileEvents ev = profile_events();
     profile_events() = ProfileEvents();
     if (ev.start) DYBIT_CUDA_TRY(cudaEventRecord(ev.start, s));
-    launch_k(kern, dim3((unsigned)(grid)), dim3((unsigned)(CONV ? 320 : 192)), (size_t)(L::kBytes), s, ta, tb, tc, p);
+    launch_k(kern, dim3((unsigned)(grid)), dim3((unsigned)(CONV ? 448 : 320)), (size_t)(L::kBytes), s, ta, tb, tc, p);
     const dybit_status st = launch_status();
     if (ev.stop) DYBIT_CUDA_TRY(cudaEventRecord(ev.stop, s));
     return st;
