@@ -414,3 +414,34 @@ void orc_conv2d_sampled(int n, int h, int w, int c, int k, int r, int s,
         if (Y) Y[e] = (float)acc * alpha;
     }
 }
+
+/* ------------------------------------------------------------------ */
+/* Quantization error metric, Eq. 2 (Section III-C.1)                  */
+/* ------------------------------------------------------------------ */
+
+/* RMSE = sqrt( (1/n) * sum_i ((x_i - xhat_i) / sigma)^2 ), where xhat is the
+ * quantize-dequantize image of x under the given format and {scale, inv}
+ * and sigma is the standard deviation of the tensor x (population form,
+ * mean of squared deviations from the mean).  Everything in double from
+ * the fp32 inputs; xhat_i itself is the fp32 value orc_dequantize returns.
+ * out[0] = RMSE, out[1] = sigma, out[2] = mean squared error (before the
+ * division by sigma^2).  n == 0 or sigma == 0 give RMSE = 0. */
+void orc_rmse(const float *x, int64_t n, int bits, int is_signed, float scale, float inv, double *out)
+{
+    double mean = 0.0, var = 0.0, se = 0.0;
+    for (int64_t i = 0; i < n; ++i) mean += (double)x[i];
+    if (n > 0) mean /= (double)n;
+    for (int64_t i = 0; i < n; ++i) {
+        double d = (double)x[i] - mean;
+        var += d * d;
+        unsigned c = orc_encode_one(x[i], inv, bits, is_signed);
+        float xhat = scale * (float)orc_decode(bits, is_signed, c);
+        double e = (double)x[i] - (double)xhat;
+        se += e * e;
+    }
+    double sigma = n > 0 ? sqrt(var / (double)n) : 0.0;
+    double mse = n > 0 ? se / (double)n : 0.0;
+    out[0] = (sigma > 0.0) ? sqrt(mse) / sigma : 0.0;
+    out[1] = sigma;
+    out[2] = mse;
+}

@@ -62,6 +62,7 @@ def _load():
         lib.orc_gemm_sampled.argtypes = [i64, i64, vp, i32, i32, f32, vp, i32, i32, f32,
                                          vp, vp, i64, vp, vp]
         lib.orc_conv2d.argtypes = [i32] * 10 + [vp, i32, i32, f32, vp, i32, i32, f32, vp, vp]
+        lib.orc_rmse.argtypes = [vp, i64, i32, i32, f32, f32, vp]
         lib.orc_conv2d_sampled.argtypes = [i32] * 10 + [vp, i32, i32, f32, f32, vp, i32, i32, f32, vp, i64, vp, vp]
         _lib = lib
     return _lib
@@ -245,3 +246,12 @@ def conv2d_sampled(x_fp32, fmt_x, scale_pair_x, codes_w, fmt_w, scale_w, flat_id
                                _p(wt), fmt_w[0], int(fmt_w[1]), float(np.float32(scale_w)),
                                _p(idx), idx.size, _p(acc), _p(y))
     return acc, y
+
+
+def rmse(x, bits: int, is_signed: bool, scale_pair):
+    """Eq. 2: (RMSE, sigma, mse) of quantizing x to the format with {scale, inv}."""
+    x = _f32(x).ravel()
+    out = np.zeros(3, dtype=np.float64)
+    _load().orc_rmse(_p(x), x.size, bits, int(is_signed), float(np.float32(scale_pair[0])),
+                     float(np.float32(scale_pair[1])), _p(out))
+    return float(out[0]), float(out[1]), float(out[2])
