@@ -366,6 +366,16 @@ def run_sweeps(dy, wl, device, peaks):
             del x
             torch.cuda.empty_cache()
     out["quantize_sweep"] = rows
+    # Eq. 2 error metric: one streaming pass, 4 B/element
+    x = wl.normal((1 << 28,), seed=5, device=device)
+    out["rmse"] = []
+    for bits in (2, 4, 8):
+        scale = dy.dybit_absmax_scale(x, (bits, 1))
+        res = torch.empty(4, dtype=torch.float64, device=device)
+        ms = time_calls_flushed(lambda: dy.dybit_rmse(x, (bits, 1), scale, out=res), 7, flush)
+        out["rmse"].append({"log2n": 28, "bits": bits, "gbs": (1 << 28) * 4 / ms / 1e6, "rmse": res[0].item()})
+    del x
+    torch.cuda.empty_cache()
     out["gemm_sweep"] = []
     for fmt in ((4, 1), (8, 1)):
         for size in (1024, 2048, 4096, 8192):

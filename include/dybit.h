@@ -191,6 +191,14 @@ dybit_status dybit_conv2d(const dybit_conv_desc *desc,
                           float *Y, int32_t *Y_raw,
                           void *ws, size_t ws_bytes, void *stream);
 
+/* Quantization error metric of Eq. 2 (Section III-C.1), the quantity the bitwidth search ranks layers by:
+ *     RMSE = sqrt( (1/n) * sum_i ((x_i - xhat_i) / sigma)^2 )
+ * with xhat_i = scale[0] * value(encode(x_i)) the quantize-dequantize image under `fmt` and {scale, 1/scale}, and
+ * sigma the standard deviation of x (population form).  One pass over x; sums are kept in fp64.
+ *   x     [dev] n floats;  scale [dev] 2 floats {scale, 1/scale}
+ *   out   [dev] 4 doubles, 8-byte aligned: {RMSE, sigma, mean squared error, n}; RMSE = 0 when sigma == 0 or n == 0 */
+dybit_status dybit_rmse(const float *x, int64_t n, dybit_fmt fmt, const float *scale, double *out, void *stream);
+
 /* GEMM / convolution with the re-quantizing epilogue of Section III-B.1 ("the FP intermediate results will be
  * quantized to DyBit format before being written back"): instead of fp32, the result leaves the kernel as packed
  * DyBit codes of format fq, ready to be the next layer's activation.  Per output element

@@ -21,7 +21,7 @@ __all__ = [
     "dybit_conv2d_out_hw", "dybit_absmax_scale", "dybit_quantize_pack", "dybit_quantize_pack_2d",
     "dybit_decode", "dybit_gemm", "dybit_conv2d", "dybit_last_device_status",
     "dybit_launch_count", "dybit_profile_next_gemm", "dybit_gemm_static_ws", "STATIC_WS_BYTES",
-    "dybit_gemm_requant", "dybit_conv2d_requant",
+    "dybit_gemm_requant", "dybit_conv2d_requant", "dybit_rmse",
 ]
 
 
@@ -97,6 +97,7 @@ def _load() -> C.CDLL:
                                        _CFmt, vp, i32, vp, i64, vp, sz, vp]
     lib.dybit_conv2d_requant.argtypes = [C.POINTER(_CConvDesc), vp, _CFmt, vp, vp, _CFmt, vp, i64,
                                          _CFmt, vp, i32, vp, vp, sz, vp]
+    lib.dybit_rmse.argtypes = [vp, i64, _CFmt, vp, vp, vp]
     lib.dybit_gemm_static_ws.argtypes = [i64, i64, i64, vp, _CFmt, vp, i64, vp, _CFmt, vp, i64, vp, i64, vp, vp]
     return lib
 
@@ -359,3 +360,12 @@ def dybit_conv2d_requant(desc: ConvDesc, X: torch.Tensor, fx, scale_x: torch.Ten
                                     W.stride(0), _fmt(fq), _ptr(scale_q), int(bool(relu)), _ptr(Q), wp, wn,
                                     _stream(stream)), "dybit_conv2d_requant")
     return Q
+
+
+def dybit_rmse(x: torch.Tensor, fmt, scale: torch.Tensor, out: Optional[torch.Tensor] = None, stream=None):
+    """Eq. 2.  Returns a float64 device tensor {RMSE, sigma, mse, n}."""
+    _dev_f32(x, "x")
+    if out is None:
+        out = torch.empty(4, dtype=torch.float64, device=x.device)
+    _check(lib.dybit_rmse(_ptr(x), x.numel(), _fmt(fmt), _ptr(scale), _ptr(out), _stream(stream)), "dybit_rmse")
+    return out

@@ -382,6 +382,106 @@ decode_kernel(const uint8_t *__restrict__ packed, int64_t n, const float *__rest
     }
 }
 
+// ------------------------------------------------------------------ RMSE (Eq. 2)
+
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// One pass over x: sum of d, d^2 (d = x - x[0], a shift that keeps the variance well conditioned and makes it
+// exactly 0 for a constant tensor) and of e^2, e = x - xhat with xhat the fp32 quantize-dequantize image.
+// acc[0..2] collect the three sums (zero on entry), acc[3] (as an integer) counts finished blocks; the last
+// block replaces them by {RMSE, sigma, mse, n}.
+template <int BITS, bool SIGNED>
+__global__ void __launch_bounds__(kStreamThreads)
+rmse_kernel(const float *__restrict__ x, int64_t n, const float *__restrict__ scale, const __grid_constant__ FloatTable table,
+            double *__restrict__ acc) {
+    __shared__ float s_lut[256];
+    __shared__ double s_part[kWarpsPerBlock][3];
+    pdl_enter();
+    const float sc = __ldg(scale), inv = __ldg(scale + 1);
+    for (int i = threadIdx.x; i < 256; i += blockDim.x) s_lut[i] = __fmul_rn(sc, table.v[i]);
+    __syncthreads();
+    const double shift = (double)__ldg(x);
+    double sd = 0.0, sd2 = 0.0, se2 = 0.0;
+    const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t nthreads = (int64_t)gridDim.x * blockDim.x;
+    int64_t head = ((16 - (reinterpret_cast<uintptr_t>(x) & 15)) & 15) / 4;
+    if (head > n) head = n;
+    const int64_t nvec = (n - head) / 4;
+    const float4 *xv = reinterpret_cast<const float4 *>(x + head);
+    auto one = [&](float v, unsigned code) {
+        const double d = (double)v - shift;
+        sd += d;
+        sd2 = fma(d, d, sd2);
+        const double e = (double)v - (double)s_lut[code];
+        se2 = fma(e, e, se2);
+    };
+    for (int64_t i = tid; i < nvec; i += nthreads) {
+        const float4 v = __ldcs(xv + i);
+        const unsigned c = encode4<BITS, SIGNED>(v, inv);
+        one(v.x, c & 0xffu);
+        one(v.y, (c >> 8) & 0xffu);
+        one(v.z, (c >> 16) & 0xffu);
+        one(v.w, c >> 24);
+    }
+    const int64_t tail0 = head + nvec * 4;
+    for (int64_t i = tid; i < head + (n - tail0); i += nthreads) {
+        const float v = x[i < head ? i : tail0 + (i - head)];
+        const unsigned c = encode4<BITS, SIGNED>(make_float4(v, 0.f, 0.f, 0.f), inv) & 0xffu;
+        one(v, c);
+    }
+    sd = warp_sum(sd);
+    sd2 = warp_sum(sd2);
+    se2 = warp_sum(se2);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) {
+        s_part[warp][0] = sd;
+        s_part[warp][1] = sd2;
+        s_part[warp][2] = se2;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double a = 0.0, b = 0.0, c = 0.0;
+        for (int w = 0; w < kWarpsPerBlock; ++w) {
+            a += s_part[w][0];
+            b += s_part[w][1];
+            c += s_part[w][2];
+        }
+        atomicAdd(acc + 0, a);
+        atomicAdd(acc + 1, b);
+        atomicAdd(acc + 2, c);
+        __threadfence();
+        unsigned long long *ticket = reinterpret_cast<unsigned long long *>(acc + 3);
+        if (atomicAdd(ticket, 1ull) == (unsigned long long)gridDim.x - 1ull) {
+            __threadfence();
+            const double sum_d = atomicAdd(acc + 0, 0.0), sum_d2 = atomicAdd(acc + 1, 0.0), sum_e2 = atomicAdd(acc + 2, 0.0);
+            const double dn = (double)n;
+            double var = (sum_d2 - sum_d * sum_d / dn) / dn;
+            if (var < 0.0) var = 0.0;
+            const double sigma = sqrt(var), mse = sum_e2 / dn;
+            acc[0] = sigma > 0.0 ? sqrt(mse) / sigma : 0.0;
+            acc[1] = sigma;
+            acc[2] = mse;
+            acc[3] = dn;
+        }
+    }
+}
+
+template <int BITS>
+static dybit_status launch_rmse_bits(const float *x, int64_t n, bool is_signed, const float *scale, const FloatTable &t,
+                                     double *out, cudaStream_t s) {
+    int64_t blocks = (n / 4 + kStreamThreads * 4 - 1) / (kStreamThreads * 4);
+    const int64_t cap = (int64_t)sm_count() * 4;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    if (is_signed) launch_k(rmse_kernel<BITS, true>, dim3((unsigned)blocks), dim3(kStreamThreads), 0, s, x, n, scale, t, out);
+    else launch_k(rmse_kernel<BITS, false>, dim3((unsigned)blocks), dim3(kStreamThreads), 0, s, x, n, scale, t, out);
+    return launch_status();
+}
+
 // ------------------------------------------------------------------ host launchers
 
 static int stream_grid(int64_t items_per_warp_unit) {
@@ -532,6 +632,28 @@ dybit_status dybit_decode(const void *packed, int64_t n, dybit_fmt fmt, const fl
         case 6: return launch_decode_bits<6>(p, n, scale, table, out, s);
         case 7: return launch_decode_bits<7>(p, n, scale, table, out, s);
         case 8: return launch_decode_bits<8>(p, n, scale, table, out, s);
+    }
+    return DYBIT_ERR_INVALID_ARG;
+}
+
+dybit_status dybit_rmse(const float *x, int64_t n, dybit_fmt fmt, const float *scale, double *out, void *stream) {
+    using namespace dybit;
+    if (!fmt_ok(fmt) || n < 0 || out == nullptr || scale == nullptr || (n > 0 && x == nullptr)) return DYBIT_ERR_INVALID_ARG;
+    if (!aligned(x, 4) || !aligned(out, 8) || !aligned(scale, 4)) return DYBIT_ERR_ALIGNMENT;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    DYBIT_CUDA_TRY(cudaMemsetAsync(out, 0, 4 * sizeof(double), s));
+    if (n == 0) return DYBIT_OK;                      // {0, 0, 0, 0}
+    FloatTable table;
+    fill_table(fmt, table.v);
+    const bool sg = fmt.is_signed != 0;
+    switch (fmt.bits) {
+        case 2: return launch_rmse_bits<2>(x, n, sg, scale, table, out, s);
+        case 3: return launch_rmse_bits<3>(x, n, sg, scale, table, out, s);
+        case 4: return launch_rmse_bits<4>(x, n, sg, scale, table, out, s);
+        case 5: return launch_rmse_bits<5>(x, n, sg, scale, table, out, s);
+        case 6: return launch_rmse_bits<6>(x, n, sg, scale, table, out, s);
+        case 7: return launch_rmse_bits<7>(x, n, sg, scale, table, out, s);
+        case 8: return launch_rmse_bits<8>(x, n, sg, scale, table, out, s);
     }
     return DYBIT_ERR_INVALID_ARG;
 }
