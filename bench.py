@@ -383,6 +383,7 @@ def run_sweeps(dy, wl, device, peaks):
             out["gemm_sweep"].append({"size": size, "bits": fmt[0], "container": r["container"],
                                       "tops_call": r["tops_call"], "tops_mma_kernel": r["tops_mma_kernel"],
                                       "library_matmul_tops": r.get("library_matmul_tops")})
+    out["bitwidth_search"] = run_search(dy, wl, device)
     layers = wl.resnet50_layers(64)
     bits = wl.mixed_bitwidths(len(layers), seed=0)
     work = LayerwiseStep(dy, wl, device, layers, bits, host_copies=False)
@@ -398,6 +399,45 @@ def run_sweeps(dy, wl, device, peaks):
                                  "containers": {c: conts.count(c) for c in sorted(set(conts))},
                                  "bits_w_a": bits}
     return out
+
+
+def run_search(dy, wl, device, batch=32, alpha=3.0, beta=3.0, top_k=4):
+    """Algorithm 1 on the ResNet-18 shapes with MEASURED per-layer latencies (quantize + conv on this GPU, in place of
+    the paper's accelerator simulator) and Eq. 2 errors (weights' RMSE + activations' RMSE) for a, w in {8, 4, 2}."""
+    layers = wl.resnet18_layers(batch)
+    levels = (8, 4, 2)
+    lat, err = [], []
+    for i, L in enumerate(layers):
+        x = wl.half_normal((L.n, L.h, L.w, L.c), seed=1000 + i, device=device)
+        w = wl.kaiming_normal(L.k, L.r, L.s, L.c, seed=2000 + i).reshape(L.k, -1).to(device)
+        d = dy.ConvDesc(L.n, L.h, L.w, L.c, L.k, L.r, L.s, L.stride, L.pad, 1)
+        y = torch.empty((L.n, L.oh, L.ow, L.k), dtype=torch.float32, device=device)
+        ra = {a: dy.dybit_rmse(x.reshape(-1), (a, 0), dy.dybit_absmax_scale(x, (a, 0)))[0].item() for a in levels}
+        rw = {b: dy.dybit_rmse(w.reshape(-1), (b, 1), dy.dybit_absmax_scale(w, (b, 1)))[0].item() for b in levels}
+        for a in levels:
+            for b in levels:
+                fa, fw = (a, 0), (b, 1)
+                pw, sw = dy.dybit_quantize_pack_2d(w, fw)
+                px = torch.empty(dy.dybit_packed_bytes(x.numel(), a), dtype=torch.uint8, device=device)
+                sx = torch.empty(2, dtype=torch.float32, device=device)
+                ws = torch.empty(dy.dybit_conv2d_workspace_bytes(d, fa, fw) + 1024, dtype=torch.uint8, device=device)
+
+                def layer_call():
+                    dy.dybit_quantize_pack(x, fa, packed=px, scale_out=sx)
+                    dy.dybit_conv2d(d, px, fa, sx, pw, fw, sw, Y=y, ws=ws)
+                lat.append(time_calls(layer_call, 5, warmup=2))
+                err.append(ra[a] + rw[b])
+    n = len(layers)
+    base = sum(lat[i * 9] for i in range(n))
+    res = {"alpha": alpha, "beta": beta, "top_k": top_k, "latency_ms_all_8bit": base}
+    for strategy, c in (("speedup", alpha), ("rmse", beta)):
+        W, A = dy.dybit_search_bitwidths(lat, err, n, strategy, c, top_k)
+        idx = {8: 0, 4: 1, 2: 2}
+        cur = sum(lat[(i * 3 + idx[A[i]]) * 3 + idx[W[i]]] for i in range(n))
+        cur_e = sum(err[(i * 3 + idx[A[i]]) * 3 + idx[W[i]]] for i in range(n))
+        res[strategy] = {"w_bits": W, "a_bits": A, "latency_ms": cur, "speedup": base / cur,
+                         "rmse_ratio": cur_e / sum(err[i * 9] for i in range(n))}
+    return res
 
 
 CONTAINERS = {0: "int8", 1: "e4m3", 2: "bf16"}

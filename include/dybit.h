@@ -199,6 +199,21 @@ dybit_status dybit_conv2d(const dybit_conv_desc *desc,
  *   out   [dev] 4 doubles, 8-byte aligned: {RMSE, sigma, mean squared error, n}; RMSE = 0 when sigma == 0 or n == 0 */
 dybit_status dybit_rmse(const float *x, int64_t n, dybit_fmt fmt, const float *scale, double *out, void *stream);
 
+/* Layer-wise bitwidth search of Algorithm 1 (Section III-C.3) -- host only.  All layers start at (8, 8); each
+ * round ranks the layers that can still be degraded (speedup strategy: the top_k slowest, re-ordered by ascending
+ * RMSE; RMSE strategy: the top_k with the smallest RMSE, re-ordered by descending latency) and degrades first the
+ * weights, then the activations of that list one layer at a time (8 -> 4 -> 2), re-evaluating the total after every
+ * single step, until the constraint is met:
+ *   strategy 0 (speedup, Eq. 3): stop when constraint * sum Lat_i(a, w) <= sum Lat_i(8, 8)        (constraint = alpha)
+ *   strategy 1 (RMSE,    Eq. 4): keep degrading while sum RMSE_i(a, w) <= constraint * sum RMSE_i(8, 8); the step
+ *                                that would exceed the budget is taken back                      (constraint = beta)
+ * or until every layer is at (2, 2).
+ *   lat, rmse  [host] num_layers * 9 doubles, index (layer * 3 + a_idx) * 3 + w_idx with idx 0, 1, 2 <-> 8, 4, 2 bits
+ *              (latencies e.g. measured per layer with dybit_conv2d, errors with dybit_rmse)
+ *   w_bits, a_bits [host] num_layers ints each, receive 8, 4 or 2 */
+dybit_status dybit_search_bitwidths(int num_layers, const double *lat, const double *rmse, int strategy,
+                                    double constraint, int top_k, int *w_bits, int *a_bits);
+
 /* GEMM / convolution with the re-quantizing epilogue of Section III-B.1 ("the FP intermediate results will be
  * quantized to DyBit format before being written back"): instead of fp32, the result leaves the kernel as packed
  * DyBit codes of format fq, ready to be the next layer's activation.  Per output element

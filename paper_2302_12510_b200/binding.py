@@ -21,7 +21,7 @@ __all__ = [
     "dybit_conv2d_out_hw", "dybit_absmax_scale", "dybit_quantize_pack", "dybit_quantize_pack_2d",
     "dybit_decode", "dybit_gemm", "dybit_conv2d", "dybit_last_device_status",
     "dybit_launch_count", "dybit_profile_next_gemm", "dybit_gemm_static_ws", "STATIC_WS_BYTES",
-    "dybit_gemm_requant", "dybit_conv2d_requant", "dybit_rmse",
+    "dybit_gemm_requant", "dybit_conv2d_requant", "dybit_rmse", "dybit_search_bitwidths",
 ]
 
 
@@ -98,6 +98,8 @@ def _load() -> C.CDLL:
     lib.dybit_conv2d_requant.argtypes = [C.POINTER(_CConvDesc), vp, _CFmt, vp, vp, _CFmt, vp, i64,
                                          _CFmt, vp, i32, vp, vp, sz, vp]
     lib.dybit_rmse.argtypes = [vp, i64, _CFmt, vp, vp, vp]
+    lib.dybit_search_bitwidths.argtypes = [i32, C.POINTER(C.c_double), C.POINTER(C.c_double), i32, C.c_double, i32,
+                                           C.POINTER(i32), C.POINTER(i32)]
     lib.dybit_gemm_static_ws.argtypes = [i64, i64, i64, vp, _CFmt, vp, i64, vp, _CFmt, vp, i64, vp, i64, vp, vp]
     return lib
 
@@ -369,3 +371,20 @@ def dybit_rmse(x: torch.Tensor, fmt, scale: torch.Tensor, out: Optional[torch.Te
         out = torch.empty(4, dtype=torch.float64, device=x.device)
     _check(lib.dybit_rmse(_ptr(x), x.numel(), _fmt(fmt), _ptr(scale), _ptr(out), _stream(stream)), "dybit_rmse")
     return out
+
+
+def dybit_search_bitwidths(lat, rmse, num_layers: int, strategy: str, constraint: float, top_k: int):
+    """Algorithm 1.  lat / rmse: flat sequences of num_layers*9 numbers, index (layer*3 + a_idx)*3 + w_idx with
+    idx 0, 1, 2 <-> 8, 4, 2 bits.  strategy "speedup" (constraint = alpha) or "rmse" (constraint = beta).
+    Returns (weight bits, activation bits) as two lists."""
+    if len(lat) != num_layers * 9 or len(rmse) != num_layers * 9:
+        raise ValueError("lat and rmse need num_layers * 9 entries")
+    if strategy not in ("speedup", "rmse"):
+        raise ValueError("strategy must be 'speedup' or 'rmse'")
+    la = (C.c_double * len(lat))(*[float(v) for v in lat])
+    ra = (C.c_double * len(rmse))(*[float(v) for v in rmse])
+    w = (C.c_int * num_layers)()
+    a = (C.c_int * num_layers)()
+    _check(lib.dybit_search_bitwidths(num_layers, la, ra, 0 if strategy == "speedup" else 1, float(constraint),
+                                      int(top_k), w, a), "dybit_search_bitwidths")
+    return list(w), list(a)

@@ -4,7 +4,9 @@
 #include <math.h>
 #include <string.h>
 
+#include <algorithm>
 #include <atomic>
+#include <vector>
 
 #include "dybit_common.cuh"
 
@@ -209,6 +211,80 @@ dybit_status dybit_conv2d_out_hw(const dybit_conv_desc *d, int *oh, int *ow) {
     if (eh < 0 || ew < 0) return DYBIT_ERR_INVALID_ARG;
     if (oh) *oh = eh / d->stride + 1;
     if (ow) *ow = ew / d->stride + 1;
+    return DYBIT_OK;
+}
+
+// Algorithm 1.  Tables are [layer][a][w] with index 0, 1, 2 <-> 8, 4, 2 bits.
+dybit_status dybit_search_bitwidths(int num_layers, const double *lat, const double *rmse, int strategy,
+                                    double constraint, int top_k, int *w_bits, int *a_bits) {
+    if (num_layers <= 0 || !lat || !rmse || !w_bits || !a_bits || top_k <= 0 || (strategy != 0 && strategy != 1) ||
+        !(constraint > 0.0))
+        return DYBIT_ERR_INVALID_ARG;
+    const int n = num_layers;
+    std::vector<int> wl(n, 0), al(n, 0);                       // level index: 0 -> 8 bits, 1 -> 4, 2 -> 2
+    auto at = [&](const double *t, int i) { return t[(i * 3 + al[i]) * 3 + wl[i]]; };
+    auto total = [&](const double *t) {
+        double s = 0.0;
+        for (int i = 0; i < n; ++i) s += at(t, i);
+        return s;
+    };
+    const double *budget = strategy == 0 ? lat : rmse;
+    const double base = total(budget);
+    auto meets = [&]() {
+        const double cur = total(budget);
+        return strategy == 0 ? constraint * cur <= base       // Eq. 3
+                             : cur > constraint * base;       // Eq. 4 budget exhausted
+    };
+    // one pass of Degrade_level over `order`; returns {changed, stop}
+    auto degrade = [&](const std::vector<int> &order, std::vector<int> &level, bool &changed) {
+        for (int i : order) {
+            if (level[i] == 2) continue;
+            level[i] += 1;
+            changed = true;
+            if (strategy == 1 && total(rmse) > constraint * base) {
+                level[i] -= 1;                                 // the step that breaks the Eq. 4 budget is taken back
+                return true;
+            }
+            if (meets()) return true;
+        }
+        return false;
+    };
+    if (!(strategy == 0 && meets())) {
+        for (;;) {
+            std::vector<int> live;
+            for (int i = 0; i < n; ++i)
+                if (wl[i] < 2 || al[i] < 2) live.push_back(i);
+            if (live.empty()) break;
+            std::vector<double> lnow(n), rnow(n);
+            for (int i = 0; i < n; ++i) {
+                lnow[i] = at(lat, i);
+                rnow[i] = at(rmse, i);
+            }
+            std::vector<int> order = live;
+            if (strategy == 0) {
+                std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return lnow[a] > lnow[b]; });
+                if ((int)order.size() > top_k) order.resize(top_k);
+                std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
+                    return rnow[a] < rnow[b] || (rnow[a] == rnow[b] && a < b);
+                });
+            } else {
+                std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return rnow[a] < rnow[b]; });
+                if ((int)order.size() > top_k) order.resize(top_k);
+                std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
+                    return lnow[a] > lnow[b] || (lnow[a] == lnow[b] && a < b);
+                });
+            }
+            bool changed = false;
+            if (degrade(order, wl, changed)) break;
+            if (degrade(order, al, changed)) break;
+            if (!changed) break;
+        }
+    }
+    static const int kBits[3] = {8, 4, 2};
+    for (int i = 0; i < n; ++i) {
+        w_bits[i] = kBits[wl[i]];
+        a_bits[i] = kBits[al[i]];
+    }
     return DYBIT_OK;
 }
 
