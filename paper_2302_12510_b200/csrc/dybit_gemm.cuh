@@ -317,7 +317,28 @@ patch_expand_kernel(const PatchParams p, const __grid_constant__ ElemTable table
                 const int64_t bit = ((((int64_t)img * p.H + ih) * p.W + (iw0 + s_lo)) * p.C) * p.bits;
                 uint8_t *dst = row + ((fr * p.S + s_lo) * p.C) * p.elem;
                 const int count = (s_hi - s_lo) * p.C;
-                // 64-bit window over the stream, refilled one word at a time
+                if ((32 % p.bits) == 0) {
+                    // 2-, 4- and 8-bit codes never straddle a 32-bit word: peel them off word by word
+                    const int per_word = 32 / p.bits;
+                    const int log_pw = p.bits == 2 ? 4 : (p.bits == 4 ? 3 : 2);
+                    int64_t ci = bit >> (5 - log_pw);                 // global code index = bit / bits
+                    int left = count, c = 0;
+                    while (left > 0) {
+                        const int k0 = (int)(ci & (per_word - 1));
+                        const int take = min(per_word - k0, left);
+                        unsigned word = __ldg(w32 + (ci >> log_pw)) >> (k0 * p.bits);
+                        for (int t = 0; t < take; ++t, ++c) {
+                            const unsigned v = s_lut[word & mask];
+                            word >>= p.bits;
+                            if (p.elem == 1) dst[c] = (uint8_t)v;
+                            else reinterpret_cast<uint16_t *>(dst)[c] = (uint16_t)v;
+                        }
+                        ci += take;
+                        left -= take;
+                    }
+                    continue;
+                }
+                // other widths: 64-bit window over the stream, refilled one word at a time
                 int64_t wi = bit >> 5;
                 const int sh = (int)(bit & 31);
                 unsigned long long buf = __ldg(w32 + wi);

@@ -145,12 +145,12 @@ absmax_kernel(const float *__restrict__ x, int64_t rows, int64_t cols, int64_t l
         unsigned b = threadIdx.x < kWarpsPerBlock ? warp_best[threadIdx.x] : 0u;
         b = __reduce_max_sync(0xffffffffu, b);
         if (threadIdx.x == 0) {
-            if (b > *reinterpret_cast<volatile unsigned *>(slot)) atomicMax(slot, b);   // the slot only ever grows
+            if (b != 0u) atomicMax(slot, b);                 // result unused: a fire-and-forget reduction
             __threadfence();
             const unsigned ticket = atomicAdd(slot + 1, 1u);
             if (ticket == gridDim.x - 1) {
                 __threadfence();
-                const float amax = __uint_as_float(atomicMax(slot, 0u));     // the final maximum
+                const float amax = __uint_as_float(atomicMax(slot, 0u));     // the final maximum, read at L2
                 float *scale = reinterpret_cast<float *>(slot);
                 if (amax == 0.0f) {
                     scale[0] = 1.0f;
