@@ -374,6 +374,24 @@ def run_sweeps(dy, wl, device, peaks):
         res = torch.empty(4, dtype=torch.float64, device=device)
         ms = time_calls_flushed(lambda: dy.dybit_rmse(x, (bits, 1), scale, out=res), 7, flush)
         out["rmse"].append({"log2n": 28, "bits": bits, "gbs": (1 << 28) * 4 / ms / 1e6, "rmse": res[0].item()})
+    # the same metric for several candidates in one pass: the 7 signed bitwidths, then 16 scales of one format
+    out["rmse_sweep"] = []
+    fmts7 = [(b, 1) for b in range(2, 9)]
+    sc7 = torch.stack([dy.dybit_absmax_scale(x, f) for f in fmts7]).contiguous()
+    base = dy.dybit_absmax_scale(x, (4, 1))
+    ratios = torch.linspace(1.0, 0.25, 16, device=device)
+    sc16 = torch.stack([base[0] * ratios, 1.0 / (base[0] * ratios)], dim=1).contiguous()
+    for what, fmts, sc in (("bitwidths 2..8 signed", fmts7, sc7), ("16 clipping ratios, 4-bit signed", [(4, 1)] * 16, sc16)):
+        holder = {}
+
+        def call():
+            holder["r"] = dy.dybit_rmse_sweep(x, fmts, sc)
+        ms = time_calls_flushed(call, 5, flush)
+        res, best = holder["r"]
+        out["rmse_sweep"].append({"log2n": 28, "candidates": what, "n_cand": len(fmts), "ms": ms,
+                                  "gbs": (1 << 28) * 4 / ms / 1e6,
+                                  "gelem_cand_per_s": (1 << 28) * len(fmts) / ms / 1e6,
+                                  "best": int(best.item()), "rmse": [float(v) for v in res[:, 0].tolist()]})
     del x
     torch.cuda.empty_cache()
     out["gemm_sweep"] = []

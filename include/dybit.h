@@ -199,6 +199,18 @@ dybit_status dybit_conv2d(const dybit_conv_desc *desc,
  *   out   [dev] 4 doubles, 8-byte aligned: {RMSE, sigma, mean squared error, n}; RMSE = 0 when sigma == 0 or n == 0 */
 dybit_status dybit_rmse(const float *x, int64_t n, dybit_fmt fmt, const float *scale, double *out, void *stream);
 
+/* Eq. 2 for up to DYBIT_RMSE_MAX_CANDIDATES candidate (format, scale) pairs in ONE pass over x: the sweep behind
+ * the choice of a tensor's bitwidth (the RMSE_i table of Algorithm 1) and of its scale (the tensor-level precision
+ * adjustment of Section III-A).  x is read once; every candidate's error is the one dybit_rmse would report.
+ *   fmts   [host] n_cand formats
+ *   scales [dev]  n_cand pairs {scale, 1/scale}, 2 * n_cand floats
+ *   out    [dev]  4 * n_cand doubles, 8-byte aligned: {RMSE, sigma, mse, n} per candidate
+ *   best   [dev]  optional (may be NULL): index of the candidate with the smallest RMSE, lowest index among equals
+ * n == 0 gives all zeros and best = 0.  n_cand outside 1..DYBIT_RMSE_MAX_CANDIDATES -> DYBIT_ERR_INVALID_ARG. */
+#define DYBIT_RMSE_MAX_CANDIDATES 16
+dybit_status dybit_rmse_sweep(const float *x, int64_t n, int n_cand, const dybit_fmt *fmts, const float *scales,
+                              double *out, int *best, void *stream);
+
 /* Layer-wise bitwidth search of Algorithm 1 (Section III-C.3) -- host only.  All layers start at (8, 8); each
  * round ranks the layers that can still be degraded (speedup strategy: the top_k slowest, re-ordered by ascending
  * RMSE; RMSE strategy: the top_k with the smallest RMSE, re-ordered by descending latency) and degrades first the
@@ -214,16 +226,19 @@ dybit_status dybit_rmse(const float *x, int64_t n, dybit_fmt fmt, const float *s
 dybit_status dybit_search_bitwidths(int num_layers, const double *lat, const double *rmse, int strategy,
                                     double constraint, int top_k, int *w_bits, int *a_bits);
 
-/* GEMM / convolution with the re-quantizing epilogue of Section III-B.1 ("the FP intermediate results will be
- * quantized to DyBit format before being written back"): instead of fp32, the result leaves the kernel as packed
- * DyBit codes of format fq, ready to be the next layer's activation.  Per output element
+/* GEMM / convolution with the re-quantizing epilogue of Section III-B.1 (the accelerator encodes its floating-point
+ * intermediate results as DyBit before it writes them to memory): instead of fp32, the result leaves the kernel as
+ * packed DyBit codes of format fq, ready to be the next layer's activation.  Per output element (row m, column j)
  *     y = fmul_rn((float)sum, alpha)            exactly as dybit_gemm / dybit_conv2d compute it
+ *     y = fadd_rn(y, bias[j])                   if bias != NULL (one fp32 per output column / channel, e.g. a
+ *                                               folded batch-norm shift)
  *     y = max(y, 0)                             if relu != 0
  *     code = encode(y, scale_q[1])              the encoder of dybit_quantize_pack (nearest value, ties to even code)
  * and row m of the output (N codes; N = desc->k for the convolution) is written as a dense little-endian bit
  * stream starting at Q + m * ldq_bytes.
  *   scale_q [dev] {scale, 1/scale} of the OUTPUT tensor, given by the caller (e.g. a calibrated or trained scale;
  *           the maximum of the result is not known before it is computed)
+ *   bias    [dev] N floats, 4-byte aligned, or NULL
  *   Q       [dev] M rows of ldq_bytes; ldq_bytes >= N*fq.bits/8 and N*fq.bits a multiple of 8 (rows that start on
  *           4-byte boundaries are written with word stores, others byte by byte).  Only the first N*fq.bits/8 bytes of each row are written: a caller that wants padded
  *           rows (ldq_bytes = dybit_row_stride_bytes(N, fq.bits), to feed dybit_gemm) zero-fills the buffer once.
@@ -233,12 +248,13 @@ dybit_status dybit_search_bitwidths(int num_layers, const double *lat, const dou
 dybit_status dybit_gemm_requant(int64_t M, int64_t N, int64_t K,
                                 const void *A, dybit_fmt fa, const float *scale_a, int64_t lda_bytes,
                                 const void *B, dybit_fmt fb, const float *scale_b, int64_t ldb_bytes,
-                                dybit_fmt fq, const float *scale_q, int relu, void *Q, int64_t ldq_bytes,
+                                dybit_fmt fq, const float *scale_q, const float *bias, int relu, void *Q,
+                                int64_t ldq_bytes,
                                 void *ws, size_t ws_bytes, void *stream);
 dybit_status dybit_conv2d_requant(const dybit_conv_desc *desc,
                                   const void *X, dybit_fmt fx, const float *scale_x,
                                   const void *W, dybit_fmt fw, const float *scale_w, int64_t ldw_bytes,
-                                  dybit_fmt fq, const float *scale_q, int relu, void *Q,
+                                  dybit_fmt fq, const float *scale_q, const float *bias, int relu, void *Q,
                                   void *ws, size_t ws_bytes, void *stream);
 
 /* (No counterpart in the paper.)  dybit_gemm for callers that cannot call

@@ -21,7 +21,7 @@ __all__ = [
     "dybit_conv2d_out_hw", "dybit_absmax_scale", "dybit_quantize_pack", "dybit_quantize_pack_2d",
     "dybit_decode", "dybit_gemm", "dybit_conv2d", "dybit_last_device_status",
     "dybit_launch_count", "dybit_profile_next_gemm", "dybit_gemm_static_ws", "STATIC_WS_BYTES",
-    "dybit_gemm_requant", "dybit_conv2d_requant", "dybit_rmse", "dybit_search_bitwidths",
+    "dybit_gemm_requant", "dybit_conv2d_requant", "dybit_rmse", "dybit_rmse_sweep", "dybit_search_bitwidths",
 ]
 
 
@@ -94,10 +94,11 @@ def _load() -> C.CDLL:
     lib.dybit_launch_count.argtypes = []
     lib.dybit_profile_next_gemm.argtypes = [vp, vp]
     lib.dybit_gemm_requant.argtypes = [i64, i64, i64, vp, _CFmt, vp, i64, vp, _CFmt, vp, i64,
-                                       _CFmt, vp, i32, vp, i64, vp, sz, vp]
+                                       _CFmt, vp, vp, i32, vp, i64, vp, sz, vp]
     lib.dybit_conv2d_requant.argtypes = [C.POINTER(_CConvDesc), vp, _CFmt, vp, vp, _CFmt, vp, i64,
-                                         _CFmt, vp, i32, vp, vp, sz, vp]
+                                         _CFmt, vp, vp, i32, vp, vp, sz, vp]
     lib.dybit_rmse.argtypes = [vp, i64, _CFmt, vp, vp, vp]
+    lib.dybit_rmse_sweep.argtypes = [vp, i64, i32, C.POINTER(_CFmt), vp, vp, vp, vp]
     lib.dybit_search_bitwidths.argtypes = [i32, C.POINTER(C.c_double), C.POINTER(C.c_double), i32, C.c_double, i32,
                                            C.POINTER(i32), C.POINTER(i32)]
     lib.dybit_gemm_static_ws.argtypes = [i64, i64, i64, vp, _CFmt, vp, i64, vp, _CFmt, vp, i64, vp, i64, vp, vp]
@@ -329,9 +330,17 @@ def _ws_ptr(ws: torch.Tensor):
     return C.c_void_p(ws.data_ptr() + off), ws.numel() - off
 
 
+def _bias_ptr(bias, n):
+    if bias is None:
+        return None
+    if not (bias.is_cuda and bias.dtype == torch.float32 and bias.is_contiguous() and bias.numel() == n):
+        raise ValueError("bias must be a contiguous float32 device tensor with one value per output column")
+    return _ptr(bias)
+
+
 def dybit_gemm_requant(M: int, N: int, K: int, A: torch.Tensor, fa, scale_a: torch.Tensor,
                        B: torch.Tensor, fb, scale_b: torch.Tensor, fq, scale_q: torch.Tensor, relu: bool = False,
-                       Q: Optional[torch.Tensor] = None, ldq_bytes: Optional[int] = None,
+                       bias: Optional[torch.Tensor] = None, Q: Optional[torch.Tensor] = None, ldq_bytes: Optional[int] = None,
                        ws: Optional[torch.Tensor] = None, stream=None):
     """GEMM whose result is written as packed DyBit codes of format fq (scale given).  Returns Q [M][ldq] uint8."""
     if ldq_bytes is None:
@@ -342,14 +351,14 @@ def dybit_gemm_requant(M: int, N: int, K: int, A: torch.Tensor, fa, scale_a: tor
         ws = torch.empty(dybit_gemm_workspace_bytes(M, N, K, fa, fb) + 1024, dtype=torch.uint8, device=A.device)
     wp, wn = _ws_ptr(ws)
     _check(lib.dybit_gemm_requant(M, N, K, _ptr(A), _fmt(fa), _ptr(scale_a), A.stride(0), _ptr(B), _fmt(fb),
-                                  _ptr(scale_b), B.stride(0), _fmt(fq), _ptr(scale_q), int(bool(relu)), _ptr(Q),
-                                  ldq_bytes, wp, wn, _stream(stream)), "dybit_gemm_requant")
+                                  _ptr(scale_b), B.stride(0), _fmt(fq), _ptr(scale_q), _bias_ptr(bias, N), int(bool(relu)),
+                                  _ptr(Q), ldq_bytes, wp, wn, _stream(stream)), "dybit_gemm_requant")
     return Q
 
 
 def dybit_conv2d_requant(desc: ConvDesc, X: torch.Tensor, fx, scale_x: torch.Tensor, W: torch.Tensor, fw,
                          scale_w: torch.Tensor, fq, scale_q: torch.Tensor, relu: bool = False,
-                         Q: Optional[torch.Tensor] = None, ws: Optional[torch.Tensor] = None, stream=None):
+                         bias: Optional[torch.Tensor] = None, Q: Optional[torch.Tensor] = None, ws: Optional[torch.Tensor] = None, stream=None):
     """Convolution whose result is the dense NHWK stream of packed codes (the next layer's X).  Returns Q (1-D uint8)."""
     oh, ow = dybit_conv2d_out_hw(desc)
     if Q is None:
@@ -359,7 +368,8 @@ def dybit_conv2d_requant(desc: ConvDesc, X: torch.Tensor, fx, scale_x: torch.Ten
     wp, wn = _ws_ptr(ws)
     cd = _cdesc(desc)
     _check(lib.dybit_conv2d_requant(C.byref(cd), _ptr(X), _fmt(fx), _ptr(scale_x), _ptr(W), _fmt(fw), _ptr(scale_w),
-                                    W.stride(0), _fmt(fq), _ptr(scale_q), int(bool(relu)), _ptr(Q), wp, wn,
+                                    W.stride(0), _fmt(fq), _ptr(scale_q), _bias_ptr(bias, desc.k), int(bool(relu)),
+                                    _ptr(Q), wp, wn,
                                     _stream(stream)), "dybit_conv2d_requant")
     return Q
 
@@ -371,6 +381,22 @@ def dybit_rmse(x: torch.Tensor, fmt, scale: torch.Tensor, out: Optional[torch.Te
         out = torch.empty(4, dtype=torch.float64, device=x.device)
     _check(lib.dybit_rmse(_ptr(x), x.numel(), _fmt(fmt), _ptr(scale), _ptr(out), _stream(stream)), "dybit_rmse")
     return out
+
+
+def dybit_rmse_sweep(x: torch.Tensor, fmts, scales: torch.Tensor, stream=None):
+    """Eq. 2 for several candidate (format, scale) pairs in one pass over x.  scales: float32 device tensor
+    [len(fmts)][2] of {scale, 1/scale}.  Returns (float64 device tensor [len(fmts)][4] of {RMSE, sigma, mse, n},
+    int32 device tensor holding the index of the smallest RMSE)."""
+    _dev_f32(x, "x")
+    nc = len(fmts)
+    if not (scales.is_cuda and scales.dtype == torch.float32 and scales.is_contiguous() and scales.numel() == 2 * nc):
+        raise ValueError("scales must be a contiguous float32 device tensor with two values per candidate")
+    arr = (_CFmt * max(nc, 1))(*[_fmt(f) for f in fmts])
+    out = torch.empty((nc, 4), dtype=torch.float64, device=x.device)
+    best = torch.empty(1, dtype=torch.int32, device=x.device)
+    _check(lib.dybit_rmse_sweep(_ptr(x), x.numel(), nc, arr, _ptr(scales), _ptr(out), _ptr(best), _stream(stream)),
+           "dybit_rmse_sweep")
+    return out, best
 
 
 def dybit_search_bitwidths(lat, rmse, num_layers: int, strategy: str, constraint: float, top_k: int):

@@ -469,6 +469,7 @@ struct GemmParams {
     int64_t ldq;
     const float *scale_q;     // {scale, 1/scale} of the output tensor
     int q_bits, q_signed, relu;
+    const float *bias;        // requant only: one fp32 per output column, or null
 };
 
 // Waits for the phase with the given parity; gives up after kWaitLimitNs, records
@@ -751,6 +752,12 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 }
                 if (p.Q) {
                     if (row < p.M) {
+                        if (p.bias) {
+                            // every lane reads the same 32 floats: one broadcast transaction each
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (col0 + j < p.N) f[j] = __fadd_rn(f[j], __ldg(p.bias + col0 + j));
+                        }
                         if (p.relu) {
 #pragma unroll
                             for (int j = 0; j < 32; ++j) f[j] = fmaxf(f[j], 0.0f);
@@ -1047,6 +1054,7 @@ static inline int64_t k_row_bytes(int64_t k_elems, int elem) { return round_up(k
 struct RequantSpec {
     dybit_fmt fq;
     const float *scale_q;
+    const float *bias;
     int relu;
     void *Q;
     int64_t ldq;
@@ -1056,7 +1064,7 @@ static dybit_status check_requant(const RequantSpec *rq, int64_t N) {
     if (rq == nullptr) return DYBIT_OK;
     if (!fmt_ok(rq->fq) || rq->Q == nullptr || rq->scale_q == nullptr) return DYBIT_ERR_INVALID_ARG;
     if ((N * rq->fq.bits) % 8 != 0 || rq->ldq < N * rq->fq.bits / 8) return DYBIT_ERR_INVALID_ARG;
-    if (!aligned(rq->scale_q, 4)) return DYBIT_ERR_ALIGNMENT;
+    if (!aligned(rq->scale_q, 4) || !aligned(rq->bias, 4)) return DYBIT_ERR_ALIGNMENT;
     return DYBIT_OK;
 }
 
@@ -1068,6 +1076,7 @@ static void apply_requant(GemmParams &p, const RequantSpec *rq) {
     p.q_bits = rq->fq.bits;
     p.q_signed = rq->fq.is_signed;
     p.relu = rq->relu;
+    p.bias = rq->bias;
 }
 
 // How a convolution is lowered, and what it needs in the workspace.
@@ -1360,18 +1369,19 @@ dybit_status dybit_conv2d(const dybit_conv_desc *d, const void *X, dybit_fmt fx,
 
 dybit_status dybit_gemm_requant(int64_t M, int64_t N, int64_t K, const void *A, dybit_fmt fa, const float *scale_a,
                                 int64_t lda_bytes, const void *B, dybit_fmt fb, const float *scale_b,
-                                int64_t ldb_bytes, dybit_fmt fq, const float *scale_q, int relu, void *Q,
+                                int64_t ldb_bytes, dybit_fmt fq, const float *scale_q, const float *bias, int relu, void *Q,
                                 int64_t ldq_bytes, void *ws, size_t ws_bytes, void *stream) {
-    const dybit::RequantSpec rq = {fq, scale_q, relu ? 1 : 0, Q, ldq_bytes};
+    const dybit::RequantSpec rq = {fq, scale_q, bias, relu ? 1 : 0, Q, ldq_bytes};
     return dybit::gemm_impl(M, N, K, A, fa, scale_a, lda_bytes, B, fb, scale_b, ldb_bytes, nullptr, 0, nullptr, &rq, ws,
                             ws_bytes, stream);
 }
 
 dybit_status dybit_conv2d_requant(const dybit_conv_desc *d, const void *X, dybit_fmt fx, const float *scale_x,
                                   const void *W, dybit_fmt fw, const float *scale_w, int64_t ldw_bytes, dybit_fmt fq,
-                                  const float *scale_q, int relu, void *Q, void *ws, size_t ws_bytes, void *stream) {
+                                  const float *scale_q, const float *bias, int relu, void *Q, void *ws,
+                                  size_t ws_bytes, void *stream) {
     if (d == nullptr) return DYBIT_ERR_INVALID_ARG;
-    const dybit::RequantSpec rq = {fq, scale_q, relu ? 1 : 0, Q, (int64_t)d->k * fq.bits / 8};
+    const dybit::RequantSpec rq = {fq, scale_q, bias, relu ? 1 : 0, Q, (int64_t)d->k * fq.bits / 8};
     return dybit::conv_impl(d, X, fx, scale_x, W, fw, scale_w, ldw_bytes, nullptr, nullptr, &rq, ws, ws_bytes, stream);
 }
 

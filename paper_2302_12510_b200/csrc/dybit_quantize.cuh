@@ -482,6 +482,190 @@ static dybit_status launch_rmse_bits(const float *x, int64_t n, bool is_signed, 
     return launch_status();
 }
 
+// ------------------------------------------------------------------ RMSE of several candidates in one pass
+
+constexpr int kSweepMaxCand = 16;
+constexpr int kSweepUnroll = 4;
+
+// Candidate formats and the magnitude tables they decode with: the table for m magnitude bits (2^m floats)
+// starts at mags[2^m - 2]; a signed code carries its sign in bit m.
+struct SweepParams {
+    int n_cand;
+    unsigned char bits[kSweepMaxCand];
+    unsigned char sgn[kSweepMaxCand];
+    float mags[512];
+};
+
+// Sum of squared errors of U float4 groups under one candidate.
+template <int BITS, bool SIGNED, int U>
+__device__ __forceinline__ double sweep_sq_err(const float4 (&v)[U], const float *__restrict__ lut, float inv) {
+    double s = 0.0;
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const unsigned c = encode4<BITS, SIGNED>(v[u], inv);
+        const double e0 = (double)v[u].x - (double)lut[c & 0xffu];
+        const double e1 = (double)v[u].y - (double)lut[(c >> 8) & 0xffu];
+        const double e2 = (double)v[u].z - (double)lut[(c >> 16) & 0xffu];
+        const double e3 = (double)v[u].w - (double)lut[c >> 24];
+        s = fma(e0, e0, s);
+        s = fma(e1, e1, s);
+        s = fma(e2, e2, s);
+        s = fma(e3, e3, s);
+    }
+    return s;
+}
+
+template <int U>
+__device__ __forceinline__ double sweep_dispatch(int bits, int sgn, const float4 (&v)[U], const float *lut, float inv) {
+    switch (bits * 2 + sgn) {
+        case 4: return sweep_sq_err<2, false, U>(v, lut, inv);
+        case 5: return sweep_sq_err<2, true, U>(v, lut, inv);
+        case 6: return sweep_sq_err<3, false, U>(v, lut, inv);
+        case 7: return sweep_sq_err<3, true, U>(v, lut, inv);
+        case 8: return sweep_sq_err<4, false, U>(v, lut, inv);
+        case 9: return sweep_sq_err<4, true, U>(v, lut, inv);
+        case 10: return sweep_sq_err<5, false, U>(v, lut, inv);
+        case 11: return sweep_sq_err<5, true, U>(v, lut, inv);
+        case 12: return sweep_sq_err<6, false, U>(v, lut, inv);
+        case 13: return sweep_sq_err<6, true, U>(v, lut, inv);
+        case 14: return sweep_sq_err<7, false, U>(v, lut, inv);
+        case 15: return sweep_sq_err<7, true, U>(v, lut, inv);
+        case 16: return sweep_sq_err<8, false, U>(v, lut, inv);
+        default: return sweep_sq_err<8, true, U>(v, lut, inv);
+    }
+}
+
+// One pass over x for n_cand candidate (format, scale) pairs: x is read once, every candidate's squared error is
+// accumulated per thread in shared memory.  acc holds 4 doubles per candidate, zero on entry; while the kernel
+// runs acc[0], acc[1] collect the sums of d and d^2 (d = x - x[0]), acc[4c + 2] candidate c's squared error and
+// acc[3] (as an integer) the finished blocks.  The last block replaces them by {RMSE, sigma, mse, n} per
+// candidate and writes the index of the smallest RMSE (lowest index among equals) to *best if that is given.
+// Dynamic shared memory: n_cand * (256 floats + blockDim doubles).
+__global__ void __launch_bounds__(kStreamThreads)
+rmse_sweep_kernel(const float *__restrict__ x, int64_t n, const float *__restrict__ scales,
+                  const __grid_constant__ SweepParams sp, double *__restrict__ acc, int *__restrict__ best) {
+    extern __shared__ __align__(16) unsigned char sweep_smem[];
+    double *s_acc = reinterpret_cast<double *>(sweep_smem);                                  // [n_cand][blockDim]
+    float *s_lut = reinterpret_cast<float *>(sweep_smem + (size_t)sp.n_cand * kStreamThreads * 8);   // [n_cand][256]
+    __shared__ double s_part[kWarpsPerBlock][2];
+    __shared__ float s_inv[kSweepMaxCand];
+    pdl_enter();
+    const int nc = sp.n_cand;
+    for (int i = threadIdx.x; i < nc * 256; i += blockDim.x) {
+        const int c = i >> 8, code = i & 255;
+        const int m = sp.bits[c] - sp.sgn[c];
+        const float mag = __fmul_rn(__ldg(scales + 2 * c), sp.mags[(1 << m) - 2 + (code & ((1 << m) - 1))]);
+        const bool valid = code < (1 << sp.bits[c]);
+        s_lut[i] = valid ? ((sp.sgn[c] && ((code >> m) & 1)) ? -mag : mag) : 0.0f;
+    }
+    for (int c = 0; c < nc; ++c) s_acc[c * kStreamThreads + threadIdx.x] = 0.0;
+    if (threadIdx.x < nc) s_inv[threadIdx.x] = __ldg(scales + 2 * threadIdx.x + 1);
+    __syncthreads();
+    const double shift = (double)__ldg(x);
+    double sd = 0.0, sd2 = 0.0;
+    const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t nthreads = (int64_t)gridDim.x * blockDim.x;
+    int64_t head = ((16 - (reinterpret_cast<uintptr_t>(x) & 15)) & 15) / 4;
+    if (head > n) head = n;
+    const int64_t nvec = (n - head) / 4;
+    const float4 *xv = reinterpret_cast<const float4 *>(x + head);
+    auto moments = [&](float v) {
+        const double d = (double)v - shift;
+        sd += d;
+        sd2 = fma(d, d, sd2);
+    };
+    int64_t i = tid;
+    for (; i + (kSweepUnroll - 1) * nthreads < nvec; i += kSweepUnroll * nthreads) {
+        float4 v[kSweepUnroll];
+#pragma unroll
+        for (int u = 0; u < kSweepUnroll; ++u) v[u] = __ldcs(xv + i + u * nthreads);
+#pragma unroll
+        for (int u = 0; u < kSweepUnroll; ++u) {
+            moments(v[u].x);
+            moments(v[u].y);
+            moments(v[u].z);
+            moments(v[u].w);
+        }
+#pragma unroll 1
+        for (int c = 0; c < nc; ++c)
+            s_acc[c * kStreamThreads + threadIdx.x] += sweep_dispatch<kSweepUnroll>(sp.bits[c], sp.sgn[c], v, s_lut + c * 256, s_inv[c]);
+    }
+    for (; i < nvec; i += nthreads) {
+        float4 v[1] = {__ldcs(xv + i)};
+        moments(v[0].x);
+        moments(v[0].y);
+        moments(v[0].z);
+        moments(v[0].w);
+#pragma unroll 1
+        for (int c = 0; c < nc; ++c)
+            s_acc[c * kStreamThreads + threadIdx.x] += sweep_dispatch<1>(sp.bits[c], sp.sgn[c], v, s_lut + c * 256, s_inv[c]);
+    }
+    // the few elements before the first and after the last aligned group of four, one per thread
+    const int64_t tail0 = head + nvec * 4;
+    for (int64_t k = tid; k < head + (n - tail0); k += nthreads) {
+        const float e = x[k < head ? k : tail0 + (k - head)];
+        moments(e);
+        // padded with zeros, which every format represents exactly: they add no error
+        float4 v[1] = {make_float4(e, 0.0f, 0.0f, 0.0f)};
+#pragma unroll 1
+        for (int c = 0; c < nc; ++c)
+            s_acc[c * kStreamThreads + threadIdx.x] += sweep_dispatch<1>(sp.bits[c], sp.sgn[c], v, s_lut + c * 256, s_inv[c]);
+    }
+    sd = warp_sum(sd);
+    sd2 = warp_sum(sd2);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) {
+        s_part[warp][0] = sd;
+        s_part[warp][1] = sd2;
+    }
+    __syncthreads();
+    // warp w adds up the candidates w, w + 8, ...
+    for (int c = warp; c < nc; c += kWarpsPerBlock) {
+        double t = 0.0;
+        for (int k = lane; k < kStreamThreads; k += 32) t += s_acc[c * kStreamThreads + k];
+        t = warp_sum(t);
+        if (lane == 0) {
+            atomicAdd(acc + 4 * c + 2, t);
+            __threadfence();
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double a = 0.0, b = 0.0;
+        for (int w = 0; w < kWarpsPerBlock; ++w) {
+            a += s_part[w][0];
+            b += s_part[w][1];
+        }
+        atomicAdd(acc + 0, a);
+        atomicAdd(acc + 1, b);
+        __threadfence();
+        unsigned long long *ticket = reinterpret_cast<unsigned long long *>(acc + 3);
+        if (atomicAdd(ticket, 1ull) == (unsigned long long)gridDim.x - 1ull) {
+            __threadfence();
+            const double sum_d = atomicAdd(acc + 0, 0.0), sum_d2 = atomicAdd(acc + 1, 0.0);
+            const double dn = (double)n;
+            double var = (sum_d2 - sum_d * sum_d / dn) / dn;
+            if (var < 0.0) var = 0.0;
+            const double sigma = sqrt(var);
+            int arg = 0;
+            double lowest = 0.0;
+            for (int c = 0; c < nc; ++c) {
+                const double mse = atomicAdd(acc + 4 * c + 2, 0.0) / dn;
+                const double r = sigma > 0.0 ? sqrt(mse) / sigma : 0.0;
+                acc[4 * c + 0] = r;
+                acc[4 * c + 1] = sigma;
+                acc[4 * c + 2] = mse;
+                acc[4 * c + 3] = dn;
+                if (c == 0 || r < lowest) {
+                    lowest = r;
+                    arg = c;
+                }
+            }
+            if (best) *best = arg;
+        }
+    }
+}
+
 // ------------------------------------------------------------------ host launchers
 
 static int stream_grid(int64_t items_per_warp_unit) {
@@ -658,4 +842,49 @@ dybit_status dybit_rmse(const float *x, int64_t n, dybit_fmt fmt, const float *s
     return DYBIT_ERR_INVALID_ARG;
 }
 
+dybit_status dybit_rmse_sweep(const float *x, int64_t n, int n_cand, const dybit_fmt *fmts, const float *scales,
+                              double *out, int *best, void *stream) {
+    using namespace dybit;
+    if (n_cand < 1 || n_cand > kSweepMaxCand || fmts == nullptr || n < 0 || out == nullptr || scales == nullptr ||
+        (n > 0 && x == nullptr))
+        return DYBIT_ERR_INVALID_ARG;
+    for (int c = 0; c < n_cand; ++c)
+        if (!fmt_ok(fmts[c])) return DYBIT_ERR_INVALID_ARG;
+    if (!aligned(x, 4) || !aligned(out, 8) || !aligned(scales, 4) || !aligned(best, 4)) return DYBIT_ERR_ALIGNMENT;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    DYBIT_CUDA_TRY(cudaMemsetAsync(out, 0, (size_t)n_cand * 4 * sizeof(double), s));
+    if (best) DYBIT_CUDA_TRY(cudaMemsetAsync(best, 0, sizeof(int), s));
+    if (n == 0) return DYBIT_OK;
+    SweepParams sp = {};
+    sp.n_cand = n_cand;
+    for (int c = 0; c < n_cand; ++c) {
+        sp.bits[c] = (unsigned char)fmts[c].bits;
+        sp.sgn[c] = fmts[c].is_signed ? 1 : 0;
+    }
+    // magnitude tables: m = 1..7 are the non-negative half of the signed (m+1)-bit format, m = 8 is unsigned 8-bit
+    float full[256];
+    for (int m = 1; m <= 8; ++m) {
+        const dybit_fmt f = {m == 8 ? 8 : m + 1, m == 8 ? 0 : 1};
+        fill_table(f, full);
+        for (int k = 0; k < (1 << m); ++k) sp.mags[(1 << m) - 2 + k] = full[k];
+    }
+    const size_t smem = (size_t)n_cand * (256 * sizeof(float) + kStreamThreads * sizeof(double));
+    static bool configured[64] = {};
+    int dev = 0;
+    DYBIT_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return DYBIT_ERR_CUDA;
+    if (!configured[dev]) {
+        DYBIT_CUDA_TRY(cudaFuncSetAttribute(rmse_sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            kSweepMaxCand * (256 * 4 + kStreamThreads * 8)));
+        configured[dev] = true;
+    }
+    int64_t blocks = (n / 4 + kStreamThreads * kSweepUnroll - 1) / (kStreamThreads * kSweepUnroll);
+    const int64_t cap = (int64_t)sm_count() * 4;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    launch_k(rmse_sweep_kernel, dim3((unsigned)blocks), dim3(kStreamThreads), smem, s, x, n, scales, sp, out, best);
+    return launch_status();
+}
+
 }  // extern "C"
+

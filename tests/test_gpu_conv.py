@@ -74,6 +74,8 @@ def test_mixed_bitwidths_small_conv(fx, fw):
     wl.ConvLayer("c20_pad_channels", 2, 8, 8, 20, 24, 3, 3, 1, 1),
     wl.ConvLayer("fc_like", 5, 1, 1, 512, 1000, 1, 1, 1, 0),
     wl.ConvLayer("one_pixel", 1, 1, 1, 16, 1, 1, 1, 1, 0),
+    wl.ConvLayer("gather_long_k_c48_7x7", 2, 12, 12, 48, 40, 7, 7, 1, 3),
+    wl.ConvLayer("gather_long_k_c128_small_image", 1, 10, 10, 128, 64, 3, 3, 2, 1),
 ], ids=lambda L: L.name)
 def test_edge_geometries(shape):
     assert run_conv(shape, (4, 0), (4, 1), seed=3) == 0

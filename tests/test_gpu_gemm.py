@@ -89,6 +89,27 @@ def test_bf16_container_within_tolerance(fa, fb):
     assert check_gemm(260, 300, 700, fa, fb, seed=fa[0] * 8 + fb[0]) == 2
 
 
+# Few output tiles and a long K: the contraction is cut into ranges that separate CTAs accumulate and the
+# last one to finish adds up (2 to 8 ranges, the last one shorter, every container, ragged M / N / K).
+@pytest.mark.parametrize("M,N,K,fa,fb,cont", [
+    (130, 70, 1100, (4, 1), (4, 1), 0),
+    (64, 1000, 4096, (4, 0), (4, 1), 0),
+    (257, 300, 5003, (3, 1), (5, 1), 0),
+    (1, 1, 3000, (2, 1), (4, 0), 0),
+    (700, 129, 2500, (4, 1), (2, 1), 0),
+    (260, 300, 3000, (5, 0), (4, 1), 1),
+    (100, 520, 1500, (8, 1), (8, 1), 2),
+    (500, 64, 2111, (6, 0), (7, 1), 2),
+])
+def test_split_k_small_outputs_long_k(M, N, K, fa, fb, cont):
+    assert check_gemm(M, N, K, fa, fb, seed=M + N + K) == cont
+
+
+def test_split_k_twice_in_a_row_reuses_the_tile_counters():
+    for seed in (1, 2, 3):
+        assert check_gemm(256, 256, 2048, (4, 1), (4, 1), seed=seed) == 0
+
+
 def test_many_tiles_persistent_schedule():
     # more tiles than SMs with ragged edges in every dimension: each CTA runs several tiles
     assert check_gemm(128 * 13 + 5, 256 * 12 + 9, 256 + 3, (4, 1), (4, 0), seed=7) == 0

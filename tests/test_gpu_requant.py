@@ -28,7 +28,8 @@ def _expect(y_ref, fq, inv_q, relu):
     return np.stack([orc.pack(r, fq[0])[: y.shape[1] * fq[0] // 8] for r in codes])
 
 
-@pytest.mark.parametrize("M,N,K", [(128, 256, 128), (300, 520, 400), (777, 64, 1153), (64, 1000, 512), (5, 8, 77)])
+@pytest.mark.parametrize("M,N,K", [(128, 256, 128), (300, 520, 400), (777, 64, 1153), (64, 1000, 512), (5, 8, 77),
+                                   (200, 264, 3100)])
 @pytest.mark.parametrize("fq,relu", [((4, 0), True), ((4, 1), False), ((8, 1), False), ((2, 0), True), ((3, 1), False),
                                      ((6, 0), True)])
 def test_gemm_requant_int8_container_bit_exact(M, N, K, fq, relu):
@@ -123,6 +124,55 @@ def test_conv_requant_chains_into_the_next_conv(layer):
     S2, y2 = orc.conv2d(q_codes, fq, sq[0], cw2, fw, spw2[0])
     assert np.array_equal(Y2_raw.cpu().numpy().astype(np.int64), S2)
     assert np.array_equal(Y2.cpu().numpy(), y2)
+
+
+@pytest.mark.parametrize("M,N,K,fq,relu", [(300, 520, 400, (4, 0), True), (130, 72, 1153, (4, 1), False),
+                                          (64, 1000, 512, (8, 1), False), (200, 264, 200, (3, 0), True)])
+def test_gemm_requant_bias_is_added_in_fp32_before_relu(M, N, K, fq, relu):
+    fa, fb = (4, 0), (4, 1)
+    a = wl.half_normal((M, K), seed=M + K)
+    b = wl.normal((N, K), seed=N + K, std=0.05)
+    pa, sa, ca, spa = _quant(a, fa)
+    pb, sb, cb, spb = _quant(b, fb)
+    _, y_ref = orc.gemm(ca, fa, spa[0], cb, fb, spb[0])
+    # biases of the size of the outputs, both signs, so that they flip codes and the ReLU decision
+    bias = (wl.normal((N,), seed=N, std=float(np.abs(y_ref).mean()))).numpy().astype(np.float32)
+    y_b = (y_ref.astype(np.float32) + bias[None, :]).astype(np.float32)
+    sq = orc.absmax_scale(y_b * 0.9, fq[0], bool(fq[1]))
+    scale_q = torch.tensor([float(sq[0]), float(sq[1])], dtype=torch.float32, device=DEV)
+    Q = dy.dybit_gemm_requant(M, N, K, pa, fa, sa, pb, fb, sb, fq, scale_q, relu=relu,
+                              bias=torch.from_numpy(bias).to(DEV))
+    torch.cuda.synchronize()
+    assert dy.dybit_last_device_status() == (0, 0)
+    assert np.array_equal(Q.cpu().numpy(), _expect(y_b, fq, sq[1], relu))
+    # and the bias does change the result
+    Q0 = dy.dybit_gemm_requant(M, N, K, pa, fa, sa, pb, fb, sb, fq, scale_q, relu=relu)
+    assert not np.array_equal(Q.cpu().numpy(), Q0.cpu().numpy())
+
+
+def test_conv_requant_bias_per_output_channel():
+    fx, fw, fq = (4, 0), (4, 1), (4, 0)
+    L = wl.ConvLayer("c64_3x3", 4, 28, 28, 64, 72, 3, 3, 1, 1)
+    x = wl.half_normal((L.n, L.h, L.w, L.c), seed=17)
+    w = wl.kaiming_normal(L.k, L.r, L.s, L.c, seed=18)
+    px, sx = dy.dybit_quantize_pack(x.to(DEV), fx)
+    pw, sw = dy.dybit_quantize_pack_2d(w.reshape(L.k, -1).to(DEV), fw)
+    spx = orc.absmax_scale(x.numpy(), 4, False)
+    spw = orc.absmax_scale(w.numpy(), 4, True)
+    cx = orc.quantize(x.numpy(), 4, False, spx[1])
+    cw = orc.quantize(w.numpy(), 4, True, spw[1])
+    _, y = orc.conv2d(cx, fx, spx[0], cw, fw, spw[0], stride=L.stride, pad=L.pad)
+    bias = wl.normal((L.k,), seed=19, std=float(np.abs(y).mean())).numpy().astype(np.float32)
+    y_b = (y.astype(np.float32) + bias.reshape(1, 1, 1, -1)).astype(np.float32)
+    sq = orc.absmax_scale(np.maximum(y_b, 0) * 0.95, 4, False)
+    scale_q = torch.tensor([float(sq[0]), float(sq[1])], dtype=torch.float32, device=DEV)
+    desc = dy.ConvDesc(L.n, L.h, L.w, L.c, L.k, L.r, L.s, L.stride, L.pad, 1)
+    Q = dy.dybit_conv2d_requant(desc, px, fx, sx, pw, fw, sw, fq, scale_q, relu=True,
+                                bias=torch.from_numpy(bias).to(DEV))
+    torch.cuda.synchronize()
+    assert dy.dybit_last_device_status() == (0, 0)
+    q_codes = orc.quantize(np.maximum(y_b, 0), 4, False, sq[1])
+    assert np.array_equal(Q.cpu().numpy(), orc.pack(q_codes, 4))
 
 
 def test_requant_argument_errors():
