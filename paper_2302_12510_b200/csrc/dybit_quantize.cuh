@@ -390,6 +390,18 @@ __device__ __forceinline__ double warp_sum(double v) {
     return v;
 }
 
+// Squared error of one element, added to s.  Only the magnitude code is needed: a signed format is symmetric, so
+// |x| is compared with the magnitude's value; an unsigned one sends negative inputs to code 0.  lut[m] is the
+// fp32 product scale * value(m), widened to double once per block.
+template <int BITS, bool SIGNED>
+__device__ __forceinline__ double sq_err_acc(float v, double dv, const double *__restrict__ lut, float inv, double s) {
+    constexpr int M = SIGNED ? BITS - 1 : BITS;
+    const float a = SIGNED ? fabsf(v) : fmaxf(v, 0.0f);
+    const unsigned m = magnitude_code_biased<M>(a, inv) & 0xffu;
+    const double e = (SIGNED ? fabs(dv) : dv) - lut[m];
+    return fma(e, e, s);
+}
+
 // One pass over x: sum of d, d^2 (d = x - x[0], a shift that keeps the variance well conditioned and makes it
 // exactly 0 for a constant tensor) and of e^2, e = x - xhat with xhat the fp32 quantize-dequantize image.
 // acc[0..2] collect the three sums (zero on entry), acc[3] (as an integer) counts finished blocks; the last
@@ -398,11 +410,12 @@ template <int BITS, bool SIGNED>
 __global__ void __launch_bounds__(kStreamThreads)
 rmse_kernel(const float *__restrict__ x, int64_t n, const float *__restrict__ scale, const __grid_constant__ FloatTable table,
             double *__restrict__ acc) {
-    __shared__ float s_lut[256];
+    __shared__ double s_lut[256];
     __shared__ double s_part[kWarpsPerBlock][3];
     pdl_enter();
     const float sc = __ldg(scale), inv = __ldg(scale + 1);
-    for (int i = threadIdx.x; i < 256; i += blockDim.x) s_lut[i] = __fmul_rn(sc, table.v[i]);
+    // the first 2^M entries of either kind of table are the magnitudes
+    for (int i = threadIdx.x; i < 256; i += blockDim.x) s_lut[i] = (double)__fmul_rn(sc, fabsf(table.v[i]));
     __syncthreads();
     const double shift = (double)__ldg(x);
     double sd = 0.0, sd2 = 0.0, se2 = 0.0;
@@ -412,27 +425,36 @@ rmse_kernel(const float *__restrict__ x, int64_t n, const float *__restrict__ sc
     if (head > n) head = n;
     const int64_t nvec = (n - head) / 4;
     const float4 *xv = reinterpret_cast<const float4 *>(x + head);
-    auto one = [&](float v, unsigned code) {
-        const double d = (double)v - shift;
+    auto one = [&](float v) {
+        const double dv = (double)v;
+        const double d = dv - shift;
         sd += d;
         sd2 = fma(d, d, sd2);
-        const double e = (double)v - (double)s_lut[code];
-        se2 = fma(e, e, se2);
+        se2 = sq_err_acc<BITS, SIGNED>(v, dv, s_lut, inv, se2);
     };
-    for (int64_t i = tid; i < nvec; i += nthreads) {
+    constexpr int kUnroll = 4;                        // loads in flight per thread
+    int64_t i = tid;
+    for (; i + (kUnroll - 1) * nthreads < nvec; i += kUnroll * nthreads) {
+        float4 v[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) v[u] = __ldcs(xv + i + u * nthreads);
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            one(v[u].x);
+            one(v[u].y);
+            one(v[u].z);
+            one(v[u].w);
+        }
+    }
+    for (; i < nvec; i += nthreads) {
         const float4 v = __ldcs(xv + i);
-        const unsigned c = encode4<BITS, SIGNED>(v, inv);
-        one(v.x, c & 0xffu);
-        one(v.y, (c >> 8) & 0xffu);
-        one(v.z, (c >> 16) & 0xffu);
-        one(v.w, c >> 24);
+        one(v.x);
+        one(v.y);
+        one(v.z);
+        one(v.w);
     }
     const int64_t tail0 = head + nvec * 4;
-    for (int64_t i = tid; i < head + (n - tail0); i += nthreads) {
-        const float v = x[i < head ? i : tail0 + (i - head)];
-        const unsigned c = encode4<BITS, SIGNED>(make_float4(v, 0.f, 0.f, 0.f), inv) & 0xffu;
-        one(v, c);
-    }
+    for (int64_t k = tid; k < head + (n - tail0); k += nthreads) one(x[k < head ? k : tail0 + (k - head)]);
     sd = warp_sum(sd);
     sd2 = warp_sum(sd2);
     se2 = warp_sum(se2);
@@ -496,42 +518,39 @@ struct SweepParams {
     float mags[512];
 };
 
-// Sum of squared errors of U float4 groups under one candidate.
+// Sum of squared errors of U float4 groups (and their widened copies) under one candidate.
 template <int BITS, bool SIGNED, int U>
-__device__ __forceinline__ double sweep_sq_err(const float4 (&v)[U], const float *__restrict__ lut, float inv) {
+__device__ __forceinline__ double sweep_sq_err(const float4 (&v)[U], const double (&dv)[U][4], const double *__restrict__ lut,
+                                               float inv) {
     double s = 0.0;
 #pragma unroll
     for (int u = 0; u < U; ++u) {
-        const unsigned c = encode4<BITS, SIGNED>(v[u], inv);
-        const double e0 = (double)v[u].x - (double)lut[c & 0xffu];
-        const double e1 = (double)v[u].y - (double)lut[(c >> 8) & 0xffu];
-        const double e2 = (double)v[u].z - (double)lut[(c >> 16) & 0xffu];
-        const double e3 = (double)v[u].w - (double)lut[c >> 24];
-        s = fma(e0, e0, s);
-        s = fma(e1, e1, s);
-        s = fma(e2, e2, s);
-        s = fma(e3, e3, s);
+        s = sq_err_acc<BITS, SIGNED>(v[u].x, dv[u][0], lut, inv, s);
+        s = sq_err_acc<BITS, SIGNED>(v[u].y, dv[u][1], lut, inv, s);
+        s = sq_err_acc<BITS, SIGNED>(v[u].z, dv[u][2], lut, inv, s);
+        s = sq_err_acc<BITS, SIGNED>(v[u].w, dv[u][3], lut, inv, s);
     }
     return s;
 }
 
 template <int U>
-__device__ __forceinline__ double sweep_dispatch(int bits, int sgn, const float4 (&v)[U], const float *lut, float inv) {
+__device__ __forceinline__ double sweep_dispatch(int bits, int sgn, const float4 (&v)[U], const double (&dv)[U][4],
+                                                 const double *lut, float inv) {
     switch (bits * 2 + sgn) {
-        case 4: return sweep_sq_err<2, false, U>(v, lut, inv);
-        case 5: return sweep_sq_err<2, true, U>(v, lut, inv);
-        case 6: return sweep_sq_err<3, false, U>(v, lut, inv);
-        case 7: return sweep_sq_err<3, true, U>(v, lut, inv);
-        case 8: return sweep_sq_err<4, false, U>(v, lut, inv);
-        case 9: return sweep_sq_err<4, true, U>(v, lut, inv);
-        case 10: return sweep_sq_err<5, false, U>(v, lut, inv);
-        case 11: return sweep_sq_err<5, true, U>(v, lut, inv);
-        case 12: return sweep_sq_err<6, false, U>(v, lut, inv);
-        case 13: return sweep_sq_err<6, true, U>(v, lut, inv);
-        case 14: return sweep_sq_err<7, false, U>(v, lut, inv);
-        case 15: return sweep_sq_err<7, true, U>(v, lut, inv);
-        case 16: return sweep_sq_err<8, false, U>(v, lut, inv);
-        default: return sweep_sq_err<8, true, U>(v, lut, inv);
+        case 4: return sweep_sq_err<2, false, U>(v, dv, lut, inv);
+        case 5: return sweep_sq_err<2, true, U>(v, dv, lut, inv);
+        case 6: return sweep_sq_err<3, false, U>(v, dv, lut, inv);
+        case 7: return sweep_sq_err<3, true, U>(v, dv, lut, inv);
+        case 8: return sweep_sq_err<4, false, U>(v, dv, lut, inv);
+        case 9: return sweep_sq_err<4, true, U>(v, dv, lut, inv);
+        case 10: return sweep_sq_err<5, false, U>(v, dv, lut, inv);
+        case 11: return sweep_sq_err<5, true, U>(v, dv, lut, inv);
+        case 12: return sweep_sq_err<6, false, U>(v, dv, lut, inv);
+        case 13: return sweep_sq_err<6, true, U>(v, dv, lut, inv);
+        case 14: return sweep_sq_err<7, false, U>(v, dv, lut, inv);
+        case 15: return sweep_sq_err<7, true, U>(v, dv, lut, inv);
+        case 16: return sweep_sq_err<8, false, U>(v, dv, lut, inv);
+        default: return sweep_sq_err<8, true, U>(v, dv, lut, inv);
     }
 }
 
@@ -540,13 +559,13 @@ __device__ __forceinline__ double sweep_dispatch(int bits, int sgn, const float4
 // runs acc[0], acc[1] collect the sums of d and d^2 (d = x - x[0]), acc[4c + 2] candidate c's squared error and
 // acc[3] (as an integer) the finished blocks.  The last block replaces them by {RMSE, sigma, mse, n} per
 // candidate and writes the index of the smallest RMSE (lowest index among equals) to *best if that is given.
-// Dynamic shared memory: n_cand * (256 floats + blockDim doubles).
+// Dynamic shared memory: n_cand * (256 + blockDim) doubles.
 __global__ void __launch_bounds__(kStreamThreads)
 rmse_sweep_kernel(const float *__restrict__ x, int64_t n, const float *__restrict__ scales,
                   const __grid_constant__ SweepParams sp, double *__restrict__ acc, int *__restrict__ best) {
     extern __shared__ __align__(16) unsigned char sweep_smem[];
     double *s_acc = reinterpret_cast<double *>(sweep_smem);                                  // [n_cand][blockDim]
-    float *s_lut = reinterpret_cast<float *>(sweep_smem + (size_t)sp.n_cand * kStreamThreads * 8);   // [n_cand][256]
+    double *s_lut = s_acc + (size_t)sp.n_cand * kStreamThreads;                              // [n_cand][256] magnitudes
     __shared__ double s_part[kWarpsPerBlock][2];
     __shared__ float s_inv[kSweepMaxCand];
     pdl_enter();
@@ -554,9 +573,7 @@ rmse_sweep_kernel(const float *__restrict__ x, int64_t n, const float *__restric
     for (int i = threadIdx.x; i < nc * 256; i += blockDim.x) {
         const int c = i >> 8, code = i & 255;
         const int m = sp.bits[c] - sp.sgn[c];
-        const float mag = __fmul_rn(__ldg(scales + 2 * c), sp.mags[(1 << m) - 2 + (code & ((1 << m) - 1))]);
-        const bool valid = code < (1 << sp.bits[c]);
-        s_lut[i] = valid ? ((sp.sgn[c] && ((code >> m) & 1)) ? -mag : mag) : 0.0f;
+        s_lut[i] = code < (1 << m) ? (double)__fmul_rn(__ldg(scales + 2 * c), sp.mags[(1 << m) - 2 + code]) : 0.0;
     }
     for (int c = 0; c < nc; ++c) s_acc[c * kStreamThreads + threadIdx.x] = 0.0;
     if (threadIdx.x < nc) s_inv[threadIdx.x] = __ldg(scales + 2 * threadIdx.x + 1);
@@ -570,46 +587,50 @@ rmse_sweep_kernel(const float *__restrict__ x, int64_t n, const float *__restric
     const int64_t nvec = (n - head) / 4;
     const float4 *xv = reinterpret_cast<const float4 *>(x + head);
     auto moments = [&](float v) {
-        const double d = (double)v - shift;
+        const double dv = (double)v;
+        const double d = dv - shift;
         sd += d;
         sd2 = fma(d, d, sd2);
+        return dv;
     };
     int64_t i = tid;
     for (; i + (kSweepUnroll - 1) * nthreads < nvec; i += kSweepUnroll * nthreads) {
         float4 v[kSweepUnroll];
 #pragma unroll
         for (int u = 0; u < kSweepUnroll; ++u) v[u] = __ldcs(xv + i + u * nthreads);
+        double dv[kSweepUnroll][4];
 #pragma unroll
         for (int u = 0; u < kSweepUnroll; ++u) {
-            moments(v[u].x);
-            moments(v[u].y);
-            moments(v[u].z);
-            moments(v[u].w);
+            dv[u][0] = moments(v[u].x);
+            dv[u][1] = moments(v[u].y);
+            dv[u][2] = moments(v[u].z);
+            dv[u][3] = moments(v[u].w);
         }
 #pragma unroll 1
         for (int c = 0; c < nc; ++c)
-            s_acc[c * kStreamThreads + threadIdx.x] += sweep_dispatch<kSweepUnroll>(sp.bits[c], sp.sgn[c], v, s_lut + c * 256, s_inv[c]);
+            s_acc[c * kStreamThreads + threadIdx.x] += sweep_dispatch<kSweepUnroll>(sp.bits[c], sp.sgn[c], v, dv, s_lut + c * 256, s_inv[c]);
     }
     for (; i < nvec; i += nthreads) {
         float4 v[1] = {__ldcs(xv + i)};
-        moments(v[0].x);
-        moments(v[0].y);
-        moments(v[0].z);
-        moments(v[0].w);
+        double dv[1][4];
+        dv[0][0] = moments(v[0].x);
+        dv[0][1] = moments(v[0].y);
+        dv[0][2] = moments(v[0].z);
+        dv[0][3] = moments(v[0].w);
 #pragma unroll 1
         for (int c = 0; c < nc; ++c)
-            s_acc[c * kStreamThreads + threadIdx.x] += sweep_dispatch<1>(sp.bits[c], sp.sgn[c], v, s_lut + c * 256, s_inv[c]);
+            s_acc[c * kStreamThreads + threadIdx.x] += sweep_dispatch<1>(sp.bits[c], sp.sgn[c], v, dv, s_lut + c * 256, s_inv[c]);
     }
     // the few elements before the first and after the last aligned group of four, one per thread
     const int64_t tail0 = head + nvec * 4;
     for (int64_t k = tid; k < head + (n - tail0); k += nthreads) {
         const float e = x[k < head ? k : tail0 + (k - head)];
-        moments(e);
         // padded with zeros, which every format represents exactly: they add no error
         float4 v[1] = {make_float4(e, 0.0f, 0.0f, 0.0f)};
+        const double dv[1][4] = {{moments(e), 0.0, 0.0, 0.0}};
 #pragma unroll 1
         for (int c = 0; c < nc; ++c)
-            s_acc[c * kStreamThreads + threadIdx.x] += sweep_dispatch<1>(sp.bits[c], sp.sgn[c], v, s_lut + c * 256, s_inv[c]);
+            s_acc[c * kStreamThreads + threadIdx.x] += sweep_dispatch<1>(sp.bits[c], sp.sgn[c], v, dv, s_lut + c * 256, s_inv[c]);
     }
     sd = warp_sum(sd);
     sd2 = warp_sum(sd2);
@@ -868,14 +889,14 @@ dybit_status dybit_rmse_sweep(const float *x, int64_t n, int n_cand, const dybit
         fill_table(f, full);
         for (int k = 0; k < (1 << m); ++k) sp.mags[(1 << m) - 2 + k] = full[k];
     }
-    const size_t smem = (size_t)n_cand * (256 * sizeof(float) + kStreamThreads * sizeof(double));
+    const size_t smem = (size_t)n_cand * (256 + kStreamThreads) * sizeof(double);
     static bool configured[64] = {};
     int dev = 0;
     DYBIT_CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64) return DYBIT_ERR_CUDA;
     if (!configured[dev]) {
         DYBIT_CUDA_TRY(cudaFuncSetAttribute(rmse_sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            kSweepMaxCand * (256 * 4 + kStreamThreads * 8)));
+                                            kSweepMaxCand * (256 + kStreamThreads) * 8));
         configured[dev] = true;
     }
     int64_t blocks = (n / 4 + kStreamThreads * kSweepUnroll - 1) / (kStreamThreads * kSweepUnroll);
