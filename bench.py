@@ -392,7 +392,19 @@ def run_sweeps(dy, wl, device, peaks):
                                   "gbs": (1 << 28) * 4 / ms / 1e6,
                                   "gelem_cand_per_s": (1 << 28) * len(fmts) / ms / 1e6,
                                   "best": int(best.item()), "rmse": [float(v) for v in res[:, 0].tolist()]})
-    del x
+    # QAT pair: quantize-dequantize image (8 B/element) and its clipped straight-through gradient (12 B/element)
+    out["fake_quant"] = []
+    y = torch.empty_like(x)
+    for fmt in ((4, 1), (8, 1), (2, 0)):
+        scale = dy.dybit_absmax_scale(x, fmt)
+        ms = time_calls_flushed(lambda: dy.dybit_fake_quant(x, fmt, scale, out=y), 5, flush)
+        out["fake_quant"].append({"log2n": 28, "fmt": list(fmt), "direction": "forward", "ms": ms,
+                                  "gbs": (1 << 28) * 8 / ms / 1e6})
+    g = torch.empty_like(x).normal_()
+    ms = time_calls_flushed(lambda: dy.dybit_fake_quant_backward(x, g, (4, 1), scale, out=y), 5, flush)
+    out["fake_quant"].append({"log2n": 28, "fmt": [4, 1], "direction": "backward", "ms": ms,
+                              "gbs": (1 << 28) * 12 / ms / 1e6})
+    del x, y, g
     torch.cuda.empty_cache()
     out["gemm_sweep"] = []
     for fmt in ((4, 1), (8, 1)):

@@ -211,6 +211,20 @@ dybit_status dybit_rmse(const float *x, int64_t n, dybit_fmt fmt, const float *s
 dybit_status dybit_rmse_sweep(const float *x, int64_t n, int n_cand, const dybit_fmt *fmts, const float *scales,
                               double *out, int *best, void *stream);
 
+/* Fake quantization, the forward of quantization-aware training (Section IV-A fine-tunes the quantized models for
+ * a few epochs; the paper does not spell the operator out, this is the usual one): the fp32 image of x under the
+ * format, y_i = fmul_rn(scale[0], value(encode(x_i, scale[1]))), i.e. dybit_decode(dybit_quantize_pack(x)) in one
+ * streaming pass that never stores the codes.  NaN -> 0, as in the encoder.
+ *   x, y [dev] n floats (y may be x);  scale [dev] {scale, 1/scale} */
+dybit_status dybit_fake_quant(const float *x, int64_t n, dybit_fmt fmt, const float *scale, float *y, void *stream);
+
+/* Backward of dybit_fake_quant by the straight-through estimator with clipping (a reading: the paper trains with
+ * QAT but gives no gradient rule): gx_i = gy_i where lo <= x_i <= hi, else 0, with hi = fmul_rn(scale[0], 2^(m-1))
+ * the largest representable value (m magnitude bits) and lo = -hi for a signed format, 0 for an unsigned one.
+ * NaN in x gives 0.   x, gy, gx [dev] n floats (gx may be gy) */
+dybit_status dybit_fake_quant_backward(const float *x, const float *gy, int64_t n, dybit_fmt fmt, const float *scale,
+                                       float *gx, void *stream);
+
 /* Layer-wise bitwidth search of Algorithm 1 (Section III-C.3) -- host only.  All layers start at (8, 8); each
  * round ranks the layers that can still be degraded (speedup strategy: the top_k slowest, re-ordered by ascending
  * RMSE; RMSE strategy: the top_k with the smallest RMSE, re-ordered by descending latency) and degrades first the

@@ -255,3 +255,24 @@ def rmse(x, bits: int, is_signed: bool, scale_pair):
     _load().orc_rmse(_p(x), x.size, bits, int(is_signed), float(np.float32(scale_pair[0])),
                      float(np.float32(scale_pair[1])), _p(out))
     return float(out[0]), float(out[1]), float(out[2])
+
+
+def fake_quant(x, bits: int, is_signed: bool, scale_pair) -> np.ndarray:
+    """QAT forward: the fp32 image of x under the format, decode(encode(x)) with {scale, inv}."""
+    x = _f32(x)
+    codes = quantize(x, bits, is_signed, scale_pair[1])
+    return dequantize(codes, bits, is_signed, scale_pair[0]).reshape(x.shape)
+
+
+def fake_quant_backward(x, grad_out, bits: int, is_signed: bool, scale_pair) -> np.ndarray:
+    """Straight-through estimator with clipping: the gradient passes where x lies inside the closed range the
+    format covers under this scale, [-hi, hi] (signed) or [0, hi] (unsigned), hi = fl32(scale * 2^(m-1)) by Eq. 1."""
+    x, g = _f32(x), _f32(grad_out)
+    m = bits - (1 if is_signed else 0)
+    hi = np.float32(scale_pair[0]) * np.float32(2.0 ** (m - 1))
+    lo = -hi if is_signed else np.float32(0.0)
+    out = np.zeros(x.shape, dtype=np.float32)
+    for i in np.ndindex(x.shape):
+        if lo <= x[i] <= hi:          # NaN compares false: no gradient
+            out[i] = g[i]
+    return out

@@ -21,7 +21,8 @@ __all__ = [
     "dybit_conv2d_out_hw", "dybit_absmax_scale", "dybit_quantize_pack", "dybit_quantize_pack_2d",
     "dybit_decode", "dybit_gemm", "dybit_conv2d", "dybit_last_device_status",
     "dybit_launch_count", "dybit_profile_next_gemm", "dybit_gemm_static_ws", "STATIC_WS_BYTES",
-    "dybit_gemm_requant", "dybit_conv2d_requant", "dybit_rmse", "dybit_rmse_sweep", "dybit_search_bitwidths",
+    "dybit_gemm_requant", "dybit_conv2d_requant", "dybit_rmse", "dybit_rmse_sweep", "dybit_fake_quant", "dybit_fake_quant_backward",
+    "dybit_search_bitwidths",
 ]
 
 
@@ -99,6 +100,8 @@ def _load() -> C.CDLL:
                                          _CFmt, vp, vp, i32, vp, vp, sz, vp]
     lib.dybit_rmse.argtypes = [vp, i64, _CFmt, vp, vp, vp]
     lib.dybit_rmse_sweep.argtypes = [vp, i64, i32, C.POINTER(_CFmt), vp, vp, vp, vp]
+    lib.dybit_fake_quant.argtypes = [vp, i64, _CFmt, vp, vp, vp]
+    lib.dybit_fake_quant_backward.argtypes = [vp, vp, i64, _CFmt, vp, vp, vp]
     lib.dybit_search_bitwidths.argtypes = [i32, C.POINTER(C.c_double), C.POINTER(C.c_double), i32, C.c_double, i32,
                                            C.POINTER(i32), C.POINTER(i32)]
     lib.dybit_gemm_static_ws.argtypes = [i64, i64, i64, vp, _CFmt, vp, i64, vp, _CFmt, vp, i64, vp, i64, vp, vp]
@@ -397,6 +400,32 @@ def dybit_rmse_sweep(x: torch.Tensor, fmts, scales: torch.Tensor, stream=None):
     _check(lib.dybit_rmse_sweep(_ptr(x), x.numel(), nc, arr, _ptr(scales), _ptr(out), _ptr(best), _stream(stream)),
            "dybit_rmse_sweep")
     return out, best
+
+
+def dybit_fake_quant(x: torch.Tensor, fmt, scale: torch.Tensor, out: Optional[torch.Tensor] = None, stream=None):
+    """Quantize-dequantize image of x (QAT forward) in one pass; returns a float32 tensor shaped like x."""
+    _dev_f32(x, "x")
+    if out is None:
+        out = torch.empty_like(x)
+    _dev_f32(out, "out")
+    _check(lib.dybit_fake_quant(_ptr(x), x.numel(), _fmt(fmt), _ptr(scale), _ptr(out), _stream(stream)),
+           "dybit_fake_quant")
+    return out
+
+
+def dybit_fake_quant_backward(x: torch.Tensor, grad_out: torch.Tensor, fmt, scale: torch.Tensor,
+                              out: Optional[torch.Tensor] = None, stream=None):
+    """Clipped straight-through gradient of dybit_fake_quant with respect to x."""
+    _dev_f32(x, "x")
+    _dev_f32(grad_out, "grad_out")
+    if grad_out.numel() != x.numel():
+        raise ValueError("grad_out must have as many elements as x")
+    if out is None:
+        out = torch.empty_like(x)
+    _dev_f32(out, "out")
+    _check(lib.dybit_fake_quant_backward(_ptr(x), _ptr(grad_out), x.numel(), _fmt(fmt), _ptr(scale), _ptr(out),
+                                         _stream(stream)), "dybit_fake_quant_backward")
+    return out
 
 
 def dybit_search_bitwidths(lat, rmse, num_layers: int, strategy: str, constraint: float, top_k: int):

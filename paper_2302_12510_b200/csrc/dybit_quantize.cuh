@@ -687,6 +687,125 @@ rmse_sweep_kernel(const float *__restrict__ x, int64_t n, const float *__restric
     }
 }
 
+// ------------------------------------------------------------------ fake quantization (QAT forward / backward)
+
+// y = scale * value(encode(x)): the quantize-dequantize image in one streaming pass, codes never stored.
+// lut[m] = fmul_rn(scale, value(m)) for the magnitude codes; a signed format mirrors them.
+template <int BITS, bool SIGNED>
+__device__ __forceinline__ float fake_quant_one(float v, const float *__restrict__ lut, float inv) {
+    constexpr int M = SIGNED ? BITS - 1 : BITS;
+    // fmaxf(., 0) maps NaN to 0, as the encoder does
+    const float a = SIGNED ? fmaxf(fabsf(v), 0.0f) : fmaxf(v, 0.0f);
+    const unsigned m = magnitude_code_biased<M>(a, inv) & 0xffu;
+    const float q = lut[m];
+    // a zero magnitude carries no sign (the encoder never emits "minus zero")
+    return (SIGNED && m != 0u) ? copysignf(q, v) : q;
+}
+
+template <int BITS, bool SIGNED>
+__global__ void __launch_bounds__(kStreamThreads)
+fake_quant_kernel(const float *__restrict__ x, int64_t n, const float *__restrict__ scale,
+                  const __grid_constant__ FloatTable table, float *__restrict__ y) {
+    __shared__ float s_lut[256];
+    pdl_enter();
+    const float sc = __ldg(scale), inv = __ldg(scale + 1);
+    for (int i = threadIdx.x; i < 256; i += blockDim.x) s_lut[i] = __fmul_rn(sc, fabsf(table.v[i]));
+    __syncthreads();
+    const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t nthreads = (int64_t)gridDim.x * blockDim.x;
+    // vector body only when x and y share their 16-byte phase
+    const bool same_phase = ((reinterpret_cast<uintptr_t>(x) ^ reinterpret_cast<uintptr_t>(y)) & 15) == 0;
+    int64_t head = same_phase ? ((16 - (reinterpret_cast<uintptr_t>(x) & 15)) & 15) / 4 : n;
+    if (head > n) head = n;
+    const int64_t nvec = (n - head) / 4;
+    const float4 *xv = reinterpret_cast<const float4 *>(x + head);
+    float4 *yv = reinterpret_cast<float4 *>(y + head);
+    constexpr int kUnroll = 4;
+    int64_t i = tid;
+    for (; i + (kUnroll - 1) * nthreads < nvec; i += kUnroll * nthreads) {
+        float4 v[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) v[u] = __ldcs(xv + i + u * nthreads);
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            float4 r;
+            r.x = fake_quant_one<BITS, SIGNED>(v[u].x, s_lut, inv);
+            r.y = fake_quant_one<BITS, SIGNED>(v[u].y, s_lut, inv);
+            r.z = fake_quant_one<BITS, SIGNED>(v[u].z, s_lut, inv);
+            r.w = fake_quant_one<BITS, SIGNED>(v[u].w, s_lut, inv);
+            __stcs(yv + i + u * nthreads, r);
+        }
+    }
+    for (; i < nvec; i += nthreads) {
+        const float4 v = __ldcs(xv + i);
+        float4 r;
+        r.x = fake_quant_one<BITS, SIGNED>(v.x, s_lut, inv);
+        r.y = fake_quant_one<BITS, SIGNED>(v.y, s_lut, inv);
+        r.z = fake_quant_one<BITS, SIGNED>(v.z, s_lut, inv);
+        r.w = fake_quant_one<BITS, SIGNED>(v.w, s_lut, inv);
+        __stcs(yv + i, r);
+    }
+    const int64_t tail0 = head + nvec * 4;
+    for (int64_t k = tid; k < head + (n - tail0); k += nthreads) {
+        const int64_t j = k < head ? k : tail0 + (k - head);
+        y[j] = fake_quant_one<BITS, SIGNED>(x[j], s_lut, inv);
+    }
+}
+
+// Straight-through backward with clipping: the gradient passes where x lies inside [lo, hi], the range the format
+// covers under this scale (lo = -hi for a signed format, 0 for an unsigned one; hi = scale * 2^(m-1)), else 0.
+__global__ void __launch_bounds__(kStreamThreads)
+fake_quant_backward_kernel(const float *__restrict__ x, const float *__restrict__ gy, int64_t n,
+                           const float *__restrict__ scale, float top, int is_signed, float *__restrict__ gx) {
+    pdl_enter();
+    const float hi = __fmul_rn(__ldg(scale), top), lo = is_signed ? -hi : 0.0f;
+    const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t nthreads = (int64_t)gridDim.x * blockDim.x;
+    const uintptr_t px = reinterpret_cast<uintptr_t>(x), pg = reinterpret_cast<uintptr_t>(gy), po = reinterpret_cast<uintptr_t>(gx);
+    const bool same_phase = (((px ^ pg) | (px ^ po)) & 15) == 0;
+    int64_t head = same_phase ? ((16 - (px & 15)) & 15) / 4 : n;
+    if (head > n) head = n;
+    const int64_t nvec = (n - head) / 4;
+    const float4 *xv = reinterpret_cast<const float4 *>(x + head);
+    const float4 *gv = reinterpret_cast<const float4 *>(gy + head);
+    float4 *ov = reinterpret_cast<float4 *>(gx + head);
+    auto pass = [&](float v, float g) { return (v >= lo && v <= hi) ? g : 0.0f; };
+    constexpr int kUnroll = 2;
+    int64_t i = tid;
+    for (; i + (kUnroll - 1) * nthreads < nvec; i += kUnroll * nthreads) {
+        float4 v[kUnroll], g[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            v[u] = __ldcs(xv + i + u * nthreads);
+            g[u] = __ldcs(gv + i + u * nthreads);
+        }
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u)
+            __stcs(ov + i + u * nthreads, make_float4(pass(v[u].x, g[u].x), pass(v[u].y, g[u].y), pass(v[u].z, g[u].z), pass(v[u].w, g[u].w)));
+    }
+    for (; i < nvec; i += nthreads) {
+        const float4 v = __ldcs(xv + i), g = __ldcs(gv + i);
+        __stcs(ov + i, make_float4(pass(v.x, g.x), pass(v.y, g.y), pass(v.z, g.z), pass(v.w, g.w)));
+    }
+    const int64_t tail0 = head + nvec * 4;
+    for (int64_t k = tid; k < head + (n - tail0); k += nthreads) {
+        const int64_t j = k < head ? k : tail0 + (k - head);
+        gx[j] = pass(x[j], gy[j]);
+    }
+}
+
+template <int BITS>
+static dybit_status launch_fake_quant_bits(const float *x, int64_t n, bool is_signed, const float *scale, const FloatTable &t,
+                                           float *y, cudaStream_t s) {
+    int64_t blocks = (n / 4 + kStreamThreads * 4 - 1) / (kStreamThreads * 4);
+    const int64_t cap = (int64_t)sm_count() * 6;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    if (is_signed) launch_k(fake_quant_kernel<BITS, true>, dim3((unsigned)blocks), dim3(kStreamThreads), 0, s, x, n, scale, t, y);
+    else launch_k(fake_quant_kernel<BITS, false>, dim3((unsigned)blocks), dim3(kStreamThreads), 0, s, x, n, scale, t, y);
+    return launch_status();
+}
+
 // ------------------------------------------------------------------ host launchers
 
 static int stream_grid(int64_t items_per_warp_unit) {
@@ -907,5 +1026,45 @@ dybit_status dybit_rmse_sweep(const float *x, int64_t n, int n_cand, const dybit
     return launch_status();
 }
 
+dybit_status dybit_fake_quant(const float *x, int64_t n, dybit_fmt fmt, const float *scale, float *y, void *stream) {
+    using namespace dybit;
+    if (!fmt_ok(fmt) || n < 0 || scale == nullptr || (n > 0 && (x == nullptr || y == nullptr))) return DYBIT_ERR_INVALID_ARG;
+    if (!aligned(x, 4) || !aligned(y, 4) || !aligned(scale, 4)) return DYBIT_ERR_ALIGNMENT;
+    if (n == 0) return DYBIT_OK;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    FloatTable table;
+    fill_table(fmt, table.v);
+    const bool sg = fmt.is_signed != 0;
+    switch (fmt.bits) {
+        case 2: return launch_fake_quant_bits<2>(x, n, sg, scale, table, y, s);
+        case 3: return launch_fake_quant_bits<3>(x, n, sg, scale, table, y, s);
+        case 4: return launch_fake_quant_bits<4>(x, n, sg, scale, table, y, s);
+        case 5: return launch_fake_quant_bits<5>(x, n, sg, scale, table, y, s);
+        case 6: return launch_fake_quant_bits<6>(x, n, sg, scale, table, y, s);
+        case 7: return launch_fake_quant_bits<7>(x, n, sg, scale, table, y, s);
+        case 8: return launch_fake_quant_bits<8>(x, n, sg, scale, table, y, s);
+    }
+    return DYBIT_ERR_INVALID_ARG;
+}
+
+dybit_status dybit_fake_quant_backward(const float *x, const float *gy, int64_t n, dybit_fmt fmt, const float *scale,
+                                       float *gx, void *stream) {
+    using namespace dybit;
+    if (!fmt_ok(fmt) || n < 0 || scale == nullptr || (n > 0 && (x == nullptr || gy == nullptr || gx == nullptr)))
+        return DYBIT_ERR_INVALID_ARG;
+    if (!aligned(x, 4) || !aligned(gy, 4) || !aligned(gx, 4) || !aligned(scale, 4)) return DYBIT_ERR_ALIGNMENT;
+    if (n == 0) return DYBIT_OK;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int64_t blocks = (n / 4 + kStreamThreads * 2 - 1) / (kStreamThreads * 2);
+    const int64_t cap = (int64_t)sm_count() * 8;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    const float top = ldexpf(1.0f, fmt.bits - (fmt.is_signed ? 1 : 0) - 1);      // Eq. 1: the largest value is 2^(m-1)
+    launch_k(fake_quant_backward_kernel, dim3((unsigned)blocks), dim3(kStreamThreads), 0, s, x, gy, n, scale, top,
+             fmt.is_signed ? 1 : 0, gx);
+    return launch_status();
+}
+
 }  // extern "C"
+
 
