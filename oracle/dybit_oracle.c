@@ -415,6 +415,49 @@ void orc_conv2d_sampled(int n, int h, int w, int c, int k, int r, int s,
     }
 }
 
+/* Depth-wise convolution (the 3x3 layers of MobileNetV2, one of the models of
+ * Section IV-A): every channel is filtered by its own r x s kernel, no sum
+ * across channels.  X: [n][h][w][c] codes; W: [c][r][s] codes; Y: [n][oh][ow][c].
+ * S is the exact integer sum over the taps, Y = (float)S * alpha as in the
+ * dense layers. */
+void orc_depthwise_conv2d(int n, int h, int w, int c, int r, int s,
+                          int stride, int pad, int dilation,
+                          const uint8_t *X, int bits_x, int signed_x, float scale_x,
+                          const uint8_t *W, int bits_w, int signed_w, float scale_w,
+                          int64_t *S, float *Y)
+{
+    int oh = (h + 2 * pad - dilation * (r - 1) - 1) / stride + 1;
+    int ow = (w + 2 * pad - dilation * (s - 1) - 1) / stride + 1;
+    float alpha = orc_alpha(scale_x, bits_x, signed_x, scale_w, bits_w, signed_w);
+    int64_t tx[256], tw[256];
+    int_table(bits_x, signed_x, tx);
+    int_table(bits_w, signed_w, tw);
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int in = 0; in < n; ++in) {
+        for (int io = 0; io < oh; ++io) {
+            for (int jo = 0; jo < ow; ++jo) {
+                for (int ic = 0; ic < c; ++ic) {
+                    int64_t acc = 0;
+                    for (int ir = 0; ir < r; ++ir) {
+                        int ih = io * stride - pad + ir * dilation;
+                        if (ih < 0 || ih >= h) continue;
+                        for (int is = 0; is < s; ++is) {
+                            int iw = jo * stride - pad + is * dilation;
+                            if (iw < 0 || iw >= w) continue;
+                            unsigned cx = X[(((int64_t)in * h + ih) * w + iw) * c + ic];
+                            unsigned cw = W[((int64_t)ic * r + ir) * s + is];
+                            acc += tx[cx] * tw[cw];
+                        }
+                    }
+                    int64_t o = (((int64_t)in * oh + io) * ow + jo) * c + ic;
+                    if (S) S[o] = acc;
+                    if (Y) Y[o] = (float)acc * alpha;
+                }
+            }
+        }
+    }
+}
+
 /* ------------------------------------------------------------------ */
 /* Quantization error metric, Eq. 2 (Section III-C.1)                  */
 /* ------------------------------------------------------------------ */

@@ -63,6 +63,7 @@ def _load():
                                          vp, vp, i64, vp, vp]
         lib.orc_conv2d.argtypes = [i32] * 10 + [vp, i32, i32, f32, vp, i32, i32, f32, vp, vp]
         lib.orc_rmse.argtypes = [vp, i64, i32, i32, f32, f32, vp]
+        lib.orc_depthwise_conv2d.argtypes = [i32] * 9 + [vp, i32, i32, f32, vp, i32, i32, f32, vp, vp]
         lib.orc_conv2d_sampled.argtypes = [i32] * 10 + [vp, i32, i32, f32, f32, vp, i32, i32, f32, vp, i64, vp, vp]
         _lib = lib
     return _lib
@@ -224,6 +225,22 @@ def conv2d(codes_x, fmt_x, scale_x, codes_w, fmt_w, scale_w, stride=1, pad=0, di
                        _p(x), fmt_x[0], int(fmt_x[1]), float(np.float32(scale_x)),
                        _p(wt), fmt_w[0], int(fmt_w[1]), float(np.float32(scale_w)),
                        _p(acc), _p(y))
+    return acc, y
+
+
+def depthwise_conv2d(codes_x, fmt_x, scale_x, codes_w, fmt_w, scale_w, stride=1, pad=0, dilation=1):
+    """codes_x: [n][h][w][c]; codes_w: [c][r][s] (one filter per channel) -> (S int64, Y fp32) [n][oh][ow][c]."""
+    x, wt = _u8(codes_x), _u8(codes_w)
+    n, h, w, c = x.shape
+    c2, r, s = wt.shape
+    assert c2 == c
+    oh, ow = conv_out_hw(h, w, r, s, stride, pad, dilation)
+    acc = np.zeros((n, oh, ow, c), dtype=np.int64)
+    y = np.zeros((n, oh, ow, c), dtype=np.float32)
+    _load().orc_depthwise_conv2d(n, h, w, c, r, s, stride, pad, dilation,
+                                 _p(x), fmt_x[0], int(fmt_x[1]), float(np.float32(scale_x)),
+                                 _p(wt), fmt_w[0], int(fmt_w[1]), float(np.float32(scale_w)),
+                                 _p(acc), _p(y))
     return acc, y
 
 
