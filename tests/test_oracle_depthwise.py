@@ -62,4 +62,7 @@ def test_hand_worked_single_channel():
     _, y = orc.depthwise_conv2d(x, (4, False), 2.0, k, (4, True), 0.5, stride=2)
     assert y.reshape(-1).tolist() == [0.5, -0.5]
     _, y = orc.depthwise_conv2d(x, (4, False), 1.0, k, (4, True), 1.0, pad=1)   # zero padding on both sides
-    assert y.reshape(-1).tolist() == [1.0, 0.5, 0.5, -0.5, -1.5]
+    # the padding also adds a row above and below the 1 x 4 image: those output rows see zeros only
+    assert y.shape == (1, 3, 5, 1)
+    assert y[0, 1, :, 0].tolist() == [1.0, 0.5, 0.5, -0.5, -1.5]
+    assert not y[0, 0].any() and not y[0, 2].any()
