@@ -191,6 +191,22 @@ dybit_status dybit_conv2d(const dybit_conv_desc *desc,
                           float *Y, int32_t *Y_raw,
                           void *ws, size_t ws_bytes, void *stream);
 
+/* Depth-wise convolution on coded operands (MobileNetV2, one of the models of Section IV-A, is built from 3x3
+ * layers of this kind): channel ch of the output is channel ch of the input filtered by its own r x s kernel,
+ *     Y[n][oh][ow][ch] = sX*sW * sum_{r,s} value(X[n][ih][iw][ch]) * value(W[ch][r][s])
+ * desc->k must equal desc->c.  There is no contraction over channels, hence no tensor-core work: the kernel decodes
+ * the packed codes itself, accumulates in fp32 on integer values (bit-exact whenever both formats have at most 4
+ * magnitude bits; wider formats may round once sums exceed 2^24: |err| <= 1e-5 * r*s * max|x| * max|w|) and is
+ * bound by the fp32 output stream.  No workspace.
+ *   X   [dev] dense NHWC code stream as for dybit_conv2d, 4-byte aligned
+ *   W   [dev] c rows of r*s codes (tap order r, s), row stride ldw_bytes >= dybit_packed_bytes(r*s, fw.bits)
+ *   Y   [dev] n*oh*ow*c floats, dense
+ * Filters or strides whose staged input patch exceeds 200 KB of shared memory -> DYBIT_ERR_UNSUPPORTED. */
+dybit_status dybit_depthwise_conv2d(const dybit_conv_desc *desc,
+                                    const void *X, dybit_fmt fx, const float *scale_x,
+                                    const void *W, dybit_fmt fw, const float *scale_w, int64_t ldw_bytes,
+                                    float *Y, void *stream);
+
 /* Quantization error metric of Eq. 2 (Section III-C.1), the quantity the bitwidth search ranks layers by:
  *     RMSE = sqrt( (1/n) * sum_i ((x_i - xhat_i) / sigma)^2 )
  * with xhat_i = scale[0] * value(encode(x_i)) the quantize-dequantize image under `fmt` and {scale, 1/scale}, and

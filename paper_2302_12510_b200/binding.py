@@ -21,7 +21,7 @@ __all__ = [
     "dybit_conv2d_out_hw", "dybit_absmax_scale", "dybit_quantize_pack", "dybit_quantize_pack_2d",
     "dybit_decode", "dybit_gemm", "dybit_conv2d", "dybit_last_device_status",
     "dybit_launch_count", "dybit_profile_next_gemm", "dybit_gemm_static_ws", "STATIC_WS_BYTES",
-    "dybit_gemm_requant", "dybit_conv2d_requant", "dybit_rmse", "dybit_rmse_sweep", "dybit_fake_quant", "dybit_fake_quant_backward",
+    "dybit_gemm_requant", "dybit_conv2d_requant", "dybit_depthwise_conv2d", "dybit_rmse", "dybit_rmse_sweep", "dybit_fake_quant", "dybit_fake_quant_backward",
     "dybit_search_bitwidths",
 ]
 
@@ -99,6 +99,7 @@ def _load() -> C.CDLL:
     lib.dybit_conv2d_requant.argtypes = [C.POINTER(_CConvDesc), vp, _CFmt, vp, vp, _CFmt, vp, i64,
                                          _CFmt, vp, vp, i32, vp, vp, sz, vp]
     lib.dybit_rmse.argtypes = [vp, i64, _CFmt, vp, vp, vp]
+    lib.dybit_depthwise_conv2d.argtypes = [C.POINTER(_CConvDesc), vp, _CFmt, vp, vp, _CFmt, vp, i64, vp, vp]
     lib.dybit_rmse_sweep.argtypes = [vp, i64, i32, C.POINTER(_CFmt), vp, vp, vp, vp]
     lib.dybit_fake_quant.argtypes = [vp, i64, _CFmt, vp, vp, vp]
     lib.dybit_fake_quant_backward.argtypes = [vp, vp, i64, _CFmt, vp, vp, vp]
@@ -375,6 +376,19 @@ def dybit_conv2d_requant(desc: ConvDesc, X: torch.Tensor, fx, scale_x: torch.Ten
                                     _ptr(Q), wp, wn,
                                     _stream(stream)), "dybit_conv2d_requant")
     return Q
+
+
+def dybit_depthwise_conv2d(desc: ConvDesc, X: torch.Tensor, fx, scale_x: torch.Tensor, W: torch.Tensor, fw,
+                           scale_w: torch.Tensor, Y: Optional[torch.Tensor] = None, stream=None):
+    """Depth-wise convolution (desc.k == desc.c).  X: dense NHWC code stream; W: [c][row bytes] rows of r*s codes
+    (dybit_quantize_pack_2d of the [c][r*s] filter matrix).  Returns Y [n][oh][ow][c] float32."""
+    oh, ow = dybit_conv2d_out_hw(desc)
+    if Y is None:
+        Y = torch.empty((desc.n, oh, ow, desc.c), dtype=torch.float32, device=X.device)
+    cd = _cdesc(desc)
+    _check(lib.dybit_depthwise_conv2d(C.byref(cd), _ptr(X), _fmt(fx), _ptr(scale_x), _ptr(W), _fmt(fw), _ptr(scale_w),
+                                      W.stride(0), _ptr(Y), _stream(stream)), "dybit_depthwise_conv2d")
+    return Y
 
 
 def dybit_rmse(x: torch.Tensor, fmt, scale: torch.Tensor, out: Optional[torch.Tensor] = None, stream=None):

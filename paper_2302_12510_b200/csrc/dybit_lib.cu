@@ -4,3 +4,4 @@
 #include "dybit_quantize.cuh"
 #include "dybit_gemm.cuh"
 #include "dybit_static_ws.cuh"
+#include "dybit_depthwise.cuh"
