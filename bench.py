@@ -344,6 +344,30 @@ def time_calls_flushed(fn, iters, flush):
     return ms[len(ms) // 2]
 
 
+def time_graph(run, replays):
+    """Device time of one replay of `run` captured as a CUDA graph (ms)."""
+    run()
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        run()
+        torch.cuda.synchronize()
+        with torch.cuda.graph(graph, stream=side):
+            run()
+    torch.cuda.synchronize()
+    for _ in range(3):
+        graph.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(replays):
+        graph.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / replays
+
+
 def run_sweeps(dy, wl, device, peaks):
     """Configs 3-5 of the workload list: quantize/pack sweep, square GEMM sweep, ResNet-50 mixed bitwidths."""
     out = {"peaks": peaks}
@@ -406,6 +430,30 @@ def run_sweeps(dy, wl, device, peaks):
                               "gbs": (1 << 28) * 12 / ms / 1e6})
     del x, y, g
     torch.cuda.empty_cache()
+    # depth-wise convolutions of MobileNetV2 at batch 32, 4-bit: one CUDA graph over buffers that rotate through
+    # more than the L2 holds, so that the output stream goes to HBM
+    out["depthwise"] = []
+    for L in wl.mobilenetv2_depthwise_layers(32):
+        if any(r["shape"] == [L.c, L.h, L.stride] for r in out["depthwise"]):
+            continue
+        fx, fw = (4, 0), (4, 1)
+        d = dy.ConvDesc(L.n, L.h, L.w, L.c, L.c, L.r, L.s, L.stride, L.pad, 1)
+        out_elems = L.n * L.oh * L.ow * L.c
+        nbuf = min(64, max(2, int(300e6 // (out_elems * 4)) + 1))
+        xs = [dy.dybit_quantize_pack(wl.half_normal((L.n, L.h, L.w, L.c), seed=i, device=device), fx) for i in range(nbuf)]
+        ys = [torch.empty((L.n, L.oh, L.ow, L.c), dtype=torch.float32, device=device) for _ in range(nbuf)]
+        pw, sw = dy.dybit_quantize_pack_2d(wl.normal((L.c, 9), seed=2, device=device), fw)
+
+        def run():
+            for (px, sx), y in zip(xs, ys):
+                dy.dybit_depthwise_conv2d(d, px, fx, sx, pw, fw, sw, Y=y)
+        ms = time_graph(run, 5) / nbuf
+        nbytes = out_elems * 4 + L.n * L.h * L.w * L.c * fx[0] / 8
+        out["depthwise"].append({"shape": [L.c, L.h, L.stride], "us": ms * 1e3, "gbs": nbytes / ms / 1e6,
+                                 "frac_hbm": nbytes / ms / 1e6 / peaks["hbm_gbs"],
+                                 "goutputs_per_s": out_elems / ms / 1e6})
+        del xs, ys
+        torch.cuda.empty_cache()
     out["gemm_sweep"] = []
     for fmt in ((4, 1), (8, 1)):
         for size in (1024, 2048, 4096, 8192):

@@ -95,6 +95,22 @@ def resnet50_layers(batch: int = 64):
     return L
 
 
+def mobilenetv2_depthwise_layers(batch: int = 32):
+    """The 17 depth-wise 3x3 convolutions of a MobileNetV2 (width 1.0, 224x224 input): the middle layer of every
+    inverted-residual block, on t * c_in channels, with the block's stride; k == c marks them as depth-wise."""
+    L = []
+    hw, cin = 112, 32
+    for t, c, n, s in ((1, 16, 1, 1), (6, 24, 2, 2), (6, 32, 3, 2), (6, 64, 4, 2), (6, 96, 3, 1), (6, 160, 3, 2),
+                       (6, 320, 1, 1)):
+        for i in range(n):
+            stride = s if i == 0 else 1
+            hidden = cin * t
+            L.append(ConvLayer(f"block{len(L)}.dw", batch, hw, hw, hidden, hidden, 3, 3, stride, 1))
+            hw //= stride
+            cin = c
+    return L
+
+
 MIXED_BITS = (2, 3, 4, 5, 6, 8)
 
 
