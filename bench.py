@@ -454,6 +454,21 @@ def run_sweeps(dy, wl, device, peaks):
                                  "goutputs_per_s": out_elems / ms / 1e6})
         del xs, ys
         torch.cuda.empty_cache()
+    # ViT-Base attention products at batch 32 (12 heads): Q K^T and (attention) V as batched GEMMs
+    out["gemm_batched"] = []
+    for fmt in ((4, 1), (8, 1)):
+        for (batch, M, N, K) in ((384, 197, 197, 64), (384, 197, 64, 197)):
+            pa, sa = dy.dybit_quantize_pack_2d(wl.normal((batch * M, K), seed=1, device=device), fmt)
+            pb, sb = dy.dybit_quantize_pack_2d(wl.normal((batch * N, K), seed=2, device=device), fmt)
+            pa, pb = pa.reshape(batch, M, -1), pb.reshape(batch, N, -1)
+            C = torch.empty((batch, M, N), dtype=torch.float32, device=device)
+            ws = torch.empty(dy.dybit_gemm_batched_workspace_bytes(batch, M, N, K, fmt, fmt) + 1024, dtype=torch.uint8,
+                             device=device)
+            ms = time_calls_flushed(lambda: dy.dybit_gemm_batched(M, N, K, pa, fmt, sa, pb, fmt, sb, C=C, ws=ws), 7, flush)
+            nbytes = batch * (M * N * 4 + (M + N) * K * fmt[0] / 8)
+            out["gemm_batched"].append({"batch": batch, "M": M, "N": N, "K": K, "bits": fmt[0], "us": ms * 1e3,
+                                        "tflops": 2 * batch * M * N * K / ms / 1e9, "gbs": nbytes / ms / 1e6,
+                                        "frac_hbm": nbytes / ms / 1e6 / peaks["hbm_gbs"]})
     out["gemm_sweep"] = []
     for fmt in ((4, 1), (8, 1)):
         for size in (1024, 2048, 4096, 8192):

@@ -176,6 +176,21 @@ dybit_status dybit_gemm(int64_t M, int64_t N, int64_t K,
                         float *C, int64_t ldc, int32_t *C_raw,
                         void *ws, size_t ws_bytes, void *stream);
 
+/* Batched GEMM: `batch` independent products of equal shape, C_b = alpha * A_b * B_b^T for b = 0..batch-1 (the
+ * attention products of ViT-Base, one of the models of Section IV-A, are of this kind: 12 heads x batch matrices of
+ * 197 x 64).  Each operand is ONE quantized tensor with one scale; entry b of A starts stride_a_bytes after entry
+ * b-1 (likewise B; C and C_raw: stride_c elements).  Every entry is tiled on its own, so no tile mixes two entries.
+ * Arguments, alignment and exactness as dybit_gemm; additionally stride_a_bytes, stride_b_bytes multiples of 16,
+ * stride_a_bytes >= M*lda_bytes, stride_b_bytes >= N*ldb_bytes, stride_c >= (M-1)*ldc + N.  Dense batches
+ * (stride == rows * ld) expand in one launch, others entry by entry.
+ *   ws [dev] dybit_gemm_batched_workspace_bytes(...) bytes, 1024-byte aligned */
+size_t dybit_gemm_batched_workspace_bytes(int64_t batch, int64_t M, int64_t N, int64_t K, dybit_fmt fa, dybit_fmt fb);
+dybit_status dybit_gemm_batched(int64_t batch, int64_t M, int64_t N, int64_t K,
+                                const void *A, dybit_fmt fa, const float *scale_a, int64_t lda_bytes, int64_t stride_a_bytes,
+                                const void *B, dybit_fmt fb, const float *scale_b, int64_t ldb_bytes, int64_t stride_b_bytes,
+                                float *C, int64_t ldc, int64_t stride_c, int32_t *C_raw,
+                                void *ws, size_t ws_bytes, void *stream);
+
 /* Convolution on coded operands as an implicit GEMM (Section III-C.4: conv
  * and FC layers run on the GEMM dataflow), M = n*oh*ow, N = k, K = r*s*c:
  *     Y[n][oh][ow][k] = sX*sW * sum_{r,s,c} value(X[n][ih][iw][c]) * value(W[k][r][s][c])

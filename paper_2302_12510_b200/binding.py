@@ -21,7 +21,8 @@ __all__ = [
     "dybit_conv2d_out_hw", "dybit_absmax_scale", "dybit_quantize_pack", "dybit_quantize_pack_2d",
     "dybit_decode", "dybit_gemm", "dybit_conv2d", "dybit_last_device_status",
     "dybit_launch_count", "dybit_profile_next_gemm", "dybit_gemm_static_ws", "STATIC_WS_BYTES",
-    "dybit_gemm_requant", "dybit_conv2d_requant", "dybit_depthwise_conv2d", "dybit_rmse", "dybit_rmse_sweep", "dybit_fake_quant", "dybit_fake_quant_backward",
+    "dybit_gemm_requant", "dybit_conv2d_requant", "dybit_depthwise_conv2d", "dybit_gemm_batched",
+    "dybit_gemm_batched_workspace_bytes", "dybit_rmse", "dybit_rmse_sweep", "dybit_fake_quant", "dybit_fake_quant_backward",
     "dybit_search_bitwidths",
 ]
 
@@ -99,6 +100,10 @@ def _load() -> C.CDLL:
     lib.dybit_conv2d_requant.argtypes = [C.POINTER(_CConvDesc), vp, _CFmt, vp, vp, _CFmt, vp, i64,
                                          _CFmt, vp, vp, i32, vp, vp, sz, vp]
     lib.dybit_rmse.argtypes = [vp, i64, _CFmt, vp, vp, vp]
+    lib.dybit_gemm_batched_workspace_bytes.restype = sz
+    lib.dybit_gemm_batched_workspace_bytes.argtypes = [i64, i64, i64, i64, _CFmt, _CFmt]
+    lib.dybit_gemm_batched.argtypes = [i64, i64, i64, i64, vp, _CFmt, vp, i64, i64, vp, _CFmt, vp, i64, i64,
+                                       vp, i64, i64, vp, vp, sz, vp]
     lib.dybit_depthwise_conv2d.argtypes = [C.POINTER(_CConvDesc), vp, _CFmt, vp, vp, _CFmt, vp, i64, vp, vp]
     lib.dybit_rmse_sweep.argtypes = [vp, i64, i32, C.POINTER(_CFmt), vp, vp, vp, vp]
     lib.dybit_fake_quant.argtypes = [vp, i64, _CFmt, vp, vp, vp]
@@ -376,6 +381,36 @@ def dybit_conv2d_requant(desc: ConvDesc, X: torch.Tensor, fx, scale_x: torch.Ten
                                     _ptr(Q), wp, wn,
                                     _stream(stream)), "dybit_conv2d_requant")
     return Q
+
+
+def dybit_gemm_batched_workspace_bytes(batch: int, M: int, N: int, K: int, fa, fb) -> int:
+    return int(lib.dybit_gemm_batched_workspace_bytes(int(batch), int(M), int(N), int(K), _fmt(fa), _fmt(fb)))
+
+
+def dybit_gemm_batched(M: int, N: int, K: int, A: torch.Tensor, fa, scale_a: torch.Tensor, B: torch.Tensor, fb,
+                       scale_b: torch.Tensor, want_raw: bool = False, C: Optional[torch.Tensor] = None,
+                       ws: Optional[torch.Tensor] = None, stream=None):
+    """C[b] = A[b] * B[b]^T for packed A [batch][M][row bytes], B [batch][N][row bytes] (uint8, one scale per operand).
+    Returns (C float32 [batch][M][N], C_raw int32 or None)."""
+    if A.dim() != 3 or B.dim() != 3 or A.shape[0] != B.shape[0] or A.shape[1] != M or B.shape[1] != N:
+        raise ValueError("A must be [batch][M][row bytes] and B [batch][N][row bytes]")
+    if A.stride(2) != 1 or B.stride(2) != 1:
+        raise ValueError("rows of A and B must be contiguous")
+    batch = A.shape[0]
+    if C is None:
+        C = torch.empty((batch, M, N), dtype=torch.float32, device=A.device)
+    raw = torch.empty(C.shape, dtype=torch.int32, device=A.device) if want_raw else None
+    if raw is not None and not C.is_contiguous():
+        raise ValueError("want_raw needs a contiguous C")
+    if ws is None:
+        ws = torch.empty(dybit_gemm_batched_workspace_bytes(batch, M, N, K, fa, fb) + 1024, dtype=torch.uint8,
+                         device=A.device)
+    wp, wn = _ws_ptr(ws)
+    _check(lib.dybit_gemm_batched(batch, M, N, K, _ptr(A), _fmt(fa), _ptr(scale_a), A.stride(1), A.stride(0),
+                                  _ptr(B), _fmt(fb), _ptr(scale_b), B.stride(1), B.stride(0),
+                                  _ptr(C), C.stride(1), C.stride(0), _ptr(raw), wp, wn, _stream(stream)),
+           "dybit_gemm_batched")
+    return C, raw
 
 
 def dybit_depthwise_conv2d(desc: ConvDesc, X: torch.Tensor, fx, scale_x: torch.Tensor, W: torch.Tensor, fw,

@@ -470,6 +470,8 @@ struct GemmParams {
     const float *scale_q;     // {scale, 1/scale} of the output tensor
     int q_bits, q_signed, relu;
     const float *bias;        // requant only: one fp32 per output column, or null
+    int bmt;                  // batched GEMM: M tiles per batch entry (0: not batched); M is then one entry's rows
+    int64_t c_bstride;        // batched GEMM: elements between consecutive entries of C / C_raw
 };
 
 // Waits for the phase with the given parity; gives up after kWaitLimitNs, records
@@ -668,7 +670,8 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     if (!wait_bounded(&empty[s], ph ^ 1u, abort_flag, 1)) { ok = false; break; }
                     mbar_arrive_expect_tx(&full[s], CONV ? L::kBStage : L::kAStage + L::kBStage);
                     if (AMODE == kATiled) {
-                        tma_load_2d(a_stages + s * L::kAStage, &tmap_a, kb * SWB, m_blk * kBM, &full[s]);
+                        if (p.bmt) tma_load_3d(a_stages + s * L::kAStage, &tmap_a, kb * SWB, (m_blk % p.bmt) * kBM, m_blk / p.bmt, &full[s]);
+                        else tma_load_2d(a_stages + s * L::kAStage, &tmap_a, kb * SWB, m_blk * kBM, &full[s]);
                     } else if (AMODE == kAIm2col) {
                         tma_load_im2col_4d(a_stages + s * L::kAStage, &tmap_a, cb * SWB, iw, ih, img, &full[s],
                                            (uint16_t)(fs * p.dil), (uint16_t)(fr * p.dil));
@@ -677,7 +680,8 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                             if (++fs == p.S) { fs = 0; ++fr; }
                         }
                     }
-                    tma_load_2d(b_stages + s * L::kBStage, &tmap_b, kb * SWB, n_blk * BN, &full[s]);
+                    if (AMODE == kATiled && p.bmt) tma_load_3d(b_stages + s * L::kBStage, &tmap_b, kb * SWB, n_blk * BN, m_blk / p.bmt, &full[s]);
+                    else tma_load_2d(b_stages + s * L::kBStage, &tmap_b, kb * SWB, n_blk * BN, &full[s]);
                 }
             }
             if (!ok) {
@@ -735,7 +739,10 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after_sync();
-            const int row = m_blk * kBM + row_in_tile;
+            // batched: the tile belongs to entry `bat`, rows count inside that entry
+            const int bat = p.bmt ? m_blk / p.bmt : 0;
+            const int m_loc = m_blk - bat * p.bmt;
+            const int row = m_loc * kBM + row_in_tile;
             const uint32_t taddr = tmem_base + as * BN + ((uint32_t)(q * 32) << 16);
 #pragma unroll 1
             for (int cc = group; cc < BN / 32; cc += kEpilogueWarps / 4) {
@@ -781,19 +788,38 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     fence_proxy_async_smem();
                     named_barrier(1 + group, 128);
                     if (issuer) {
-                        tma_store_2d(&tmap_c, stage, col0, m_blk * kBM);
+                        if (p.bmt) tma_store_3d(&tmap_c, stage, col0, m_loc * kBM, bat);
+                        else tma_store_2d(&tmap_c, stage, col0, m_blk * kBM);
                         bulk_commit_group();
                     }
                 }
-                if (row < p.M) {
-                    float *crow = p.C + (int64_t)row * p.ldc + col0;
-                    int32_t *rrow = p.C_raw ? p.C_raw + (int64_t)row * p.ldc + col0 : nullptr;
-                    if (vec_ok && col0 + 32 <= p.N) {
-                        if (!p.tma_store) {
+                if (!p.tma_store) {
+                    // C cannot be described to the TMA (rows or base not 16-byte aligned): each warp stages its own
+                    // 32 rows in the same buffer and writes them out row by row, 32 consecutive floats per store
+                    uint8_t *stage = c_stages + group * L::kCStage;
+                    __syncwarp();
+                    uint8_t *srow = stage + row_in_tile * 128;
 #pragma unroll
-                            for (int j = 0; j < 8; ++j)
-                                __stcs(reinterpret_cast<float4 *>(crow) + j, make_float4(f[4 * j], f[4 * j + 1], f[4 * j + 2], f[4 * j + 3]));
+                    for (int j = 0; j < 8; ++j)
+                        *reinterpret_cast<float4 *>(srow + ((j ^ (row_in_tile & 7)) << 4)) =
+                            make_float4(f[4 * j], f[4 * j + 1], f[4 * j + 2], f[4 * j + 3]);
+                    __syncwarp();
+                    const int col = col0 + lane;
+                    const int r_first = m_loc * kBM + q * 32;
+                    if (col < p.N) {
+                        float *cout = p.C + (int64_t)bat * p.c_bstride + (int64_t)r_first * p.ldc + col;
+                        const int rows_here = min(32, p.M - r_first);
+                        for (int rr = 0; rr < rows_here; ++rr) {
+                            const int rt = q * 32 + rr;
+                            const float v = *reinterpret_cast<const float *>(stage + rt * 128 + (((lane >> 2) ^ (rt & 7)) << 4) + ((lane & 3) << 2));
+                            __stcs(cout + (int64_t)rr * p.ldc, v);
                         }
+                    }
+                }
+                if (row < p.M) {
+                    const int64_t coff = (int64_t)bat * p.c_bstride + (int64_t)row * p.ldc + col0;
+                    int32_t *rrow = p.C_raw ? p.C_raw + coff : nullptr;
+                    if (vec_ok && col0 + 32 <= p.N) {
                         if (KIND == Kind::I8 && rrow) {
 #pragma unroll
                             for (int j = 0; j < 8; ++j)
@@ -803,7 +829,6 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
 #pragma unroll
                         for (int j = 0; j < 32; ++j) {
                             if (col0 + j < p.N) {
-                                if (!p.tma_store) crow[j] = f[j];
                                 if (KIND == Kind::I8 && rrow) rrow[j] = (int)r[j];
                             }
                         }
@@ -927,6 +952,22 @@ static dybit_status make_operand_map(CUtensorMap *map, const void *base, int64_t
     return r == CUDA_SUCCESS ? DYBIT_OK : DYBIT_ERR_CUDA;
 }
 
+// Batched operand [batch][rows][row_bytes] (entries `bstride` bytes apart): box = 128 bytes x box_rows x 1 entry, so
+// a tile never reaches into the next entry and rows past `rows` read as zeros.
+static dybit_status make_operand_map_batched(CUtensorMap *map, const void *base, int64_t rows, int64_t row_bytes,
+                                             int64_t stride, int64_t batch, int64_t bstride, int box_rows) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (fn == nullptr) return DYBIT_ERR_CUDA;
+    cuuint64_t dims[3] = {(cuuint64_t)row_bytes, (cuuint64_t)rows, (cuuint64_t)batch};
+    cuuint64_t strides[2] = {(cuuint64_t)stride, (cuuint64_t)bstride};
+    cuuint32_t box[3] = {128, (cuuint32_t)box_rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void *>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? DYBIT_OK : DYBIT_ERR_CUDA;
+}
+
 typedef CUresult (*EncodeIm2colFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                    const cuuint64_t *, const int *, const int *, cuuint32_t, cuuint32_t,
                                    const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
@@ -964,17 +1005,20 @@ static dybit_status make_im2col_map(CUtensorMap *map, const void *xe, const dybi
     return r == CUDA_SUCCESS ? DYBIT_OK : DYBIT_ERR_CUDA;
 }
 
-// fp32 output [M][ldc] as a map whose box is 32 columns x 128 rows, 128-byte swizzle (the staging layout).
-static bool make_output_map(CUtensorMap *map, float *C, int64_t M, int64_t N, int64_t ldc) {
+// fp32 output [M][ldc] (batched: [batch][M][ldc] with `bstride` elements between entries) as a map whose box is
+// 32 columns x 128 rows (x 1 entry), 128-byte swizzle (the staging layout).
+static bool make_output_map(CUtensorMap *map, float *C, int64_t M, int64_t N, int64_t ldc, int64_t batch, int64_t bstride) {
     if ((reinterpret_cast<uintptr_t>(C) & 15) != 0 || (ldc * 4) % 16 != 0) return false;
+    if (batch > 0 && (bstride * 4) % 16 != 0) return false;
     EncodeTiledFn fn = encode_tiled_fn();
     if (fn == nullptr) return false;
-    cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)M};
-    cuuint64_t strides[1] = {(cuuint64_t)ldc * 4};
-    cuuint32_t box[2] = {32, (cuuint32_t)kBM};
-    cuuint32_t estr[2] = {1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, C, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    cuuint64_t dims[3] = {(cuuint64_t)N, (cuuint64_t)M, (cuuint64_t)(batch > 0 ? batch : 1)};
+    cuuint64_t strides[2] = {(cuuint64_t)ldc * 4, (cuuint64_t)bstride * 4};
+    cuuint32_t box[3] = {32, (cuuint32_t)kBM, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, batch > 0 ? 3 : 2, C, dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 template <Kind KIND, int BN, int AMODE, int SWB>
@@ -982,7 +1026,7 @@ static dybit_status launch_gemm_inst(const CUtensorMap &ta, const CUtensorMap &t
     GemmParams p = p_in;
     CUtensorMap tc;
     memset(&tc, 0, sizeof(tc));
-    p.tma_store = (p.Q == nullptr && make_output_map(&tc, p.C, p.M, p.N, p.ldc)) ? 1 : 0;
+    p.tma_store = (p.Q == nullptr && make_output_map(&tc, p.C, p.M, p.N, p.ldc, p.bmt ? p.m_tiles / p.bmt : 0, p.c_bstride)) ? 1 : 0;
     using L = GemmSmem<BN, SWB>;
     auto kern = dybit_gemm_kernel<KIND, BN, AMODE, SWB>;
     constexpr bool CONV = AMODE == kAGather;
@@ -1137,6 +1181,15 @@ size_t dybit_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K, dybit_fmt fa,
     return (size_t)(round_up(M * rb, 1024) + round_up(N * rb, 1024) + 1024);
 }
 
+size_t dybit_gemm_batched_workspace_bytes(int64_t batch, int64_t M, int64_t N, int64_t K, dybit_fmt fa, dybit_fmt fb) {
+    using namespace dybit;
+    ContainerPlan plan;
+    if (batch <= 0 || M <= 0 || N <= 0 || K <= 0 || plan_container(fa, fb, &plan) != DYBIT_OK) return 0;
+    const int elem = container_elem_bytes(plan.container);
+    const int64_t rb = k_row_bytes(round_up(K, 128), elem);
+    return (size_t)(round_up(batch * M * rb, 1024) + round_up(batch * N * rb, 1024) + 1024);
+}
+
 size_t dybit_conv2d_workspace_bytes(const dybit_conv_desc *d, dybit_fmt fx, dybit_fmt fw) {
     using namespace dybit;
     ContainerPlan plan;
@@ -1209,6 +1262,84 @@ static dybit_status gemm_impl(int64_t M, int64_t N, int64_t K, const void *A, dy
     p.scale_b = scale_b;
     p.pow2 = ldexp(1.0, -(plan.exp_a + plan.exp_b));
     apply_requant(p, rq);
+    return launch_gemm_kind<kATiled, 128>(plan.container, bn, map_a, map_b, p, s);
+}
+
+// Batched GEMM: `batch` independent products C_b = A_b * B_b^T of equal shape, one scale per operand tensor (the
+// whole batch is one quantized tensor).  Every entry gets its own tiles: tile rows count over batch * m_tiles and
+// the kernel's 3-D tensor maps keep a tile inside its entry.
+static dybit_status gemm_batched_impl(int64_t batch, int64_t M, int64_t N, int64_t K, const void *A, dybit_fmt fa,
+                                      const float *scale_a, int64_t lda_bytes, int64_t stride_a_bytes, const void *B,
+                                      dybit_fmt fb, const float *scale_b, int64_t ldb_bytes, int64_t stride_b_bytes,
+                                      float *C, int64_t ldc, int64_t stride_c, int32_t *C_raw, void *ws, size_t ws_bytes,
+                                      void *stream) {
+    if (batch <= 0 || M <= 0 || N <= 0 || K <= 0 || !fmt_ok(fa) || !fmt_ok(fb)) return DYBIT_ERR_INVALID_ARG;
+    if (!A || !B || !scale_a || !scale_b || !C || ldc < N || stride_c < (M - 1) * ldc + N) return DYBIT_ERR_INVALID_ARG;
+    if (M > (1 << 24) || N > (1 << 24) || K > (1 << 24) || batch > (1 << 24)) return DYBIT_ERR_UNSUPPORTED;
+    const int64_t m_tiles = (M + kBM - 1) / kBM;
+    if (batch * m_tiles > (1 << 24)) return DYBIT_ERR_UNSUPPORTED;
+    if (lda_bytes < (int64_t)dybit_row_stride_bytes(K, fa.bits) || ldb_bytes < (int64_t)dybit_row_stride_bytes(K, fb.bits) ||
+        stride_a_bytes < M * lda_bytes || stride_b_bytes < N * ldb_bytes)
+        return DYBIT_ERR_INVALID_ARG;
+    if (lda_bytes % 16 || ldb_bytes % 16 || stride_a_bytes % 16 || stride_b_bytes % 16 || !aligned(A, 16) || !aligned(B, 16) ||
+        !aligned(C, 4) || !aligned(C_raw, 4) || !aligned(scale_a, 4) || !aligned(scale_b, 4))
+        return DYBIT_ERR_ALIGNMENT;
+    ContainerPlan plan;
+    dybit_status st = plan_container(fa, fb, &plan);
+    if (st != DYBIT_OK) return st;
+    if (C_raw && plan.container != DYBIT_CONTAINER_I8) return DYBIT_ERR_UNSUPPORTED;
+    if (plan.container == DYBIT_CONTAINER_I8 && (K > (1 << 19) || K * plan.max_product > (int64_t)INT32_MAX))
+        return DYBIT_ERR_UNSUPPORTED;
+    const size_t need = dybit_gemm_batched_workspace_bytes(batch, M, N, K, fa, fb);
+    if (need == 0) return DYBIT_ERR_INVALID_ARG;
+    if (!ws || ws_bytes < need) return DYBIT_ERR_WORKSPACE;
+    if (!aligned(ws, 1024)) return DYBIT_ERR_ALIGNMENT;
+
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int elem = container_elem_bytes(plan.container);
+    const int64_t kp = round_up(K, 128);
+    const int64_t rb = k_row_bytes(kp, elem);
+    uint8_t *ae = static_cast<uint8_t *>(ws);
+    uint8_t *be = ae + round_up(batch * M * rb, 1024);
+    const ElemTable &ta = make_elem_table(fa, plan.container, plan.exp_a);
+    const ElemTable &tb = make_elem_table(fb, plan.container, plan.exp_b);
+    const bool i8 = plan.container == DYBIT_CONTAINER_I8;
+    if (stride_a_bytes == M * lda_bytes && stride_b_bytes == N * ldb_bytes) {
+        // dense batches: all entries of an operand are one run of rows
+        const ExpandOperand opa = {static_cast<const uint8_t *>(A), fa.bits, batch * M, lda_bytes, kp, ae, rb, &ta};
+        const ExpandOperand opb = {static_cast<const uint8_t *>(B), fb.bits, batch * N, ldb_bytes, kp, be, rb, &tb};
+        st = launch_expand_pair(opa, opb, elem, i8, s);
+        if (st != DYBIT_OK) return st;
+    } else {
+        for (int64_t b = 0; b < batch; ++b) {
+            const ExpandOperand opa = {static_cast<const uint8_t *>(A) + b * stride_a_bytes, fa.bits, M, lda_bytes, kp,
+                                       ae + b * M * rb, rb, &ta};
+            const ExpandOperand opb = {static_cast<const uint8_t *>(B) + b * stride_b_bytes, fb.bits, N, ldb_bytes, kp,
+                                       be + b * N * rb, rb, &tb};
+            st = launch_expand_pair(opa, opb, elem, i8, s);
+            if (st != DYBIT_OK) return st;
+        }
+    }
+    const int bn = choose_bn(batch * m_tiles * kBM, N);
+    CUtensorMap map_a, map_b;
+    st = make_operand_map_batched(&map_a, ae, M, rb, rb, batch, M * rb, kBM);
+    if (st != DYBIT_OK) return st;
+    st = make_operand_map_batched(&map_b, be, N, rb, rb, batch, N * rb, bn);
+    if (st != DYBIT_OK) return st;
+    GemmParams p = {};
+    p.M = (int)M;
+    p.N = (int)N;
+    p.k_blocks = (int)(rb / kBKBytes);
+    p.bmt = (int)m_tiles;
+    p.m_tiles = (int)(batch * m_tiles);
+    p.n_tiles = (int)((N + bn - 1) / bn);
+    p.C = C;
+    p.C_raw = C_raw;
+    p.ldc = ldc;
+    p.c_bstride = stride_c;
+    p.scale_a = scale_a;
+    p.scale_b = scale_b;
+    p.pow2 = ldexp(1.0, -(plan.exp_a + plan.exp_b));
     return launch_gemm_kind<kATiled, 128>(plan.container, bn, map_a, map_b, p, s);
 }
 
@@ -1359,6 +1490,14 @@ dybit_status dybit_gemm(int64_t M, int64_t N, int64_t K, const void *A, dybit_fm
                         float *C, int64_t ldc, int32_t *C_raw, void *ws, size_t ws_bytes, void *stream) {
     return dybit::gemm_impl(M, N, K, A, fa, scale_a, lda_bytes, B, fb, scale_b, ldb_bytes, C, ldc, C_raw, nullptr, ws,
                             ws_bytes, stream);
+}
+
+dybit_status dybit_gemm_batched(int64_t batch, int64_t M, int64_t N, int64_t K, const void *A, dybit_fmt fa,
+                                const float *scale_a, int64_t lda_bytes, int64_t stride_a_bytes, const void *B,
+                                dybit_fmt fb, const float *scale_b, int64_t ldb_bytes, int64_t stride_b_bytes, float *C,
+                                int64_t ldc, int64_t stride_c, int32_t *C_raw, void *ws, size_t ws_bytes, void *stream) {
+    return dybit::gemm_batched_impl(batch, M, N, K, A, fa, scale_a, lda_bytes, stride_a_bytes, B, fb, scale_b, ldb_bytes,
+                                    stride_b_bytes, C, ldc, stride_c, C_raw, ws, ws_bytes, stream);
 }
 
 dybit_status dybit_conv2d(const dybit_conv_desc *d, const void *X, dybit_fmt fx, const float *scale_x, const void *W,
