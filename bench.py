@@ -368,10 +368,52 @@ def time_graph(run, replays):
     return e0.elapsed_time(e1) / replays
 
 
-def run_sweeps(dy, wl, device, peaks):
-    """Configs 3-5 of the workload list: quantize/pack sweep, square GEMM sweep, ResNet-50 mixed bitwidths."""
+SWEEP_SECTIONS = ("quantize_sweep", "rmse", "rmse_sweep", "fake_quant", "depthwise", "gemm_batched", "gemm_sweep",
+                  "bitwidth_search", "resnet50_b64_mixed")
+
+
+def run_sweeps(dy, wl, device, peaks, only=None, log2n=28):
+    """Configs 3-5 of the workload list (quantize/pack sweep, square GEMM sweep, ResNet-50 mixed bitwidths) and the
+    kernels beyond the hot path.  `only`: names from SWEEP_SECTIONS to run (default all); `log2n`: size of the
+    streaming-kernel cases (a smaller one keeps a profiler capture short)."""
+    want = set(SWEEP_SECTIONS if not only else only)
+    unknown = want - set(SWEEP_SECTIONS)
+    if unknown:
+        raise SystemExit(f"unknown sweep section(s) {sorted(unknown)}; choose from {SWEEP_SECTIONS}")
     out = {"peaks": peaks}
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+    if "quantize_sweep" in want:
+        out["quantize_sweep"] = sweep_quantize(dy, wl, device, flush)
+    if want & {"rmse", "rmse_sweep", "fake_quant"}:
+        x = wl.normal((1 << log2n,), seed=5, device=device)
+        if "rmse" in want:
+            out["rmse"] = sweep_rmse(dy, x, log2n, flush)
+        if "rmse_sweep" in want:
+            out["rmse_sweep"] = sweep_rmse_candidates(dy, x, log2n, flush)
+        if "fake_quant" in want:
+            out["fake_quant"] = sweep_fake_quant(dy, x, log2n, flush)
+        del x
+        torch.cuda.empty_cache()
+    if "depthwise" in want:
+        out["depthwise"] = sweep_depthwise(dy, wl, device, peaks)
+    if "gemm_batched" in want:
+        out["gemm_batched"] = sweep_gemm_batched(dy, wl, device, peaks, flush)
+    if "gemm_sweep" in want:
+        out["gemm_sweep"] = []
+        for fmt in ((4, 1), (8, 1)):
+            for size in (1024, 2048, 4096, 8192):
+                r = target_gemm(dy, wl, device, peaks, size=size, fmt=fmt)
+                out["gemm_sweep"].append({"size": size, "bits": fmt[0], "container": r["container"],
+                                          "tops_call": r["tops_call"], "tops_mma_kernel": r["tops_mma_kernel"],
+                                          "library_matmul_tops": r.get("library_matmul_tops")})
+    if "bitwidth_search" in want:
+        out["bitwidth_search"] = run_search(dy, wl, device)
+    if "resnet50_b64_mixed" in want:
+        out["resnet50_b64_mixed"] = sweep_resnet50(dy, wl, device)
+    return out
+
+
+def sweep_quantize(dy, wl, device, flush):
     rows = []
     for log2n in (20, 22, 24, 26, 28, 30):
         n = 1 << log2n
@@ -389,21 +431,27 @@ def run_sweeps(dy, wl, device, peaks):
                              "gbs_with_max_abs": n * (8 + bits / 8) / ms_m / 1e6})
             del x
             torch.cuda.empty_cache()
-    out["quantize_sweep"] = rows
-    # Eq. 2 error metric: one streaming pass, 4 B/element
-    x = wl.normal((1 << 28,), seed=5, device=device)
-    out["rmse"] = []
+    return rows
+
+
+def sweep_rmse(dy, x, log2n, flush):
+    """Eq. 2 error metric: one streaming pass, 4 B/element."""
+    rows = []
     for bits in (2, 4, 8):
         scale = dy.dybit_absmax_scale(x, (bits, 1))
-        res = torch.empty(4, dtype=torch.float64, device=device)
+        res = torch.empty(4, dtype=torch.float64, device=x.device)
         ms = time_calls_flushed(lambda: dy.dybit_rmse(x, (bits, 1), scale, out=res), 7, flush)
-        out["rmse"].append({"log2n": 28, "bits": bits, "gbs": (1 << 28) * 4 / ms / 1e6, "rmse": res[0].item()})
-    # the same metric for several candidates in one pass: the 7 signed bitwidths, then 16 scales of one format
-    out["rmse_sweep"] = []
+        rows.append({"log2n": log2n, "bits": bits, "gbs": x.numel() * 4 / ms / 1e6, "rmse": res[0].item()})
+    return rows
+
+
+def sweep_rmse_candidates(dy, x, log2n, flush):
+    """The same metric for several candidates in one pass: the 7 signed bitwidths, then 16 scales of one format."""
+    rows = []
     fmts7 = [(b, 1) for b in range(2, 9)]
     sc7 = torch.stack([dy.dybit_absmax_scale(x, f) for f in fmts7]).contiguous()
     base = dy.dybit_absmax_scale(x, (4, 1))
-    ratios = torch.linspace(1.0, 0.25, 16, device=device)
+    ratios = torch.linspace(1.0, 0.25, 16, device=x.device)
     sc16 = torch.stack([base[0] * ratios, 1.0 / (base[0] * ratios)], dim=1).contiguous()
     for what, fmts, sc in (("bitwidths 2..8 signed", fmts7, sc7), ("16 clipping ratios, 4-bit signed", [(4, 1)] * 16, sc16)):
         holder = {}
@@ -412,29 +460,32 @@ def run_sweeps(dy, wl, device, peaks):
             holder["r"] = dy.dybit_rmse_sweep(x, fmts, sc)
         ms = time_calls_flushed(call, 5, flush)
         res, best = holder["r"]
-        out["rmse_sweep"].append({"log2n": 28, "candidates": what, "n_cand": len(fmts), "ms": ms,
-                                  "gbs": (1 << 28) * 4 / ms / 1e6,
-                                  "gelem_cand_per_s": (1 << 28) * len(fmts) / ms / 1e6,
-                                  "best": int(best.item()), "rmse": [float(v) for v in res[:, 0].tolist()]})
-    # QAT pair: quantize-dequantize image (8 B/element) and its clipped straight-through gradient (12 B/element)
-    out["fake_quant"] = []
+        rows.append({"log2n": log2n, "candidates": what, "n_cand": len(fmts), "ms": ms,
+                     "gbs": x.numel() * 4 / ms / 1e6, "gelem_cand_per_s": x.numel() * len(fmts) / ms / 1e6,
+                     "best": int(best.item()), "rmse": [float(v) for v in res[:, 0].tolist()]})
+    return rows
+
+
+def sweep_fake_quant(dy, x, log2n, flush):
+    """QAT pair: quantize-dequantize image (8 B/element) and its clipped straight-through gradient (12 B/element)."""
+    rows = []
     y = torch.empty_like(x)
     for fmt in ((4, 1), (8, 1), (2, 0)):
         scale = dy.dybit_absmax_scale(x, fmt)
         ms = time_calls_flushed(lambda: dy.dybit_fake_quant(x, fmt, scale, out=y), 5, flush)
-        out["fake_quant"].append({"log2n": 28, "fmt": list(fmt), "direction": "forward", "ms": ms,
-                                  "gbs": (1 << 28) * 8 / ms / 1e6})
+        rows.append({"log2n": log2n, "fmt": list(fmt), "direction": "forward", "ms": ms, "gbs": x.numel() * 8 / ms / 1e6})
     g = torch.empty_like(x).normal_()
     ms = time_calls_flushed(lambda: dy.dybit_fake_quant_backward(x, g, (4, 1), scale, out=y), 5, flush)
-    out["fake_quant"].append({"log2n": 28, "fmt": [4, 1], "direction": "backward", "ms": ms,
-                              "gbs": (1 << 28) * 12 / ms / 1e6})
-    del x, y, g
-    torch.cuda.empty_cache()
-    # depth-wise convolutions of MobileNetV2 at batch 32, 4-bit: one CUDA graph over buffers that rotate through
-    # more than the L2 holds, so that the output stream goes to HBM
-    out["depthwise"] = []
+    rows.append({"log2n": log2n, "fmt": [4, 1], "direction": "backward", "ms": ms, "gbs": x.numel() * 12 / ms / 1e6})
+    return rows
+
+
+def sweep_depthwise(dy, wl, device, peaks):
+    """Depth-wise convolutions of MobileNetV2 at batch 32, 4-bit: one CUDA graph over buffers that rotate through
+    more than the L2 holds, so that the output stream goes to HBM."""
+    rows = []
     for L in wl.mobilenetv2_depthwise_layers(32):
-        if any(r["shape"] == [L.c, L.h, L.stride] for r in out["depthwise"]):
+        if any(r["shape"] == [L.c, L.h, L.stride] for r in rows):
             continue
         fx, fw = (4, 0), (4, 1)
         d = dy.ConvDesc(L.n, L.h, L.w, L.c, L.c, L.r, L.s, L.stride, L.pad, 1)
@@ -449,13 +500,16 @@ def run_sweeps(dy, wl, device, peaks):
                 dy.dybit_depthwise_conv2d(d, px, fx, sx, pw, fw, sw, Y=y)
         ms = time_graph(run, 5) / nbuf
         nbytes = out_elems * 4 + L.n * L.h * L.w * L.c * fx[0] / 8
-        out["depthwise"].append({"shape": [L.c, L.h, L.stride], "us": ms * 1e3, "gbs": nbytes / ms / 1e6,
-                                 "frac_hbm": nbytes / ms / 1e6 / peaks["hbm_gbs"],
-                                 "goutputs_per_s": out_elems / ms / 1e6})
+        rows.append({"shape": [L.c, L.h, L.stride], "us": ms * 1e3, "gbs": nbytes / ms / 1e6,
+                     "frac_hbm": nbytes / ms / 1e6 / peaks["hbm_gbs"], "goutputs_per_s": out_elems / ms / 1e6})
         del xs, ys
         torch.cuda.empty_cache()
-    # ViT-Base attention products at batch 32 (12 heads): Q K^T and (attention) V as batched GEMMs
-    out["gemm_batched"] = []
+    return rows
+
+
+def sweep_gemm_batched(dy, wl, device, peaks, flush):
+    """ViT-Base attention products at batch 32 (12 heads): Q K^T and (attention) V as batched GEMMs."""
+    rows = []
     for fmt in ((4, 1), (8, 1)):
         for (batch, M, N, K) in ((384, 197, 197, 64), (384, 197, 64, 197)):
             pa, sa = dy.dybit_quantize_pack_2d(wl.normal((batch * M, K), seed=1, device=device), fmt)
@@ -466,17 +520,13 @@ def run_sweeps(dy, wl, device, peaks):
                              device=device)
             ms = time_calls_flushed(lambda: dy.dybit_gemm_batched(M, N, K, pa, fmt, sa, pb, fmt, sb, C=C, ws=ws), 7, flush)
             nbytes = batch * (M * N * 4 + (M + N) * K * fmt[0] / 8)
-            out["gemm_batched"].append({"batch": batch, "M": M, "N": N, "K": K, "bits": fmt[0], "us": ms * 1e3,
-                                        "tflops": 2 * batch * M * N * K / ms / 1e9, "gbs": nbytes / ms / 1e6,
-                                        "frac_hbm": nbytes / ms / 1e6 / peaks["hbm_gbs"]})
-    out["gemm_sweep"] = []
-    for fmt in ((4, 1), (8, 1)):
-        for size in (1024, 2048, 4096, 8192):
-            r = target_gemm(dy, wl, device, peaks, size=size, fmt=fmt)
-            out["gemm_sweep"].append({"size": size, "bits": fmt[0], "container": r["container"],
-                                      "tops_call": r["tops_call"], "tops_mma_kernel": r["tops_mma_kernel"],
-                                      "library_matmul_tops": r.get("library_matmul_tops")})
-    out["bitwidth_search"] = run_search(dy, wl, device)
+            rows.append({"batch": batch, "M": M, "N": N, "K": K, "bits": fmt[0], "us": ms * 1e3,
+                         "tflops": 2 * batch * M * N * K / ms / 1e9, "gbs": nbytes / ms / 1e6,
+                         "frac_hbm": nbytes / ms / 1e6 / peaks["hbm_gbs"]})
+    return rows
+
+
+def sweep_resnet50(dy, wl, device):
     layers = wl.resnet50_layers(64)
     bits = wl.mixed_bitwidths(len(layers), seed=0)
     work = LayerwiseStep(dy, wl, device, layers, bits, host_copies=False)
@@ -487,11 +537,8 @@ def run_sweeps(dy, wl, device, peaks):
         graph.replay()
     ms = timed_region(graph.replay, 10, None, device) / 10
     conts = [CONTAINERS[dy.dybit_choose_container(fa, fw)[0]] for fa, fw in zip(work.fa, work.fw)]
-    out["resnet50_b64_mixed"] = {"ms_per_step": ms, "tops": 2.0 * work.macs / (ms * 1e-3) / 1e12,
-                                 "layers": len(layers), "seed": 0,
-                                 "containers": {c: conts.count(c) for c in sorted(set(conts))},
-                                 "bits_w_a": bits}
-    return out
+    return {"ms_per_step": ms, "tops": 2.0 * work.macs / (ms * 1e-3) / 1e12, "layers": len(layers), "seed": 0,
+            "containers": {c: conts.count(c) for c in sorted(set(conts))}, "bits_w_a": bits}
 
 
 def run_search(dy, wl, device, batch=32, alpha=3.0, beta=3.0, top_k=4):
@@ -618,6 +665,10 @@ def main():
     ap.add_argument("--sweeps", action="store_true",
                     help="measure the other configurations instead (quantize sweep, square GEMM sweep, "
                          "ResNet-50 batch 64 with mixed bitwidths) and print them as one JSON object")
+    ap.add_argument("--only", default="",
+                    help="with --sweeps: comma-separated sections to run (" + ", ".join(SWEEP_SECTIONS) + ")")
+    ap.add_argument("--sweep-log2n", type=int, default=28,
+                    help="with --sweeps: log2 of the element count of the rmse / fake_quant cases")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
@@ -641,7 +692,8 @@ def main():
     peaks = load_peaks()
     warmup = max(3, args.warmup)
     if args.sweeps:
-        print(json.dumps({"sweeps": run_sweeps(dy, wl, device, peaks)}))
+        only = [t for t in args.only.split(",") if t] if args.only else None
+        print(json.dumps({"sweeps": run_sweeps(dy, wl, device, peaks, only=only, log2n=args.sweep_log2n)}))
         return
     if args.targets_only:
         out = {}
