@@ -703,7 +703,7 @@ __device__ __forceinline__ float fake_quant_one(float v, const float *__restrict
 }
 
 template <int BITS, bool SIGNED>
-__global__ void __launch_bounds__(kStreamThreads)
+__global__ void __launch_bounds__(kStreamThreads, 8)
 fake_quant_kernel(const float *__restrict__ x, int64_t n, const float *__restrict__ scale,
                   const __grid_constant__ FloatTable table, float *__restrict__ y) {
     __shared__ float s_lut[256];
@@ -798,7 +798,7 @@ template <int BITS>
 static dybit_status launch_fake_quant_bits(const float *x, int64_t n, bool is_signed, const float *scale, const FloatTable &t,
                                            float *y, cudaStream_t s) {
     int64_t blocks = (n / 4 + kStreamThreads * 4 - 1) / (kStreamThreads * 4);
-    const int64_t cap = (int64_t)sm_count() * 6;
+    const int64_t cap = (int64_t)sm_count() * 8;
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
     if (is_signed) launch_k(fake_quant_kernel<BITS, true>, dim3((unsigned)blocks), dim3(kStreamThreads), 0, s, x, n, scale, t, y);
