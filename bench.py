@@ -117,8 +117,9 @@ class LayerwiseStep:
 
     bits[i] = (weight bits, activation bits) of layer i; weights are signed, activations unsigned."""
 
-    def __init__(self, dy, wl, device, layers, bits, host_copies=True):
+    def __init__(self, dy, wl, device, layers, bits, host_copies=True, two_calls=False):
         self.dy, self.device = dy, device
+        self.two_calls = two_calls          # quantize_pack + conv2d as two library calls instead of one
         self.layers = layers
         self.fw = [(wb, 1) for wb, _ in bits]
         self.fa = [(ab, 0) for _, ab in bits]
@@ -155,13 +156,18 @@ class LayerwiseStep:
     def step(self, events=None):
         dy = self.dy
         for i in range(len(self.layers)):
-            dy.dybit_quantize_pack(self.x_dev[i], self.fa[i], packed=self.px[i], scale_out=self.sx[i])
             if events is not None:
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 dy.dybit_profile_next_gemm(e0, e1)
                 events[i].append((e0, e1))
-            dy.dybit_conv2d(self.desc[i], self.px[i], self.fa[i], self.sx[i], self.pw[i], self.fw[i], self.sw[i],
-                            Y=self.y[i], ws=self.ws)
+            if self.two_calls:
+                dy.dybit_quantize_pack(self.x_dev[i], self.fa[i], packed=self.px[i], scale_out=self.sx[i])
+                dy.dybit_conv2d(self.desc[i], self.px[i], self.fa[i], self.sx[i], self.pw[i], self.fw[i], self.sw[i],
+                                Y=self.y[i], ws=self.ws)
+            else:
+                # same results (codes, scale, layer output) from one library call that saves a launch per layer
+                dy.dybit_quantize_conv2d(self.desc[i], self.x_dev[i], self.fa[i], self.pw[i], self.fw[i], self.sw[i],
+                                         scale_out=self.sx[i], packed=self.px[i], Y=self.y[i], ws=self.ws)
 
     def prepare_requant(self, fq=(4, 0)):
         """Output scales for the re-quantizing epilogue: max-abs of each layer's fp32 output from one normal step
@@ -781,7 +787,8 @@ def main():
         "steps": args.steps, "warmup": warmup, "ms_per_step": ms_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
         "config": {"workload": f"resnet18_b{args.batch}_w4a4: 20 convs + FC as implicit GEMM, per layer "
-                               "max-abs + quantize/pack of the fp32 activation then conv; weights pre-quantized",
+                               "max-abs + quantize/pack of the fp32 activation then conv (one dybit_quantize_conv2d "
+                               "call per layer); weights pre-quantized",
                    "parallelism": "replicas only" if world > 1 else "single GPU",
                    "launch": "one step captured once as a CUDA graph, timed region = K replays",
                    "l2": "per-step footprint (fp32 inputs %.0f MB + fp32 outputs %.0f MB) exceeds the 126 MB L2"
@@ -802,6 +809,19 @@ def main():
                 "given output scales) instead of fp32",
         "ms_per_step": ms_q, "value": whole_job_tops(work.macs, world, ms_q), "unit": "TOPS",
         "output_bytes_per_step": work.q_bytes, "fp32_output_bytes_per_step": work.d2h_bytes}
+    # ---- the same step as two library calls per layer (dybit_quantize_pack, then dybit_conv2d): one more launch each
+    work.two_calls = True
+    for _ in range(3):
+        work.step()
+    launches0 = dy.dybit_launch_count()
+    graph_2 = capture_step(work, device)
+    launches_2 = dy.dybit_launch_count() - launches0
+    for _ in range(3):
+        graph_2.replay()
+    ms_2 = timed_region(graph_2.replay, args.steps, dist, device) / args.steps
+    result["two_call_step"] = {"what": "dybit_quantize_pack + dybit_conv2d per layer instead of dybit_quantize_conv2d",
+                               "ms_per_step": ms_2, "value": whole_job_tops(work.macs, world, ms_2), "unit": "TOPS",
+                               "gpu_launches_per_step": launches_2}
     del work
     torch.cuda.empty_cache()
 

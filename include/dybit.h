@@ -206,6 +206,21 @@ dybit_status dybit_conv2d(const dybit_conv_desc *desc,
                           float *Y, int32_t *Y_raw,
                           void *ws, size_t ws_bytes, void *stream);
 
+/* The two halves of the path in one call: quantize + pack an fp32 NHWC activation (Section III-A) and run the
+ * convolution on its codes (Section III-C.4).  Results are those of dybit_quantize_pack(X) followed by dybit_conv2d,
+ * bit for bit: X_packed receives the dense code stream, scale_x_out the pair it was made with, Y the layer's output.
+ * What is saved is launches: where the expanded activation is the code order itself (channels a multiple of 16, no
+ * patch matrix), one kernel writes the codes, their tensor-core elements and the expanded weights.
+ *   X           [dev] n*h*w*c floats, NHWC, 4-byte aligned
+ *   scale_x     [dev] {scale, 1/scale} to use, or NULL for the max-abs scale of X
+ *   scale_x_out [dev] 2 floats, required (may be scale_x itself)
+ *   X_packed    [dev] dybit_packed_bytes(n*h*w*c, fx.bits) bytes, 16-byte aligned, required
+ * Everything else as in dybit_conv2d (same workspace size). */
+dybit_status dybit_quantize_conv2d(const dybit_conv_desc *desc,
+                                   const float *X, dybit_fmt fx, const float *scale_x, float *scale_x_out, void *X_packed,
+                                   const void *W, dybit_fmt fw, const float *scale_w, int64_t ldw_bytes,
+                                   float *Y, int32_t *Y_raw, void *ws, size_t ws_bytes, void *stream);
+
 /* Depth-wise convolution on coded operands (MobileNetV2, one of the models of Section IV-A, is built from 3x3
  * layers of this kind): channel ch of the output is channel ch of the input filtered by its own r x s kernel,
  *     Y[n][oh][ow][ch] = sX*sW * sum_{r,s} value(X[n][ih][iw][ch]) * value(W[ch][r][s])

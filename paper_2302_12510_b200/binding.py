@@ -22,6 +22,7 @@ __all__ = [
     "dybit_decode", "dybit_gemm", "dybit_conv2d", "dybit_last_device_status",
     "dybit_launch_count", "dybit_profile_next_gemm", "dybit_gemm_static_ws", "STATIC_WS_BYTES",
     "dybit_gemm_requant", "dybit_conv2d_requant", "dybit_depthwise_conv2d", "dybit_gemm_batched",
+    "dybit_quantize_conv2d",
     "dybit_gemm_batched_workspace_bytes", "dybit_rmse", "dybit_rmse_sweep", "dybit_fake_quant", "dybit_fake_quant_backward",
     "dybit_search_bitwidths",
 ]
@@ -100,6 +101,8 @@ def _load() -> C.CDLL:
     lib.dybit_conv2d_requant.argtypes = [C.POINTER(_CConvDesc), vp, _CFmt, vp, vp, _CFmt, vp, i64,
                                          _CFmt, vp, vp, i32, vp, vp, sz, vp]
     lib.dybit_rmse.argtypes = [vp, i64, _CFmt, vp, vp, vp]
+    lib.dybit_quantize_conv2d.argtypes = [C.POINTER(_CConvDesc), vp, _CFmt, vp, vp, vp, vp, _CFmt, vp, i64,
+                                          vp, vp, vp, sz, vp]
     lib.dybit_gemm_batched_workspace_bytes.restype = sz
     lib.dybit_gemm_batched_workspace_bytes.argtypes = [i64, i64, i64, i64, _CFmt, _CFmt]
     lib.dybit_gemm_batched.argtypes = [i64, i64, i64, i64, vp, _CFmt, vp, i64, i64, vp, _CFmt, vp, i64, i64,
@@ -411,6 +414,33 @@ def dybit_gemm_batched(M: int, N: int, K: int, A: torch.Tensor, fa, scale_a: tor
                                   _ptr(C), C.stride(1), C.stride(0), _ptr(raw), wp, wn, _stream(stream)),
            "dybit_gemm_batched")
     return C, raw
+
+
+def dybit_quantize_conv2d(desc: ConvDesc, X: torch.Tensor, fx, W: torch.Tensor, fw, scale_w: torch.Tensor,
+                          scale_x: Optional[torch.Tensor] = None, scale_out: Optional[torch.Tensor] = None,
+                          packed: Optional[torch.Tensor] = None, want_raw: bool = False,
+                          Y: Optional[torch.Tensor] = None, ws: Optional[torch.Tensor] = None, stream=None):
+    """Quantize + pack the fp32 NHWC activation X and convolve its codes with the packed weights W in one call.
+    Returns (Y float32 [n][oh][ow][k], Y_raw int32 or None, packed codes uint8, scale float32[2])."""
+    _dev_f32(X, "X")
+    if X.numel() != desc.n * desc.h * desc.w * desc.c:
+        raise ValueError("X does not match the descriptor")
+    oh, ow = dybit_conv2d_out_hw(desc)
+    if Y is None:
+        Y = torch.empty((desc.n, oh, ow, desc.k), dtype=torch.float32, device=X.device)
+    raw = torch.empty(Y.shape, dtype=torch.int32, device=X.device) if want_raw else None
+    if packed is None:
+        packed = torch.empty(dybit_packed_bytes(X.numel(), fx[0]), dtype=torch.uint8, device=X.device)
+    if scale_out is None:
+        scale_out = torch.empty(2, dtype=torch.float32, device=X.device)
+    if ws is None:
+        ws = torch.empty(dybit_conv2d_workspace_bytes(desc, fx, fw) + 1024, dtype=torch.uint8, device=X.device)
+    wp, wn = _ws_ptr(ws)
+    cd = _cdesc(desc)
+    _check(lib.dybit_quantize_conv2d(C.byref(cd), _ptr(X), _fmt(fx), _ptr(scale_x), _ptr(scale_out), _ptr(packed),
+                                     _ptr(W), _fmt(fw), _ptr(scale_w), W.stride(0), _ptr(Y), _ptr(raw), wp, wn,
+                                     _stream(stream)), "dybit_quantize_conv2d")
+    return Y, raw, packed, scale_out
 
 
 def dybit_depthwise_conv2d(desc: ConvDesc, X: torch.Tensor, fx, scale_x: torch.Tensor, W: torch.Tensor, fw,

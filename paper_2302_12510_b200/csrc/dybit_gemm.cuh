@@ -232,6 +232,181 @@ __global__ void expand_pad_kernel(const uint8_t *__restrict__ packed, int bits, 
     }
 }
 
+// ------------------------------------------------------------------ quantize + expand in one launch
+
+// A weight matrix to expand alongside: rows of `cols` container elements from rows of packed codes.
+struct FusedWeights {
+    const uint8_t *packed;
+    int bits;
+    int64_t rows, in_stride, cols;
+    uint8_t *out;
+    int64_t out_stride;
+};
+
+// fp32 activation -> packed codes AND their container elements, plus the layer's weights expanded by the
+// last blocks of the same grid: what dybit_quantize_pack followed by the expand launch of dybit_conv2d
+// compute, in one launch instead of two.  The activation is one flat run of n elements whose expanded
+// layout is the code order itself (channels a multiple of 16).  Blocks [0, x_blocks) take the activation,
+// a warp 1024 elements at a time exactly as quantize_pack_kernel does; the others the weights, one
+// 16-byte output chunk per thread.
+template <int BITS, bool SIGNED, int ELEM>
+__global__ void __launch_bounds__(kStreamThreads, 3)
+quantize_expand_kernel(const float *__restrict__ x, int64_t n, const float *__restrict__ scale,
+                       uint8_t *__restrict__ packed, int64_t packed_bytes, uint8_t *__restrict__ xe, int64_t xe_bytes,
+                       const __grid_constant__ ElemTable tx, const FusedWeights wj, const __grid_constant__ ElemTable tw,
+                       int x_blocks) {
+    __shared__ __align__(16) unsigned s_codes[kWarpsPerBlock][kChunkCodes / 4];
+    __shared__ __align__(16) unsigned s_words[kWarpsPerBlock][32 * BITS];
+    __shared__ uint16_t s_lut[256];
+    const bool weights = (int)blockIdx.x >= x_blocks;
+    for (int i = threadIdx.x; i < 256; i += blockDim.x) s_lut[i] = weights ? tw.v[i] : tx.v[i];
+    __syncthreads();
+    pdl_enter();
+    if (weights) {
+        constexpr int per_chunk = 16 / ELEM;
+        const int64_t chunks_per_row = wj.cols / per_chunk;
+        const int64_t total = wj.rows * chunks_per_row;
+        const unsigned mask = (1u << wj.bits) - 1u;
+        for (int64_t idx = (int64_t)(blockIdx.x - x_blocks) * blockDim.x + threadIdx.x; idx < total;
+             idx += (int64_t)(gridDim.x - x_blocks) * blockDim.x) {
+            const int64_t row = idx / chunks_per_row, g = idx - row * chunks_per_row;
+            const uint8_t *src = wj.packed + row * wj.in_stride;
+            unsigned o[4] = {0, 0, 0, 0};
+#pragma unroll
+            for (int e = 0; e < per_chunk; ++e) {
+                const int64_t bit = (g * per_chunk + e) * wj.bits;
+                const int sh = (int)(bit & 7);
+                unsigned two = __ldg(src + (bit >> 3));
+                if (sh + wj.bits > 8) two |= (unsigned)__ldg(src + (bit >> 3) + 1) << 8;
+                const unsigned v = s_lut[(two >> sh) & mask];
+                if (ELEM == 1) o[e >> 2] |= (v & 0xffu) << ((e & 3) * 8);
+                else o[e >> 1] |= v << ((e & 1) * 16);
+            }
+            *reinterpret_cast<uint4 *>(wj.out + row * wj.out_stride + g * 16) = make_uint4(o[0], o[1], o[2], o[3]);
+        }
+        return;
+    }
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const float inv = __ldg(scale + 1);
+    constexpr int kChunkBytes = kChunkCodes * BITS / 8;
+    constexpr int kChunkVecs = kChunkBytes / 16;
+    const int64_t items = (packed_bytes + kChunkBytes - 1) / kChunkBytes;
+    const bool vec_ok = (reinterpret_cast<uintptr_t>(x) & 15) == 0;
+    for (int64_t item = (int64_t)blockIdx.x * kWarpsPerBlock + warp; item < items; item += (int64_t)x_blocks * kWarpsPerBlock) {
+        const int64_t c0 = item * kChunkCodes;
+        const float *src = x + c0;
+        const int64_t valid = min((int64_t)kChunkCodes, max((int64_t)0, n - c0));
+        const int nvec = (int)min((int64_t)kChunkVecs, (packed_bytes - item * kChunkBytes) / 16);
+        float4 v[8];
+        if (valid == kChunkCodes && vec_ok) {
+            const float4 *s4 = reinterpret_cast<const float4 *>(src);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) v[j] = __ldcs(s4 + j * 32 + lane);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int64_t i0 = j * 128 + lane * 4;
+                v[j].x = (i0 + 0 < valid) ? src[i0 + 0] : 0.0f;
+                v[j].y = (i0 + 1 < valid) ? src[i0 + 1] : 0.0f;
+                v[j].z = (i0 + 2 < valid) ? src[i0 + 2] : 0.0f;
+                v[j].w = (i0 + 3 < valid) ? src[i0 + 3] : 0.0f;
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) s_codes[warp][j * 32 + lane] = encode4<BITS, SIGNED>(v[j], inv);
+        __syncwarp();
+        // lane takes codes [32*lane, 32*lane + 32)
+        unsigned cw[8];
+        {
+            const uint4 *s4 = reinterpret_cast<const uint4 *>(&s_codes[warp][lane * 8]);
+            const int first = (lane >> 2) & 1;
+            uint4 a = s4[first], b = s4[first ^ 1];
+            if (first) { uint4 t = a; a = b; b = t; }
+            cw[0] = a.x; cw[1] = a.y; cw[2] = a.z; cw[3] = a.w;
+            cw[4] = b.x; cw[5] = b.y; cw[6] = b.z; cw[7] = b.w;
+        }
+        // container elements of the same 32 codes
+        {
+            const int64_t off = (c0 + lane * 32) * ELEM;
+            if constexpr (ELEM == 1) {
+                unsigned o[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    o[i] = (unsigned)(s_lut[cw[i] & 0xffu] & 0xffu) | ((unsigned)(s_lut[(cw[i] >> 8) & 0xffu] & 0xffu) << 8) |
+                           ((unsigned)(s_lut[(cw[i] >> 16) & 0xffu] & 0xffu) << 16) | ((unsigned)(s_lut[cw[i] >> 24] & 0xffu) << 24);
+                if (off + 16 <= xe_bytes) reinterpret_cast<uint4 *>(xe + off)[0] = make_uint4(o[0], o[1], o[2], o[3]);
+                if (off + 32 <= xe_bytes) reinterpret_cast<uint4 *>(xe + off)[1] = make_uint4(o[4], o[5], o[6], o[7]);
+            } else {
+                unsigned o[16];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    o[2 * i] = (unsigned)s_lut[cw[i] & 0xffu] | ((unsigned)s_lut[(cw[i] >> 8) & 0xffu] << 16);
+                    o[2 * i + 1] = (unsigned)s_lut[(cw[i] >> 16) & 0xffu] | ((unsigned)s_lut[cw[i] >> 24] << 16);
+                }
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    if (off + 16 * (i + 1) <= xe_bytes)
+                        reinterpret_cast<uint4 *>(xe + off)[i] = make_uint4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
+            }
+        }
+        unsigned w[BITS];
+        pack32<BITS>(cw, w);
+        uint8_t *dst = packed + item * kChunkBytes;
+        if constexpr (BITS == 4) {
+            if (lane < nvec) reinterpret_cast<uint4 *>(dst)[lane] = make_uint4(w[0], w[1], w[2], w[3]);
+        } else if constexpr (BITS == 8) {
+            if (2 * lane < nvec) reinterpret_cast<uint4 *>(dst)[2 * lane] = make_uint4(w[0], w[1], w[2], w[3]);
+            if (2 * lane + 1 < nvec) reinterpret_cast<uint4 *>(dst)[2 * lane + 1] = make_uint4(w[4], w[5], w[6], w[7]);
+        } else if constexpr (BITS == 2) {
+            if ((lane >> 1) < nvec) reinterpret_cast<uint2 *>(dst)[lane] = make_uint2(w[0], w[1]);
+        } else {
+#pragma unroll
+            for (int i = 0; i < BITS; ++i) s_words[warp][lane * BITS + i] = w[i];
+            __syncwarp();
+            const uint4 *s4 = reinterpret_cast<const uint4 *>(&s_words[warp][0]);
+            for (int i = lane; i < nvec; i += 32) reinterpret_cast<uint4 *>(dst)[i] = s4[i];
+        }
+        __syncwarp();
+    }
+}
+
+template <int BITS, int ELEM>
+static dybit_status launch_quantize_expand_bits(const float *x, int64_t n, bool is_signed, const float *scale, uint8_t *packed,
+                                                int64_t packed_bytes, uint8_t *xe, int64_t xe_bytes, const ElemTable &tx,
+                                                const FusedWeights &wj, const ElemTable &tw, cudaStream_t s) {
+    constexpr int kChunkBytes = kChunkCodes * BITS / 8;
+    const int x_blocks = stream_grid((packed_bytes + kChunkBytes - 1) / kChunkBytes);
+    int64_t w_blocks = (wj.rows * (wj.cols * ELEM / 16) + kStreamThreads - 1) / kStreamThreads;
+    if (w_blocks > sm_count()) w_blocks = sm_count();
+    if (w_blocks < 1) w_blocks = 1;
+    const unsigned grid = (unsigned)(x_blocks + w_blocks);
+    if (is_signed)
+        launch_k(quantize_expand_kernel<BITS, true, ELEM>, dim3(grid), dim3((unsigned)kStreamThreads), (size_t)0, s, x, n, scale, packed,
+                 packed_bytes, xe, xe_bytes, tx, wj, tw, x_blocks);
+    else
+        launch_k(quantize_expand_kernel<BITS, false, ELEM>, dim3(grid), dim3((unsigned)kStreamThreads), (size_t)0, s, x, n, scale, packed,
+                 packed_bytes, xe, xe_bytes, tx, wj, tw, x_blocks);
+    return launch_status();
+}
+
+template <int ELEM>
+static dybit_status launch_quantize_expand(const float *x, int64_t n, dybit_fmt fx, const float *scale, uint8_t *packed,
+                                           int64_t packed_bytes, uint8_t *xe, int64_t xe_bytes, const ElemTable &tx,
+                                           const FusedWeights &wj, const ElemTable &tw, cudaStream_t s) {
+    const bool sg = fx.is_signed != 0;
+    switch (fx.bits) {
+        case 2: return launch_quantize_expand_bits<2, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, s);
+        case 3: return launch_quantize_expand_bits<3, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, s);
+        case 4: return launch_quantize_expand_bits<4, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, s);
+        case 5: return launch_quantize_expand_bits<5, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, s);
+        case 6: return launch_quantize_expand_bits<6, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, s);
+        case 7: return launch_quantize_expand_bits<7, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, s);
+        case 8: return launch_quantize_expand_bits<8, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, s);
+    }
+    return DYBIT_ERR_INVALID_ARG;
+}
+
 // One operand's expand job: rows of `cols` codes -> rows of container elements.
 struct ExpandOperand {
     const uint8_t *packed;
@@ -1343,13 +1518,22 @@ static dybit_status gemm_batched_impl(int64_t batch, int64_t M, int64_t N, int64
     return launch_gemm_kind<kATiled, 128>(plan.container, bn, map_a, map_b, p, s);
 }
 
+// An fp32 activation to quantize on the way in (dybit_quantize_conv2d): X then is the buffer that receives its
+// packed codes and scale_x the pair the codes are made with (written first when `given` is null).
+struct QuantInput {
+    const float *x;
+    const float *given;       // scale to use, or null for the max-abs scale
+};
+
 static dybit_status conv_impl(const dybit_conv_desc *d, const void *X, dybit_fmt fx, const float *scale_x, const void *W,
                               dybit_fmt fw, const float *scale_w, int64_t ldw_bytes, float *Y, int32_t *Y_raw,
-                              const RequantSpec *rq, void *ws, size_t ws_bytes, void *stream) {
+                              const RequantSpec *rq, void *ws, size_t ws_bytes, void *stream,
+                              const QuantInput *xq = nullptr) {
     int oh, ow;
     dybit_status st = dybit_conv2d_out_hw(d, &oh, &ow);
     if (st != DYBIT_OK) return st;
     if (!fmt_ok(fx) || !fmt_ok(fw) || !X || !W || !scale_x || !scale_w) return DYBIT_ERR_INVALID_ARG;
+    if (xq && (!xq->x || !aligned(xq->x, 4) || !aligned(xq->given, 4))) return xq->x ? DYBIT_ERR_ALIGNMENT : DYBIT_ERR_INVALID_ARG;
     if (rq == nullptr && !Y) return DYBIT_ERR_INVALID_ARG;
     {
         const dybit_status rs = check_requant(rq, d->k);
@@ -1382,7 +1566,34 @@ static dybit_status conv_impl(const dybit_conv_desc *d, const void *X, dybit_fmt
     const ElemTable &tx = make_elem_table(fx, plan.container, plan.exp_a);
     const ElemTable &tw = make_elem_table(fw, plan.container, plan.exp_b);
     const bool i8 = plan.container == DYBIT_CONTAINER_I8;
-    if (cv.mode == kConvPatch) {
+    bool expanded = false;
+    if (xq) {
+        // scale first (max-abs, or a copy of the given pair), then codes; where the expanded activation is the code
+        // order itself, one launch writes the codes, their container elements and the expanded weights
+        const int64_t n_x = pixels * d->c;
+        float *scale_dst = const_cast<float *>(scale_x);
+        if (xq->given == nullptr) {
+            st = launch_absmax(xq->x, 1, n_x, n_x, fx, scale_dst, s);
+            if (st != DYBIT_OK) return st;
+        } else if (xq->given != scale_x) {
+            DYBIT_CUDA_TRY(cudaMemcpyAsync(scale_dst, xq->given, 2 * sizeof(float), cudaMemcpyDeviceToDevice, s));
+        }
+        uint8_t *packed = static_cast<uint8_t *>(const_cast<void *>(X));
+        const int64_t packed_bytes = (int64_t)dybit_packed_bytes(n_x, fx.bits);
+        if (cv.mode != kConvPatch && !cv.pad_channels) {
+            const FusedWeights wj = {static_cast<const uint8_t *>(W), fw.bits, N, ldw_bytes, wrb / elem, we, wrb};
+            st = elem == 1 ? launch_quantize_expand<1>(xq->x, n_x, fx, scale_x, packed, packed_bytes, xe, cv.a_bytes, tx, wj, tw, s)
+                           : launch_quantize_expand<2>(xq->x, n_x, fx, scale_x, packed, packed_bytes, xe, cv.a_bytes, tx, wj, tw, s);
+            if (st != DYBIT_OK) return st;
+            expanded = true;
+        } else {
+            st = launch_quantize(xq->x, 1, n_x, n_x, fx, scale_x, packed, packed_bytes, s);
+            if (st != DYBIT_OK) return st;
+        }
+    }
+    if (expanded) {
+        // nothing left to expand
+    } else if (cv.mode == kConvPatch) {
         // patch matrix from the packed activation in one kernel; weights expand as plain rows (K order r, s, c)
         PatchParams pp = {};
         pp.packed = static_cast<const uint8_t *>(X);
@@ -1504,6 +1715,14 @@ dybit_status dybit_conv2d(const dybit_conv_desc *d, const void *X, dybit_fmt fx,
                           dybit_fmt fw, const float *scale_w, int64_t ldw_bytes, float *Y, int32_t *Y_raw, void *ws,
                           size_t ws_bytes, void *stream) {
     return dybit::conv_impl(d, X, fx, scale_x, W, fw, scale_w, ldw_bytes, Y, Y_raw, nullptr, ws, ws_bytes, stream);
+}
+
+dybit_status dybit_quantize_conv2d(const dybit_conv_desc *d, const float *X, dybit_fmt fx, const float *scale_x,
+                                   float *scale_x_out, void *X_packed, const void *W, dybit_fmt fw, const float *scale_w,
+                                   int64_t ldw_bytes, float *Y, int32_t *Y_raw, void *ws, size_t ws_bytes, void *stream) {
+    if (scale_x_out == nullptr || X_packed == nullptr) return DYBIT_ERR_INVALID_ARG;
+    const dybit::QuantInput xq = {X, scale_x};
+    return dybit::conv_impl(d, X_packed, fx, scale_x_out, W, fw, scale_w, ldw_bytes, Y, Y_raw, nullptr, ws, ws_bytes, stream, &xq);
 }
 
 dybit_status dybit_gemm_requant(int64_t M, int64_t N, int64_t K, const void *A, dybit_fmt fa, const float *scale_a,

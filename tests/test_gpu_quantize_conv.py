@@ -1,0 +1,118 @@
+"""GPU parity of dybit_quantize_conv2d (fp32 activation in, codes + layer output out) against the oracle: the codes
+and the scale must be those of the oracle's quantizer, the output that of the oracle's convolution on those codes."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2302_12510_b200 as dy
+from paper_2302_12510_b200 import workloads as wl
+from oracle import dybit_oracle as orc
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def run(layer, fx, fw, seed=0, given_scale=False):
+    x = wl.half_normal((layer.n, layer.h, layer.w, layer.c), seed=seed)
+    if fx[1]:
+        x = x - 0.5
+    w = wl.kaiming_normal(layer.k, layer.r, layer.s, layer.c, seed=seed + 1)
+    pw, sw = dy.dybit_quantize_pack_2d(w.reshape(layer.k, -1).to(DEV), fw)
+    spw = orc.absmax_scale(w.numpy(), fw[0], bool(fw[1]))
+    cw = orc.quantize(w.numpy(), fw[0], bool(fw[1]), spw[1])
+    if given_scale:
+        # a calibrated scale below the maximum: the largest activations saturate
+        full = orc.absmax_scale(x.numpy(), fx[0], bool(fx[1]))
+        s0 = np.float32(full[0]) * np.float32(0.6)
+        spx = (float(s0), float(np.float32(1.0) / s0))
+        scale_x = torch.tensor(spx, dtype=torch.float32, device=DEV)
+    else:
+        spx = orc.absmax_scale(x.numpy(), fx[0], bool(fx[1]))
+        scale_x = None
+    cx = orc.quantize(x.numpy(), fx[0], bool(fx[1]), spx[1])
+    desc = dy.ConvDesc(layer.n, layer.h, layer.w, layer.c, layer.k, layer.r, layer.s, layer.stride, layer.pad, 1)
+    cont, _, _ = dy.dybit_choose_container(fx, fw)
+    Y, Y_raw, packed, scale = dy.dybit_quantize_conv2d(desc, x.to(DEV), fx, pw, fw, sw, scale_x=scale_x,
+                                                       want_raw=(cont == 0))
+    torch.cuda.synchronize()
+    assert dy.dybit_last_device_status() == (0, 0)
+    assert scale.cpu().numpy().tolist() == [float(np.float32(spx[0])), float(np.float32(spx[1]))]
+    assert np.array_equal(packed.cpu().numpy(), orc.pack(cx, fx[0]))
+    S, Y_ref = orc.conv2d(cx, fx, spx[0], cw, fw, spw[0], stride=layer.stride, pad=layer.pad)
+    if cont == 0:
+        assert np.array_equal(Y_raw.cpu().numpy().astype(np.int64), S)
+        assert np.array_equal(Y.cpu().numpy(), Y_ref)
+    else:
+        amax = float(spx[0]) * float(np.abs(orc.decode_table(fx[0], bool(fx[1]))).max())
+        bmax = float(spw[0]) * float(np.abs(orc.decode_table(fw[0], bool(fw[1]))).max())
+        err = np.abs(Y.cpu().numpy().astype(np.float64) - Y_ref.astype(np.float64)).max()
+        assert err <= 1e-5 * layer.gemm_k * amax * bmax
+    # and the two-call path gives the same bits
+    px, sx = dy.dybit_quantize_pack(x.to(DEV), fx, scale=scale_x)
+    Y2, _ = dy.dybit_conv2d(desc, px, fx, sx, pw, fw, sw)
+    assert np.array_equal(Y.cpu().numpy().view(np.uint32), Y2.cpu().numpy().view(np.uint32))
+    return cont
+
+
+# one launch for codes + elements + weights: im2col (64-byte and 128-byte pixels), pointwise, cp.async gather
+@pytest.mark.parametrize("layer", [
+    wl.ConvLayer("c64_3x3_im2col", 8, 28, 28, 64, 64, 3, 3, 1, 1),
+    wl.ConvLayer("c128_3x3_s2_im2col", 6, 20, 20, 128, 96, 3, 3, 2, 1),
+    wl.ConvLayer("c256_pointwise_ragged", 3, 13, 11, 256, 100, 1, 1, 1, 0),
+    wl.ConvLayer("c64_1x1_s2", 6, 28, 28, 64, 128, 1, 1, 2, 0),
+    wl.ConvLayer("c48_gather", 2, 9, 9, 48, 64, 3, 3, 1, 1),
+    wl.ConvLayer("c16_tiny", 1, 3, 5, 16, 8, 3, 3, 1, 1),
+    wl.ConvLayer("fc_like", 5, 1, 1, 512, 1000, 1, 1, 1, 0),
+], ids=lambda L: L.name)
+def test_fused_layouts_4bit(layer):
+    assert run(layer, (4, 0), (4, 1), seed=len(layer.name)) == 0
+    assert run(layer, (4, 0), (4, 1), seed=len(layer.name) + 1, given_scale=True) == 0
+
+
+# separate quantize + patch / padded expand: few channels, channels not a multiple of 16
+@pytest.mark.parametrize("layer", [
+    wl.ConvLayer("c3_7x7_patch", 2, 32, 32, 3, 64, 7, 7, 2, 3),
+    wl.ConvLayer("c20_pad_channels", 2, 8, 8, 20, 24, 3, 3, 1, 1),
+], ids=lambda L: L.name)
+def test_unfused_layouts(layer):
+    assert run(layer, (4, 0), (4, 1), seed=3) == 0
+
+
+@pytest.mark.parametrize("fx,fw,cont", [((2, 0), (2, 1), 0), ((3, 0), (5, 1), 0), ((5, 0), (4, 1), 1), ((6, 0), (3, 1), 2),
+                                        ((8, 0), (8, 1), 2), ((4, 1), (6, 1), 1), ((7, 1), (2, 1), 2)])
+def test_every_container_and_odd_widths(fx, fw, cont):
+    L = wl.ConvLayer("t", 2, 14, 14, 64, 96, 3, 3, 1, 1)
+    assert run(L, fx, fw, seed=fx[0] * 10 + fw[0]) == cont
+    L = wl.ConvLayer("t_big", 6, 20, 20, 64, 96, 3, 3, 1, 1)       # large enough for the TMA im2col path
+    assert run(L, fx, fw, seed=fx[0] * 10 + fw[0] + 1, given_scale=True) == cont
+
+
+def test_resnet18_layer_at_bench_batch_sampled():
+    L = [l for l in wl.resnet18_layers(32) if l.name == "layer2.0.conv2"][0]
+    fx, fw = (4, 0), (4, 1)
+    x = wl.half_normal((L.n, L.h, L.w, L.c), seed=1, device=DEV)
+    w = wl.kaiming_normal(L.k, L.r, L.s, L.c, seed=2)
+    pw, sw = dy.dybit_quantize_pack_2d(w.reshape(L.k, -1).to(DEV), fw)
+    spw = orc.absmax_scale(w.numpy(), 4, True)
+    cw = orc.quantize(w.numpy(), 4, True, spw[1])
+    desc = dy.ConvDesc(L.n, L.h, L.w, L.c, L.k, L.r, L.s, L.stride, L.pad, 1)
+    Y, _, packed, scale = dy.dybit_quantize_conv2d(desc, x, fx, pw, fw, sw)
+    xh = x.cpu().numpy()
+    spx = orc.absmax_scale(xh, 4, False)
+    assert scale.cpu().numpy().tolist() == [float(np.float32(spx[0])), float(np.float32(spx[1]))]
+    rng = np.random.default_rng(0)
+    idx = np.concatenate([rng.integers(0, Y.numel(), 1500), [Y.numel() - 1]]).astype(np.int64)
+    _, y_ref = orc.conv2d_sampled(xh, fx, spx, cw, fw, spw[0], idx, stride=L.stride, pad=L.pad)
+    assert np.array_equal(Y.cpu().numpy().reshape(-1)[idx], y_ref)
+    first = orc.pack(orc.quantize(xh.reshape(-1)[: 1 << 16], 4, False, spx[1]), 4)
+    assert np.array_equal(packed.cpu().numpy()[: first.size], first)
+
+
+def test_argument_errors():
+    one = torch.tensor([1.0, 1.0], device=DEV)
+    d = dy.ConvDesc(1, 4, 4, 16, 8, 3, 3, 1, 1, 1)
+    W = torch.zeros((8, 80), dtype=torch.uint8, device=DEV)
+    with pytest.raises(Exception):                       # wrong element count
+        dy.dybit_quantize_conv2d(d, torch.zeros(100, device=DEV), (4, 0), W, (4, 1), one)
+    with pytest.raises(Exception):                       # not fp32
+        dy.dybit_quantize_conv2d(d, torch.zeros(256, device=DEV, dtype=torch.float16), (4, 0), W, (4, 1), one)
