@@ -248,13 +248,14 @@ struct FusedWeights {
 // compute, in one launch instead of two.  The activation is one flat run of n elements whose expanded
 // layout is the code order itself (channels a multiple of 16).  Blocks [0, x_blocks) take the activation,
 // a warp 1024 elements at a time exactly as quantize_pack_kernel does; the others the weights, one
-// 16-byte output chunk per thread.
+// 16-byte output chunk per thread.  With `partials` the max-abs reduction is finished here as well (see
+// scale_from_partials) and block 0 stores the {scale, 1/scale} pair in scale_out.
 template <int BITS, bool SIGNED, int ELEM>
 __global__ void __launch_bounds__(kStreamThreads, 3)
 quantize_expand_kernel(const float *__restrict__ x, int64_t n, const float *__restrict__ scale,
                        uint8_t *__restrict__ packed, int64_t packed_bytes, uint8_t *__restrict__ xe, int64_t xe_bytes,
                        const __grid_constant__ ElemTable tx, const FusedWeights wj, const __grid_constant__ ElemTable tw,
-                       int x_blocks) {
+                       int x_blocks, const unsigned *__restrict__ partials, int n_partials, int m, float *__restrict__ scale_out) {
     __shared__ __align__(16) unsigned s_codes[kWarpsPerBlock][kChunkCodes / 4];
     __shared__ __align__(16) unsigned s_words[kWarpsPerBlock][32 * BITS];
     __shared__ uint16_t s_lut[256];
@@ -288,7 +289,8 @@ quantize_expand_kernel(const float *__restrict__ x, int64_t n, const float *__re
     }
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
-    const float inv = __ldg(scale + 1);
+    // the scale is either there already, or made here from the per-block maxima the preceding absmax launch left
+    const float inv = partials ? scale_from_partials(partials, n_partials, m, scale_out) : __ldg(scale + 1);
     constexpr int kChunkBytes = kChunkCodes * BITS / 8;
     constexpr int kChunkVecs = kChunkBytes / 16;
     const int64_t items = (packed_bytes + kChunkBytes - 1) / kChunkBytes;
@@ -374,7 +376,9 @@ quantize_expand_kernel(const float *__restrict__ x, int64_t n, const float *__re
 template <int BITS, int ELEM>
 static dybit_status launch_quantize_expand_bits(const float *x, int64_t n, bool is_signed, const float *scale, uint8_t *packed,
                                                 int64_t packed_bytes, uint8_t *xe, int64_t xe_bytes, const ElemTable &tx,
-                                                const FusedWeights &wj, const ElemTable &tw, cudaStream_t s) {
+                                                const FusedWeights &wj, const ElemTable &tw, const unsigned *partials,
+                                                int n_partials, float *scale_out, cudaStream_t s) {
+    const int m = is_signed ? BITS - 1 : BITS;
     constexpr int kChunkBytes = kChunkCodes * BITS / 8;
     const int x_blocks = stream_grid((packed_bytes + kChunkBytes - 1) / kChunkBytes);
     int64_t w_blocks = (wj.rows * (wj.cols * ELEM / 16) + kStreamThreads - 1) / kStreamThreads;
@@ -383,26 +387,27 @@ static dybit_status launch_quantize_expand_bits(const float *x, int64_t n, bool 
     const unsigned grid = (unsigned)(x_blocks + w_blocks);
     if (is_signed)
         launch_k(quantize_expand_kernel<BITS, true, ELEM>, dim3(grid), dim3((unsigned)kStreamThreads), (size_t)0, s, x, n, scale, packed,
-                 packed_bytes, xe, xe_bytes, tx, wj, tw, x_blocks);
+                 packed_bytes, xe, xe_bytes, tx, wj, tw, x_blocks, partials, n_partials, m, scale_out);
     else
         launch_k(quantize_expand_kernel<BITS, false, ELEM>, dim3(grid), dim3((unsigned)kStreamThreads), (size_t)0, s, x, n, scale, packed,
-                 packed_bytes, xe, xe_bytes, tx, wj, tw, x_blocks);
+                 packed_bytes, xe, xe_bytes, tx, wj, tw, x_blocks, partials, n_partials, m, scale_out);
     return launch_status();
 }
 
 template <int ELEM>
 static dybit_status launch_quantize_expand(const float *x, int64_t n, dybit_fmt fx, const float *scale, uint8_t *packed,
                                            int64_t packed_bytes, uint8_t *xe, int64_t xe_bytes, const ElemTable &tx,
-                                           const FusedWeights &wj, const ElemTable &tw, cudaStream_t s) {
+                                           const FusedWeights &wj, const ElemTable &tw, const unsigned *partials,
+                                           int n_partials, float *scale_out, cudaStream_t s) {
     const bool sg = fx.is_signed != 0;
     switch (fx.bits) {
-        case 2: return launch_quantize_expand_bits<2, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, s);
-        case 3: return launch_quantize_expand_bits<3, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, s);
-        case 4: return launch_quantize_expand_bits<4, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, s);
-        case 5: return launch_quantize_expand_bits<5, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, s);
-        case 6: return launch_quantize_expand_bits<6, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, s);
-        case 7: return launch_quantize_expand_bits<7, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, s);
-        case 8: return launch_quantize_expand_bits<8, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, s);
+        case 2: return launch_quantize_expand_bits<2, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, s);
+        case 3: return launch_quantize_expand_bits<3, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, s);
+        case 4: return launch_quantize_expand_bits<4, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, s);
+        case 5: return launch_quantize_expand_bits<5, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, s);
+        case 6: return launch_quantize_expand_bits<6, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, s);
+        case 7: return launch_quantize_expand_bits<7, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, s);
+        case 8: return launch_quantize_expand_bits<8, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, s);
     }
     return DYBIT_ERR_INVALID_ARG;
 }
@@ -553,6 +558,88 @@ patch_expand_kernel(const PatchParams p, const __grid_constant__ ElemTable table
     }
     __syncthreads();
     // rows [blockIdx*128, +128) x krow bytes, 16 bytes per thread per step
+    const int vec_per_row = p.krow / 16;
+    const int rows_here = min(128, p.M - blockIdx.x * 128);
+    for (int i = threadIdx.x; i < rows_here * vec_per_row; i += blockDim.x) {
+        const int r = i / vec_per_row, v = i - r * vec_per_row;
+        const unsigned *src = reinterpret_cast<const unsigned *>(s_rows + r * p.row_pitch + v * 16);
+        const uint4 val = make_uint4(src[0], src[1], src[2], src[3]);
+        *reinterpret_cast<uint4 *>(p.out + ((int64_t)blockIdx.x * 128 + r) * p.krow + v * 16) = val;
+    }
+}
+
+// The same patch matrix from the activation's container elements in dense NHWC order (one element per code,
+// no channel padding), for dilation 1: the taps of one filter row that fall inside the image are one
+// contiguous byte run there, copied with aligned 32-bit loads and a funnel shift; the row is assembled
+// word by word through a 64-bit accumulator (no byte stores, no table lookups), zeros where taps fall outside.
+// The source must be readable up to 7 bytes past its last element.
+struct PatchGatherParams {
+    const uint8_t *xd;         // dense NHWC container elements
+    uint8_t *out;              // [M][krow] container bytes
+    int elem;
+    int H, W, C, R, S, OH, OW, stride, pad;
+    int M, krow, row_pitch;    // row_pitch = krow + 4: odd word count, so threads hit distinct banks
+};
+
+__global__ void __launch_bounds__(128)
+patch_gather_kernel(const PatchGatherParams p) {
+    extern __shared__ __align__(16) uint8_t s_rows[];
+    pdl_enter();
+    const int m = blockIdx.x * 128 + threadIdx.x;
+    if (m < p.M) {
+        const int img = m / (p.OH * p.OW);
+        const int rem = m - img * (p.OH * p.OW);
+        const int oh = rem / p.OW, ow = rem - oh * p.OW;
+        const int ih0 = oh * p.stride - p.pad, iw0 = ow * p.stride - p.pad;
+        const int tapb = p.C * p.elem;             // bytes per tap
+        const int rowb = p.S * tapb;               // bytes per filter row
+        const int s_lo = max(0, -iw0), s_hi = min(p.S, p.W - iw0);
+        unsigned *wp = reinterpret_cast<unsigned *>(s_rows + threadIdx.x * p.row_pitch);
+        unsigned long long acc = 0;
+        int nb = 0;                                // bytes waiting in acc (always < 4 between steps)
+        int zeros = 0;                             // zero bytes owed before the next run
+        for (int fr = 0; fr < p.R; ++fr) {
+            const int ih = ih0 + fr;
+            if ((unsigned)ih >= (unsigned)p.H || s_lo >= s_hi) {
+                zeros += rowb;
+                continue;
+            }
+            nb += zeros + s_lo * tapb;
+            while (nb >= 4) {
+                *wp++ = (unsigned)acc;
+                acc >>= 32;
+                nb -= 4;
+            }
+            const int len = (s_hi - s_lo) * tapb;
+            const int64_t a = (((int64_t)img * p.H + ih) * p.W + (iw0 + s_lo)) * tapb;
+            const unsigned *src = reinterpret_cast<const unsigned *>(p.xd + (a & ~(int64_t)3));
+            const unsigned sh = (unsigned)(a & 3) * 8u;
+            unsigned w0 = __ldg(src);
+            for (int j = 0; j < len; j += 4) {
+                const unsigned w1 = __ldg(++src);
+                unsigned v = __funnelshift_r(w0, w1, sh);
+                w0 = w1;
+                const int k = min(4, len - j);
+                if (k < 4) v &= (1u << (8 * k)) - 1u;
+                acc |= (unsigned long long)v << (8 * nb);
+                nb += k;
+                if (nb >= 4) {
+                    *wp++ = (unsigned)acc;
+                    acc >>= 32;
+                    nb -= 4;
+                }
+            }
+            zeros = (p.S - s_hi) * tapb;
+        }
+        // zeros owed, then the row's zero tail up to krow (a multiple of 16, so nothing is left over)
+        nb += zeros + p.krow - p.R * rowb;
+        while (nb >= 4) {
+            *wp++ = (unsigned)acc;
+            acc >>= 32;
+            nb -= 4;
+        }
+    }
+    __syncthreads();
     const int vec_per_row = p.krow / 16;
     const int rows_here = min(128, p.M - blockIdx.x * 128);
     for (int i = threadIdx.x; i < rows_here * vec_per_row; i += blockDim.x) {
@@ -1316,6 +1403,7 @@ struct ConvPlan {
     int64_t krow;                  // patch mode: bytes per patch row
     int64_t wrb;                   // bytes per expanded weight row
     bool pad_channels;             // expanded activation / weights carry zero channels c..cp-1
+    int64_t xd_bytes;              // patch mode, dilation 1: dense container elements of the activation (third region)
 };
 
 static ConvPlan plan_conv(const dybit_conv_desc *d, int oh, int ow, int elem) {
@@ -1343,6 +1431,7 @@ static ConvPlan plan_conv(const dybit_conv_desc *d, int oh, int ow, int elem) {
         c.a_bytes = round_up(M * krow, 1024);
         c.wrb = k_row_bytes(taps * d->c, elem);
         c.pad_channels = false;
+        if (d->dilation == 1) c.xd_bytes = round_up(round_up(c.pixels * d->c, kChunkCodes) * elem, 1024) + 1024;
     } else {
         c.a_bytes = round_up(c.pixels * c.cpb, 1024);
         c.wrb = k_row_bytes(taps * c.cp, elem);
@@ -1379,7 +1468,9 @@ size_t dybit_conv2d_workspace_bytes(const dybit_conv_desc *d, dybit_fmt fx, dybi
     int oh, ow;
     if (dybit_conv2d_out_hw(d, &oh, &ow) != DYBIT_OK || plan_container(fx, fw, &plan) != DYBIT_OK) return 0;
     const ConvPlan c = plan_conv(d, oh, ow, container_elem_bytes(plan.container));
-    return (size_t)(c.a_bytes + round_up((int64_t)d->k * c.wrb, 1024) + 2048);
+    // expanded activation (or patch matrix), expanded weights, dense activation elements (patch mode), slack,
+    // per-block maxima of the max-abs reduction
+    return (size_t)(c.a_bytes + round_up((int64_t)d->k * c.wrb, 1024) + c.xd_bytes + 2048 + kMaxAbsmaxPartials * sizeof(unsigned));
 }
 
 }  // extern "C"
@@ -1571,6 +1662,8 @@ static dybit_status conv_impl(const dybit_conv_desc *d, const void *X, dybit_fmt
     const int64_t cp = cv.cp, pixels = cv.pixels, wrb = cv.wrb;
     uint8_t *xe = static_cast<uint8_t *>(ws);
     uint8_t *we = xe + cv.a_bytes;
+    uint8_t *xd = we + round_up(N * wrb, 1024);              // patch mode: dense container elements of the activation
+    const bool patch_dense = cv.mode == kConvPatch && cv.xd_bytes > 0;
     const ElemTable &tx = make_elem_table(fx, plan.container, plan.exp_a);
     const ElemTable &tw = make_elem_table(fw, plan.container, plan.exp_b);
     const bool i8 = plan.container == DYBIT_CONTAINER_I8;
@@ -1580,7 +1673,16 @@ static dybit_status conv_impl(const dybit_conv_desc *d, const void *X, dybit_fmt
         // order itself, one launch writes the codes, their container elements and the expanded weights
         const int64_t n_x = pixels * d->c;
         float *scale_dst = const_cast<float *>(scale_x);
-        if (xq->given == nullptr) {
+        const bool fused = patch_dense || (cv.mode != kConvPatch && !cv.pad_channels);
+        // max-abs scale: in the fused case the absmax launch leaves one maximum per block in the workspace and the
+        // quantize launch folds them (nothing to zero first, no atomics); otherwise the ticket version writes the pair
+        unsigned *partials = nullptr;
+        int n_partials = 0;
+        if (xq->given == nullptr && fused && n_x > 0) {
+            partials = reinterpret_cast<unsigned *>(static_cast<uint8_t *>(ws) + need - kMaxAbsmaxPartials * sizeof(unsigned));
+            st = launch_absmax(xq->x, 1, n_x, n_x, fx, scale_dst, s, partials, &n_partials);
+            if (st != DYBIT_OK) return st;
+        } else if (xq->given == nullptr) {
             st = launch_absmax(xq->x, 1, n_x, n_x, fx, scale_dst, s);
             if (st != DYBIT_OK) return st;
         } else if (xq->given != scale_x) {
@@ -1588,10 +1690,14 @@ static dybit_status conv_impl(const dybit_conv_desc *d, const void *X, dybit_fmt
         }
         uint8_t *packed = static_cast<uint8_t *>(const_cast<void *>(X));
         const int64_t packed_bytes = (int64_t)dybit_packed_bytes(n_x, fx.bits);
-        if (cv.mode != kConvPatch && !cv.pad_channels) {
+        if (fused) {
             const FusedWeights wj = {static_cast<const uint8_t *>(W), fw.bits, N, ldw_bytes, wrb / elem, we, wrb};
-            st = elem == 1 ? launch_quantize_expand<1>(xq->x, n_x, fx, scale_x, packed, packed_bytes, xe, cv.a_bytes, tx, wj, tw, s)
-                           : launch_quantize_expand<2>(xq->x, n_x, fx, scale_x, packed, packed_bytes, xe, cv.a_bytes, tx, wj, tw, s);
+            uint8_t *const dense = patch_dense ? xd : xe;         // code order either way
+            const int64_t dense_bytes = patch_dense ? cv.xd_bytes : cv.a_bytes;
+            st = elem == 1 ? launch_quantize_expand<1>(xq->x, n_x, fx, scale_x, packed, packed_bytes, dense, dense_bytes, tx, wj, tw,
+                                                       partials, n_partials, scale_dst, s)
+                           : launch_quantize_expand<2>(xq->x, n_x, fx, scale_x, packed, packed_bytes, dense, dense_bytes, tx, wj, tw,
+                                                       partials, n_partials, scale_dst, s);
             if (st != DYBIT_OK) return st;
             expanded = true;
         } else {
@@ -1599,7 +1705,37 @@ static dybit_status conv_impl(const dybit_conv_desc *d, const void *X, dybit_fmt
             if (st != DYBIT_OK) return st;
         }
     }
-    if (expanded) {
+    if (patch_dense) {
+        // dense container elements first (unless the quantize launch wrote them), then the patch matrix from those
+        if (!expanded) {
+            const int64_t n_codes = pixels * d->c;
+            const ExpandOperand opx = {static_cast<const uint8_t *>(X), fx.bits, 1, 0,
+                                       fx.bits == 4 ? round_up(n_codes, 32) : n_codes, xd, 0, &tx};
+            const ExpandOperand opw = {static_cast<const uint8_t *>(W), fw.bits, N, ldw_bytes, wrb / elem, we, wrb, &tw};
+            st = launch_expand_pair(opx, opw, elem, i8, s);
+            if (st != DYBIT_OK) return st;
+        }
+        PatchGatherParams pg = {};
+        pg.xd = xd;
+        pg.out = xe;
+        pg.elem = elem;
+        pg.H = d->h; pg.W = d->w; pg.C = d->c; pg.R = d->r; pg.S = d->s;
+        pg.OH = oh; pg.OW = ow; pg.stride = d->stride; pg.pad = d->pad;
+        pg.M = (int)M;
+        pg.krow = (int)cv.krow;
+        pg.row_pitch = (int)cv.krow + 4;
+        const size_t smem = (size_t)128 * pg.row_pitch;
+        static bool gather_configured[64] = {};
+        int dev = 0;
+        DYBIT_CUDA_TRY(cudaGetDevice(&dev));
+        if (dev >= 0 && dev < 64 && !gather_configured[dev]) {
+            DYBIT_CUDA_TRY(cudaFuncSetAttribute(patch_gather_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                128 * (1024 + 4)));
+            gather_configured[dev] = true;
+        }
+        launch_k(patch_gather_kernel, dim3((unsigned)((int)((M + 127) / 128))), dim3((unsigned)(128)), (size_t)(smem), s, pg);
+        if (launch_status() != DYBIT_OK) return DYBIT_ERR_CUDA;
+    } else if (expanded) {
         // nothing left to expand
     } else if (cv.mode == kConvPatch) {
         // patch matrix from the packed activation in one kernel; weights expand as plain rows (K order r, s, c)

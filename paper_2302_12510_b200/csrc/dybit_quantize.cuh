@@ -95,10 +95,13 @@ __device__ __forceinline__ unsigned finite_abs_bits(float v) {
 // pair into {scale, 1/scale} for m magnitude bits: amax / 2^(m-1) and one IEEE
 // division 2^(m-1) / amax ({1, 1} for an all-zero tensor).
 // Handles rows x cols with leading dimension ld (ld == cols: one flat run).
+// With `partials` set the kernel stops one step earlier: block b stores its own maximum in partials[b] (no
+// atomics, no ticket, nothing to zero beforehand) and the consumer folds the gridDim.x words itself
+// (scale_from_partials); `slot` is then unused.
 template <bool STREAM>   // STREAM: evict-first loads (tensor larger than L2); otherwise leave it in L2 for the next pass
 __global__ void __launch_bounds__(kStreamThreads)
 absmax_kernel(const float *__restrict__ x, int64_t rows, int64_t cols, int64_t ld,
-              unsigned *__restrict__ slot, int m) {
+              unsigned *__restrict__ slot, int m, unsigned *__restrict__ partials) {
     unsigned best = 0;
     pdl_enter();
     const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -144,7 +147,9 @@ absmax_kernel(const float *__restrict__ x, int64_t rows, int64_t cols, int64_t l
     if (threadIdx.x < 32) {
         unsigned b = threadIdx.x < kWarpsPerBlock ? warp_best[threadIdx.x] : 0u;
         b = __reduce_max_sync(0xffffffffu, b);
-        if (threadIdx.x == 0) {
+        if (threadIdx.x == 0 && partials != nullptr) {
+            partials[blockIdx.x] = b;
+        } else if (threadIdx.x == 0) {
             if (b != 0u) atomicMax(slot, b);                 // result unused: a fire-and-forget reduction
             __threadfence();
             const unsigned ticket = atomicAdd(slot + 1, 1u);
@@ -163,6 +168,39 @@ absmax_kernel(const float *__restrict__ x, int64_t rows, int64_t cols, int64_t l
             }
         }
     }
+}
+
+// Consumer side of the partials mode of absmax_kernel: every block folds the per-block maxima (written by the
+// previous kernel of the stream) into the tensor's maximum and derives the same {scale, 1/scale} pair with the
+// same two IEEE operations as the ticket path; block 0 also stores the pair for later kernels.  Returns 1/scale.
+// Must be called by all threads of the block, after pdl_enter().
+constexpr int kMaxAbsmaxPartials = 1024;
+__device__ __forceinline__ float scale_from_partials(const unsigned *__restrict__ partials, int n_partials, int m,
+                                                     float *__restrict__ scale_out) {
+    __shared__ unsigned s_part[kWarpsPerBlock];
+    __shared__ float s_inv;
+    unsigned b = 0;
+    for (int i = threadIdx.x; i < n_partials; i += blockDim.x) b = max(b, __ldcg(partials + i));
+    b = __reduce_max_sync(0xffffffffu, b);
+    if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = b;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < (int)(blockDim.x >> 5); ++w) b = max(b, s_part[w]);
+        const float amax = __uint_as_float(b);
+        float sc = 1.0f, inv = 1.0f;
+        if (amax != 0.0f) {
+            const float vmax = (float)(1u << (m - 1));
+            sc = __fdiv_rn(amax, vmax);
+            inv = __fdiv_rn(vmax, amax);
+        }
+        s_inv = inv;
+        if (blockIdx.x == 0) {
+            scale_out[0] = sc;
+            scale_out[1] = inv;
+        }
+    }
+    __syncthreads();
+    return s_inv;
 }
 
 // Empty tensor: no reduction runs, the scale is {1, 1}.
@@ -817,22 +855,28 @@ static int stream_grid(int64_t items_per_warp_unit) {
     return (int)blocks;
 }
 
+// With `partials` (room for kMaxAbsmaxPartials words) the kernel leaves one maximum per block there and
+// *n_partials says how many; the consumer finishes the reduction (scale_from_partials) and scale_out is not touched.
 static dybit_status launch_absmax(const float *x, int64_t rows, int64_t cols, int64_t ld, dybit_fmt fmt,
-                                  float *scale_out, cudaStream_t s) {
-    DYBIT_CUDA_TRY(cudaMemsetAsync(scale_out, 0, 2 * sizeof(float), s));
+                                  float *scale_out, cudaStream_t s, unsigned *partials = nullptr,
+                                  int *n_partials = nullptr) {
     const int64_t n = rows * cols;
+    if (partials == nullptr) DYBIT_CUDA_TRY(cudaMemsetAsync(scale_out, 0, 2 * sizeof(float), s));
+    else if (n <= 0) return DYBIT_ERR_INVALID_ARG;
     if (n > 0) {
         // few, fat blocks: every block ends with two atomics on the same words
         int64_t blocks = (n / 4 + kStreamThreads * 8 - 1) / (kStreamThreads * 8);
         int64_t cap = (int64_t)sm_count() * 4;
+        if (cap > kMaxAbsmaxPartials) cap = kMaxAbsmaxPartials;
         if (blocks > cap) blocks = cap;
         if (blocks < 1) blocks = 1;
+        if (n_partials) *n_partials = (int)blocks;
         if (n * 4 > ((int64_t)64 << 20))
             launch_k(absmax_kernel<true>, dim3((unsigned)((int)blocks)), dim3((unsigned)(kStreamThreads)), (size_t)(0), s, x, rows, cols, ld,
-                                                                       reinterpret_cast<unsigned *>(scale_out), mag_bits(fmt));
+                                                                       reinterpret_cast<unsigned *>(scale_out), mag_bits(fmt), partials);
         else
             launch_k(absmax_kernel<false>, dim3((unsigned)((int)blocks)), dim3((unsigned)(kStreamThreads)), (size_t)(0), s, x, rows, cols, ld,
-                                                                        reinterpret_cast<unsigned *>(scale_out), mag_bits(fmt));
+                                                                        reinterpret_cast<unsigned *>(scale_out), mag_bits(fmt), partials);
         return launch_status();
     }
     launch_k(unit_scale_kernel, dim3((unsigned)(1)), dim3((unsigned)(1)), (size_t)(0), s, scale_out);
