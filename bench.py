@@ -737,9 +737,19 @@ def main():
     ms_step = ms_total / args.steps
     value = whole_job_tops(work.macs, world, ms_step)
 
-    # ---- the same K steps launched directly, with events around each layer's tensor-core kernel
+    # ---- the same K steps launched directly (host-bound: every launch goes through the Python binding)
+    ms_eager = timed_region(work.step, args.steps, dist, device) / args.steps
+    # ---- and with events around each layer's tensor-core kernel.  A spin kernel is queued in front of every
+    #      profiled step so that the host has submitted the whole step before the GPU starts it: the event pairs
+    #      then bracket the kernel itself, not the wait for its launch to arrive.
     events = [[] for _ in work.layers]
-    ms_eager = timed_region(lambda: work.step(events), args.steps, dist, device) / args.steps
+    prof_steps = max(3, min(args.steps, 20))
+
+    def profiled_step():
+        torch.cuda._sleep(5_000_000)        # ~2.5 ms at 1965 MHz; one directly launched step takes ~1 ms of host time
+        work.step(events)
+
+    timed_region(profiled_step, prof_steps, dist, device)
     st, detail = dy.dybit_last_device_status()
     if st != 0:
         raise SystemExit(f"device status {st} detail {detail:#x}")
@@ -763,9 +773,9 @@ def main():
         # (profiles/dybit_gemm_kernel_conv_resnet18_b32_dram_traffic.txt); only valid for the batch-32 workload
         "traffic": GEMM_KERNEL_DRAM_BYTES_PER_LAUNCH if args.batch == 32 else None,
         "peak_how": (f"2 x sustained bf16 ({peaks['source']})" if tensor_bound else f"copy bandwidth ({peaks['source']})"),
-        "how": "CUDA events recorded by the library around this kernel alone, same K steps launched directly "
-               "(not as a graph) right after the timed region",
-        "ms_per_step_in_kernel": mma_total_ms, "share_of_step": mma_total_ms / ms_eager,
+        "how": "CUDA events recorded by the library around this kernel alone, in %d directly launched steps right "
+               "after the timed region, each queued behind a spin kernel so that launches never arrive late" % prof_steps,
+        "ms_per_step_in_kernel": mma_total_ms, "share_of_step": mma_total_ms / ms_step,
         "ms_per_step_direct_launch": ms_eager,
         "layers_us": {L.name: [round(t * 1e3, 1), round(b[2] * 1e6, 1)] for L, t, b in zip(work.layers, mma_ms, bounds)},
         "frac_of_layerwise_bound": ideal_s / (mma_total_ms * 1e-3),

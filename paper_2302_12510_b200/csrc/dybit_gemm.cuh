@@ -241,6 +241,8 @@ struct FusedWeights {
     int64_t rows, in_stride, cols;
     uint8_t *out;
     int64_t out_stride;
+    int use4;                 // 1: job4 describes the same rows for the 4-bit register-table expansion
+    Expand4Job job4;
 };
 
 // fp32 activation -> packed codes AND their container elements, plus the layer's weights expanded by the
@@ -262,8 +264,60 @@ quantize_expand_kernel(const float *__restrict__ x, int64_t n, const float *__re
     const bool weights = (int)blockIdx.x >= x_blocks;
     for (int i = threadIdx.x; i < 256; i += blockDim.x) s_lut[i] = weights ? tw.v[i] : tx.v[i];
     __syncthreads();
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    constexpr int kChunkBytes = kChunkCodes * BITS / 8;
+    constexpr int kChunkVecs = kChunkBytes / 16;
+    const int64_t items = (packed_bytes + kChunkBytes - 1) / kChunkBytes;
+    const bool vec_ok = (reinterpret_cast<uintptr_t>(x) & 15) == 0;
+    const int64_t first_item = (int64_t)blockIdx.x * kWarpsPerBlock + warp;
+    float4 v[8];
+    auto load_item = [&](int64_t item) {
+        const int64_t c0 = item * kChunkCodes;
+        const float *src = x + c0;
+        const int64_t valid = min((int64_t)kChunkCodes, max((int64_t)0, n - c0));
+        if (valid == kChunkCodes && vec_ok) {
+            const float4 *s4 = reinterpret_cast<const float4 *>(src);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) v[j] = __ldcs(s4 + j * 32 + lane);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int64_t i0 = j * 128 + lane * 4;
+                v[j].x = (i0 + 0 < valid) ? src[i0 + 0] : 0.0f;
+                v[j].y = (i0 + 1 < valid) ? src[i0 + 1] : 0.0f;
+                v[j].z = (i0 + 2 < valid) ? src[i0 + 2] : 0.0f;
+                v[j].w = (i0 + 3 < valid) ? src[i0 + 3] : 0.0f;
+            }
+        }
+    };
+    // With `partials` the kernel in front of this one is the max-abs pass over the same x, which only reads it: x
+    // itself was complete before that pass began, so the first chunk can be fetched while it is still draining.
+    const bool early = partials != nullptr && !weights && first_item < items;
+    if (early) load_item(first_item);
     pdl_enter();
     if (weights) {
+        if (wj.use4) {
+            // 4-bit codes through the 16-entry register table: one 16-byte vector of codes per step
+            const Expand4Job &j = wj.job4;
+            const int64_t total = j.rows * j.vecs_per_row;
+            const unsigned t[4] = {j.tab[0], j.tab[1], j.tab[2], j.tab[3]};
+            const bool ng = j.neg_high != 0;
+            for (int64_t i = (int64_t)(blockIdx.x - x_blocks) * blockDim.x + threadIdx.x; i < total;
+                 i += (int64_t)(gridDim.x - x_blocks) * blockDim.x) {
+                const int64_t row = i / j.vecs_per_row, col = i - row * j.vecs_per_row;
+                const uint4 w = __ldg(reinterpret_cast<const uint4 *>(j.packed + row * j.in_stride) + col);
+                uint4 o0, o1;
+                o0.x = expand4_lookup(w.x, t, ng); o0.y = expand4_lookup(w.x >> 16, t, ng);
+                o0.z = expand4_lookup(w.y, t, ng); o0.w = expand4_lookup(w.y >> 16, t, ng);
+                o1.x = expand4_lookup(w.z, t, ng); o1.y = expand4_lookup(w.z >> 16, t, ng);
+                o1.z = expand4_lookup(w.w, t, ng); o1.w = expand4_lookup(w.w >> 16, t, ng);
+                uint4 *dst = reinterpret_cast<uint4 *>(j.out + row * j.out_stride + col * 32);
+                dst[0] = o0;
+                dst[1] = o1;
+            }
+            return;
+        }
         constexpr int per_chunk = 16 / ELEM;
         const int64_t chunks_per_row = wj.cols / per_chunk;
         const int64_t total = wj.rows * chunks_per_row;
@@ -287,34 +341,12 @@ quantize_expand_kernel(const float *__restrict__ x, int64_t n, const float *__re
         }
         return;
     }
-    const int lane = threadIdx.x & 31;
-    const int warp = threadIdx.x >> 5;
     // the scale is either there already, or made here from the per-block maxima the preceding absmax launch left
     const float inv = partials ? scale_from_partials(partials, n_partials, m, scale_out) : __ldg(scale + 1);
-    constexpr int kChunkBytes = kChunkCodes * BITS / 8;
-    constexpr int kChunkVecs = kChunkBytes / 16;
-    const int64_t items = (packed_bytes + kChunkBytes - 1) / kChunkBytes;
-    const bool vec_ok = (reinterpret_cast<uintptr_t>(x) & 15) == 0;
-    for (int64_t item = (int64_t)blockIdx.x * kWarpsPerBlock + warp; item < items; item += (int64_t)x_blocks * kWarpsPerBlock) {
+    for (int64_t item = first_item; item < items; item += (int64_t)x_blocks * kWarpsPerBlock) {
         const int64_t c0 = item * kChunkCodes;
-        const float *src = x + c0;
-        const int64_t valid = min((int64_t)kChunkCodes, max((int64_t)0, n - c0));
         const int nvec = (int)min((int64_t)kChunkVecs, (packed_bytes - item * kChunkBytes) / 16);
-        float4 v[8];
-        if (valid == kChunkCodes && vec_ok) {
-            const float4 *s4 = reinterpret_cast<const float4 *>(src);
-#pragma unroll
-            for (int j = 0; j < 8; ++j) v[j] = __ldcs(s4 + j * 32 + lane);
-        } else {
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const int64_t i0 = j * 128 + lane * 4;
-                v[j].x = (i0 + 0 < valid) ? src[i0 + 0] : 0.0f;
-                v[j].y = (i0 + 1 < valid) ? src[i0 + 1] : 0.0f;
-                v[j].z = (i0 + 2 < valid) ? src[i0 + 2] : 0.0f;
-                v[j].w = (i0 + 3 < valid) ? src[i0 + 3] : 0.0f;
-            }
-        }
+        if (!(early && item == first_item)) load_item(item);
 #pragma unroll
         for (int j = 0; j < 8; ++j) s_codes[warp][j * 32 + lane] = encode4<BITS, SIGNED>(v[j], inv);
         __syncwarp();
@@ -380,10 +412,16 @@ static dybit_status launch_quantize_expand_bits(const float *x, int64_t n, bool 
                                                 int n_partials, float *scale_out, cudaStream_t s) {
     const int m = is_signed ? BITS - 1 : BITS;
     constexpr int kChunkBytes = kChunkCodes * BITS / 8;
-    const int x_blocks = stream_grid((packed_bytes + kChunkBytes - 1) / kChunkBytes);
-    int64_t w_blocks = (wj.rows * (wj.cols * ELEM / 16) + kStreamThreads - 1) / kStreamThreads;
+    // one wave: three blocks fit an SM, the weights' blocks (a few 16-byte chunks per thread) take their share of
+    // it and the activation's blocks loop over what is left of the chunks
+    const int64_t resident = (int64_t)sm_count() * 3;
+    int64_t w_blocks = (wj.rows * (wj.cols * ELEM / 16) + kStreamThreads * 4 - 1) / (kStreamThreads * 4);
     if (w_blocks > sm_count()) w_blocks = sm_count();
     if (w_blocks < 1) w_blocks = 1;
+    int64_t x_blocks64 = ((packed_bytes + kChunkBytes - 1) / kChunkBytes + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    if (x_blocks64 > resident - w_blocks) x_blocks64 = resident - w_blocks;
+    if (x_blocks64 < 1) x_blocks64 = 1;
+    const int x_blocks = (int)x_blocks64;
     const unsigned grid = (unsigned)(x_blocks + w_blocks);
     if (is_signed)
         launch_k(quantize_expand_kernel<BITS, true, ELEM>, dim3(grid), dim3((unsigned)kStreamThreads), (size_t)0, s, x, n, scale, packed,
@@ -905,6 +943,28 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    // The producer's coordinates of its first tile (a few integer divisions, ~0.7 us in a single thread) are worked
+    // out before the wait below, so they overlap the predecessor's tail.  im2col mode: window origin of the
+    // tile's first output pixel.
+    struct TileOrigin { int m_blk, n_blk, iw, ih, img; };
+    auto tile_origin = [&](int tile) {
+        TileOrigin o = {0, 0, 0, 0, 0};
+        tile_coords(tile, p.m_tiles, p.n_tiles, o.m_blk, o.n_blk);
+        if (AMODE == kAIm2col) {
+            const int m0 = o.m_blk * kBM;
+            o.img = m0 / (p.OH * p.OW);
+            const int rem = m0 - o.img * (p.OH * p.OW);
+            const int oh = rem / p.OW;
+            o.ih = oh * p.stride - p.pad;
+            o.iw = (rem - oh * p.OW) * p.stride - p.pad;
+        }
+        return o;
+    };
+    TileOrigin first = {0, 0, 0, 0, 0};
+    if (threadIdx.x == 0 && (int)blockIdx.x < total_tiles) {
+        first = tile_origin(blockIdx.x);
+        asm volatile("" : "+r"(first.m_blk), "+r"(first.n_blk), "+r"(first.iw), "+r"(first.ih), "+r"(first.img));
+    }
     // everything above touched only this CTA's own resources; operands, scales and outputs come next
     pdl_enter();
 
@@ -914,18 +974,9 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             uint32_t it = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-                int m_blk, n_blk;
-                tile_coords(tile, p.m_tiles, p.n_tiles, m_blk, n_blk);
-                // im2col mode: window origin of the tile's first output pixel, and the running filter tap
-                int iw = 0, ih = 0, img = 0, fr = 0, fs = 0, cb = 0;
-                if (AMODE == kAIm2col) {
-                    const int m0 = m_blk * kBM;
-                    img = m0 / (p.OH * p.OW);
-                    const int rem = m0 - img * (p.OH * p.OW);
-                    const int oh = rem / p.OW;
-                    ih = oh * p.stride - p.pad;
-                    iw = (rem - oh * p.OW) * p.stride - p.pad;
-                }
+                const TileOrigin o = tile == (int)blockIdx.x ? first : tile_origin(tile);
+                const int m_blk = o.m_blk, n_blk = o.n_blk, iw = o.iw, ih = o.ih, img = o.img;
+                int fr = 0, fs = 0, cb = 0;                     // im2col mode: the running filter tap
                 for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
                     const int s = it % kStages;
                     const uint32_t ph = (it / kStages) & 1u;
@@ -1038,9 +1089,12 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 }
                 if (p.tma_store) {
                     // stage 128 rows x 128 bytes in the TMA's 128-byte swizzle, then one thread stores the box;
-                    // rows / columns beyond C are clipped by the tensor map
-                    uint8_t *stage = c_stages + group * L::kCStage;
-                    if (issuer) bulk_wait_group_read<0>();        // the store that last read this buffer is done with it
+                    // rows / columns beyond C are clipped by the tensor map.  In the CTA's last tile the operand
+                    // stages are idle (the commit that published this accumulator followed the last MMA), so every
+                    // chunk takes a buffer of its own there and no store waits for the one before it.
+                    const bool last_tile = tile + (int)gridDim.x >= total_tiles;
+                    uint8_t *stage = last_tile ? a_stages + cc * L::kCStage : c_stages + group * L::kCStage;
+                    if (issuer && !last_tile) bulk_wait_group_read<0>();   // the store that last read this buffer is done with it
                     named_barrier(1 + group, 128);
                     uint8_t *srow = stage + row_in_tile * 128;
 #pragma unroll
@@ -1691,7 +1745,9 @@ static dybit_status conv_impl(const dybit_conv_desc *d, const void *X, dybit_fmt
         uint8_t *packed = static_cast<uint8_t *>(const_cast<void *>(X));
         const int64_t packed_bytes = (int64_t)dybit_packed_bytes(n_x, fx.bits);
         if (fused) {
-            const FusedWeights wj = {static_cast<const uint8_t *>(W), fw.bits, N, ldw_bytes, wrb / elem, we, wrb};
+            FusedWeights wj = {static_cast<const uint8_t *>(W), fw.bits, N, ldw_bytes, wrb / elem, we, wrb, 0, {}};
+            const ExpandOperand opw = {static_cast<const uint8_t *>(W), fw.bits, N, ldw_bytes, wrb / elem, we, wrb, &tw};
+            wj.use4 = expand4_job(opw, elem, i8, &wj.job4) ? 1 : 0;
             uint8_t *const dense = patch_dense ? xd : xe;         // code order either way
             const int64_t dense_bytes = patch_dense ? cv.xd_bytes : cv.a_bytes;
             st = elem == 1 ? launch_quantize_expand<1>(xq->x, n_x, fx, scale_x, packed, packed_bytes, dense, dense_bytes, tx, wj, tw,

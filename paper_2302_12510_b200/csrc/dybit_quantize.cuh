@@ -113,22 +113,20 @@ absmax_kernel(const float *__restrict__ x, int64_t rows, int64_t cols, int64_t l
         if (head > n) head = n;
         const int64_t nvec = (n - head) / 4;
         const float4 *xv = reinterpret_cast<const float4 *>(x + head);
-        constexpr int kUnroll = 4;
-        int64_t i = tid;
-        for (; i + (kUnroll - 1) * nthreads < nvec; i += kUnroll * nthreads) {
+        // eight independent 16-byte loads per thread and round trip (the ragged end reads zeros instead)
+        constexpr int kUnroll = 8;
+        for (int64_t i = tid; i < nvec; i += kUnroll * nthreads) {
             float4 v[kUnroll];
 #pragma unroll
-            for (int u = 0; u < kUnroll; ++u) v[u] = STREAM ? __ldcs(xv + i + u * nthreads) : __ldg(xv + i + u * nthreads);
+            for (int u = 0; u < kUnroll; ++u) {
+                const int64_t iu = i + u * nthreads;
+                v[u] = iu < nvec ? (STREAM ? __ldcs(xv + iu) : __ldg(xv + iu)) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
 #pragma unroll
             for (int u = 0; u < kUnroll; ++u) {
                 best = max(best, max(max(finite_abs_bits(v[u].x), finite_abs_bits(v[u].y)),
                                      max(finite_abs_bits(v[u].z), finite_abs_bits(v[u].w))));
             }
-        }
-        for (; i < nvec; i += nthreads) {
-            float4 v = STREAM ? __ldcs(xv + i) : __ldg(xv + i);
-            best = max(best, max(max(finite_abs_bits(v.x), finite_abs_bits(v.y)),
-                                 max(finite_abs_bits(v.z), finite_abs_bits(v.w))));
         }
         if (tid < head) best = max(best, finite_abs_bits(x[tid]));
         const int64_t tail0 = head + nvec * 4;
@@ -866,7 +864,7 @@ static dybit_status launch_absmax(const float *x, int64_t rows, int64_t cols, in
     if (n > 0) {
         // few, fat blocks: every block ends with two atomics on the same words
         int64_t blocks = (n / 4 + kStreamThreads * 8 - 1) / (kStreamThreads * 8);
-        int64_t cap = (int64_t)sm_count() * 4;
+        int64_t cap = (int64_t)sm_count() * 4;          // what the register file holds at once
         if (cap > kMaxAbsmaxPartials) cap = kMaxAbsmaxPartials;
         if (blocks > cap) blocks = cap;
         if (blocks < 1) blocks = 1;
