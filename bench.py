@@ -153,9 +153,11 @@ class LayerwiseStep:
     def alloc_host_outputs(self):
         self.y_host = [torch.empty(y.shape, dtype=torch.float32).pin_memory() for y in self.y]
 
-    def step(self, events=None):
+    def step(self, events=None, clocks=None):
         dy = self.dy
         for i in range(len(self.layers)):
+            if clocks is not None:
+                dy.dybit_profile_next_gemm_clock(clocks[i])
             if events is not None:
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 dy.dybit_profile_next_gemm(e0, e1)
@@ -753,6 +755,21 @@ def main():
     st, detail = dy.dybit_last_device_status()
     if st != 0:
         raise SystemExit(f"device status {st} detail {detail:#x}")
+    # ---- and on the device's own clock inside graph replays: per layer, first CTA past the dependency wait to last
+    #      CTA retired (the event pairs above also contain the launch latency that the graph's overlapped launches hide)
+    clk = torch.empty((len(work.layers), 2), dtype=torch.int64, device=device)
+    graph_c = capture_step(work, device, lambda: work.step(clocks=clk))
+    clock_us = [0.0] * len(work.layers)
+    clock_reps = 10
+    for rep in range(clock_reps + 2):
+        clk[:, 0] = -1
+        clk[:, 1] = 0
+        graph_c.replay()
+        torch.cuda.synchronize(device)
+        if rep >= 2:
+            span = (clk[:, 1] - clk[:, 0]).cpu().tolist()
+            clock_us = [a + s * 1e-3 / clock_reps for a, s in zip(clock_us, span)]
+    del graph_c
     mma_ms = [sum(e0.elapsed_time(e1) for e0, e1 in ev) / len(ev) for ev in events]
     mma_total_ms = sum(mma_ms)
     peak_tensor = 2.0 * peaks["bf16_tflops_sustained"]      # int8 = 2 x bf16 (nominal ratio), sustained: inside a long step
@@ -779,6 +796,14 @@ def main():
         "ms_per_step_direct_launch": ms_eager,
         "layers_us": {L.name: [round(t * 1e3, 1), round(b[2] * 1e6, 1)] for L, t, b in zip(work.layers, mma_ms, bounds)},
         "frac_of_layerwise_bound": ideal_s / (mma_total_ms * 1e-3),
+        "device_clock": {
+            "what": "the same kernel timed by %%globaltimer inside CUDA-graph replays of the step (dybit_profile_next_gemm_clock): "
+                    "first CTA past its dependency wait to last CTA retired, mean of %d replays" % clock_reps,
+            "ms_per_step_in_kernel": sum(clock_us) * 1e-3, "share_of_step": sum(clock_us) * 1e-3 / ms_step,
+            "achieved": (flops_total / 1e12 if tensor_bound else bytes_total / 1e9) / (sum(clock_us) * 1e-6),
+            "frac": (flops_total / 1e12 if tensor_bound else bytes_total / 1e9) / (sum(clock_us) * 1e-6) / peak,
+            "frac_of_layerwise_bound": ideal_s / (sum(clock_us) * 1e-6),
+            "layers_us": {L.name: round(t, 1) for L, t in zip(work.layers, clock_us)}},
         "algorithmic_flops_per_step": flops_total, "algorithmic_bytes_per_step": bytes_total,
     }
 

@@ -365,6 +365,16 @@ uint64_t dybit_launch_count(void);
  * then disarms.  Both are cudaEvent_t passed as void*; NULL, NULL disarms. */
 dybit_status dybit_profile_next_gemm(void *ev_start, void *ev_stop);
 
+/* The same arming for the device's own clock: the CTAs of the next
+ * tensor-core kernel min-reduce the time at which they pass the dependency
+ * wait into t2[0] and max-reduce the time at which they retire into t2[1]
+ * (nanoseconds of %globaltimer; device memory, 8-byte aligned, initialised
+ * by the caller to {UINT64_MAX, 0}).  Unlike an event pair this brackets the
+ * kernel's own run even inside a CUDA graph replay, where neighbouring
+ * launches overlap its prologue; stores still in flight when the last CTA
+ * retires are not covered.  NULL disarms. */
+dybit_status dybit_profile_next_gemm_clock(unsigned long long *t2);
+
 #ifdef __cplusplus
 }
 #endif

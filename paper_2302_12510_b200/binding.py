@@ -20,7 +20,7 @@ __all__ = [
     "dybit_choose_container", "dybit_gemm_workspace_bytes", "dybit_conv2d_workspace_bytes",
     "dybit_conv2d_out_hw", "dybit_absmax_scale", "dybit_quantize_pack", "dybit_quantize_pack_2d",
     "dybit_decode", "dybit_gemm", "dybit_conv2d", "dybit_last_device_status",
-    "dybit_launch_count", "dybit_profile_next_gemm", "dybit_gemm_static_ws", "STATIC_WS_BYTES",
+    "dybit_launch_count", "dybit_profile_next_gemm", "dybit_profile_next_gemm_clock", "dybit_gemm_static_ws", "STATIC_WS_BYTES",
     "dybit_gemm_requant", "dybit_conv2d_requant", "dybit_depthwise_conv2d", "dybit_gemm_batched",
     "dybit_quantize_conv2d",
     "dybit_gemm_batched_workspace_bytes", "dybit_rmse", "dybit_rmse_sweep", "dybit_fake_quant", "dybit_fake_quant_backward",
@@ -96,6 +96,7 @@ def _load() -> C.CDLL:
     lib.dybit_launch_count.restype = C.c_uint64
     lib.dybit_launch_count.argtypes = []
     lib.dybit_profile_next_gemm.argtypes = [vp, vp]
+    lib.dybit_profile_next_gemm_clock.argtypes = [vp]
     lib.dybit_gemm_requant.argtypes = [i64, i64, i64, vp, _CFmt, vp, i64, vp, _CFmt, vp, i64,
                                        _CFmt, vp, vp, i32, vp, i64, vp, sz, vp]
     lib.dybit_conv2d_requant.argtypes = [C.POINTER(_CConvDesc), vp, _CFmt, vp, vp, _CFmt, vp, i64,
@@ -313,6 +314,14 @@ def dybit_profile_next_gemm(ev_start: Optional[torch.cuda.Event], ev_stop: Optio
             ev.record()
     _check(lib.dybit_profile_next_gemm(C.c_void_p(ev_start.cuda_event), C.c_void_p(ev_stop.cuda_event)),
            "dybit_profile_next_gemm")
+
+
+def dybit_profile_next_gemm_clock(t2: Optional[torch.Tensor]):
+    """Arms device-clock recording for the next GEMM/conv tensor-core kernel: t2 is an int64 device tensor of two
+    elements, initialised to {-1 (all ones), 0}, that receives {first start, last end} in nanoseconds."""
+    if t2 is not None and (t2.dtype != torch.int64 or t2.numel() < 2 or not t2.is_cuda):
+        raise ValueError("t2 must be an int64 CUDA tensor of two elements")
+    _check(lib.dybit_profile_next_gemm_clock(_ptr(t2)), "dybit_profile_next_gemm_clock")
 
 
 STATIC_WS_BYTES = 16 * 1024 * 1024   # DYBIT_STATIC_WS_BYTES in include/dybit.h

@@ -67,6 +67,7 @@ __device__ __forceinline__ void pdl_enter() {
 
 struct ProfileEvents {
     cudaEvent_t start = nullptr, stop = nullptr;
+    unsigned long long *clock = nullptr;      // device pair {first start, last end} in %globaltimer ns
 };
 inline ProfileEvents &profile_events() {
     static thread_local ProfileEvents ev;

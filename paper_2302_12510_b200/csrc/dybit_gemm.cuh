@@ -770,6 +770,7 @@ struct GemmParams {
     const float *scale_q;     // {scale, 1/scale} of the output tensor
     int q_bits, q_signed, relu;
     const float *bias;        // requant only: one fp32 per output column, or null
+    unsigned long long *clock; // profiling: {min start after the dependency wait, max end} in %globaltimer ns, or null
     int bmt;                  // batched GEMM: M tiles per batch entry (0: not batched); M is then one entry's rows
     int64_t c_bstride;        // batched GEMM: elements between consecutive entries of C / C_raw
 };
@@ -967,6 +968,7 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     }
     // everything above touched only this CTA's own resources; operands, scales and outputs come next
     pdl_enter();
+    if (p.clock != nullptr && threadIdx.x == 32) atomicMin(p.clock, (unsigned long long)global_timer_ns());
 
     if (warp == 0) {
         // ------------------------------------------------ TMA producer
@@ -1227,6 +1229,7 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
 
     tc_fence_before_sync();
     __syncthreads();
+    if (p.clock != nullptr && threadIdx.x == 32) atomicMax(p.clock + 1, (unsigned long long)global_timer_ns());
     if (warp == 1) {
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, kTmemCols);
@@ -1358,6 +1361,7 @@ static dybit_status launch_gemm_inst(const CUtensorMap &ta, const CUtensorMap &t
     const int grid = tiles < sm_count() ? tiles : sm_count();
     ProfileEvents ev = profile_events();
     profile_events() = ProfileEvents();
+    p.clock = ev.clock;
     if (ev.start) DYBIT_CUDA_TRY(cudaEventRecord(ev.start, s));
     launch_k(kern, dim3((unsigned)(grid)), dim3((unsigned)(CONV ? 448 : 320)), (size_t)(L::kBytes), s, ta, tb, tc, p);
     const dybit_status st = launch_status();

@@ -297,6 +297,12 @@ dybit_status dybit_profile_next_gemm(void *ev_start, void *ev_stop) {
     return DYBIT_OK;
 }
 
+dybit_status dybit_profile_next_gemm_clock(unsigned long long *t2) {
+    if (!dybit::aligned(t2, 8)) return DYBIT_ERR_ALIGNMENT;
+    dybit::profile_events().clock = t2;
+    return DYBIT_OK;
+}
+
 dybit_status dybit_last_device_status(void *stream, uint32_t *detail) {
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     unsigned int word = 0, zero = 0;

@@ -144,3 +144,26 @@ def test_gemm_argument_errors():
         dy.dybit_gemm(4, 4, 128, pa, (8, 1), one, pa, (8, 1), one, want_raw=True, lda_bytes=128, ldb_bytes=128)
     assert e.value.status in (1, 2)
     del ws
+
+
+def test_profile_clock_brackets_the_kernel():
+    # the device-clock hook: start and end stamps of the tensor-core kernel, result unchanged
+    fa = fb = (4, 1)
+    M, N, K = 300, 200, 384
+    a = wl.normal((M, K), seed=11)
+    b = wl.normal((N, K), seed=12)
+    pa, sa = dy.dybit_quantize_pack_2d(a.to(DEV), fa)
+    pb, sb = dy.dybit_quantize_pack_2d(b.to(DEV), fb)
+    C0, _ = dy.dybit_gemm(M, N, K, pa, fa, sa, pb, fb, sb)
+    t2 = torch.tensor([-1, 0], dtype=torch.int64, device=DEV)
+    dy.dybit_profile_next_gemm_clock(t2)
+    C1, _ = dy.dybit_gemm(M, N, K, pa, fa, sa, pb, fb, sb)
+    torch.cuda.synchronize()
+    start, end = t2.cpu().tolist()
+    assert start > 0 and end > start and end - start < 10_000_000        # nanoseconds
+    assert torch.equal(C0, C1)
+    # disarmed after one kernel: the pair stays as it is
+    before = t2.clone()
+    dy.dybit_gemm(M, N, K, pa, fa, sa, pb, fb, sb)
+    torch.cuda.synchronize()
+    assert torch.equal(before, t2)
