@@ -243,7 +243,33 @@ struct FusedWeights {
     int64_t out_stride;
     int use4;                 // 1: job4 describes the same rows for the 4-bit register-table expansion
     Expand4Job job4;
+    int pix_c, pix_r, pix_s;  // pix_c > 0: filter rows of 8 taps x 4 bytes instead (see expand_weights_pix4)
 };
+
+// Weights for the few-channel lowering (ConvMode kConvPix4): row n of the output holds, for each filter row r,
+// eight taps of four bytes: tap s < S carries its C <= 4 one-byte elements, everything else is zero; rows are
+// padded with zeros to out_stride.  Thread `idx` writes one 16-byte chunk (four taps).
+__device__ __forceinline__ void expand_weights_pix4(const FusedWeights &wj, const uint16_t *s_lut, int64_t idx) {
+    const int64_t chunks_per_row = wj.out_stride / 16;
+    const int64_t row = idx / chunks_per_row;
+    const int g = (int)(idx - row * chunks_per_row);
+    const int r = g >> 1, s0 = (g & 1) * 4;
+    const uint8_t *src = wj.packed + row * wj.in_stride;
+    const unsigned mask = (1u << wj.bits) - 1u;
+    unsigned o[4] = {0, 0, 0, 0};
+    for (int t = 0; t < 4; ++t) {
+        const int s = s0 + t;
+        if (r >= wj.pix_r || s >= wj.pix_s) continue;
+        for (int c = 0; c < wj.pix_c; ++c) {
+            const int64_t bit = (int64_t)((r * wj.pix_s + s) * wj.pix_c + c) * wj.bits;
+            const int sh = (int)(bit & 7);
+            unsigned two = __ldg(src + (bit >> 3));
+            if (sh + wj.bits > 8) two |= (unsigned)__ldg(src + (bit >> 3) + 1) << 8;
+            o[t] |= (unsigned)(s_lut[(two >> sh) & mask] & 0xffu) << (8 * c);
+        }
+    }
+    *reinterpret_cast<uint4 *>(wj.out + row * wj.out_stride + g * 16) = make_uint4(o[0], o[1], o[2], o[3]);
+}
 
 // fp32 activation -> packed codes AND their container elements, plus the layer's weights expanded by the
 // last blocks of the same grid: what dybit_quantize_pack followed by the expand launch of dybit_conv2d
@@ -257,7 +283,8 @@ __global__ void __launch_bounds__(kStreamThreads, 3)
 quantize_expand_kernel(const float *__restrict__ x, int64_t n, const float *__restrict__ scale,
                        uint8_t *__restrict__ packed, int64_t packed_bytes, uint8_t *__restrict__ xe, int64_t xe_bytes,
                        const __grid_constant__ ElemTable tx, const FusedWeights wj, const __grid_constant__ ElemTable tw,
-                       int x_blocks, const unsigned *__restrict__ partials, int n_partials, int m, float *__restrict__ scale_out) {
+                       int x_blocks, const unsigned *__restrict__ partials, int n_partials, int m, float *__restrict__ scale_out,
+                       int pix_c) {
     __shared__ __align__(16) unsigned s_codes[kWarpsPerBlock][kChunkCodes / 4];
     __shared__ __align__(16) unsigned s_words[kWarpsPerBlock][32 * BITS];
     __shared__ uint16_t s_lut[256];
@@ -297,6 +324,13 @@ quantize_expand_kernel(const float *__restrict__ x, int64_t n, const float *__re
     if (early) load_item(first_item);
     pdl_enter();
     if (weights) {
+        if (wj.pix_c > 0) {
+            const int64_t total = wj.rows * (wj.out_stride / 16);
+            for (int64_t idx = (int64_t)(blockIdx.x - x_blocks) * blockDim.x + threadIdx.x; idx < total;
+                 idx += (int64_t)(gridDim.x - x_blocks) * blockDim.x)
+                expand_weights_pix4(wj, s_lut, idx);
+            return;
+        }
         if (wj.use4) {
             // 4-bit codes through the 16-entry register table: one 16-byte vector of codes per step
             const Expand4Job &j = wj.job4;
@@ -369,8 +403,42 @@ quantize_expand_kernel(const float *__restrict__ x, int64_t n, const float *__re
                 for (int i = 0; i < 8; ++i)
                     o[i] = (unsigned)(s_lut[cw[i] & 0xffu] & 0xffu) | ((unsigned)(s_lut[(cw[i] >> 8) & 0xffu] & 0xffu) << 8) |
                            ((unsigned)(s_lut[(cw[i] >> 16) & 0xffu] & 0xffu) << 16) | ((unsigned)(s_lut[cw[i] >> 24] & 0xffu) << 24);
+                if (pix_c > 0) {
+                    // pixels of pix_c < 4 one-byte elements, each padded to a 32-bit word: the chunk's 1024 bytes go
+                    // back to shared memory in element order, lanes then assemble whole pixels; the (at most two)
+                    // pixels that straddle the chunk's ends are completed byte by byte by both chunks involved
+                    __syncwarp();
+                    uint4 *mine = reinterpret_cast<uint4 *>(&s_codes[warp][lane * 8]);
+                    mine[0] = make_uint4(o[0], o[1], o[2], o[3]);
+                    mine[1] = make_uint4(o[4], o[5], o[6], o[7]);
+                    __syncwarp();
+                    const uint8_t *sb = reinterpret_cast<const uint8_t *>(&s_codes[warp][0]);
+                    const int64_t e_end = min(c0 + (int64_t)kChunkCodes, n);
+                    const int64_t p_lo = (c0 + pix_c - 1) / pix_c;      // first pixel that starts in this chunk
+                    const int64_t p_hi = e_end / pix_c;                 // one past the last pixel that ends in it
+                    unsigned *x4 = reinterpret_cast<unsigned *>(xe);
+                    for (int64_t px = p_lo + lane; px < p_hi; px += 32) {
+                        const int o0 = (int)(px * pix_c - c0);
+                        unsigned w = sb[o0];
+                        if (pix_c > 1) w |= (unsigned)sb[o0 + 1] << 8;
+                        if (pix_c > 2) w |= (unsigned)sb[o0 + 2] << 16;
+                        x4[px] = w;
+                    }
+                    if (lane == 0 && p_lo * pix_c > c0 && c0 < e_end) {
+                        // tail of the pixel that began in the previous chunk
+                        const int64_t px = p_lo - 1;
+                        for (int64_t e = c0; e < min(p_lo * pix_c, e_end); ++e) xe[px * 4 + (e - px * pix_c)] = sb[e - c0];
+                    }
+                    if (lane == 1 && p_hi * pix_c < e_end && p_hi >= p_lo) {
+                        // head of the pixel that ends in the next chunk, and its padding bytes
+                        const int64_t px = p_hi;
+                        for (int64_t e = px * pix_c; e < e_end; ++e) xe[px * 4 + (e - px * pix_c)] = sb[e - c0];
+                        for (int b = pix_c; b < 4; ++b) xe[px * 4 + b] = 0;
+                    }
+                } else {
                 if (off + 16 <= xe_bytes) reinterpret_cast<uint4 *>(xe + off)[0] = make_uint4(o[0], o[1], o[2], o[3]);
                 if (off + 32 <= xe_bytes) reinterpret_cast<uint4 *>(xe + off)[1] = make_uint4(o[4], o[5], o[6], o[7]);
+                }
             } else {
                 unsigned o[16];
 #pragma unroll
@@ -409,13 +477,14 @@ template <int BITS, int ELEM>
 static dybit_status launch_quantize_expand_bits(const float *x, int64_t n, bool is_signed, const float *scale, uint8_t *packed,
                                                 int64_t packed_bytes, uint8_t *xe, int64_t xe_bytes, const ElemTable &tx,
                                                 const FusedWeights &wj, const ElemTable &tw, const unsigned *partials,
-                                                int n_partials, float *scale_out, cudaStream_t s) {
+                                                int n_partials, float *scale_out, int pix_c, cudaStream_t s) {
     const int m = is_signed ? BITS - 1 : BITS;
     constexpr int kChunkBytes = kChunkCodes * BITS / 8;
     // one wave: three blocks fit an SM, the weights' blocks (a few 16-byte chunks per thread) take their share of
     // it and the activation's blocks loop over what is left of the chunks
     const int64_t resident = (int64_t)sm_count() * 3;
-    int64_t w_blocks = (wj.rows * (wj.cols * ELEM / 16) + kStreamThreads * 4 - 1) / (kStreamThreads * 4);
+    const int64_t w_chunks = wj.pix_c > 0 ? wj.rows * (wj.out_stride / 16) : wj.rows * (wj.cols * ELEM / 16);
+    int64_t w_blocks = (w_chunks + kStreamThreads * 4 - 1) / (kStreamThreads * 4);
     if (w_blocks > sm_count()) w_blocks = sm_count();
     if (w_blocks < 1) w_blocks = 1;
     int64_t x_blocks64 = ((packed_bytes + kChunkBytes - 1) / kChunkBytes + kWarpsPerBlock - 1) / kWarpsPerBlock;
@@ -425,10 +494,10 @@ static dybit_status launch_quantize_expand_bits(const float *x, int64_t n, bool 
     const unsigned grid = (unsigned)(x_blocks + w_blocks);
     if (is_signed)
         launch_k(quantize_expand_kernel<BITS, true, ELEM>, dim3(grid), dim3((unsigned)kStreamThreads), (size_t)0, s, x, n, scale, packed,
-                 packed_bytes, xe, xe_bytes, tx, wj, tw, x_blocks, partials, n_partials, m, scale_out);
+                 packed_bytes, xe, xe_bytes, tx, wj, tw, x_blocks, partials, n_partials, m, scale_out, pix_c);
     else
         launch_k(quantize_expand_kernel<BITS, false, ELEM>, dim3(grid), dim3((unsigned)kStreamThreads), (size_t)0, s, x, n, scale, packed,
-                 packed_bytes, xe, xe_bytes, tx, wj, tw, x_blocks, partials, n_partials, m, scale_out);
+                 packed_bytes, xe, xe_bytes, tx, wj, tw, x_blocks, partials, n_partials, m, scale_out, pix_c);
     return launch_status();
 }
 
@@ -436,16 +505,16 @@ template <int ELEM>
 static dybit_status launch_quantize_expand(const float *x, int64_t n, dybit_fmt fx, const float *scale, uint8_t *packed,
                                            int64_t packed_bytes, uint8_t *xe, int64_t xe_bytes, const ElemTable &tx,
                                            const FusedWeights &wj, const ElemTable &tw, const unsigned *partials,
-                                           int n_partials, float *scale_out, cudaStream_t s) {
+                                           int n_partials, float *scale_out, int pix_c, cudaStream_t s) {
     const bool sg = fx.is_signed != 0;
     switch (fx.bits) {
-        case 2: return launch_quantize_expand_bits<2, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, s);
-        case 3: return launch_quantize_expand_bits<3, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, s);
-        case 4: return launch_quantize_expand_bits<4, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, s);
-        case 5: return launch_quantize_expand_bits<5, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, s);
-        case 6: return launch_quantize_expand_bits<6, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, s);
-        case 7: return launch_quantize_expand_bits<7, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, s);
-        case 8: return launch_quantize_expand_bits<8, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, s);
+        case 2: return launch_quantize_expand_bits<2, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pix_c, s);
+        case 3: return launch_quantize_expand_bits<3, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pix_c, s);
+        case 4: return launch_quantize_expand_bits<4, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pix_c, s);
+        case 5: return launch_quantize_expand_bits<5, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pix_c, s);
+        case 6: return launch_quantize_expand_bits<6, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pix_c, s);
+        case 7: return launch_quantize_expand_bits<7, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pix_c, s);
+        case 8: return launch_quantize_expand_bits<8, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pix_c, s);
     }
     return DYBIT_ERR_INVALID_ARG;
 }
@@ -688,6 +757,38 @@ patch_gather_kernel(const PatchGatherParams p) {
     }
 }
 
+// Packed NHWC codes with C <= 4 channels -> one 32-bit word per pixel (C one-byte elements, zero padding), and the
+// weights in the matching filter-row layout (expand_weights_pix4), in one launch: blocks [0, x_blocks) take pixels.
+__global__ void __launch_bounds__(256)
+expand_pix4_kernel(const uint8_t *__restrict__ packed, int bits, int64_t pixels, int c, unsigned *__restrict__ x4,
+                   const __grid_constant__ ElemTable tx, const FusedWeights wj, const __grid_constant__ ElemTable tw,
+                   int x_blocks) {
+    __shared__ uint16_t s_lut[256];
+    const bool weights = (int)blockIdx.x >= x_blocks;
+    for (int i = threadIdx.x; i < 256; i += blockDim.x) s_lut[i] = weights ? tw.v[i] : tx.v[i];
+    __syncthreads();
+    pdl_enter();
+    if (weights) {
+        const int64_t total = wj.rows * (wj.out_stride / 16);
+        for (int64_t idx = (int64_t)(blockIdx.x - x_blocks) * blockDim.x + threadIdx.x; idx < total;
+             idx += (int64_t)(gridDim.x - x_blocks) * blockDim.x)
+            expand_weights_pix4(wj, s_lut, idx);
+        return;
+    }
+    const unsigned mask = (1u << bits) - 1u;
+    for (int64_t px = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; px < pixels; px += (int64_t)x_blocks * blockDim.x) {
+        unsigned w = 0;
+        int64_t bit = px * c * bits;
+        for (int ch = 0; ch < c; ++ch, bit += bits) {
+            const int sh = (int)(bit & 7);
+            unsigned two = __ldg(packed + (bit >> 3));
+            if (sh + bits > 8) two |= (unsigned)__ldg(packed + (bit >> 3) + 1) << 8;
+            w |= (unsigned)(s_lut[(two >> sh) & mask] & 0xffu) << (8 * ch);
+        }
+        x4[px] = w;
+    }
+}
+
 template <int ELEM>
 static dybit_status launch_expand_rows(const uint8_t *packed, int bits, int64_t rows, int64_t in_stride, int64_t cols,
                                        uint8_t *out, int64_t out_stride, const ElemTable &t, cudaStream_t s) {
@@ -798,7 +899,9 @@ __device__ __forceinline__ bool wait_bounded(uint64_t *bar, uint32_t parity, vol
 // How the A tile reaches shared memory.
 enum AMode { kATiled = 0,    // GEMM: 2-D tiled TMA
              kAGather = 1,   // conv: four warps gather 16-byte chunks with cp.async (any channel count)
-             kAIm2col = 2 }; // conv: one im2col TMA per stage (pixel = a whole number of SWB-byte blocks)
+             kAIm2col = 2,   // conv: one im2col TMA per stage (pixel = a whole number of SWB-byte blocks)
+             kAGather4 = 3 };// conv with <= 4 one-byte channels: pixels are 32-bit words, a K block = four filter rows of
+                             // eight taps, gathered with 4-byte cp.async
 
 // Re-quantizing epilogue (Section III-B.1: results are quantized to DyBit before they are written back):
 // 32 consecutive outputs of one row -> 32 codes of the output format -> 4*BITS bytes at dst.
@@ -895,11 +998,11 @@ __device__ __forceinline__ void tile_coords(int tile, int m_tiles, int n_tiles, 
 }
 
 template <Kind KIND, int BN, int AMODE, int SWB>
-__global__ void __launch_bounds__(AMODE == kAGather ? 448 : 320, 1)
+__global__ void __launch_bounds__((AMODE == kAGather || AMODE == kAGather4) ? 448 : 320, 1)
 dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                   const __grid_constant__ CUtensorMap tmap_c, const GemmParams p) {
-    static_assert(AMODE != kAGather || SWB == 128, "the cp.async gather writes 128-byte rows");
-    constexpr bool CONV = AMODE == kAGather;          // extra gather warps present
+    static_assert((AMODE != kAGather && AMODE != kAGather4) || SWB == 128, "the cp.async gather writes 128-byte rows");
+    constexpr bool CONV = AMODE == kAGather || AMODE == kAGather4;          // extra gather warps present
     using L = GemmSmem<BN, SWB>;
     constexpr int kStages = L::kStages;
     constexpr int kGatherThreads = 128;
@@ -932,7 +1035,7 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         }
         *abort_flag = 0;
         fence_mbar_init();
-        if (AMODE != kAGather) prefetch_tensormap(&tmap_a);
+        if (!CONV) prefetch_tensormap(&tmap_a);
         prefetch_tensormap(&tmap_b);
         if (p.tma_store) prefetch_tensormap(&tmap_c);
     }
@@ -1175,6 +1278,15 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             const int oh = rem / p.OW, ow = rem - oh * p.OW;
             const int ih0 = oh * p.stride - p.pad, iw0 = ow * p.stride - p.pad;
             const uint8_t *img_base = p.xe + (int64_t)img * p.H * p.W * p.cpb;
+            // pixel-word mode: pointer to the window's first column in image row 0 (only dereferenced where the mask
+            // allows), and the taps of a filter row that exist and fall inside the image horizontally
+            const unsigned *pix_base = reinterpret_cast<const unsigned *>(p.xe) + (int64_t)img * p.H * p.W + iw0;
+            unsigned col_mask = 0;
+            if (AMODE == kAGather4) {
+#pragma unroll
+                for (int fs4 = 0; fs4 < 8; ++fs4)
+                    if (fs4 < p.S && (unsigned)(iw0 + fs4) < (unsigned)p.W) col_mask |= 1u << fs4;
+            }
             // filter tap (fr, fs) and byte offset inside the pixel, advanced chunk by chunk: K runs (r, s, c)
             int fr = 0, fs = 0, cb = 0;
             for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
@@ -1182,7 +1294,29 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 const uint32_t ph = (it / kStages) & 1u;
                 if (!wait_bounded(&empty[s], ph ^ 1u, abort_flag, 5)) { ok = false; break; }
                 const uint32_t dst_row = smem_u32(a_stages + s * L::kAStage) + (uint32_t)t * kBKBytes;
-                if (p.cpb % kBKBytes == 0) {
+                if (AMODE == kAGather4) {
+                    // the row = four filter rows (4*kb ..) of eight 4-byte slots, slot s = tap s: every slot is
+                    // written, with the pixel it points at where that tap exists and lies inside the image, with
+                    // zeros otherwise (straight-line code: the zero fill is a copy of size 0, not a branch)
+                    const unsigned *zero_src = reinterpret_cast<const unsigned *>(p.xe);
+#pragma unroll
+                    for (int jj = 0; jj < 4; ++jj) {
+                        const int r = kb * 4 + jj;
+                        const int ih = ih0 + r;
+                        const bool row_in = row_ok && r < p.R && (unsigned)ih < (unsigned)p.H;
+                        const unsigned *src_row = row_in ? pix_base + (int64_t)ih * p.W : zero_src;
+                        const unsigned mask = row_in ? col_mask : 0u;
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            const uint32_t dst = dst_row + (uint32_t)(((jj * 2 + h) ^ sw) << 4);
+#pragma unroll
+                            for (int w = 0; w < 4; ++w) {
+                                const bool in = (mask >> (h * 4 + w)) & 1u;
+                                cp_async_4(dst + w * 4, in ? src_row + (h * 4 + w) : zero_src, in ? 4u : 0u);
+                            }
+                        }
+                    }
+                } else if (p.cpb % kBKBytes == 0) {
                     // a pixel holds whole 128-byte blocks: the eight chunks share one tap and are contiguous
                     const int ih = ih0 + fr * p.dil, iw = iw0 + fs * p.dil;
                     const bool in = row_ok && fr < p.R && (unsigned)ih < (unsigned)p.H && (unsigned)iw < (unsigned)p.W;
@@ -1348,7 +1482,7 @@ static dybit_status launch_gemm_inst(const CUtensorMap &ta, const CUtensorMap &t
     p.tma_store = (p.Q == nullptr && make_output_map(&tc, p.C, p.M, p.N, p.ldc, p.bmt ? p.m_tiles / p.bmt : 0, p.c_bstride)) ? 1 : 0;
     using L = GemmSmem<BN, SWB>;
     auto kern = dybit_gemm_kernel<KIND, BN, AMODE, SWB>;
-    constexpr bool CONV = AMODE == kAGather;
+    constexpr bool CONV = AMODE == kAGather || AMODE == kAGather4;
     static bool configured[64] = {};
     int dev = 0;
     DYBIT_CUDA_TRY(cudaGetDevice(&dev));
@@ -1385,7 +1519,9 @@ static dybit_status launch_gemm_kind(dybit_container cont, int bn, const CUtenso
     switch (cont) {
         case DYBIT_CONTAINER_I8: return launch_gemm_bn<Kind::I8, AMODE, SWB>(bn, ta, tb, p, s);
         case DYBIT_CONTAINER_E4M3: return launch_gemm_bn<Kind::F8F6F4, AMODE, SWB>(bn, ta, tb, p, s);
-        default: return launch_gemm_bn<Kind::F16, AMODE, SWB>(bn, ta, tb, p, s);
+        default:
+            if constexpr (AMODE == kAGather4) return DYBIT_ERR_UNSUPPORTED;     // one-byte elements only
+            else return launch_gemm_bn<Kind::F16, AMODE, SWB>(bn, ta, tb, p, s);
     }
 }
 
@@ -1452,7 +1588,7 @@ static void apply_requant(GemmParams &p, const RequantSpec *rq) {
 }
 
 // How a convolution is lowered, and what it needs in the workspace.
-enum ConvMode { kConvPointwise, kConvIm2col, kConvPatch, kConvGather };
+enum ConvMode { kConvPointwise, kConvIm2col, kConvPix4, kConvPatch, kConvGather };
 struct ConvPlan {
     ConvMode mode;
     int elem, swb;
@@ -1480,11 +1616,19 @@ static ConvPlan plan_conv(const dybit_conv_desc *d, int oh, int ow, int elem) {
     const bool im2col_ok = c.swb != 0 && c.pixels * c.cpb >= 131072 && d->pad <= 127 && up_w >= -128 && up_h >= -128 &&
                            (d->s - 1) * d->dilation <= 255 && (d->r - 1) * d->dilation <= 255 && d->stride <= 8;
     const int64_t krow = round_up(taps * d->c * elem, 16);
+    // at most four one-byte channels (the 3-channel stem): pixels become 32-bit words and the tensor-core kernel
+    // gathers its A tile from them, four filter rows of eight taps per K block; no patch matrix is written
+    const bool pix4_ok = elem == 1 && d->c <= 4 && d->dilation == 1 && d->s <= 8 && d->r <= 64;
     if (pointwise) c.mode = kConvPointwise;
     else if (im2col_ok) c.mode = kConvIm2col;
+    else if (pix4_ok) c.mode = kConvPix4;
     else if (krow <= 1024 && M * krow <= ((int64_t)1 << 32)) c.mode = kConvPatch;
     else c.mode = kConvGather;
-    if (c.mode == kConvPatch) {
+    if (c.mode == kConvPix4) {
+        c.a_bytes = round_up(c.pixels * 4, 1024) + 1024;
+        c.wrb = round_up((int64_t)d->r * 32, kBKBytes);
+        c.pad_channels = false;
+    } else if (c.mode == kConvPatch) {
         c.krow = krow;
         c.a_bytes = round_up(M * krow, 1024);
         c.wrb = k_row_bytes(taps * d->c, elem);
@@ -1722,6 +1866,8 @@ static dybit_status conv_impl(const dybit_conv_desc *d, const void *X, dybit_fmt
     uint8_t *we = xe + cv.a_bytes;
     uint8_t *xd = we + round_up(N * wrb, 1024);              // patch mode: dense container elements of the activation
     const bool patch_dense = cv.mode == kConvPatch && cv.xd_bytes > 0;
+    const bool pix4 = cv.mode == kConvPix4;
+    FusedWeights wpix = {static_cast<const uint8_t *>(W), fw.bits, N, ldw_bytes, wrb, we, wrb, 0, {}, d->c, d->r, d->s};
     const ElemTable &tx = make_elem_table(fx, plan.container, plan.exp_a);
     const ElemTable &tw = make_elem_table(fw, plan.container, plan.exp_b);
     const bool i8 = plan.container == DYBIT_CONTAINER_I8;
@@ -1731,7 +1877,7 @@ static dybit_status conv_impl(const dybit_conv_desc *d, const void *X, dybit_fmt
         // order itself, one launch writes the codes, their container elements and the expanded weights
         const int64_t n_x = pixels * d->c;
         float *scale_dst = const_cast<float *>(scale_x);
-        const bool fused = patch_dense || (cv.mode != kConvPatch && !cv.pad_channels);
+        const bool fused = patch_dense || pix4 || (cv.mode != kConvPatch && !cv.pad_channels);
         // max-abs scale: in the fused case the absmax launch leaves one maximum per block in the workspace and the
         // quantize launch folds them (nothing to zero first, no atomics); otherwise the ticket version writes the pair
         unsigned *partials = nullptr;
@@ -1749,15 +1895,17 @@ static dybit_status conv_impl(const dybit_conv_desc *d, const void *X, dybit_fmt
         uint8_t *packed = static_cast<uint8_t *>(const_cast<void *>(X));
         const int64_t packed_bytes = (int64_t)dybit_packed_bytes(n_x, fx.bits);
         if (fused) {
-            FusedWeights wj = {static_cast<const uint8_t *>(W), fw.bits, N, ldw_bytes, wrb / elem, we, wrb, 0, {}};
+            FusedWeights wj = {static_cast<const uint8_t *>(W), fw.bits, N, ldw_bytes, wrb / elem, we, wrb, 0, {}, 0, 0, 0};
             const ExpandOperand opw = {static_cast<const uint8_t *>(W), fw.bits, N, ldw_bytes, wrb / elem, we, wrb, &tw};
             wj.use4 = expand4_job(opw, elem, i8, &wj.job4) ? 1 : 0;
+            if (pix4) wj = wpix;
+            const int pix_c = (pix4 && d->c < 4) ? d->c : 0;     // four channels: the code order is the pixel-word layout already
             uint8_t *const dense = patch_dense ? xd : xe;         // code order either way
             const int64_t dense_bytes = patch_dense ? cv.xd_bytes : cv.a_bytes;
             st = elem == 1 ? launch_quantize_expand<1>(xq->x, n_x, fx, scale_x, packed, packed_bytes, dense, dense_bytes, tx, wj, tw,
-                                                       partials, n_partials, scale_dst, s)
+                                                       partials, n_partials, scale_dst, pix_c, s)
                            : launch_quantize_expand<2>(xq->x, n_x, fx, scale_x, packed, packed_bytes, dense, dense_bytes, tx, wj, tw,
-                                                       partials, n_partials, scale_dst, s);
+                                                       partials, n_partials, scale_dst, 0, s);
             if (st != DYBIT_OK) return st;
             expanded = true;
         } else {
@@ -1765,7 +1913,18 @@ static dybit_status conv_impl(const dybit_conv_desc *d, const void *X, dybit_fmt
             if (st != DYBIT_OK) return st;
         }
     }
-    if (patch_dense) {
+    if (pix4) {
+        if (!expanded) {
+            // pixels to 32-bit words and the weights to filter rows of eight taps, in one launch
+            int64_t x_blocks = (pixels + 256 * 8 - 1) / (256 * 8), w_blocks = (N * (wrb / 16) + 1023) / 1024;
+            if (x_blocks > (int64_t)sm_count() * 8) x_blocks = (int64_t)sm_count() * 8;
+            if (w_blocks > sm_count()) w_blocks = sm_count();
+            launch_k(expand_pix4_kernel, dim3((unsigned)(x_blocks + w_blocks)), dim3(256u), (size_t)0, s,
+                     static_cast<const uint8_t *>(X), fx.bits, pixels, d->c, reinterpret_cast<unsigned *>(xe), tx, wpix, tw,
+                     (int)x_blocks);
+            if (launch_status() != DYBIT_OK) return DYBIT_ERR_CUDA;
+        }
+    } else if (patch_dense) {
         // dense container elements first (unless the quantize launch wrote them), then the patch matrix from those
         if (!expanded) {
             const int64_t n_codes = pixels * d->c;
@@ -1893,6 +2052,7 @@ static dybit_status conv_impl(const dybit_conv_desc *d, const void *X, dybit_fmt
     st = make_operand_map(&map_b, we, N, wrb, wrb, bn);
     if (st != DYBIT_OK) return st;
     p.k_blocks = (int)(wrb / kBKBytes);
+    if (pix4) return launch_gemm_kind<kAGather4, 128>(plan.container, bn, map_b, map_b, p, s);
     return launch_gemm_kind<kAGather, 128>(plan.container, bn, map_b, map_b, p, s);
 }
 

@@ -136,6 +136,12 @@ __device__ __forceinline__ void cp_async_16(uint32_t smem_dst, const void *gsrc,
                  : "memory");
 }
 
+// 4-byte variant (only .ca moves fewer than 16 bytes); src_bytes = 0 stores zeros.
+__device__ __forceinline__ void cp_async_4(uint32_t smem_dst, const void *gsrc, uint32_t src_bytes) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(smem_dst), "l"(gsrc), "r"(src_bytes)
+                 : "memory");
+}
+
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 
 template <int N>

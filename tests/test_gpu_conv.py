@@ -108,3 +108,18 @@ def test_im2col_tma_path(shape, fx, fw):
 def test_pointwise_conv_runs_as_plain_gemm(shape):
     run_conv(shape, (4, 0), (4, 1), seed=5)
     run_conv(shape, (8, 0), (6, 1), seed=6)
+
+
+# at most four one-byte channels: pixels as 32-bit words gathered by the tensor-core kernel (no patch matrix);
+# two-byte elements (6 or more magnitude bits) take the patch-matrix path instead
+@pytest.mark.parametrize("shape", [
+    wl.ConvLayer("c3_7x7_s2_ragged", 2, 37, 41, 3, 64, 7, 7, 2, 3),
+    wl.ConvLayer("c3_3x3", 3, 19, 23, 3, 40, 3, 3, 1, 1),
+    wl.ConvLayer("c1_5x5_s2", 2, 30, 28, 1, 24, 5, 5, 2, 2),
+    wl.ConvLayer("c2_8x8_nopad", 1, 26, 26, 2, 72, 8, 8, 1, 0),
+    wl.ConvLayer("c4_9x3_s3", 2, 33, 21, 4, 130, 9, 3, 3, 1),
+    wl.ConvLayer("c3_1x7", 2, 12, 40, 3, 16, 1, 7, 1, 3),
+], ids=lambda L: L.name)
+@pytest.mark.parametrize("fx,fw", [((4, 0), (4, 1)), ((3, 1), (2, 1)), ((5, 0), (4, 1)), ((8, 0), (4, 1))])
+def test_few_channel_geometries(shape, fx, fw):
+    run_conv(shape, fx, fw, seed=len(shape.name) + fx[0])

@@ -116,3 +116,19 @@ def test_argument_errors():
         dy.dybit_quantize_conv2d(d, torch.zeros(100, device=DEV), (4, 0), W, (4, 1), one)
     with pytest.raises(Exception):                       # not fp32
         dy.dybit_quantize_conv2d(d, torch.zeros(256, device=DEV, dtype=torch.float16), (4, 0), W, (4, 1), one)
+
+
+# few channels: the quantize launch writes one 32-bit word per pixel; element counts that are not multiples of
+# the 1024-element chunk make pixels straddle chunk boundaries
+@pytest.mark.parametrize("layer", [
+    wl.ConvLayer("c3_7x7_s2_ragged", 2, 37, 41, 3, 64, 7, 7, 2, 3),
+    wl.ConvLayer("c3_stem_small", 2, 64, 64, 3, 64, 7, 7, 2, 3),
+    wl.ConvLayer("c1_5x5", 3, 30, 31, 1, 24, 5, 5, 1, 2),
+    wl.ConvLayer("c2_3x3_s2", 5, 17, 29, 2, 48, 3, 3, 2, 1),
+    wl.ConvLayer("c4_3x3", 2, 21, 21, 4, 32, 3, 3, 1, 1),
+    wl.ConvLayer("c3_tiny", 1, 3, 5, 3, 8, 3, 3, 1, 1),
+], ids=lambda L: L.name)
+@pytest.mark.parametrize("fx,fw,given", [((4, 0), (4, 1), False), ((4, 1), (3, 1), True), ((5, 0), (5, 1), False),
+                                         ((7, 0), (4, 1), False)])
+def test_few_channels_pixel_words(layer, fx, fw, given):
+    run(layer, fx, fw, seed=len(layer.name) * 3 + fx[0], given_scale=given)
