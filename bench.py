@@ -36,7 +36,7 @@ import torch  # noqa: E402
 FMT_W = (4, 1)      # weights: signed 4-bit
 FMT_A = (4, 0)      # post-ReLU activations: unsigned 4-bit
 NOMINAL = {"hbm_gbs": 7700.0, "bf16_tflops": 2250.0, "int8_tops": 4500.0, "fp8_tflops": 4500.0}
-GEMM_KERNEL_DRAM_BYTES_PER_LAUNCH = 8.53e6   # ncu capture of the current dybit_gemm_kernel, see profiles/
+GEMM_KERNEL_DRAM_BYTES_PER_LAUNCH = 5.78e6   # ncu capture of the current dybit_gemm_kernel, see profiles/
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -665,6 +665,9 @@ def main():
     ap.add_argument("--batch", type=int, default=32, help="images per step (32 = the quoted configuration)")
     ap.add_argument("--no-targets", action="store_true", help="skip the single-kernel target measurements")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--step-only", action="store_true",
+                    help="only the step itself (graph replays, direct launches, end to end): no device-clock pass, no "
+                         "re-quantizing or two-call variants, no targets, no CPU baseline (for profiler captures)")
     ap.add_argument("--targets-only", action="store_true",
                     help="run only the single-kernel target measurements (small cases for profiler captures)")
     ap.add_argument("--gemm-size", type=int, default=8192, help="M=N=K of the square 4-bit GEMM target")
@@ -760,13 +763,13 @@ def main():
     clk = torch.empty((len(work.layers), 2), dtype=torch.int64, device=device)
     graph_c = capture_step(work, device, lambda: work.step(clocks=clk))
     clock_us = [0.0] * len(work.layers)
-    clock_reps = 10
-    for rep in range(clock_reps + 2):
+    clock_reps = 1 if args.step_only else 10
+    for rep in range(clock_reps + (0 if args.step_only else 2)):
         clk[:, 0] = -1
         clk[:, 1] = 0
         graph_c.replay()
         torch.cuda.synchronize(device)
-        if rep >= 2:
+        if rep >= 2 or args.step_only:
             span = (clk[:, 1] - clk[:, 0]).cpu().tolist()
             clock_us = [a + s * 1e-3 / clock_reps for a, s in zip(clock_us, span)]
     del graph_c
@@ -831,6 +834,13 @@ def main():
         "gpu_launches": launches, "clocks": clocks, "e2e": e2e, "roofline": roofline,
         "quantize_elems_per_step": work.quant_elems,
     }
+    if args.step_only:
+        if rank == 0:
+            print(json.dumps(result))
+        if dist is not None:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
     # ---- the same step with the re-quantizing epilogue (results leave as 4-bit codes instead of fp32)
     work.prepare_requant()
     for _ in range(3):
