@@ -99,7 +99,7 @@ __device__ __forceinline__ unsigned finite_abs_bits(float v) {
 // atomics, no ticket, nothing to zero beforehand) and the consumer folds the gridDim.x words itself
 // (scale_from_partials); `slot` is then unused.
 template <bool STREAM>   // STREAM: evict-first loads (tensor larger than L2); otherwise leave it in L2 for the next pass
-__global__ void __launch_bounds__(kStreamThreads)
+__global__ void __launch_bounds__(kStreamThreads, 3)
 absmax_kernel(const float *__restrict__ x, int64_t rows, int64_t cols, int64_t ld,
               unsigned *__restrict__ slot, int m, unsigned *__restrict__ partials) {
     unsigned best = 0;
@@ -113,8 +113,9 @@ absmax_kernel(const float *__restrict__ x, int64_t rows, int64_t cols, int64_t l
         if (head > n) head = n;
         const int64_t nvec = (n - head) / 4;
         const float4 *xv = reinterpret_cast<const float4 *>(x + head);
-        // eight independent 16-byte loads per thread and round trip (the ragged end reads zeros instead)
-        constexpr int kUnroll = 8;
+        // sixteen independent 16-byte loads per thread and round trip (the ragged end reads zeros instead): with
+        // three blocks per SM one round covers 29 MB, so the activations of a ResNet layer take a single round
+        constexpr int kUnroll = 16;
         for (int64_t i = tid; i < nvec; i += kUnroll * nthreads) {
             float4 v[kUnroll];
 #pragma unroll
@@ -863,8 +864,8 @@ static dybit_status launch_absmax(const float *x, int64_t rows, int64_t cols, in
     else if (n <= 0) return DYBIT_ERR_INVALID_ARG;
     if (n > 0) {
         // few, fat blocks: every block ends with two atomics on the same words
-        int64_t blocks = (n / 4 + kStreamThreads * 8 - 1) / (kStreamThreads * 8);
-        int64_t cap = (int64_t)sm_count() * 4;          // what the register file holds at once
+        int64_t blocks = (n / 4 + kStreamThreads * 16 - 1) / (kStreamThreads * 16);
+        int64_t cap = (int64_t)sm_count() * 3;          // what the register file holds at once
         if (cap > kMaxAbsmaxPartials) cap = kMaxAbsmaxPartials;
         if (blocks > cap) blocks = cap;
         if (blocks < 1) blocks = 1;
