@@ -864,6 +864,8 @@ struct GemmParams {
     int H, W, OH, OW, R, S, stride, pad, dil;
     int cpb;                  // bytes per pixel in xe (padded channels * element size)
     int kb_per_tap;           // im2col mode: SWB-byte blocks per filter tap (cpb / SWB)
+    int b_resident;           // 1: one tile column and k_blocks <= stages: the whole B panel is loaded once per CTA
+                              //    into the B stage slots (slot = K block) and the ring carries A only
     int tma_store;            // 1: C leaves through shared memory and TMA stores (needs 16-byte aligned C rows)
     // re-quantizing epilogue: when Q is set the result is encoded and packed instead of stored as fp32
     uint8_t *Q;               // row m starts at Q + m * ldq; N codes of q_bits each
@@ -1016,7 +1018,8 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     uint64_t *empty = bars + kStages;
     uint64_t *acc_full = bars + 2 * kStages;
     uint64_t *acc_empty = acc_full + 2;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_empty + 2);
+    uint64_t *b_full = acc_empty + 2;                    // resident-B mode: the panel has landed
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(b_full + 1);
     volatile uint32_t *abort_flag = tmem_slot + 1;
 
     const int warp = threadIdx.x >> 5;
@@ -1033,6 +1036,7 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             mbar_init(&acc_full[a], 1);
             mbar_init(&acc_empty[a], kEpilogueWarps);
         }
+        mbar_init(b_full, 1);
         *abort_flag = 0;
         fence_mbar_init();
         if (!CONV) prefetch_tensormap(&tmap_a);
@@ -1078,6 +1082,13 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
+            const bool b_res = !CONV && p.b_resident != 0;
+            if (b_res && (int)blockIdx.x < total_tiles) {
+                // every tile of this CTA multiplies by the same B panel: fetch it once, K block kb into slot kb
+                mbar_arrive_expect_tx(b_full, (uint32_t)p.k_blocks * L::kBStage);
+                for (int kb = 0; kb < p.k_blocks; ++kb)
+                    tma_load_2d(b_stages + kb * L::kBStage, &tmap_b, kb * SWB, 0, b_full);
+            }
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
                 const TileOrigin o = tile == (int)blockIdx.x ? first : tile_origin(tile);
                 const int m_blk = o.m_blk, n_blk = o.n_blk, iw = o.iw, ih = o.ih, img = o.img;
@@ -1086,7 +1097,7 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     const int s = it % kStages;
                     const uint32_t ph = (it / kStages) & 1u;
                     if (!wait_bounded(&empty[s], ph ^ 1u, abort_flag, 1)) { ok = false; break; }
-                    mbar_arrive_expect_tx(&full[s], CONV ? L::kBStage : L::kAStage + L::kBStage);
+                    mbar_arrive_expect_tx(&full[s], CONV ? L::kBStage : (b_res ? L::kAStage : L::kAStage + L::kBStage));
                     if (AMODE == kATiled) {
                         if (p.bmt) tma_load_3d(a_stages + s * L::kAStage, &tmap_a, kb * SWB, (m_blk % p.bmt) * kBM, m_blk / p.bmt, &full[s]);
                         else tma_load_2d(a_stages + s * L::kAStage, &tmap_a, kb * SWB, m_blk * kBM, &full[s]);
@@ -1098,6 +1109,7 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                             if (++fs == p.S) { fs = 0; ++fr; }
                         }
                     }
+                    if (b_res) continue;
                     if (AMODE == kATiled && p.bmt) tma_load_3d(b_stages + s * L::kBStage, &tmap_b, kb * SWB, n_blk * BN, m_blk / p.bmt, &full[s]);
                     else tma_load_2d(b_stages + s * L::kBStage, &tmap_b, kb * SWB, n_blk * BN, &full[s]);
                 }
@@ -1115,6 +1127,8 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             constexpr uint32_t idesc = umma_idesc(kCFormat, kABFormat, kBM, BN);
             uint32_t it = 0, lt = 0;
             bool ok = true;
+            const bool b_res = !CONV && p.b_resident != 0;
+            if (b_res && (int)blockIdx.x < total_tiles) ok = wait_bounded(b_full, 0u, abort_flag, 6);
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++lt) {
                 const uint32_t as = lt & 1u, aph = (lt >> 1) & 1u;
                 if (!wait_bounded(&acc_empty[as], aph ^ 1u, abort_flag, 2)) { ok = false; break; }
@@ -1126,7 +1140,7 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     if (!wait_bounded(&full[s], ph, abort_flag, 3)) { ok = false; break; }
                     tc_fence_after_sync();
                     const uint64_t adesc = umma_desc_kmajor<SWB>(smem_u32(a_stages + s * L::kAStage));
-                    const uint64_t bdesc = umma_desc_kmajor<SWB>(smem_u32(b_stages + s * L::kBStage));
+                    const uint64_t bdesc = umma_desc_kmajor<SWB>(smem_u32(b_stages + (b_res ? kb : s) * L::kBStage));
 #pragma unroll
                     for (int k = 0; k < SWB / kUmmaKBytes; ++k) {
                         umma<KIND>(d, adesc + (uint64_t)(k * (kUmmaKBytes >> 4)), bdesc + (uint64_t)(k * (kUmmaKBytes >> 4)),
@@ -1496,6 +1510,8 @@ static dybit_status launch_gemm_inst(const CUtensorMap &ta, const CUtensorMap &t
     ProfileEvents ev = profile_events();
     profile_events() = ProfileEvents();
     p.clock = ev.clock;
+    // a B panel that fits the B stage slots is fetched once per CTA when every tile shares it and CTAs take several tiles
+    p.b_resident = (!CONV && p.bmt == 0 && p.n_tiles == 1 && p.k_blocks <= L::kStages && tiles > sm_count()) ? 1 : 0;
     if (ev.start) DYBIT_CUDA_TRY(cudaEventRecord(ev.start, s));
     launch_k(kern, dim3((unsigned)(grid)), dim3((unsigned)(CONV ? 448 : 320)), (size_t)(L::kBytes), s, ta, tb, tc, p);
     const dybit_status st = launch_status();
