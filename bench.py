@@ -186,9 +186,9 @@ class LayerwiseStep:
         """The same step with results written back as packed DyBit codes (ReLU + encode in the epilogue)."""
         dy = self.dy
         for i in range(len(self.layers)):
-            dy.dybit_quantize_pack(self.x_dev[i], self.fa[i], packed=self.px[i], scale_out=self.sx[i])
-            dy.dybit_conv2d_requant(self.desc[i], self.px[i], self.fa[i], self.sx[i], self.pw[i], self.fw[i], self.sw[i],
-                                    self.fq, self.sq[i], relu=True, Q=self.q[i], ws=self.ws)
+            dy.dybit_quantize_conv2d_requant(self.desc[i], self.x_dev[i], self.fa[i], self.pw[i], self.fw[i], self.sw[i],
+                                             self.fq, self.sq[i], relu=True, scale_out=self.sx[i], packed=self.px[i],
+                                             Q=self.q[i], ws=self.ws)
 
     def step_e2e(self):
         for i in range(len(self.layers)):

@@ -317,6 +317,17 @@ dybit_status dybit_conv2d_requant(const dybit_conv_desc *desc,
                                   dybit_fmt fq, const float *scale_q, const float *bias, int relu, void *Q,
                                   void *ws, size_t ws_bytes, void *stream);
 
+/* One whole layer of Section III-B.1 in one call: the fp32 NHWC activation is quantized and packed
+ * (dybit_quantize_conv2d's arguments X, scale_x, scale_x_out, X_packed), convolved on its codes, and the result leaves
+ * as packed DyBit codes (dybit_conv2d_requant's arguments fq, scale_q, bias, relu, Q).  Bit for bit the results of
+ * dybit_quantize_pack followed by dybit_conv2d_requant; same workspace size as dybit_conv2d. */
+dybit_status dybit_quantize_conv2d_requant(const dybit_conv_desc *desc,
+                                           const float *X, dybit_fmt fx, const float *scale_x, float *scale_x_out,
+                                           void *X_packed,
+                                           const void *W, dybit_fmt fw, const float *scale_w, int64_t ldw_bytes,
+                                           dybit_fmt fq, const float *scale_q, const float *bias, int relu, void *Q,
+                                           void *ws, size_t ws_bytes, void *stream);
+
 /* (No counterpart in the paper.)  dybit_gemm for callers that cannot call
  * cudaMalloc -- or any allocator built on it -- at the point where they need
  * a GEMM: code running under a fixed memory budget that was handed out at

@@ -22,7 +22,7 @@ __all__ = [
     "dybit_decode", "dybit_gemm", "dybit_conv2d", "dybit_last_device_status",
     "dybit_launch_count", "dybit_profile_next_gemm", "dybit_profile_next_gemm_clock", "dybit_gemm_static_ws", "STATIC_WS_BYTES",
     "dybit_gemm_requant", "dybit_conv2d_requant", "dybit_depthwise_conv2d", "dybit_gemm_batched",
-    "dybit_quantize_conv2d",
+    "dybit_quantize_conv2d", "dybit_quantize_conv2d_requant",
     "dybit_gemm_batched_workspace_bytes", "dybit_rmse", "dybit_rmse_sweep", "dybit_fake_quant", "dybit_fake_quant_backward",
     "dybit_search_bitwidths",
 ]
@@ -101,6 +101,8 @@ def _load() -> C.CDLL:
                                        _CFmt, vp, vp, i32, vp, i64, vp, sz, vp]
     lib.dybit_conv2d_requant.argtypes = [C.POINTER(_CConvDesc), vp, _CFmt, vp, vp, _CFmt, vp, i64,
                                          _CFmt, vp, vp, i32, vp, vp, sz, vp]
+    lib.dybit_quantize_conv2d_requant.argtypes = [C.POINTER(_CConvDesc), vp, _CFmt, vp, vp, vp, vp, _CFmt, vp, i64,
+                                                  _CFmt, vp, vp, i32, vp, vp, sz, vp]
     lib.dybit_rmse.argtypes = [vp, i64, _CFmt, vp, vp, vp]
     lib.dybit_quantize_conv2d.argtypes = [C.POINTER(_CConvDesc), vp, _CFmt, vp, vp, vp, vp, _CFmt, vp, i64,
                                           vp, vp, vp, sz, vp]
@@ -393,6 +395,34 @@ def dybit_conv2d_requant(desc: ConvDesc, X: torch.Tensor, fx, scale_x: torch.Ten
                                     _ptr(Q), wp, wn,
                                     _stream(stream)), "dybit_conv2d_requant")
     return Q
+
+
+def dybit_quantize_conv2d_requant(desc: ConvDesc, X: torch.Tensor, fx, W: torch.Tensor, fw, scale_w: torch.Tensor,
+                                  fq, scale_q: torch.Tensor, relu: bool = False, bias: Optional[torch.Tensor] = None,
+                                  scale_x: Optional[torch.Tensor] = None, scale_out: Optional[torch.Tensor] = None,
+                                  packed: Optional[torch.Tensor] = None, Q: Optional[torch.Tensor] = None,
+                                  ws: Optional[torch.Tensor] = None, stream=None):
+    """Quantize + pack the fp32 NHWC activation X, convolve its codes with W and write the result as packed codes.
+    Returns (Q uint8 dense NHWK stream, packed codes of X uint8, scale of X float32[2])."""
+    _dev_f32(X, "X")
+    if X.numel() != desc.n * desc.h * desc.w * desc.c:
+        raise ValueError("X does not match the descriptor")
+    oh, ow = dybit_conv2d_out_hw(desc)
+    if Q is None:
+        Q = torch.zeros(dybit_packed_bytes(desc.n * oh * ow * desc.k, fq[0]), dtype=torch.uint8, device=X.device)
+    if packed is None:
+        packed = torch.empty(dybit_packed_bytes(X.numel(), fx[0]), dtype=torch.uint8, device=X.device)
+    if scale_out is None:
+        scale_out = torch.empty(2, dtype=torch.float32, device=X.device)
+    if ws is None:
+        ws = torch.empty(dybit_conv2d_workspace_bytes(desc, fx, fw) + 1024, dtype=torch.uint8, device=X.device)
+    wp, wn = _ws_ptr(ws)
+    cd = _cdesc(desc)
+    _check(lib.dybit_quantize_conv2d_requant(C.byref(cd), _ptr(X), _fmt(fx), _ptr(scale_x), _ptr(scale_out), _ptr(packed),
+                                             _ptr(W), _fmt(fw), _ptr(scale_w), W.stride(0), _fmt(fq), _ptr(scale_q),
+                                             _bias_ptr(bias, desc.k), int(bool(relu)), _ptr(Q), wp, wn, _stream(stream)),
+           "dybit_quantize_conv2d_requant")
+    return Q, packed, scale_out
 
 
 def dybit_gemm_batched_workspace_bytes(batch: int, M: int, N: int, K: int, fa, fb) -> int:

@@ -2123,4 +2123,15 @@ dybit_status dybit_conv2d_requant(const dybit_conv_desc *d, const void *X, dybit
     return dybit::conv_impl(d, X, fx, scale_x, W, fw, scale_w, ldw_bytes, nullptr, nullptr, &rq, ws, ws_bytes, stream);
 }
 
+dybit_status dybit_quantize_conv2d_requant(const dybit_conv_desc *d, const float *X, dybit_fmt fx, const float *scale_x,
+                                           float *scale_x_out, void *X_packed, const void *W, dybit_fmt fw,
+                                           const float *scale_w, int64_t ldw_bytes, dybit_fmt fq, const float *scale_q,
+                                           const float *bias, int relu, void *Q, void *ws, size_t ws_bytes, void *stream) {
+    if (d == nullptr || scale_x_out == nullptr || X_packed == nullptr) return DYBIT_ERR_INVALID_ARG;
+    const dybit::QuantInput xq = {X, scale_x};
+    const dybit::RequantSpec rq = {fq, scale_q, bias, relu ? 1 : 0, Q, (int64_t)d->k * fq.bits / 8};
+    return dybit::conv_impl(d, X_packed, fx, scale_x_out, W, fw, scale_w, ldw_bytes, nullptr, nullptr, &rq, ws, ws_bytes,
+                            stream, &xq);
+}
+
 }  // extern "C"

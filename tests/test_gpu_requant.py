@@ -184,3 +184,39 @@ def test_requant_argument_errors():
     with pytest.raises(dy.DybitError) as e:       # rows shorter than N codes
         dy.dybit_gemm_requant(4, 4, 128, pa, (4, 1), one, pa, (4, 1), one, (8, 0), one, Q=torch.zeros((4, 4), dtype=torch.uint8, device=DEV), ldq_bytes=0)
     assert e.value.status == 1
+
+
+# the whole layer in one call: fp32 activation -> codes -> conv -> bias + ReLU -> packed output codes
+@pytest.mark.parametrize("layer", [
+    wl.ConvLayer("c64_3x3_im2col", 4, 28, 28, 64, 72, 3, 3, 1, 1),
+    wl.ConvLayer("c3_7x7_stem", 2, 40, 40, 3, 64, 7, 7, 2, 3),
+    wl.ConvLayer("c256_1x1", 3, 14, 14, 256, 128, 1, 1, 1, 0),
+    wl.ConvLayer("c20_patch", 2, 9, 11, 20, 24, 3, 3, 1, 1),
+], ids=lambda L: L.name)
+def test_quantize_conv_requant_one_call(layer):
+    fx, fw, fq = (4, 0), (4, 1), (4, 0)
+    L = layer
+    x = wl.half_normal((L.n, L.h, L.w, L.c), seed=31)
+    w = wl.kaiming_normal(L.k, L.r, L.s, L.c, seed=32)
+    pw, sw = dy.dybit_quantize_pack_2d(w.reshape(L.k, -1).to(DEV), fw)
+    spx = orc.absmax_scale(x.numpy(), 4, False)
+    spw = orc.absmax_scale(w.numpy(), 4, True)
+    cx = orc.quantize(x.numpy(), 4, False, spx[1])
+    cw = orc.quantize(w.numpy(), 4, True, spw[1])
+    _, y = orc.conv2d(cx, fx, spx[0], cw, fw, spw[0], stride=L.stride, pad=L.pad)
+    bias = wl.normal((L.k,), seed=33, std=float(np.abs(y).mean())).numpy().astype(np.float32)
+    y_b = (y.astype(np.float32) + bias.reshape(1, 1, 1, -1)).astype(np.float32)
+    sq = orc.absmax_scale(np.maximum(y_b, 0) * 0.9, 4, False)
+    scale_q = torch.tensor([float(sq[0]), float(sq[1])], dtype=torch.float32, device=DEV)
+    desc = dy.ConvDesc(L.n, L.h, L.w, L.c, L.k, L.r, L.s, L.stride, L.pad, 1)
+    Q, packed, scale = dy.dybit_quantize_conv2d_requant(desc, x.to(DEV), fx, pw, fw, sw, fq, scale_q, relu=True,
+                                                        bias=torch.from_numpy(bias).to(DEV))
+    torch.cuda.synchronize()
+    assert dy.dybit_last_device_status() == (0, 0)
+    assert scale.cpu().numpy().tolist() == [float(np.float32(spx[0])), float(np.float32(spx[1]))]
+    assert np.array_equal(packed.cpu().numpy(), orc.pack(cx, 4))
+    assert np.array_equal(Q.cpu().numpy(), orc.pack(orc.quantize(np.maximum(y_b, 0), 4, False, sq[1]), 4))
+    # and the same bits as the two-call path
+    px, sx = dy.dybit_quantize_pack(x.to(DEV), fx)
+    Q2 = dy.dybit_conv2d_requant(desc, px, fx, sx, pw, fw, sw, fq, scale_q, relu=True, bias=torch.from_numpy(bias).to(DEV))
+    assert torch.equal(Q, Q2)
