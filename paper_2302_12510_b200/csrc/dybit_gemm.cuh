@@ -1695,6 +1695,11 @@ size_t dybit_conv2d_workspace_bytes(const dybit_conv_desc *d, dybit_fmt fx, dybi
 
 namespace dybit {
 
+// CTA-pair variant of the plain GEMM (dybit_gemm_pair.cuh).
+static bool gemm_pair_eligible(int64_t M, int64_t N, const GemmParams &p);
+static dybit_status launch_gemm_pair(dybit_container cont, const void *ae, const void *be, int64_t M, int64_t N,
+                                     int64_t rb, const GemmParams &p_in, cudaStream_t s);
+
 static dybit_status gemm_impl(int64_t M, int64_t N, int64_t K, const void *A, dybit_fmt fa, const float *scale_a,
                               int64_t lda_bytes, const void *B, dybit_fmt fb, const float *scale_b, int64_t ldb_bytes,
                               float *C, int64_t ldc, int32_t *C_raw, const RequantSpec *rq, void *ws, size_t ws_bytes,
@@ -1754,6 +1759,11 @@ static dybit_status gemm_impl(int64_t M, int64_t N, int64_t K, const void *A, dy
     p.scale_b = scale_b;
     p.pow2 = ldexp(1.0, -(plan.exp_a + plan.exp_b));
     apply_requant(p, rq);
+    if (gemm_pair_eligible(M, N, p)) {
+        // large plain products: 256 x 256 tiles on pairs of SMs (falls through when C cannot be described to the TMA)
+        st = launch_gemm_pair(plan.container, ae, be, M, N, rb, p, s);
+        if (st != DYBIT_ERR_UNSUPPORTED) return st;
+    }
     return launch_gemm_kind<kATiled, 128>(plan.container, bn, map_a, map_b, p, s);
 }
 

@@ -167,3 +167,37 @@ def test_profile_clock_brackets_the_kernel():
     dy.dybit_gemm(M, N, K, pa, fa, sa, pb, fb, sb)
     torch.cuda.synchronize()
     assert torch.equal(before, t2)
+
+
+# Large plain products without raw sums run on CTA pairs (256 x 256 tiles, cta_group::2); with raw sums the same
+# product runs on the single-CTA kernel.  Both must give the oracle's fp32 result, and therefore each other's.
+@pytest.mark.parametrize("M,N,K,fa,fb", [
+    (2304, 2304, 256, (4, 1), (4, 1)),        # whole tiles
+    (2500, 2400, 384, (4, 1), (4, 0)),        # ragged in M (196 rows in the last block: both CTAs of the pair have rows) and N
+    (2404, 2308, 130, (3, 1), (4, 1)),        # last block has 100 rows: the pair's second CTA has none
+    (2304, 2304, 200, (5, 1), (5, 0)),        # e4m3 container
+    (2304, 2560, 136, (8, 1), (6, 0)),        # bf16 container
+], ids=["whole", "ragged", "half_empty_pair", "e4m3", "bf16"])
+def test_cta_pair_kernel(M, N, K, fa, fb):
+    a = wl.normal((M, K), seed=M + K)
+    if not fa[1]:
+        a = a.abs()
+    b = wl.normal((N, K), seed=N + K)
+    if not fb[1]:
+        b = b.abs()
+    pa, sa, ca, spa = quantize_operand(a, fa)
+    pb, sb, cb, spb = quantize_operand(b, fb)
+    cont, _, _ = dy.dybit_choose_container(fa, fb)
+    C, _ = dy.dybit_gemm(M, N, K, pa, fa, sa, pb, fb, sb)                       # no raw sums: CTA pairs
+    torch.cuda.synchronize()
+    assert dy.dybit_last_device_status() == (0, 0)
+    _, C_ref = orc.gemm(ca, fa, spa[0], cb, fb, spb[0])
+    if cont == 0:
+        assert np.array_equal(C.cpu().numpy(), C_ref)
+        C1, C_raw = dy.dybit_gemm(M, N, K, pa, fa, sa, pb, fb, sb, want_raw=True)   # single-CTA kernel
+        assert torch.equal(C, C1)
+    else:
+        amax = float(spa[0]) * float(np.abs(orc.decode_table(fa[0], bool(fa[1]))).max())
+        bmax = float(spb[0]) * float(np.abs(orc.decode_table(fb[0], bool(fb[1]))).max())
+        err = np.abs(C.cpu().numpy().astype(np.float64) - C_ref.astype(np.float64)).max()
+        assert err <= 1e-5 * K * amax * bmax, err
