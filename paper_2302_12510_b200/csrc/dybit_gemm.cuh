@@ -1697,8 +1697,8 @@ namespace dybit {
 
 // CTA-pair variant of the plain GEMM (dybit_gemm_pair.cuh).
 static bool gemm_pair_eligible(int64_t M, int64_t N, const GemmParams &p);
-static dybit_status launch_gemm_pair(dybit_container cont, const void *ae, const void *be, int64_t M, int64_t N,
-                                     int64_t rb, const GemmParams &p_in, cudaStream_t s);
+static dybit_status launch_gemm_pair(dybit_container cont, const void *ae, int64_t a_row_bytes, const void *be,
+                                     int64_t b_row_bytes, int64_t M, int64_t N, const GemmParams &p_in, cudaStream_t s);
 
 static dybit_status gemm_impl(int64_t M, int64_t N, int64_t K, const void *A, dybit_fmt fa, const float *scale_a,
                               int64_t lda_bytes, const void *B, dybit_fmt fb, const float *scale_b, int64_t ldb_bytes,
@@ -1761,7 +1761,7 @@ static dybit_status gemm_impl(int64_t M, int64_t N, int64_t K, const void *A, dy
     apply_requant(p, rq);
     if (gemm_pair_eligible(M, N, p)) {
         // large plain products: 256 x 256 tiles on pairs of SMs (falls through when C cannot be described to the TMA)
-        st = launch_gemm_pair(plan.container, ae, be, M, N, rb, p, s);
+        st = launch_gemm_pair(plan.container, ae, rb, be, rb, M, N, p, s);
         if (st != DYBIT_ERR_UNSUPPORTED) return st;
     }
     return launch_gemm_kind<kATiled, 128>(plan.container, bn, map_a, map_b, p, s);
@@ -2062,6 +2062,10 @@ static dybit_status conv_impl(const dybit_conv_desc *d, const void *X, dybit_fmt
         st = make_operand_map(&map_b, we, N, wrb, wrb, bn);
         if (st != DYBIT_OK) return st;
         p.k_blocks = (int)(wrb / kBKBytes);
+        if (gemm_pair_eligible(M, N, p)) {
+            st = launch_gemm_pair(plan.container, xe, arow, we, wrb, M, N, p, s);
+            if (st != DYBIT_ERR_UNSUPPORTED) return st;
+        }
         return launch_gemm_kind<kATiled, 128>(plan.container, bn, map_a, map_b, p, s);
     }
     if (cv.mode == kConvIm2col) {

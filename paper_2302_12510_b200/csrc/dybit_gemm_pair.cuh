@@ -248,15 +248,16 @@ static bool gemm_pair_eligible(int64_t M, int64_t N, const GemmParams &p) {
     return M >= 256 && N >= 256 && tiles * 2 >= sm_count();
 }
 
-static dybit_status launch_gemm_pair(dybit_container cont, const void *ae, const void *be, int64_t M, int64_t N,
-                                     int64_t rb, const GemmParams &p_in, cudaStream_t s) {
+static dybit_status launch_gemm_pair(dybit_container cont, const void *ae, int64_t a_row_bytes, const void *be,
+                                     int64_t b_row_bytes, int64_t M, int64_t N, const GemmParams &p_in, cudaStream_t s) {
     GemmParams p = p_in;
     p.m_tiles = (int)((M + 255) / 256);
     p.n_tiles = (int)((N + kPairBN - 1) / kPairBN);
     CUtensorMap ta, tb, tc;
-    dybit_status st = make_operand_map(&ta, ae, M, rb, rb, kBM);
+    // (a row of A may be shorter than a whole number of K blocks: the TMA reads zeros past its end)
+    dybit_status st = make_operand_map(&ta, ae, M, a_row_bytes, a_row_bytes, kBM);
     if (st != DYBIT_OK) return st;
-    st = make_operand_map(&tb, be, N, rb, rb, kPairBN / 2);
+    st = make_operand_map(&tb, be, N, b_row_bytes, b_row_bytes, kPairBN / 2);
     if (st != DYBIT_OK) return st;
     memset(&tc, 0, sizeof(tc));
     if (!make_output_map(&tc, p.C, p.M, p.N, p.ldc, 0, 0)) return DYBIT_ERR_UNSUPPORTED;

@@ -104,6 +104,13 @@ def _square_gemm(size, fmt, rng, n_rows, n_cols, n_points):
         raw = C_raw.cpu().numpy().astype(np.int64)
         assert np.array_equal(raw.sum(axis=0), IA.sum(axis=0) @ IB.T)
         assert np.array_equal(raw.sum(axis=1), IA @ IB.sum(axis=0))
+        del raw, C_raw
+        # the call as bench.py times it (no raw sums: products of this size then run on CTA pairs): same fp32 bits
+        C2, _ = dy.dybit_gemm(size, size, size, pa, fmt, sa, pb, fmt, sb)
+        torch.cuda.synchronize()
+        assert dy.dybit_last_device_status() == (0, 0)
+        assert np.array_equal(C2[torch.from_numpy(ri).to(DEV), torch.from_numpy(ci).to(DEV)].cpu().numpy(), Cref)
+        assert torch.equal(C, C2)
     else:
         amax = float(spa[0]) * float(np.abs(orc.decode_table(fmt[0], bool(fmt[1]))).max())
         bmax = float(spb[0]) * float(np.abs(orc.decode_table(fmt[0], bool(fmt[1]))).max())
