@@ -246,6 +246,13 @@ struct FusedWeights {
     int pix_c, pix_r, pix_s;  // pix_c > 0: filter rows of 8 taps x 4 bytes instead (see expand_weights_pix4)
 };
 
+// The activation's own 16-entry table for the register-table expansion of 4-bit codes (see expand4_lookup); use = 0
+// keeps the shared-memory table.
+struct XTab4 {
+    unsigned tab[4];
+    int use, neg_high;
+};
+
 // Weights for the few-channel lowering (ConvMode kConvPix4): row n of the output holds, for each filter row r,
 // eight taps of four bytes: tap s < S carries its C <= 4 one-byte elements, everything else is zero; rows are
 // padded with zeros to out_stride.  Thread `idx` writes one 16-byte chunk (four taps).
@@ -284,7 +291,7 @@ quantize_expand_kernel(const float *__restrict__ x, int64_t n, const float *__re
                        uint8_t *__restrict__ packed, int64_t packed_bytes, uint8_t *__restrict__ xe, int64_t xe_bytes,
                        const __grid_constant__ ElemTable tx, const FusedWeights wj, const __grid_constant__ ElemTable tw,
                        int x_blocks, const unsigned *__restrict__ partials, int n_partials, int m, float *__restrict__ scale_out,
-                       int pix_c) {
+                       int pix_c, const XTab4 xt) {
     __shared__ __align__(16) unsigned s_codes[kWarpsPerBlock][kChunkCodes / 4];
     __shared__ __align__(16) unsigned s_words[kWarpsPerBlock][32 * BITS];
     __shared__ uint16_t s_lut[256];
@@ -399,10 +406,28 @@ quantize_expand_kernel(const float *__restrict__ x, int64_t n, const float *__re
             const int64_t off = (c0 + lane * 32) * ELEM;
             if constexpr (ELEM == 1) {
                 unsigned o[8];
+                bool looked_up = false;
+                if constexpr (BITS == 4) {
+                    if (xt.use) {
+                        // eight codes per packed word -> two words of elements, through the table held in registers
+                        unsigned w4[4];
+                        pack32<4>(cw, w4);
+                        const unsigned t4[4] = {xt.tab[0], xt.tab[1], xt.tab[2], xt.tab[3]};
+                        const bool ng = xt.neg_high != 0;
 #pragma unroll
-                for (int i = 0; i < 8; ++i)
-                    o[i] = (unsigned)(s_lut[cw[i] & 0xffu] & 0xffu) | ((unsigned)(s_lut[(cw[i] >> 8) & 0xffu] & 0xffu) << 8) |
-                           ((unsigned)(s_lut[(cw[i] >> 16) & 0xffu] & 0xffu) << 16) | ((unsigned)(s_lut[cw[i] >> 24] & 0xffu) << 24);
+                        for (int i = 0; i < 4; ++i) {
+                            o[2 * i] = expand4_lookup(w4[i], t4, ng);
+                            o[2 * i + 1] = expand4_lookup(w4[i] >> 16, t4, ng);
+                        }
+                        looked_up = true;
+                    }
+                }
+                if (!looked_up) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        o[i] = (unsigned)(s_lut[cw[i] & 0xffu] & 0xffu) | ((unsigned)(s_lut[(cw[i] >> 8) & 0xffu] & 0xffu) << 8) |
+                               ((unsigned)(s_lut[(cw[i] >> 16) & 0xffu] & 0xffu) << 16) | ((unsigned)(s_lut[cw[i] >> 24] & 0xffu) << 24);
+                }
                 if (pix_c > 0) {
                     // pixels of pix_c < 4 one-byte elements, each padded to a 32-bit word: the chunk's 1024 bytes go
                     // back to shared memory in element order, lanes then assemble whole pixels; the (at most two)
@@ -477,7 +502,7 @@ template <int BITS, int ELEM>
 static dybit_status launch_quantize_expand_bits(const float *x, int64_t n, bool is_signed, const float *scale, uint8_t *packed,
                                                 int64_t packed_bytes, uint8_t *xe, int64_t xe_bytes, const ElemTable &tx,
                                                 const FusedWeights &wj, const ElemTable &tw, const unsigned *partials,
-                                                int n_partials, float *scale_out, int pix_c, cudaStream_t s) {
+                                                int n_partials, float *scale_out, int pix_c, const XTab4 &xt, cudaStream_t s) {
     const int m = is_signed ? BITS - 1 : BITS;
     constexpr int kChunkBytes = kChunkCodes * BITS / 8;
     // one wave: three blocks fit an SM, the weights' blocks (a few 16-byte chunks per thread) take their share of
@@ -494,10 +519,10 @@ static dybit_status launch_quantize_expand_bits(const float *x, int64_t n, bool 
     const unsigned grid = (unsigned)(x_blocks + w_blocks);
     if (is_signed)
         launch_k(quantize_expand_kernel<BITS, true, ELEM>, dim3(grid), dim3((unsigned)kStreamThreads), (size_t)0, s, x, n, scale, packed,
-                 packed_bytes, xe, xe_bytes, tx, wj, tw, x_blocks, partials, n_partials, m, scale_out, pix_c);
+                 packed_bytes, xe, xe_bytes, tx, wj, tw, x_blocks, partials, n_partials, m, scale_out, pix_c, xt);
     else
         launch_k(quantize_expand_kernel<BITS, false, ELEM>, dim3(grid), dim3((unsigned)kStreamThreads), (size_t)0, s, x, n, scale, packed,
-                 packed_bytes, xe, xe_bytes, tx, wj, tw, x_blocks, partials, n_partials, m, scale_out, pix_c);
+                 packed_bytes, xe, xe_bytes, tx, wj, tw, x_blocks, partials, n_partials, m, scale_out, pix_c, xt);
     return launch_status();
 }
 
@@ -505,16 +530,16 @@ template <int ELEM>
 static dybit_status launch_quantize_expand(const float *x, int64_t n, dybit_fmt fx, const float *scale, uint8_t *packed,
                                            int64_t packed_bytes, uint8_t *xe, int64_t xe_bytes, const ElemTable &tx,
                                            const FusedWeights &wj, const ElemTable &tw, const unsigned *partials,
-                                           int n_partials, float *scale_out, int pix_c, cudaStream_t s) {
+                                           int n_partials, float *scale_out, int pix_c, const XTab4 &xt, cudaStream_t s) {
     const bool sg = fx.is_signed != 0;
     switch (fx.bits) {
-        case 2: return launch_quantize_expand_bits<2, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pix_c, s);
-        case 3: return launch_quantize_expand_bits<3, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pix_c, s);
-        case 4: return launch_quantize_expand_bits<4, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pix_c, s);
-        case 5: return launch_quantize_expand_bits<5, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pix_c, s);
-        case 6: return launch_quantize_expand_bits<6, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pix_c, s);
-        case 7: return launch_quantize_expand_bits<7, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pix_c, s);
-        case 8: return launch_quantize_expand_bits<8, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pix_c, s);
+        case 2: return launch_quantize_expand_bits<2, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pix_c, xt, s);
+        case 3: return launch_quantize_expand_bits<3, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pix_c, xt, s);
+        case 4: return launch_quantize_expand_bits<4, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pix_c, xt, s);
+        case 5: return launch_quantize_expand_bits<5, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pix_c, xt, s);
+        case 6: return launch_quantize_expand_bits<6, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pix_c, xt, s);
+        case 7: return launch_quantize_expand_bits<7, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pix_c, xt, s);
+        case 8: return launch_quantize_expand_bits<8, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pix_c, xt, s);
     }
     return DYBIT_ERR_INVALID_ARG;
 }
@@ -1926,12 +1951,22 @@ static dybit_status conv_impl(const dybit_conv_desc *d, const void *X, dybit_fmt
             wj.use4 = expand4_job(opw, elem, i8, &wj.job4) ? 1 : 0;
             if (pix4) wj = wpix;
             const int pix_c = (pix4 && d->c < 4) ? d->c : 0;     // four channels: the code order is the pixel-word layout already
+            XTab4 xt = {};
+            {
+                Expand4Job xj;
+                const ExpandOperand opx = {packed, fx.bits, 1, 0, 32, xe, 0, &tx};
+                if (expand4_job(opx, elem, i8, &xj)) {
+                    for (int i = 0; i < 4; ++i) xt.tab[i] = xj.tab[i];
+                    xt.use = 1;
+                    xt.neg_high = xj.neg_high;
+                }
+            }
             uint8_t *const dense = patch_dense ? xd : xe;         // code order either way
             const int64_t dense_bytes = patch_dense ? cv.xd_bytes : cv.a_bytes;
             st = elem == 1 ? launch_quantize_expand<1>(xq->x, n_x, fx, scale_x, packed, packed_bytes, dense, dense_bytes, tx, wj, tw,
-                                                       partials, n_partials, scale_dst, pix_c, s)
+                                                       partials, n_partials, scale_dst, pix_c, xt, s)
                            : launch_quantize_expand<2>(xq->x, n_x, fx, scale_x, packed, packed_bytes, dense, dense_bytes, tx, wj, tw,
-                                                       partials, n_partials, scale_dst, 0, s);
+                                                       partials, n_partials, scale_dst, 0, xt, s);
             if (st != DYBIT_OK) return st;
             expanded = true;
         } else {
