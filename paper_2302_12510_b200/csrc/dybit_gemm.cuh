@@ -1025,14 +1025,14 @@ __device__ __forceinline__ void tile_coords(int tile, int m_tiles, int n_tiles, 
 }
 
 template <Kind KIND, int BN, int AMODE, int SWB>
-__global__ void __launch_bounds__((AMODE == kAGather || AMODE == kAGather4) ? 448 : 320, 1)
+__global__ void __launch_bounds__(AMODE == kAGather4 ? 576 : (AMODE == kAGather ? 448 : 320), 1)
 dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                   const __grid_constant__ CUtensorMap tmap_c, const GemmParams p) {
     static_assert((AMODE != kAGather && AMODE != kAGather4) || SWB == 128, "the cp.async gather writes 128-byte rows");
     constexpr bool CONV = AMODE == kAGather || AMODE == kAGather4;          // extra gather warps present
     using L = GemmSmem<BN, SWB>;
     constexpr int kStages = L::kStages;
-    constexpr int kGatherThreads = 128;
+    constexpr int kGatherThreads = AMODE == kAGather4 ? 256 : 128;     // pixel-word mode: two threads per tile row
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t *a_stages = smem;
@@ -1054,7 +1054,7 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
-            mbar_init(&full[s], CONV ? 1 + kGatherThreads : 1);
+            mbar_init(&full[s], CONV ? 1 + (AMODE == kAGather4 ? kGatherThreads / 32 : kGatherThreads) : 1);
             mbar_init(&empty[s], 1);
         }
         for (int a = 0; a < 2; ++a) {
@@ -1302,7 +1302,8 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         if (issuer) bulk_wait_group_read<0>();             // shared memory must outlive the last store's read
     } else if (CONV) {
         // ------------------------------------------------ im2col gather of the A tile (4 warps, one row per thread)
-        const int t = threadIdx.x - 32 * (2 + kEpilogueWarps);   // tile row 0..127
+        const int t = (threadIdx.x - 32 * (2 + kEpilogueWarps)) & 127;   // tile row 0..127
+        const int half = (threadIdx.x - 32 * (2 + kEpilogueWarps)) >> 7;   // pixel-word mode: which two of a K block's four filter rows
         const int sw = t & 7;
         constexpr int kAhead = 2;                     // stages issued but not yet published
         uint32_t it = 0, issued = 0, published = 0;
@@ -1331,30 +1332,45 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
                 const int s = it % kStages;
                 const uint32_t ph = (it / kStages) & 1u;
-                if (!wait_bounded(&empty[s], ph ^ 1u, abort_flag, 5)) { ok = false; break; }
+                if (AMODE == kAGather4) {
+                    // one lane of each warp watches the barrier (256 threads polling it slow everything else down)
+                    bool got = true;
+                    if ((threadIdx.x & 31) == 0) got = wait_bounded(&empty[s], ph ^ 1u, abort_flag, 5);
+                    got = __shfl_sync(0xffffffffu, got, 0);
+                    if (!got) { ok = false; break; }
+                } else if (!wait_bounded(&empty[s], ph ^ 1u, abort_flag, 5)) { ok = false; break; }
                 const uint32_t dst_row = smem_u32(a_stages + s * L::kAStage) + (uint32_t)t * kBKBytes;
                 if (AMODE == kAGather4) {
-                    // the row = four filter rows (4*kb ..) of eight 4-byte slots, slot s = tap s: every slot is
-                    // written, with the pixel it points at where that tap exists and lies inside the image, with
-                    // zeros otherwise (straight-line code: the zero fill is a copy of size 0, not a branch)
-                    const unsigned *zero_src = reinterpret_cast<const unsigned *>(p.xe);
+                    // the row = four filter rows (4*kb ..) of eight 4-byte slots, slot s = tap s; this thread fills two
+                    // of the four.  Plain loads (the pixel words are reused by many windows and sit in L1) into
+                    // registers, zeros where the tap does not exist or lies outside the image, then one 16-byte
+                    // shared-memory store per chunk: 4-byte cp.async copies, tried first, ran at about two copies per
+                    // clock and SM and bounded the whole kernel.
+                    unsigned v[2][8];
 #pragma unroll
-                    for (int jj = 0; jj < 4; ++jj) {
-                        const int r = kb * 4 + jj;
+                    for (int j2 = 0; j2 < 2; ++j2) {
+                        const int r = kb * 4 + half * 2 + j2;
                         const int ih = ih0 + r;
                         const bool row_in = row_ok && r < p.R && (unsigned)ih < (unsigned)p.H;
-                        const unsigned *src_row = row_in ? pix_base + (int64_t)ih * p.W : zero_src;
+                        const unsigned *src_row = pix_base + (int64_t)(row_in ? ih : 0) * p.W;
                         const unsigned mask = row_in ? col_mask : 0u;
 #pragma unroll
-                        for (int h = 0; h < 2; ++h) {
-                            const uint32_t dst = dst_row + (uint32_t)(((jj * 2 + h) ^ sw) << 4);
+                        for (int w = 0; w < 8; ++w) v[j2][w] = ((mask >> w) & 1u) ? __ldg(src_row + w) : 0u;
+                    }
 #pragma unroll
-                            for (int w = 0; w < 4; ++w) {
-                                const bool in = (mask >> (h * 4 + w)) & 1u;
-                                cp_async_4(dst + w * 4, in ? src_row + (h * 4 + w) : zero_src, in ? 4u : 0u);
-                            }
+                    for (int j2 = 0; j2 < 2; ++j2) {
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            const uint32_t dst = dst_row + (uint32_t)((((half * 2 + j2) * 2 + h) ^ sw) << 4);
+                            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(v[j2][4 * h]),
+                                         "r"(v[j2][4 * h + 1]), "r"(v[j2][4 * h + 2]), "r"(v[j2][4 * h + 3])
+                                         : "memory");
                         }
                     }
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if ((threadIdx.x & 31) == 0) mbar_arrive(&full[s]);        // one arrival per warp
+                    continue;
                 } else if (p.cpb % kBKBytes == 0) {
                     // a pixel holds whole 128-byte blocks: the eight chunks share one tap and are contiguous
                     const int ih = ih0 + fr * p.dil, iw = iw0 + fs * p.dil;
@@ -1538,7 +1554,8 @@ static dybit_status launch_gemm_inst(const CUtensorMap &ta, const CUtensorMap &t
     // a B panel that fits the B stage slots is fetched once per CTA when every tile shares it and CTAs take several tiles
     p.b_resident = (!CONV && p.bmt == 0 && p.n_tiles == 1 && p.k_blocks <= L::kStages && tiles > sm_count()) ? 1 : 0;
     if (ev.start) DYBIT_CUDA_TRY(cudaEventRecord(ev.start, s));
-    launch_k(kern, dim3((unsigned)(grid)), dim3((unsigned)(CONV ? 448 : 320)), (size_t)(L::kBytes), s, ta, tb, tc, p);
+    launch_k(kern, dim3((unsigned)(grid)), dim3((unsigned)(AMODE == kAGather4 ? 576 : (CONV ? 448 : 320))), (size_t)(L::kBytes), s, ta, tb,
+             tc, p);
     const dybit_status st = launch_status();
     if (ev.stop) DYBIT_CUDA_TRY(cudaEventRecord(ev.stop, s));
     return st;
