@@ -1308,55 +1308,72 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         constexpr int kAhead = 2;                     // stages issued but not yet published
         uint32_t it = 0, issued = 0, published = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-            int m_blk, n_blk;
-            tile_coords(tile, p.m_tiles, p.n_tiles, m_blk, n_blk);
-            const int m = m_blk * kBM + t;
-            const bool row_ok = m < p.M;
-            const int img = row_ok ? m / (p.OH * p.OW) : 0;
-            const int rem = row_ok ? m - img * (p.OH * p.OW) : 0;
-            const int oh = rem / p.OW, ow = rem - oh * p.OW;
-            const int ih0 = oh * p.stride - p.pad, iw0 = ow * p.stride - p.pad;
-            const uint8_t *img_base = p.xe + (int64_t)img * p.H * p.W * p.cpb;
-            // pixel-word mode: pointer to the window's first column in image row 0 (only dereferenced where the mask
-            // allows), and the taps of a filter row that exist and fall inside the image horizontally
-            const unsigned *pix_base = reinterpret_cast<const unsigned *>(p.xe) + (int64_t)img * p.H * p.W + iw0;
-            unsigned col_mask = 0;
-            if (AMODE == kAGather4) {
+        if (AMODE == kAGather4) {
+            // Pixel-word mode.  A K block of the A tile = four filter rows (4*kb ..) of eight 4-byte slots, slot s =
+            // tap s; this thread fills two of the four rows of its tile row: plain loads (the pixel words are reused
+            // by many windows and sit in L1) into registers, zeros where the tap does not exist or lies outside the
+            // image, then one 16-byte shared-memory store per chunk.  The loads of the NEXT K block (possibly of the
+            // next tile) are issued before this one's stage is waited for, so their latency hides behind the wait,
+            // the stores and the proxy fence.  One lane per warp polls the stage's barrier and arrives for the warp.
+            struct RowState {
+                int ih0;
+                unsigned col_mask;
+                const unsigned *pix_base;     // window's first column in image row 0 (dereferenced only under the mask)
+                bool row_ok;
+            };
+            auto row_state = [&](int tile) {
+                int m_blk, n_blk;
+                tile_coords(tile, p.m_tiles, p.n_tiles, m_blk, n_blk);
+                const int m = m_blk * kBM + t;
+                RowState rs;
+                rs.row_ok = m < p.M;
+                const int img = rs.row_ok ? m / (p.OH * p.OW) : 0;
+                const int rem = rs.row_ok ? m - img * (p.OH * p.OW) : 0;
+                const int oh = rem / p.OW, ow = rem - oh * p.OW;
+                const int iw0 = ow * p.stride - p.pad;
+                rs.ih0 = oh * p.stride - p.pad;
+                rs.pix_base = reinterpret_cast<const unsigned *>(p.xe) + (int64_t)img * p.H * p.W + iw0;
+                rs.col_mask = 0;
 #pragma unroll
                 for (int fs4 = 0; fs4 < 8; ++fs4)
-                    if (fs4 < p.S && (unsigned)(iw0 + fs4) < (unsigned)p.W) col_mask |= 1u << fs4;
-            }
-            // filter tap (fr, fs) and byte offset inside the pixel, advanced chunk by chunk: K runs (r, s, c)
-            int fr = 0, fs = 0, cb = 0;
-            for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
-                const int s = it % kStages;
-                const uint32_t ph = (it / kStages) & 1u;
-                if (AMODE == kAGather4) {
-                    // one lane of each warp watches the barrier (256 threads polling it slow everything else down)
+                    if (fs4 < p.S && (unsigned)(iw0 + fs4) < (unsigned)p.W) rs.col_mask |= 1u << fs4;
+                return rs;
+            };
+            auto load_rows = [&](const RowState &rs, int kb, unsigned (&v)[2][8]) {
+#pragma unroll
+                for (int j2 = 0; j2 < 2; ++j2) {
+                    const int r = kb * 4 + half * 2 + j2;
+                    const int ih = rs.ih0 + r;
+                    const bool row_in = rs.row_ok && r < p.R && (unsigned)ih < (unsigned)p.H;
+                    const unsigned *src_row = rs.pix_base + (int64_t)(row_in ? ih : 0) * p.W;
+                    const unsigned mask = row_in ? rs.col_mask : 0u;
+#pragma unroll
+                    for (int w = 0; w < 8; ++w) v[j2][w] = ((mask >> w) & 1u) ? __ldg(src_row + w) : 0u;
+                }
+            };
+            int tile = blockIdx.x, kb = 0;
+            if (tile < total_tiles) {
+                RowState cur = row_state(tile);
+                unsigned v[2][8], vn[2][8];
+                load_rows(cur, 0, v);
+                for (;; ++it) {
+                    int ntile = tile, nkb = kb + 1;
+                    if (nkb == p.k_blocks) {
+                        nkb = 0;
+                        ntile = tile + gridDim.x;
+                    }
+                    const bool has_next = ntile < total_tiles;
+                    if (has_next) {
+                        if (ntile != tile) cur = row_state(ntile);      // (the current block's values are in v already)
+                        load_rows(cur, nkb, vn);
+                    }
+                    const int s = it % kStages;
+                    const uint32_t ph = (it / kStages) & 1u;
                     bool got = true;
                     if ((threadIdx.x & 31) == 0) got = wait_bounded(&empty[s], ph ^ 1u, abort_flag, 5);
                     got = __shfl_sync(0xffffffffu, got, 0);
-                    if (!got) { ok = false; break; }
-                } else if (!wait_bounded(&empty[s], ph ^ 1u, abort_flag, 5)) { ok = false; break; }
-                const uint32_t dst_row = smem_u32(a_stages + s * L::kAStage) + (uint32_t)t * kBKBytes;
-                if (AMODE == kAGather4) {
-                    // the row = four filter rows (4*kb ..) of eight 4-byte slots, slot s = tap s; this thread fills two
-                    // of the four.  Plain loads (the pixel words are reused by many windows and sit in L1) into
-                    // registers, zeros where the tap does not exist or lies outside the image, then one 16-byte
-                    // shared-memory store per chunk: 4-byte cp.async copies, tried first, ran at about two copies per
-                    // clock and SM and bounded the whole kernel.
-                    unsigned v[2][8];
-#pragma unroll
-                    for (int j2 = 0; j2 < 2; ++j2) {
-                        const int r = kb * 4 + half * 2 + j2;
-                        const int ih = ih0 + r;
-                        const bool row_in = row_ok && r < p.R && (unsigned)ih < (unsigned)p.H;
-                        const unsigned *src_row = pix_base + (int64_t)(row_in ? ih : 0) * p.W;
-                        const unsigned mask = row_in ? col_mask : 0u;
-#pragma unroll
-                        for (int w = 0; w < 8; ++w) v[j2][w] = ((mask >> w) & 1u) ? __ldg(src_row + w) : 0u;
-                    }
+                    if (!got) break;
+                    const uint32_t dst_row = smem_u32(a_stages + s * L::kAStage) + (uint32_t)t * kBKBytes;
 #pragma unroll
                     for (int j2 = 0; j2 < 2; ++j2) {
 #pragma unroll
@@ -1370,7 +1387,35 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     fence_proxy_async_smem();
                     __syncwarp();
                     if ((threadIdx.x & 31) == 0) mbar_arrive(&full[s]);        // one arrival per warp
-                    continue;
+                    if (!has_next) break;
+#pragma unroll
+                    for (int j2 = 0; j2 < 2; ++j2)
+#pragma unroll
+                        for (int w = 0; w < 8; ++w) v[j2][w] = vn[j2][w];
+                    tile = ntile;
+                    kb = nkb;
+                }
+            }
+        }
+        for (int tile = blockIdx.x; AMODE != kAGather4 && tile < total_tiles && ok; tile += gridDim.x) {
+            int m_blk, n_blk;
+            tile_coords(tile, p.m_tiles, p.n_tiles, m_blk, n_blk);
+            const int m = m_blk * kBM + t;
+            const bool row_ok = m < p.M;
+            const int img = row_ok ? m / (p.OH * p.OW) : 0;
+            const int rem = row_ok ? m - img * (p.OH * p.OW) : 0;
+            const int oh = rem / p.OW, ow = rem - oh * p.OW;
+            const int ih0 = oh * p.stride - p.pad, iw0 = ow * p.stride - p.pad;
+            const uint8_t *img_base = p.xe + (int64_t)img * p.H * p.W * p.cpb;
+            // filter tap (fr, fs) and byte offset inside the pixel, advanced chunk by chunk: K runs (r, s, c)
+            int fr = 0, fs = 0, cb = 0;
+            for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+                const int s = it % kStages;
+                const uint32_t ph = (it / kStages) & 1u;
+                if (!wait_bounded(&empty[s], ph ^ 1u, abort_flag, 5)) { ok = false; break; }
+                const uint32_t dst_row = smem_u32(a_stages + s * L::kAStage) + (uint32_t)t * kBKBytes;
+                if (AMODE == kAGather4) {
+                    // handled above
                 } else if (p.cpb % kBKBytes == 0) {
                     // a pixel holds whole 128-byte blocks: the eight chunks share one tap and are contiguous
                     const int ih = ih0 + fr * p.dil, iw = iw0 + fs * p.dil;
