@@ -36,7 +36,7 @@ import torch  # noqa: E402
 FMT_W = (4, 1)      # weights: signed 4-bit
 FMT_A = (4, 0)      # post-ReLU activations: unsigned 4-bit
 NOMINAL = {"hbm_gbs": 7700.0, "bf16_tflops": 2250.0, "int8_tops": 4500.0, "fp8_tflops": 4500.0}
-GEMM_KERNEL_DRAM_BYTES_PER_LAUNCH = 5.78e6   # ncu capture of the current dybit_gemm_kernel, see profiles/
+GEMM_KERNEL_DRAM_BYTES_PER_LAUNCH = 5.77e6   # ncu capture of the current dybit_gemm_kernel, see profiles/
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
