@@ -2,8 +2,8 @@
 // Each CTA loads its own 128 rows of A and HALF of the tile's 256 B rows; the tensor cores of both SMs read
 // B from both shared memories, so a CTA moves 256 shared-memory rows per K block instead of the 384 that a
 // 128 x 256 tile of its own needs -- the TMA unit's row rate is what bounds the single-CTA kernel.
-// Plain fp32 output through TMA stores only (no raw sums, no re-quantizing epilogue, no batches): everything
-// else stays on dybit_gemm_kernel.
+// fp32 output through TMA stores (optionally with the raw integer sums beside it) or the re-quantizing epilogue;
+// batches, convolution gathers and outputs the TMA cannot describe stay on dybit_gemm_kernel.
 #pragma once
 
 #include "dybit_gemm.cuh"
@@ -60,7 +60,7 @@ dybit_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
         fence_mbar_init();
         prefetch_tensormap(&tmap_a);
         prefetch_tensormap(&tmap_b);
-        prefetch_tensormap(&tmap_c);
+        if (p.tma_store) prefetch_tensormap(&tmap_c);
     }
     if (warp == 1) {
         tmem_alloc_pair(tmem_slot, kTmemCols);
@@ -136,6 +136,7 @@ dybit_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
         const int group = (warp - 2) >> 2;
         const bool issuer = (threadIdx.x & 127) == 64;
         const float alpha = (float)((double)__ldg(p.scale_a) * (double)__ldg(p.scale_b) * p.pow2);
+        const float inv_q = p.Q ? __ldg(p.scale_q + 1) : 1.0f;
         uint32_t lt = 0;
         for (int tile = pair; tile < total_tiles; tile += num_pairs, ++lt) {
             int m_blk, n_blk;
@@ -160,6 +161,36 @@ dybit_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
                 for (int j = 0; j < 32; ++j) {
                     const float acc = (KIND == Kind::I8) ? __int2float_rn((int)r[j]) : __uint_as_float(r[j]);
                     f[j] = __fmul_rn(acc, alpha);
+                }
+                const int row = row0 + row_in_tile;
+                if (p.Q) {
+                    // re-quantizing epilogue: + bias, ReLU, encode, pack; 32 codes of this thread's row
+                    if (row < p.M) {
+                        if (p.bias) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (col0 + j < p.N) f[j] = __fadd_rn(f[j], __ldg(p.bias + col0 + j));
+                        }
+                        if (p.relu) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) f[j] = fmaxf(f[j], 0.0f);
+                        }
+                        requant_dispatch(p.q_bits, p.q_signed, f, inv_q,
+                                         p.Q + (int64_t)row * p.ldq + (int64_t)col0 * p.q_bits / 8, p.N - col0);
+                    }
+                    continue;
+                }
+                if (KIND == Kind::I8 && p.C_raw != nullptr && row < p.M) {
+                    // raw integer sums beside the fp32 result (rows are 16-byte aligned: checked on the host)
+                    int32_t *rrow = p.C_raw + (int64_t)row * p.ldc + col0;
+                    if (col0 + 32 <= p.N) {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+                            __stcs(reinterpret_cast<int4 *>(rrow) + j, make_int4((int)r[4 * j], (int)r[4 * j + 1], (int)r[4 * j + 2], (int)r[4 * j + 3]));
+                    } else {
+                        for (int j = 0; j < 32; ++j)
+                            if (col0 + j < p.N) rrow[j] = (int)r[j];
+                    }
                 }
                 // in the CTA's last tile the operand stages are idle: every chunk takes a buffer of its own
                 uint8_t *stage = last_tile ? a_stages + cc * kPairCStage : c_stages + group * kPairCStage;
@@ -243,7 +274,8 @@ static dybit_status launch_gemm_pair_kind(const CUtensorMap &ta, const CUtensorM
 // Whether a plain GEMM goes to the pair kernel: fp32 output that the TMA can describe, nothing else asked for,
 // and at least one 256 x 256 tile per pair of SMs.
 static bool gemm_pair_eligible(int64_t M, int64_t N, const GemmParams &p) {
-    if (p.C_raw != nullptr || p.Q != nullptr || p.bmt != 0) return false;
+    if (p.bmt != 0) return false;
+    if (p.C_raw != nullptr && ((reinterpret_cast<uintptr_t>(p.C_raw) & 15) != 0 || p.ldc % 4 != 0)) return false;
     const int64_t tiles = ((M + 255) / 256) * ((N + 255) / 256);
     return M >= 256 && N >= 256 && tiles * 2 >= sm_count();
 }
@@ -260,8 +292,8 @@ static dybit_status launch_gemm_pair(dybit_container cont, const void *ae, int64
     st = make_operand_map(&tb, be, N, b_row_bytes, b_row_bytes, kPairBN / 2);
     if (st != DYBIT_OK) return st;
     memset(&tc, 0, sizeof(tc));
-    if (!make_output_map(&tc, p.C, p.M, p.N, p.ldc, 0, 0)) return DYBIT_ERR_UNSUPPORTED;
-    p.tma_store = 1;
+    if (p.Q == nullptr && !make_output_map(&tc, p.C, p.M, p.N, p.ldc, 0, 0)) return DYBIT_ERR_UNSUPPORTED;
+    p.tma_store = p.Q == nullptr ? 1 : 0;
     switch (cont) {
         case DYBIT_CONTAINER_I8: return launch_gemm_pair_kind<Kind::I8>(ta, tb, tc, p, s);
         case DYBIT_CONTAINER_E4M3: return launch_gemm_pair_kind<Kind::F8F6F4>(ta, tb, tc, p, s);

@@ -105,7 +105,7 @@ def _square_gemm(size, fmt, rng, n_rows, n_cols, n_points):
         assert np.array_equal(raw.sum(axis=0), IA.sum(axis=0) @ IB.T)
         assert np.array_equal(raw.sum(axis=1), IA @ IB.sum(axis=0))
         del raw, C_raw
-        # the call as bench.py times it (no raw sums: products of this size then run on CTA pairs): same fp32 bits
+        # the call as bench.py times it (no raw sums): same fp32 bits
         C2, _ = dy.dybit_gemm(size, size, size, pa, fmt, sa, pb, fmt, sb)
         torch.cuda.synchronize()
         assert dy.dybit_last_device_status() == (0, 0)

@@ -169,8 +169,8 @@ def test_profile_clock_brackets_the_kernel():
     assert torch.equal(before, t2)
 
 
-# Large plain products without raw sums run on CTA pairs (256 x 256 tiles, cta_group::2); with raw sums the same
-# product runs on the single-CTA kernel.  Both must give the oracle's fp32 result, and therefore each other's.
+# Large products run on CTA pairs (256 x 256 tiles, cta_group::2), with or without raw sums; both calls must give
+# the oracle's results.
 @pytest.mark.parametrize("M,N,K,fa,fb", [
     (2304, 2304, 256, (4, 1), (4, 1)),        # whole tiles
     (2500, 2400, 384, (4, 1), (4, 0)),        # ragged in M (196 rows in the last block: both CTAs of the pair have rows) and N
@@ -188,14 +188,15 @@ def test_cta_pair_kernel(M, N, K, fa, fb):
     pa, sa, ca, spa = quantize_operand(a, fa)
     pb, sb, cb, spb = quantize_operand(b, fb)
     cont, _, _ = dy.dybit_choose_container(fa, fb)
-    C, _ = dy.dybit_gemm(M, N, K, pa, fa, sa, pb, fb, sb)                       # no raw sums: CTA pairs
+    C, _ = dy.dybit_gemm(M, N, K, pa, fa, sa, pb, fb, sb)
     torch.cuda.synchronize()
     assert dy.dybit_last_device_status() == (0, 0)
-    _, C_ref = orc.gemm(ca, fa, spa[0], cb, fb, spb[0])
+    S, C_ref = orc.gemm(ca, fa, spa[0], cb, fb, spb[0])
     if cont == 0:
         assert np.array_equal(C.cpu().numpy(), C_ref)
-        C1, C_raw = dy.dybit_gemm(M, N, K, pa, fa, sa, pb, fb, sb, want_raw=True)   # single-CTA kernel
+        C1, C_raw = dy.dybit_gemm(M, N, K, pa, fa, sa, pb, fb, sb, want_raw=True)
         assert torch.equal(C, C1)
+        assert np.array_equal(C_raw.cpu().numpy().astype(np.int64), S)
     else:
         amax = float(spa[0]) * float(np.abs(orc.decode_table(fa[0], bool(fa[1]))).max())
         bmax = float(spb[0]) * float(np.abs(orc.decode_table(fb[0], bool(fb[1]))).max())

@@ -220,3 +220,27 @@ def test_quantize_conv_requant_one_call(layer):
     px, sx = dy.dybit_quantize_pack(x.to(DEV), fx)
     Q2 = dy.dybit_conv2d_requant(desc, px, fx, sx, pw, fw, sw, fq, scale_q, relu=True, bias=torch.from_numpy(bias).to(DEV))
     assert torch.equal(Q, Q2)
+
+
+# products large enough for the CTA-pair kernel: its epilogue re-quantizes too (bias, ReLU, ragged last tiles)
+@pytest.mark.parametrize("M,N,K,fq,relu,with_bias", [(2304, 2304, 256, (4, 0), True, False),
+                                                      (2400, 2344, 200, (8, 1), False, True),
+                                                      (2404, 2312, 130, (2, 0), True, True)])
+def test_gemm_requant_on_cta_pairs(M, N, K, fq, relu, with_bias):
+    fa, fb = (4, 0), (4, 1)
+    a = wl.half_normal((M, K), seed=M + K)
+    b = wl.normal((N, K), seed=N + K, std=0.05)
+    pa, sa, ca, spa = _quant(a, fa)
+    pb, sb, cb, spb = _quant(b, fb)
+    _, y_ref = orc.gemm(ca, fa, spa[0], cb, fb, spb[0])
+    bias = None
+    if with_bias:
+        bias = wl.normal((N,), seed=7, std=float(np.abs(y_ref).mean())).numpy().astype(np.float32)
+        y_ref = (y_ref.astype(np.float32) + bias.reshape(1, -1)).astype(np.float32)
+    sq = orc.absmax_scale(y_ref * 0.9, fq[0], bool(fq[1]))
+    scale_q = torch.tensor([float(sq[0]), float(sq[1])], dtype=torch.float32, device=DEV)
+    Q = dy.dybit_gemm_requant(M, N, K, pa, fa, sa, pb, fb, sb, fq, scale_q, relu=relu,
+                              bias=None if bias is None else torch.from_numpy(bias).to(DEV))
+    torch.cuda.synchronize()
+    assert dy.dybit_last_device_status() == (0, 0)
+    assert np.array_equal(Q.cpu().numpy(), _expect(y_ref, fq, sq[1], relu))
