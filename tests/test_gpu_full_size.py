@@ -128,7 +128,7 @@ def test_square_gemm_sweep(size, fmt):
     _square_gemm(size, fmt, np.random.default_rng(size), n_rows=8, n_cols=8, n_points=5000)
 
 
-def _conv_layer_sampled(L, fx, fw, seed, n_samples=1500):
+def _conv_layer_sampled(L, fx, fw, seed, n_samples=1500, one_call_too=False):
     x = wl.half_normal((L.n, L.h, L.w, L.c), seed=seed, device=DEV)
     w = wl.kaiming_normal(L.k, L.r, L.s, L.c, seed=seed + 1)
     px, sx = dy.dybit_quantize_pack(x, fx)
@@ -157,6 +157,13 @@ def _conv_layer_sampled(L, fx, fw, seed, n_samples=1500):
         amax = float(spx[0]) * float(np.abs(orc.decode_table(fx[0], bool(fx[1]))).max())
         bmax = float(spw[0]) * float(np.abs(orc.decode_table(fw[0], bool(fw[1]))).max())
         assert np.abs(got.astype(np.float64) - Yref.astype(np.float64)).max() <= 1e-5 * L.gemm_k * amax * bmax, L.name
+    if one_call_too:
+        # the call bench.py times (fp32 activation in, no raw sums): same codes, same scale, same output bits
+        Y1, _, packed1, scale1 = dy.dybit_quantize_conv2d(desc, x, fx, pw, fw, sw)
+        torch.cuda.synchronize()
+        assert dy.dybit_last_device_status() == (0, 0)
+        assert torch.equal(packed1, px) and torch.equal(scale1, sx), L.name
+        assert torch.equal(Y1, Y), L.name
     return cont
 
 
@@ -172,7 +179,7 @@ def _distinct(layers):
 
 @pytest.mark.parametrize("i,L", _distinct(wl.resnet18_layers(32)), ids=lambda v: getattr(v, "name", str(v)))
 def test_resnet18_batch32_uniform_4bit_sampled(i, L):
-    assert _conv_layer_sampled(L, (4, 0), (4, 1), seed=1000 + i) == 0
+    assert _conv_layer_sampled(L, (4, 0), (4, 1), seed=1000 + i, one_call_too=True) == 0
 
 
 _R50 = wl.resnet50_layers(64)
