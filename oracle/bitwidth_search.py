@@ -1,66 +1,114 @@
-"""Algorithm 1 (layer-wise bitwidth search), plain Python -- test infrastructure, not a product path.
+"""Layer-wise bitwidth search (Section III-C.3, Algorithm 1; Eq. 3 and Eq. 4) -- test infrastructure, not a
+product path.  Only tests/ and the benchmark's CPU legs may import this file.
 
-Follows the paper's search flow step by step (Section III-C.3, Algorithm 1) with Eq. 3 / Eq. 4 as the stopping
-rules.  Inputs are two tables per layer, indexed by (activation bits, weight bits) over {8, 4, 2}: latency
-Lat_i(a, w) and error RMSE_i(a, w).  Readings where the paper is silent are stated next to the code.
+The search is written here as a walk over an explicit "schedule" of single moves.  A move lowers ONE operand
+(weights or activations) of ONE layer by one level, 8 -> 4 or 4 -> 2.  Every round of the search
+
+  1. reads the current per-layer latency and error (they depend on the layers' current bitwidths),
+  2. picks k candidate layers and orders them (by the strategy's two keys),
+  3. lays the moves out as: weights of the candidates in that order, then activations in the same order,
+  4. plays the moves one at a time, re-evaluating the whole-model total after each, and stops the whole
+     search at the first move after which the strategy's stopping rule holds.
+
+Strategy "speedup" (Eq. 3): candidates = the k slowest layers, ordered by ascending error; stop as soon as
+alpha * total latency <= total latency at (8, 8).
+Strategy "rmse" (Eq. 4): candidates = the k layers with the least error, ordered by descending latency; the total
+error may never exceed beta * total error at (8, 8).
+
+Readings where the paper is silent (each one is pinned by a hand-traced case in tests/test_bitwidth_search.py):
+  * Eq. 4 is a budget: the first move that would push the total error above it is not taken, and the search ends
+    there (the model returned always satisfies Eq. 4).
+  * An operand already at 2 bits has no move; a layer with both operands at 2 bits is not a candidate.
+  * Equal keys are ordered by layer index.
+  * A round in which no move exists ends the search (everything is at 2 bits).
+
+Tables are arrays of shape [N, 3, 3]: layer, activation level, weight level, with level 0 / 1 / 2 = 8 / 4 / 2 bits.
 """
 from __future__ import annotations
 
-LEVELS = (8, 4, 2)
+import numpy as np
+
+BITS_OF_LEVEL = (8, 4, 2)
+LOWEST = len(BITS_OF_LEVEL) - 1
 
 
-def _total(table, W, A):
-    return sum(table[i][(A[i], W[i])] for i in range(len(W)))
+def as_table(per_layer_dicts) -> np.ndarray:
+    """[{(a_bits, w_bits): value}] -> array [N, 3, 3] indexed by level."""
+    t = np.empty((len(per_layer_dicts), 3, 3), dtype=np.float64)
+    for i, d in enumerate(per_layer_dicts):
+        for ia, a in enumerate(BITS_OF_LEVEL):
+            for iw, w in enumerate(BITS_OF_LEVEL):
+                t[i, ia, iw] = d[(a, w)]
+    return t
 
 
-def search(lat, rmse, strategy: str, constraint: float, k: int):
-    """lat[i][(a, w)], rmse[i][(a, w)] for a, w in {8, 4, 2}.  strategy: "speedup" (Eq. 3, constraint = alpha)
-    or "rmse" (Eq. 4, constraint = beta).  Returns (W, A) lists of bitwidths."""
-    n = len(lat)
-    W, A = [8] * n, [8] * n                                   # all layers start at (8, 8)
-    total_table = lat if strategy == "speedup" else rmse
-    base = _total(total_table, W, A)                          # metric_base
+class _Model:
+    """Current level of every layer's activations and weights, and the tables they index."""
 
-    def meets():
-        cur = _total(total_table, W, A)
-        if strategy == "speedup":
-            return constraint * cur <= base                   # Eq. 3: alpha * sum Lat <= sum Lat(8,8)
-        return cur > constraint * base                        # Eq. 4 budget used up (see degrade below)
+    def __init__(self, lat: np.ndarray, err: np.ndarray):
+        self.lat, self.err = lat, err
+        self.n = lat.shape[0]
+        self.level = {"W": np.zeros(self.n, dtype=int), "A": np.zeros(self.n, dtype=int)}
+        self.rows = np.arange(self.n)
 
-    def degrade(layer_list, bits):
-        """Degrade_level: one layer at a time, 8 -> 4 or 4 -> 2, stop as soon as the constraint is met."""
-        changed = False
-        for i in layer_list:
-            if bits[i] == 2:
-                continue
-            old = bits[i]
-            bits[i] = 4 if old == 8 else 2
-            changed = True
-            if strategy == "rmse" and _total(rmse, W, A) > constraint * base:
-                bits[i] = old                                 # reading: Eq. 4 is a hard budget -> undo the step that breaks it
-                return changed, True
-            if meets():
-                return changed, True
-        return changed, False
+    def per_layer(self, table):
+        return table[self.rows, self.level["A"], self.level["W"]]
 
-    if meets() and strategy == "speedup":
-        return W, A
+    def total(self, table) -> float:
+        # summed in layer order, one addition per layer
+        s = 0.0
+        for v in self.per_layer(table):
+            s += float(v)
+        return s
+
+    def bits(self, operand):
+        return [BITS_OF_LEVEL[v] for v in self.level[operand]]
+
+
+def _candidates(model: _Model, strategy: str, k: int):
+    lat_now, err_now = model.per_layer(model.lat), model.per_layer(model.err)
+    movable = [i for i in range(model.n) if model.level["W"][i] < LOWEST or model.level["A"][i] < LOWEST]
+    if strategy == "speedup":
+        first_key = {i: (-lat_now[i], i) for i in movable}         # slowest first
+        second_key = {i: (err_now[i], i) for i in movable}         # then least error first
+    else:
+        first_key = {i: (err_now[i], i) for i in movable}          # least error first
+        second_key = {i: (-lat_now[i], i) for i in movable}        # then slowest first
+    chosen = sorted(movable, key=first_key.get)[:k]
+    return sorted(chosen, key=second_key.get)
+
+
+def search(lat, rmse, strategy: str, constraint: float, k: int, trace: list | None = None):
+    """lat, rmse: arrays [N, 3, 3] (or lists of {(a_bits, w_bits): value} dicts).  Returns (W, A) as lists of
+    bitwidths.  `trace`, if given, receives one (layer, operand, new_bits, total_after) tuple per move taken."""
+    if strategy not in ("speedup", "rmse"):
+        raise ValueError(strategy)
+    lat = lat if isinstance(lat, np.ndarray) else as_table(lat)
+    rmse = rmse if isinstance(rmse, np.ndarray) else as_table(rmse)
+    model = _Model(lat, rmse)
+    watched = lat if strategy == "speedup" else rmse
+    reference = model.total(watched)                                # the (8, 8) model
+
+    if strategy == "speedup" and constraint * reference <= reference:
+        return model.bits("W"), model.bits("A")                     # alpha <= 1: nothing to do
+
     while True:
-        lat_now = [lat[i][(A[i], W[i])] for i in range(n)]    # Layerwise_metric
-        rmse_now = [rmse[i][(A[i], W[i])] for i in range(n)]
-        live = [i for i in range(n) if W[i] > 2 or A[i] > 2]
-        if not live:
-            break
-        if strategy == "speedup":
-            top = sorted(live, key=lambda i: (-lat_now[i], i))[:k]          # Lat_rank: the k slowest layers
-            order = sorted(top, key=lambda i: (rmse_now[i], i))             # RMSE_rerank: least error first
-        else:
-            top = sorted(live, key=lambda i: (rmse_now[i], i))[:k]          # RMSE_rank: the k least-error layers
-            order = sorted(top, key=lambda i: (-lat_now[i], i))             # Lat_rerank: slowest first
-        c1, done = degrade(order, W)
-        if done:
-            break
-        c2, done = degrade(order, A)
-        if done or not (c1 or c2):
-            break
-    return W, A
+        order = _candidates(model, strategy, k)
+        schedule = [(i, "W") for i in order] + [(i, "A") for i in order]
+        moved = False
+        for layer, operand in schedule:
+            lv = model.level[operand]
+            if lv[layer] == LOWEST:
+                continue
+            lv[layer] += 1
+            after = model.total(watched)
+            if strategy == "rmse" and after > constraint * reference:
+                lv[layer] -= 1                                      # over the Eq. 4 budget: not taken, search over
+                return model.bits("W"), model.bits("A")
+            moved = True
+            if trace is not None:
+                trace.append((layer, operand, BITS_OF_LEVEL[lv[layer]], after))
+            if strategy == "speedup" and constraint * after <= reference:
+                return model.bits("W"), model.bits("A")             # Eq. 3 holds
+        if not moved:
+            return model.bits("W"), model.bits("A")                 # every operand is at 2 bits

@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "dybit.h"
 
 namespace dybit {
@@ -30,13 +32,13 @@ inline int64_t round_up(int64_t v, int64_t a) { return (v + a - 1) / a * a; }
 
 // Every kernel launch of the library is followed by launch_status(), which
 // also counts it.
-inline unsigned long long &launch_counter() {
-    static unsigned long long n = 0;
+inline std::atomic<unsigned long long> &launch_counter() {
+    static std::atomic<unsigned long long> n{0};
     return n;
 }
 
 inline dybit_status launch_status() {
-    ++launch_counter();
+    launch_counter().fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? DYBIT_OK : DYBIT_ERR_CUDA;
 }
 

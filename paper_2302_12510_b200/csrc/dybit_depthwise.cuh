@@ -227,7 +227,7 @@ depthwise_kernel(const __grid_constant__ DwParams p, const __grid_constant__ DwT
 
 template <int XB>
 static dybit_status launch_depthwise(const DwParams &p, const DwTables &tab, size_t smem, int64_t tiles, cudaStream_t s) {
-    static bool configured[64] = {};
+    static std::atomic<bool> configured[64];
     int dev = 0;
     DYBIT_CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64) return DYBIT_ERR_CUDA;

@@ -12,6 +12,8 @@
 // expanded NHWC activation (im2col addressing, zero fill for padding taps).
 #pragma once
 
+#include <thread>
+
 #include "dybit_common.cuh"
 #include "dybit_host.cuh"
 #include "dybit_quantize.cuh"
@@ -70,7 +72,6 @@ static const ElemTable &make_elem_table(dybit_fmt f, dybit_container cont, int i
         ElemTable table;
     };
     static Entry cache[14][3];
-    static thread_local ElemTable scratch;
     Entry &e = cache[fmt_index(f)][(int)cont];
     if (e.state.load(std::memory_order_acquire) != 2) {
         int expected = 0;
@@ -78,8 +79,8 @@ static const ElemTable &make_elem_table(dybit_fmt f, dybit_container cont, int i
             e.table = make_elem_table_uncached(f, cont, int_exp);
             e.state.store(2, std::memory_order_release);
         } else {
-            scratch = make_elem_table_uncached(f, cont, int_exp);
-            return scratch;
+            // another thread is filling this entry (a few microseconds of host work): wait for it
+            while (e.state.load(std::memory_order_acquire) != 2) std::this_thread::yield();
         }
     }
     return e.table;
@@ -1192,8 +1193,9 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             int m_blk, n_blk;
             tile_coords(tile, p.m_tiles, p.n_tiles, m_blk, n_blk);
             const uint32_t as = lt & 1u, aph = (lt >> 1) & 1u;
-            bool ok = wait_bounded(&acc_full[as], aph, abort_flag, 4);
-            ok = __all_sync(0xffffffffu, ok);
+            // The four warps of a group meet in named barriers below, so they must leave this loop together: the
+            // outcome of the wait is AND-reduced over the group's 128 threads (every warp gets here in bounded time).
+            const bool ok = named_barrier_and(1 + group, 128, wait_bounded(&acc_full[as], aph, abort_flag, 4));
             if (!ok) break;
             tc_fence_after_sync();
             // batched: the tile belongs to entry `bat`, rows count inside that entry
@@ -1477,17 +1479,20 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 static EncodeTiledFn encode_tiled_fn() {
-    static EncodeTiledFn fn = nullptr;
-    if (fn == nullptr) {
+    static std::atomic<EncodeTiledFn> fn{nullptr};
+    EncodeTiledFn f = fn.load(std::memory_order_acquire);
+    if (f == nullptr) {
         void *ptr = nullptr;
         cudaDriverEntryPointQueryResult qres;
         if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(ptr);
-        else
+            qres == cudaDriverEntryPointSuccess) {
+            f = reinterpret_cast<EncodeTiledFn>(ptr);
+            fn.store(f, std::memory_order_release);
+        } else {
             (void)cudaGetLastError();
+        }
     }
-    return fn;
+    return f;
 }
 
 // Byte matrix [rows][row_bytes] with row stride `stride`; box = swb bytes x box_rows, swb-byte swizzle.
@@ -1527,17 +1532,20 @@ typedef CUresult (*EncodeIm2colFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_
                                    CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 static EncodeIm2colFn encode_im2col_fn() {
-    static EncodeIm2colFn fn = nullptr;
-    if (fn == nullptr) {
+    static std::atomic<EncodeIm2colFn> fn{nullptr};
+    EncodeIm2colFn f = fn.load(std::memory_order_acquire);
+    if (f == nullptr) {
         void *ptr = nullptr;
         cudaDriverEntryPointQueryResult qres;
         if (cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeIm2colFn>(ptr);
-        else
+            qres == cudaDriverEntryPointSuccess) {
+            f = reinterpret_cast<EncodeIm2colFn>(ptr);
+            fn.store(f, std::memory_order_release);
+        } else {
             (void)cudaGetLastError();
+        }
     }
-    return fn;
+    return f;
 }
 
 // Expanded activation [n][h][w][cpb bytes] as an im2col map: one load brings 128 consecutive output
@@ -1583,7 +1591,7 @@ static dybit_status launch_gemm_inst(const CUtensorMap &ta, const CUtensorMap &t
     using L = GemmSmem<BN, SWB>;
     auto kern = dybit_gemm_kernel<KIND, BN, AMODE, SWB>;
     constexpr bool CONV = AMODE == kAGather || AMODE == kAGather4;
-    static bool configured[64] = {};
+    static std::atomic<bool> configured[64];
     int dev = 0;
     DYBIT_CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64) return DYBIT_ERR_CUDA;
@@ -2067,7 +2075,7 @@ static dybit_status conv_impl(const dybit_conv_desc *d, const void *X, dybit_fmt
         pg.krow = (int)cv.krow;
         pg.row_pitch = (int)cv.krow + 4;
         const size_t smem = (size_t)128 * pg.row_pitch;
-        static bool gather_configured[64] = {};
+        static std::atomic<bool> gather_configured[64];
         int dev = 0;
         DYBIT_CUDA_TRY(cudaGetDevice(&dev));
         if (dev >= 0 && dev < 64 && !gather_configured[dev]) {
@@ -2093,7 +2101,7 @@ static dybit_status conv_impl(const dybit_conv_desc *d, const void *X, dybit_fmt
         pp.krow = (int)cv.krow;
         pp.row_pitch = (int)cv.krow + 4;
         const size_t smem = (size_t)128 * pp.row_pitch;
-        static bool patch_configured[64] = {};
+        static std::atomic<bool> patch_configured[64];
         int dev = 0;
         DYBIT_CUDA_TRY(cudaGetDevice(&dev));
         if (dev >= 0 && dev < 64 && !patch_configured[dev]) {

@@ -142,8 +142,8 @@ dybit_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
             int m_blk, n_blk;
             tile_coords(tile, p.m_tiles, p.n_tiles, m_blk, n_blk);
             const uint32_t as = lt & 1u, aph = (lt >> 1) & 1u;
-            bool ok = wait_bounded(&acc_full[as], aph, abort_flag, 4);
-            ok = __all_sync(0xffffffffu, ok);
+            // one outcome for the group's 128 threads, which meet in named barriers below
+            const bool ok = named_barrier_and(1 + group, 128, wait_bounded(&acc_full[as], aph, abort_flag, 4));
             if (!ok) break;
             tc_fence_after_sync();
             const int row0 = m_blk * 2 * kBM + (int)rank * kBM;          // this CTA's first output row
@@ -232,7 +232,7 @@ static dybit_status launch_gemm_pair_kind(const CUtensorMap &ta, const CUtensorM
                                           const GemmParams &p_in, cudaStream_t s) {
     GemmParams p = p_in;
     auto kern = dybit_gemm_pair_kernel<KIND>;
-    static int max_clusters[64] = {};
+    static std::atomic<int> max_clusters[64];
     int dev = 0;
     DYBIT_CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64) return DYBIT_ERR_CUDA;
@@ -258,7 +258,8 @@ static dybit_status launch_gemm_pair_kind(const CUtensorMap &ta, const CUtensorM
         max_clusters[dev] = n;
     }
     const int tiles = p.m_tiles * p.n_tiles;
-    const int pairs = tiles < max_clusters[dev] ? tiles : max_clusters[dev];
+    const int resident = max_clusters[dev];
+    const int pairs = tiles < resident ? tiles : resident;
     cfg.gridDim = dim3((unsigned)(2 * pairs));
     cfg.numAttrs = 2;
     ProfileEvents ev = profile_events();

@@ -13,7 +13,7 @@
 namespace dybit {
 
 int sm_count() {
-    static int cached[64];
+    static std::atomic<int> cached[64];     // filled on first use; every thread computes the same value
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
     if (cached[dev] == 0) {
@@ -288,7 +288,7 @@ dybit_status dybit_search_bitwidths(int num_layers, const double *lat, const dou
     return DYBIT_OK;
 }
 
-uint64_t dybit_launch_count(void) { return dybit::launch_counter(); }
+uint64_t dybit_launch_count(void) { return dybit::launch_counter().load(std::memory_order_relaxed); }
 
 dybit_status dybit_profile_next_gemm(void *ev_start, void *ev_stop) {
     if ((ev_start == nullptr) != (ev_stop == nullptr)) return DYBIT_ERR_INVALID_ARG;

@@ -40,7 +40,8 @@ __device__ __forceinline__ unsigned magnitude_code_biased(float a, float inv) {
     constexpr float kMagic = 12582912.0f;                                  // 1.5 * 2^23: ulp 1 on both sides
     // largest float below the top value 2^(M-1): everything from 1.5 * 2^(M-2) up rounds to all-ones anyway
     const float below_top = __uint_as_float(((unsigned)(127 + M - 1) << 23) - 1u);
-    const float t = fminf(__fmul_rn(a, inv), below_top);
+    // (0 * inf = NaN when the reciprocal scale overflowed: fmaxf folds it to 0, the code of a zero element)
+    const float t = fminf(fmaxf(__fmul_rn(a, inv), 0.0f), below_top);
     const unsigned sub = __float_as_uint(__fmaf_rn(t, (float)(1u << (M - 1)), kMagic));
     if constexpr (M == 1) {
         return sub;
@@ -1052,7 +1053,7 @@ dybit_status dybit_rmse_sweep(const float *x, int64_t n, int n_cand, const dybit
         for (int k = 0; k < (1 << m); ++k) sp.mags[(1 << m) - 2 + k] = full[k];
     }
     const size_t smem = (size_t)n_cand * (256 + kStreamThreads) * sizeof(double);
-    static bool configured[64] = {};
+    static std::atomic<bool> configured[64];
     int dev = 0;
     DYBIT_CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64) return DYBIT_ERR_CUDA;

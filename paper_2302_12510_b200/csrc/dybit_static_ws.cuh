@@ -15,17 +15,17 @@ namespace dybit {
 // The symbol above is only a host-side handle; kernels need the address the
 // module was given on the current device.  Looked up once per device.
 static dybit_status static_ws_device_pointer(unsigned char **out) {
-    static unsigned char *cached[64] = {};
+    static std::atomic<unsigned char *> cached[64];   // filled on first use; a race stores the same address twice
     int dev = 0;
     DYBIT_CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64) return DYBIT_ERR_CUDA;
-    if (cached[dev] == nullptr) {
-        unsigned char *ptr = nullptr;
+    unsigned char *ptr = cached[dev].load(std::memory_order_acquire);
+    if (ptr == nullptr) {
         DYBIT_CUDA_TRY(cudaGetSymbolAddress(reinterpret_cast<void **>(&ptr), g_static_gemm_ws));
         if (ptr == nullptr) return DYBIT_ERR_CUDA;
-        cached[dev] = ptr;
+        cached[dev].store(ptr, std::memory_order_release);
     }
-    *out = cached[dev];
+    *out = ptr;
     return DYBIT_OK;
 }
 

@@ -73,6 +73,22 @@ def test_quantize_empty_zero_and_nonfinite():
     assert np.array_equal(packed.cpu().numpy(), want)
 
 
+@pytest.mark.parametrize("fmt", [(8, 0), (8, 1), (4, 1), (2, 1)])
+def test_quantize_tiny_tensor_whose_reciprocal_scale_overflows(fmt):
+    # max |x| = 1e-38: 2^(m-1) / amax is +inf in fp32, so a zero element meets 0 * inf = NaN, which must still encode to 0
+    x = np.array([0.0, 1e-38, -1e-38, 0.0, -0.0, 5e-39] * 50, dtype=np.float32)
+    packed, scale = dy.dybit_quantize_pack(torch.from_numpy(x).to(DEV), fmt)
+    want, _, sp = _oracle_pack(x, fmt)
+    assert np.isinf(sp[1])
+    assert np.array_equal(scale.cpu().numpy(), np.array(sp, dtype=np.float32))
+    assert np.array_equal(packed.cpu().numpy(), want)
+    # the same with a caller-given pair whose reciprocal is +inf
+    given = torch.tensor([1e-39, float("inf")], dtype=torch.float32, device=DEV)
+    packed, _ = dy.dybit_quantize_pack(torch.from_numpy(x).to(DEV), fmt, scale=given)
+    want, _, _ = _oracle_pack(x, fmt, (np.float32(1e-39), np.float32(np.inf)))
+    assert np.array_equal(packed.cpu().numpy(), want)
+
+
 def test_quantize_unaligned_input_pointer():
     fmt = (5, 1)
     base = wl.normal((10001,), 8)
