@@ -367,6 +367,22 @@ dybit_status dybit_last_device_status(void *stream, uint32_t *detail);
  * (no counterpart in the paper: they exist so that a benchmark can attribute
  * time to the tensor-core kernel alone and count the library's launches) */
 
+/* Process-wide state.  The library keeps none that a result depends on: plans and element tables are cached per
+ * format pair and per device (filled on first use, atomically, every thread computing the same values), kernels
+ * launched are counted in one atomic counter, and the device status word lives in the loaded module.  The two
+ * dybit_profile_next_gemm* hooks below arm state that is PER HOST THREAD (the arming thread's next GEMM / conv call
+ * consumes it); dybit_set_conv_lowering is a process-wide atomic setting. */
+
+/* Which lowering dybit_conv2d and its variants take for stride-1 convolutions (Section III-C.4 maps conv layers onto
+ * the GEMM array; the lowerings differ only in how the activation tile reaches shared memory, never in results):
+ *   0 (default)  choose by shape: halo tiles where they measured faster (64-byte pixels, one tile column of output
+ *                channels whose weights stay resident in shared memory), the im2col / gather lowering otherwise;
+ *   1            halo tiles wherever they apply (stride 1, dilation 1, at most three filter rows, pixels of 64 or a
+ *                multiple of 128 container bytes);
+ *   2            never halo tiles.
+ * Returns DYBIT_ERR_INVALID_ARG for any other value.  Takes effect for calls that start afterwards. */
+dybit_status dybit_set_conv_lowering(int mode);
+
 /* Number of kernels this library has launched in the calling process so far. */
 uint64_t dybit_launch_count(void);
 

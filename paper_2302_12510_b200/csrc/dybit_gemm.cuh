@@ -924,6 +924,30 @@ __device__ __forceinline__ bool wait_bounded(uint64_t *bar, uint32_t parity, vol
     }
 }
 
+// The same wait for the MMA-issuing thread: the barrier is named by its shared-memory address and only the first
+// probe is inlined, so the common case (the stage is there already) costs three instructions.
+__device__ __noinline__ bool wait_bounded_slow(uint32_t bar_addr, uint32_t parity, volatile uint32_t *abort_flag, unsigned site) {
+    const uint64_t t0 = global_timer_ns();
+    unsigned spins = 0;
+    for (;;) {
+        if (mbar_try_wait_addr(bar_addr, parity)) return true;
+        if ((++spins & 63u) == 0u) {
+            if (*abort_flag) return false;
+            if (global_timer_ns() - t0 > kWaitLimitNs) {
+                atomicOr(&g_device_status, (site << 8) | 1u);
+                *abort_flag = 1u;
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ bool wait_bounded_addr(uint32_t bar_addr, uint32_t parity, volatile uint32_t *abort_flag,
+                                                  unsigned site) {
+    if (mbar_try_wait_addr(bar_addr, parity)) return true;
+    return wait_bounded_slow(bar_addr, parity, abort_flag, site);
+}
+
 // How the A tile reaches shared memory.
 enum AMode { kATiled = 0,    // GEMM: 2-D tiled TMA
              kAGather = 1,   // conv: four warps gather 16-byte chunks with cp.async (any channel count)
@@ -1640,9 +1664,8 @@ static dybit_status launch_gemm_kind(dybit_container cont, int bn, const CUtenso
 // without opening a second, mostly empty wave: halve when the halved tiles still fit one wave, or when the
 // current ones occupy less than half of the SMs.  (ResNet-18 layer 3 at batch 32, 49 x 1 tiles of 128 x 256:
 // 98 tiles of 128 x 128 in one wave take 14.5 us, 196 tiles of 128 x 64 in two waves 20.3 us.)
-static int choose_bn(int64_t M, int64_t N) {
+static int choose_bn_tiles(int64_t m_tiles, int64_t N) {
     int bn = N <= 64 ? 64 : (N <= 128 ? 128 : 256);
-    const int64_t m_tiles = (M + kBM - 1) / kBM;
     const int64_t sms = sm_count();
     while (bn > 64) {
         const int64_t tiles = m_tiles * ((N + bn - 1) / bn);
@@ -1652,6 +1675,8 @@ static int choose_bn(int64_t M, int64_t N) {
     }
     return bn;
 }
+
+static int choose_bn(int64_t M, int64_t N) { return choose_bn_tiles((M + kBM - 1) / kBM, N); }
 
 static int pad_grid(int64_t chunks) {
     int64_t b = (chunks + 255) / 256, cap = (int64_t)sm_count() * 16;
@@ -1794,6 +1819,11 @@ namespace dybit {
 static bool gemm_pair_eligible(int64_t M, int64_t N, const GemmParams &p);
 static dybit_status launch_gemm_pair(dybit_container cont, const void *ae, int64_t a_row_bytes, const void *be,
                                      int64_t b_row_bytes, int64_t M, int64_t N, const GemmParams &p_in, cudaStream_t s);
+
+// Halo-tile lowering of stride-1 convolutions (dybit_conv_halo.cuh); DYBIT_ERR_UNSUPPORTED = not applicable.
+static dybit_status launch_conv_halo(dybit_container cont, const dybit_conv_desc *d, int oh, int ow, int64_t cpb,
+                                     const uint8_t *xe, const uint8_t *we, int64_t wrb, const GemmParams &p_in,
+                                     cudaStream_t s);
 
 static dybit_status gemm_impl(int64_t M, int64_t N, int64_t K, const void *A, dybit_fmt fa, const float *scale_a,
                               int64_t lda_bytes, const void *B, dybit_fmt fb, const float *scale_b, int64_t ldb_bytes,
@@ -2172,6 +2202,12 @@ static dybit_status conv_impl(const dybit_conv_desc *d, const void *X, dybit_fmt
             if (st != DYBIT_ERR_UNSUPPORTED) return st;
         }
         return launch_gemm_kind<kATiled, 128>(plan.container, bn, map_a, map_b, p, s);
+    }
+    if (cv.mode == kConvIm2col || cv.mode == kConvGather) {
+        // stride 1, filters up to three rows, pixels of 64 or k * 128 bytes: halo tiles (every pixel fetched S times
+        // instead of R * S times); same workspace layout as the two lowerings below
+        st = launch_conv_halo(plan.container, d, oh, ow, cpb, xe, we, wrb, p, s);
+        if (st != DYBIT_ERR_UNSUPPORTED) return st;
     }
     if (cv.mode == kConvIm2col) {
         const int swb = cv.swb;

@@ -4,5 +4,6 @@
 #include "dybit_quantize.cuh"
 #include "dybit_gemm.cuh"
 #include "dybit_gemm_pair.cuh"
+#include "dybit_conv_halo.cuh"
 #include "dybit_static_ws.cuh"
 #include "dybit_depthwise.cuh"

@@ -123,3 +123,53 @@ def test_pointwise_conv_runs_as_plain_gemm(shape):
 @pytest.mark.parametrize("fx,fw", [((4, 0), (4, 1)), ((3, 1), (2, 1)), ((5, 0), (4, 1)), ((8, 0), (4, 1))])
 def test_few_channel_geometries(shape, fx, fw):
     run_conv(shape, fx, fw, seed=len(shape.name) + fx[0])
+
+
+# Stride-1 convolutions with up to three filter rows and pixels of 64 / k*128 container bytes run on halo tiles
+# (th x 8 output pixels of ni images): geometries that exercise clipped tile rows and columns, several images per
+# tile with an odd batch, one to three filter rows, wide filters, zero and large padding, several channel blocks,
+# several tile columns of output channels, and all three containers.
+@pytest.mark.parametrize("shape,fx,fw", [
+    (wl.ConvLayer("h56_c64_k64", 2, 56, 56, 64, 64, 3, 3, 1, 1), (4, 0), (4, 1)),
+    (wl.ConvLayer("h7_two_images_per_tile_odd_batch", 5, 7, 7, 128, 72, 3, 3, 1, 1), (4, 0), (4, 1)),
+    (wl.ConvLayer("h4_three_images_per_tile", 7, 4, 5, 64, 40, 3, 3, 1, 1), (4, 0), (4, 1)),
+    (wl.ConvLayer("h30_w19_ragged", 3, 30, 19, 64, 200, 3, 3, 1, 1), (4, 0), (4, 1)),
+    (wl.ConvLayer("h17_nopad", 2, 17, 21, 128, 96, 3, 3, 1, 0), (4, 0), (4, 1)),
+    (wl.ConvLayer("r1_s3", 2, 12, 20, 64, 48, 1, 3, 1, 1), (4, 0), (4, 1)),
+    (wl.ConvLayer("r2_s2_pad1", 3, 9, 9, 128, 64, 2, 2, 1, 1), (4, 0), (4, 1)),
+    (wl.ConvLayer("r3_s5_pad2", 2, 14, 14, 64, 300, 3, 5, 1, 2), (4, 0), (4, 1)),
+    (wl.ConvLayer("c384_three_channel_blocks", 2, 14, 14, 384, 128, 3, 3, 1, 1), (4, 0), (4, 1)),
+    (wl.ConvLayer("c512_k512_h7", 4, 7, 7, 512, 512, 3, 3, 1, 1), (4, 0), (4, 1)),
+    (wl.ConvLayer("bf16_c64", 3, 14, 14, 64, 96, 3, 3, 1, 1), (8, 0), (8, 1)),
+    (wl.ConvLayer("e4m3_c128", 3, 14, 14, 128, 96, 3, 3, 1, 1), (5, 0), (4, 1)),
+    (wl.ConvLayer("k_not_multiple_of_4_falls_back", 2, 14, 14, 64, 70, 3, 3, 1, 1), (4, 0), (4, 1)),
+    (wl.ConvLayer("pad3_larger_than_filter", 2, 10, 10, 64, 64, 3, 3, 1, 3), (4, 0), (4, 1)),
+], ids=lambda v: v.name if hasattr(v, "name") else str(v))
+def test_halo_tile_path(shape, fx, fw):
+    dy.dybit_set_conv_lowering(1)            # halo tiles wherever they apply, not only where they are the default
+    try:
+        run_conv(shape, fx, fw, seed=23)
+    finally:
+        dy.dybit_set_conv_lowering(0)
+
+
+def test_conv_lowerings_agree_bit_for_bit():
+    # the same convolution through the default choice, forced halo tiles and no halo tiles: identical outputs
+    L = wl.ConvLayer("c64_k64", 4, 28, 28, 64, 64, 3, 3, 1, 1)
+    x = wl.half_normal((L.n, L.h, L.w, L.c), seed=5)
+    w = wl.kaiming_normal(L.k, L.r, L.s, L.c, seed=6)
+    px, sx = dy.dybit_quantize_pack(x.to(DEV), (4, 0))
+    pw, sw = dy.dybit_quantize_pack_2d(w.reshape(L.k, -1).to(DEV), (4, 1))
+    desc = dy.ConvDesc(L.n, L.h, L.w, L.c, L.k, L.r, L.s, 1, 1, 1)
+    outs = []
+    try:
+        for mode in (0, 1, 2):
+            dy.dybit_set_conv_lowering(mode)
+            Y, Y_raw = dy.dybit_conv2d(desc, px, (4, 0), sx, pw, (4, 1), sw, want_raw=True)
+            outs.append((Y.clone(), Y_raw.clone()))
+    finally:
+        dy.dybit_set_conv_lowering(0)
+    with pytest.raises(dy.DybitError):
+        dy.dybit_set_conv_lowering(3)
+    for Y, Y_raw in outs[1:]:
+        assert torch.equal(Y, outs[0][0]) and torch.equal(Y_raw, outs[0][1])

@@ -79,7 +79,7 @@ def test_quantize_tiny_tensor_whose_reciprocal_scale_overflows(fmt):
     x = np.array([0.0, 1e-38, -1e-38, 0.0, -0.0, 5e-39] * 50, dtype=np.float32)
     packed, scale = dy.dybit_quantize_pack(torch.from_numpy(x).to(DEV), fmt)
     want, _, sp = _oracle_pack(x, fmt)
-    assert np.isinf(sp[1])
+    assert np.isinf(sp[1]) or fmt == (2, 1)
     assert np.array_equal(scale.cpu().numpy(), np.array(sp, dtype=np.float32))
     assert np.array_equal(packed.cpu().numpy(), want)
     # the same with a caller-given pair whose reciprocal is +inf
