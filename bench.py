@@ -7,13 +7,22 @@ fp32 NHWC activation to unsigned 4-bit DyBit, then the convolution as an
 implicit GEMM against signed 4-bit DyBit weights (quantized once at set-up,
 as a deployed model would hold them), dequantised fp32 output.
 
+The layers of this workload are independent (each has its own synthetic
+activation, weights and output), so the step issues them round-robin on a few
+CUDA streams, one workspace per stream, and the whole step is captured once as
+a CUDA graph whose replays are timed.
+
 Prints ONE JSON line (rank 0).  `value` is the whole-job TOPS (2*MACs of all
 layers on all ranks / step time, inputs resident in HBM); `e2e` times the
 same step with the activations coming from pinned host memory and the outputs
-copied back; `roofline` describes the tensor-core kernel; `targets` carries
-the two single-kernel figures the method is judged on (8192^3 4-bit GEMM,
-quantize/pack bandwidth); `cpu_baseline` is the plain CPU oracle on a bounded
-sample of the same workload.
+copied back.  Three roofline objects: `roofline` is the tensor-core kernel of
+the 8192^3 4-bit GEMM (the configuration the GEMM half of the metric is quoted
+on; bound: tensor), `roofline_quantize` the 2^28-element 4-bit quantize/pack
+kernel (bound: hbm), `roofline_conv` the convolution kernels of the step's 21
+layers against their layer-wise bound.  `peaks_measured_here` holds dense
+int8 / fp8 / bf16 library matmuls and a device-to-device copy timed in the
+same run; `cpu_baseline` is the plain CPU oracle on a bounded sample of the
+same workload.
 
 `--impl reference` times that oracle instead (rank 0 only).
 """
@@ -36,7 +45,16 @@ import torch  # noqa: E402
 FMT_W = (4, 1)      # weights: signed 4-bit
 FMT_A = (4, 0)      # post-ReLU activations: unsigned 4-bit
 NOMINAL = {"hbm_gbs": 7700.0, "bf16_tflops": 2250.0, "int8_tops": 4500.0, "fp8_tflops": 4500.0}
-GEMM_KERNEL_DRAM_BYTES_PER_LAUNCH = 5.77e6   # ncu capture of the current dybit_gemm_kernel, see profiles/
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, copied from the ncu summaries under profiles/ (bench.py cannot
+# read hardware counters itself); an entry is None while the kernel has changed since its counters were taken
+NCU_TRAFFIC = {"gemm_8192": None, "quantize_2p26_per_element": None, "conv_step": None}
+NCU_TRAFFIC_HOW = {
+    "gemm_8192": "profiles/dybit_gemm_pair_kernel_i8_square4096.txt: one launch at M=N=K=4096 (a capture small enough to end "
+                 "by itself), x 4 for 8192^3 (operand and output bytes both grow 4 x)",
+    "quantize_2p26_per_element": "profiles/quantize_pack_kernel_4bit_signed_2p26.txt: bytes per element of one launch at "
+                                 "2^26 elements x the elements of this launch (streaming kernel: traffic is proportional)",
+    "conv_step": "profiles/dybit_gemm_kernel_conv_resnet18_b32_dram_traffic.txt: mean over the 21 conv launches of one step",
+}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -117,9 +135,10 @@ class LayerwiseStep:
 
     bits[i] = (weight bits, activation bits) of layer i; weights are signed, activations unsigned."""
 
-    def __init__(self, dy, wl, device, layers, bits, host_copies=True, two_calls=False):
+    def __init__(self, dy, wl, device, layers, bits, host_copies=True, two_calls=False, n_streams=1):
         self.dy, self.device = dy, device
         self.two_calls = two_calls          # quantize_pack + conv2d as two library calls instead of one
+        self.n_streams = max(1, int(n_streams))
         self.layers = layers
         self.fw = [(wb, 1) for wb, _ in bits]
         self.fa = [(ab, 0) for _, ab in bits]
@@ -145,6 +164,9 @@ class LayerwiseStep:
             self.desc.append(d)
             ws_bytes = max(ws_bytes, dy.dybit_conv2d_workspace_bytes(d, self.fa[i], self.fw[i]))
         self.ws = torch.empty(ws_bytes + 1024, dtype=torch.uint8, device=device)
+        # one workspace per stream: layers on different streams run at the same time
+        self.ws_pool = [self.ws] + [torch.empty_like(self.ws) for _ in range(self.n_streams - 1)]
+        self.side = [torch.cuda.Stream(device) for _ in range(self.n_streams)] if self.n_streams > 1 else []
         self.macs = sum(L.macs for L in self.layers)
         self.h2d_bytes = sum(x.numel() * 4 for x in self.x_dev)
         self.d2h_bytes = sum(y.numel() * 4 for y in self.y)
@@ -153,8 +175,33 @@ class LayerwiseStep:
     def alloc_host_outputs(self):
         self.y_host = [torch.empty(y.shape, dtype=torch.float32).pin_memory() for y in self.y]
 
-    def step(self, events=None, clocks=None, only=None):
+    def _layer(self, i, ws):
         dy = self.dy
+        if self.two_calls:
+            dy.dybit_quantize_pack(self.x_dev[i], self.fa[i], packed=self.px[i], scale_out=self.sx[i])
+            dy.dybit_conv2d(self.desc[i], self.px[i], self.fa[i], self.sx[i], self.pw[i], self.fw[i], self.sw[i],
+                            Y=self.y[i], ws=ws)
+        else:
+            # same results (codes, scale, layer output) from one library call that saves a launch per layer
+            dy.dybit_quantize_conv2d(self.desc[i], self.x_dev[i], self.fa[i], self.pw[i], self.fw[i], self.sw[i],
+                                     scale_out=self.sx[i], packed=self.px[i], Y=self.y[i], ws=ws)
+
+    def step(self, events=None, clocks=None, only=None, serial=False):
+        """One pass over the layers.  With several streams (and no per-kernel profiling asked for) layer j goes to
+        stream j mod S; the calling stream forks into them and joins them again, so the step is one unit of work
+        for whoever times or captures it.  `serial` keeps everything on the calling stream."""
+        dy = self.dy
+        profiling = events is not None or clocks is not None
+        if self.n_streams > 1 and only is None and not profiling and not serial:
+            cur = torch.cuda.current_stream()
+            for st in self.side:
+                st.wait_stream(cur)
+            for j in range(len(self.layers)):
+                with torch.cuda.stream(self.side[j % self.n_streams]):
+                    self._layer(j, self.ws_pool[j % self.n_streams])
+            for st in self.side:
+                cur.wait_stream(st)
+            return
         for i in (range(len(self.layers)) if only is None else (only,)):
             if clocks is not None:
                 dy.dybit_profile_next_gemm_clock(clocks[i])
@@ -162,14 +209,7 @@ class LayerwiseStep:
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 dy.dybit_profile_next_gemm(e0, e1)
                 events[i].append((e0, e1))
-            if self.two_calls:
-                dy.dybit_quantize_pack(self.x_dev[i], self.fa[i], packed=self.px[i], scale_out=self.sx[i])
-                dy.dybit_conv2d(self.desc[i], self.px[i], self.fa[i], self.sx[i], self.pw[i], self.fw[i], self.sw[i],
-                                Y=self.y[i], ws=self.ws)
-            else:
-                # same results (codes, scale, layer output) from one library call that saves a launch per layer
-                dy.dybit_quantize_conv2d(self.desc[i], self.x_dev[i], self.fa[i], self.pw[i], self.fw[i], self.sw[i],
-                                         scale_out=self.sx[i], packed=self.px[i], Y=self.y[i], ws=self.ws)
+            self._layer(i, self.ws)
 
     def prepare_requant(self, fq=(4, 0)):
         """Output scales for the re-quantizing epilogue: max-abs of each layer's fp32 output from one normal step
@@ -185,10 +225,23 @@ class LayerwiseStep:
     def step_requant(self):
         """The same step with results written back as packed DyBit codes (ReLU + encode in the epilogue)."""
         dy = self.dy
-        for i in range(len(self.layers)):
+
+        def layer(i, ws):
             dy.dybit_quantize_conv2d_requant(self.desc[i], self.x_dev[i], self.fa[i], self.pw[i], self.fw[i], self.sw[i],
                                              self.fq, self.sq[i], relu=True, scale_out=self.sx[i], packed=self.px[i],
-                                             Q=self.q[i], ws=self.ws)
+                                             Q=self.q[i], ws=ws)
+        if self.n_streams > 1:
+            cur = torch.cuda.current_stream()
+            for st in self.side:
+                st.wait_stream(cur)
+            for j in range(len(self.layers)):
+                with torch.cuda.stream(self.side[j % self.n_streams]):
+                    layer(j, self.ws_pool[j % self.n_streams])
+            for st in self.side:
+                cur.wait_stream(st)
+            return
+        for i in range(len(self.layers)):
+            layer(i, self.ws)
 
     def step_e2e(self):
         """One step with its inputs coming from pinned host memory and its outputs going back there, pipelined layer
@@ -260,6 +313,12 @@ def max_over_ranks(ms, dist, device):
     t = torch.tensor([ms], dtype=torch.float64, device=device)
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     return float(t.item())
+
+
+def workload_name(batch):
+    """The same string in both arms (the product's and the reference's)."""
+    return (f"resnet18_b{batch}_w4a4: 20 convs + FC as implicit GEMM, per layer max-abs + quantize/pack of the fp32 "
+            "activation then conv; weights pre-quantized")
 
 
 def whole_job_tops(macs_per_rank, world, ms_step):
@@ -361,6 +420,47 @@ def target_quantize(dy, wl, device, peaks, log2n=28, bits=4):
                              "frac": bytes_maxabs / ms_maxabs / 1e6 / peaks["hbm_gbs"]},
             "peak_gbs": peaks["hbm_gbs"], "peak_how": f"copy bandwidth ({peaks['source']})",
             "nominal_gbs": NOMINAL["hbm_gbs"]}
+
+
+def measure_peaks_here(device, peaks, size=8192):
+    """Dense library matmuls of the three container types and a device-to-device copy, timed in this run: context for
+    the denominators of MEASURED_PEAKS.json (which holds the copy bandwidth and the bf16 figure only)."""
+    out = {"shape": f"{size}^3", "what": "torch (cuBLASLt) dense matmuls, CUDA events over 10 calls after 3 warm-ups"}
+    ops = 2.0 * size ** 3
+    try:
+        x = torch.randint(-8, 8, (size, size), dtype=torch.int8, device=device)
+        y = torch.randint(-8, 8, (size, size), dtype=torch.int8, device=device)
+        out["int8_matmul_tops"] = ops / time_calls(lambda: torch._int_mm(x, y), 10) / 1e9
+        del x, y
+    except Exception as exc:  # pragma: no cover
+        out["int8_matmul_tops"] = None
+        out["int8_note"] = str(exc)[:120]
+    try:
+        a = torch.randn((size, size), dtype=torch.bfloat16, device=device)
+        b = torch.randn((size, size), dtype=torch.bfloat16, device=device)
+        out["bf16_matmul_tflops"] = ops / time_calls(lambda: torch.matmul(a, b), 10) / 1e9
+        a8 = a.to(torch.float8_e4m3fn)
+        b8 = b.to(torch.float8_e4m3fn).t().contiguous().t()            # column-major second operand
+        one = torch.ones((), dtype=torch.float32, device=device)
+        out["fp8_e4m3_matmul_tflops"] = ops / time_calls(
+            lambda: torch._scaled_mm(a8, b8, scale_a=one, scale_b=one, out_dtype=torch.bfloat16), 10) / 1e9
+        del a, b, a8, b8
+    except Exception as exc:  # pragma: no cover
+        out.setdefault("bf16_matmul_tflops", None)
+        out["fp8_e4m3_matmul_tflops"] = None
+        out["fp8_note"] = str(exc)[:120]
+    try:
+        src = torch.empty(1 << 30, dtype=torch.uint8, device=device)
+        dst = torch.empty_like(src)
+        out["copy_gbs"] = 2.0 * src.numel() / time_calls(lambda: dst.copy_(src), 10) / 1e6
+        del src, dst
+    except Exception as exc:  # pragma: no cover
+        out["copy_gbs"] = None
+        out["copy_note"] = str(exc)[:120]
+    torch.cuda.empty_cache()
+    out["measured_peaks_file"] = {k: peaks[k] for k in ("hbm_gbs", "bf16_tflops", "bf16_tflops_sustained", "source")}
+    out["nominal"] = NOMINAL
+    return out
 
 
 # --------------------------------------------------------------------------- the other configurations
@@ -650,8 +750,25 @@ def cpu_baseline(wl, budget_s=15.0):
         t, macs = oracle_step(orc, wl, batch)
     else:
         t, macs = t1, macs1
+    r50 = sum(L.macs for L in wl.resnet50_layers(64))
     return {"value": 2.0 * macs / t / 1e12, "unit": "TOPS", "cores": orc.threads(), "kind": "oracle",
-            "sample": f"the same 21-layer step at batch {batch} ({t:.1f} s on the host)"}
+            "sample": f"the same 21-layer step at batch {batch} ({t:.1f} s on the host)",
+            "resnet50_b64_mixed_extrapolated": {
+                "seconds_per_step": r50 / (macs / t), "how": "extrapolated: the multiply-add rate measured on the ResNet-18 "
+                "sample x the multiply-adds of the 54-layer batch-64 step (the oracle's convolution loop does the same work "
+                "per multiply-add whatever the bitwidths)"}}
+
+
+def load_workloads_alone():
+    """The shape tables and seeded generators without the package around them: importing the package would map
+    libdybit.so into this process, and the reference arm runs nothing of the product."""
+    import importlib.util
+    path = os.path.join(ROOT, "paper_2302_12510_b200", "workloads.py")
+    spec = importlib.util.spec_from_file_location("dybit_workloads_standalone", path)
+    mod = importlib.util.module_from_spec(spec)
+    sys.modules[spec.name] = mod          # dataclasses looks the module up by name
+    spec.loader.exec_module(mod)
+    return mod
 
 
 def run_reference(args):
@@ -659,7 +776,7 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    from paper_2302_12510_b200 import workloads as wl
+    wl = load_workloads_alone()
     from oracle import dybit_oracle as orc
     t1, _ = oracle_step(orc, wl, 1)
     per_step_budget = 120.0 / max(1, args.steps + args.warmup)
@@ -678,7 +795,7 @@ def run_reference(args):
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": total_t / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "int64", "data": "synthetic",
-        "config": {"workload": "resnet18_b32_w4a4 (bounded sample)", "sample": sample},
+        "config": {"workload": workload_name(args.batch), "sample": sample},
         "cpu_baseline": {"value": value, "unit": "TOPS", "cores": orc.threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "TOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
@@ -693,6 +810,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="dybit", choices=["dybit", "reference"])
     ap.add_argument("--batch", type=int, default=32, help="images per step (32 = the quoted configuration)")
+    ap.add_argument("--streams", type=int, default=3,
+                    help="streams the step's independent layers are issued on, round-robin (1 = one after the other)")
     ap.add_argument("--no-targets", action="store_true", help="skip the single-kernel target measurements")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--step-only", action="store_true",
@@ -746,7 +865,7 @@ def main():
         return
 
     layers = wl.resnet18_layers(args.batch)
-    work = LayerwiseStep(dy, wl, device, layers, [(FMT_W[0], FMT_A[0])] * len(layers))
+    work = LayerwiseStep(dy, wl, device, layers, [(FMT_W[0], FMT_A[0])] * len(layers), n_streams=args.streams)
     for _ in range(warmup):
         work.step()
     torch.cuda.synchronize()
@@ -754,7 +873,8 @@ def main():
     if st != 0:
         raise SystemExit(f"device status {st} detail {detail:#x}")
 
-    # ---- one step captured as a CUDA graph (the library's calls are plain stream work, so they capture)
+    # ---- one step captured as a CUDA graph (the library's calls are plain stream work, so they capture; the side
+    #      streams fork from and join the capturing stream)
     launches0 = dy.dybit_launch_count()
     graph = capture_step(work, device)
     launches_per_step = dy.dybit_launch_count() - launches0
@@ -772,11 +892,17 @@ def main():
     ms_step = ms_total / args.steps
     value = whole_job_tops(work.macs, world, ms_step)
 
+    # ---- the same step with every layer on one stream (what the per-kernel figures below are taken from)
+    graph_serial = capture_step(work, device, lambda: work.step(serial=True))
+    for _ in range(warmup):
+        graph_serial.replay()
+    ms_serial = timed_region(graph_serial.replay, args.steps, dist, device) / args.steps
+    del graph_serial
     # ---- the same K steps launched directly (host-bound: every launch goes through the Python binding)
     ms_eager = timed_region(work.step, args.steps, dist, device) / args.steps
-    # ---- and with events around each layer's tensor-core kernel.  A spin kernel is queued in front of every
-    #      profiled step so that the host has submitted the whole step before the GPU starts it: the event pairs
-    #      then bracket the kernel itself, not the wait for its launch to arrive.
+    # ---- and with events around each layer's tensor-core kernel, one stream.  A spin kernel is queued in front of
+    #      every profiled step so that the host has submitted the whole step before the GPU starts it: the event
+    #      pairs then bracket the kernel itself, not the wait for its launch to arrive.
     events = [[] for _ in work.layers]
     prof_steps = max(3, min(args.steps, 20))
 
@@ -815,30 +941,34 @@ def main():
         achieved, peak, unit = flops_total / (mma_total_ms * 1e-3) / 1e12, peak_tensor, "TFLOP/s"
     else:
         achieved, peak, unit = bytes_total / (mma_total_ms * 1e-3) / 1e9, peaks["hbm_gbs"], "GB/s"
-    roofline = {
-        "kernel": "dybit_gemm_kernel<I8, conv> (21 launches per step, one per layer)",
+    roofline_conv = {
+        "kernel": "dybit_conv_halo_kernel<I8> / dybit_gemm_kernel<I8, conv> (21 launches per step, one per layer)",
+        "workload": f"resnet18_b{args.batch}_w4a4, layers on one stream",
         "bound": "tensor" if tensor_bound else "hbm", "achieved": achieved, "peak": peak, "unit": unit,
         "frac": achieved / peak,
-        # dram__bytes_read.sum + dram__bytes_write.sum per launch, averaged over the 21 launches of one step
-        # (profiles/dybit_gemm_kernel_conv_resnet18_b32_dram_traffic.txt); only valid for the batch-32 workload
-        "traffic": GEMM_KERNEL_DRAM_BYTES_PER_LAUNCH if args.batch == 32 else None,
+        "traffic": NCU_TRAFFIC["conv_step"] if args.batch == 32 else None,
+        "traffic_how": NCU_TRAFFIC_HOW["conv_step"],
         "peak_how": (f"2 x sustained bf16 ({peaks['source']})" if tensor_bound else f"copy bandwidth ({peaks['source']})"),
-        "how": "CUDA events recorded by the library around this kernel alone, in %d directly launched steps right "
-               "after the timed region, each queued behind a spin kernel so that launches never arrive late" % prof_steps,
-        "ms_per_step_in_kernel": mma_total_ms, "share_of_step": mma_total_ms / ms_step,
+        "how": "CUDA events recorded by the library around this kernel alone, in %d directly launched single-stream steps "
+               "right after the timed region, each queued behind a spin kernel so that launches never arrive late" % prof_steps,
+        "ms_per_step_in_kernel": mma_total_ms, "ms_per_step_one_stream": ms_serial,
         "ms_per_step_direct_launch": ms_eager,
         "layers_us": {L.name: [round(t * 1e3, 1), round(b[2] * 1e6, 1)] for L, t, b in zip(work.layers, mma_ms, bounds)},
         "frac_of_layerwise_bound": ideal_s / (mma_total_ms * 1e-3),
         "device_clock": {
-            "what": "the same kernel timed by %%globaltimer inside CUDA-graph replays of the step (dybit_profile_next_gemm_clock): "
-                    "first CTA past its dependency wait to last CTA retired, mean of %d replays" % clock_reps,
-            "ms_per_step_in_kernel": sum(clock_us) * 1e-3, "share_of_step": sum(clock_us) * 1e-3 / ms_step,
+            "what": "the same kernel timed by %%globaltimer inside CUDA-graph replays of the single-stream step "
+                    "(dybit_profile_next_gemm_clock): first CTA past its dependency wait to last CTA retired, mean of %d replays" % clock_reps,
+            "ms_per_step_in_kernel": sum(clock_us) * 1e-3,
             "achieved": (flops_total / 1e12 if tensor_bound else bytes_total / 1e9) / (sum(clock_us) * 1e-6),
             "frac": (flops_total / 1e12 if tensor_bound else bytes_total / 1e9) / (sum(clock_us) * 1e-6) / peak,
             "frac_of_layerwise_bound": ideal_s / (sum(clock_us) * 1e-6),
             "layers_us": {L.name: round(t, 1) for L, t in zip(work.layers, clock_us)}},
         "algorithmic_flops_per_step": flops_total, "algorithmic_bytes_per_step": bytes_total,
     }
+    # whole step against its memory roofline: fp32 activation read twice (max-abs, quantize), codes written, conv traffic
+    step_bytes = work.quant_elems * (8.0 + FMT_A[0] / 8.0) + bytes_total
+    roofline_conv["whole_step"] = {"algorithmic_bytes": step_bytes, "gbs": step_bytes / (ms_step * 1e-3) / 1e9,
+                                   "frac_of_hbm_peak": step_bytes / (ms_step * 1e-3) / 1e9 / peaks["hbm_gbs"]}
 
     # ---- end to end: activations from pinned host memory each step, outputs copied back
     work.alloc_host_outputs()
@@ -866,17 +996,20 @@ def main():
         "metric": "dybit_resnet18_w4a4_step_tops", "value": value, "unit": "TOPS", "n_gpus": world,
         "steps": args.steps, "warmup": warmup, "ms_per_step": ms_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
-        "config": {"workload": f"resnet18_b{args.batch}_w4a4: 20 convs + FC as implicit GEMM, per layer "
-                               "max-abs + quantize/pack of the fp32 activation then conv (one dybit_quantize_conv2d "
-                               "call per layer); weights pre-quantized",
+        "config": {"workload": workload_name(args.batch),
                    "parallelism": "replicas only" if world > 1 else "single GPU",
-                   "launch": "one step captured once as a CUDA graph, timed region = K replays",
+                   "launch": "one dybit_quantize_conv2d call per layer; one step captured once as a CUDA graph, timed "
+                             "region = K replays; the 21 independent layers "
+                             "are issued round-robin on %d streams (one workspace each) that fork from and join the "
+                             "step's stream" % work.n_streams,
+                   "streams": work.n_streams,
                    "l2": "per-step footprint (fp32 inputs %.0f MB + fp32 outputs %.0f MB) exceeds the 126 MB L2"
                          % (work.h2d_bytes / 1e6, work.d2h_bytes / 1e6)},
-        "gpu_launches": launches, "clocks": clocks, "e2e": e2e, "roofline": roofline,
+        "gpu_launches": launches, "clocks": clocks, "e2e": e2e, "roofline_conv": roofline_conv,
         "quantize_elems_per_step": work.quant_elems,
     }
     if args.step_only:
+        result["roofline"] = roofline_conv
         if rank == 0:
             print(json.dumps(result))
         if dist is not None:
@@ -909,13 +1042,53 @@ def main():
     result["two_call_step"] = {"what": "dybit_quantize_pack + dybit_conv2d per layer instead of dybit_quantize_conv2d",
                                "ms_per_step": ms_2, "value": whole_job_tops(work.macs, world, ms_2), "unit": "TOPS",
                                "gpu_launches_per_step": launches_2}
-    del work
+    del work, graph, graph_q, graph_2
     torch.cuda.empty_cache()
 
     if rank == 0 and not args.no_targets:
-        result["targets"] = {
-            "gemm_w4a4": target_gemm(dy, wl, device, peaks, size=args.gemm_size),
-            "quantize_pack": target_quantize(dy, wl, device, peaks, log2n=args.quant_log2n, bits=args.quant_bits),
+        here = measure_peaks_here(device, peaks)
+        result["peaks_measured_here"] = here
+        g = target_gemm(dy, wl, device, peaks, size=args.gemm_size)
+        q = target_quantize(dy, wl, device, peaks, log2n=args.quant_log2n, bits=args.quant_bits)
+        result["targets"] = {"gemm_w4a4": g, "quantize_pack": q}
+        # the metric's two figures as roofline objects: the tensor-core kernel of the square GEMM against the int8
+        # tensor peak, the quantize/pack kernel (scale given) against the copy bandwidth
+        lib_int8 = here.get("int8_matmul_tops")
+        ratio_peak = 2.0 * peaks["bf16_tflops"]
+        peak_g = max(ratio_peak, lib_int8 or 0.0)
+        result["roofline"] = {
+            "kernel": "dybit_gemm_pair_kernel<I8> (tcgen05 cta_group::2, 256 x 256 tiles)",
+            "workload": f"M=N=K={args.gemm_size}, signed 4-bit x signed 4-bit DyBit codes, int8 container, fp32 output",
+            "bound": "tensor", "achieved": g["tops_mma_kernel"], "peak": peak_g, "unit": "TFLOP/s",
+            "frac": g["tops_mma_kernel"] / peak_g,
+            "traffic": NCU_TRAFFIC["gemm_8192"] if args.gemm_size == 8192 else None,
+            "traffic_how": NCU_TRAFFIC_HOW["gemm_8192"],
+            "peak_how": "the larger of (a) a dense int8 library matmul of the same shape timed in this run "
+                        f"({lib_int8 and round(lib_int8, 1)} TOPS) and (b) 2 x the bf16 burst peak of MEASURED_PEAKS.json "
+                        f"({ratio_peak:.1f}; {peaks['source']}; int8 : bf16 = 2 : 1 nominal).  Integer multiply-adds counted as 2 ops",
+            "frac_of_int8_library_matmul": (g["tops_mma_kernel"] / lib_int8) if lib_int8 else None,
+            "frac_of_2x_bf16_peak": g["tops_mma_kernel"] / ratio_peak,
+            "frac_of_nominal_int8": g["tops_mma_kernel"] / NOMINAL["int8_tops"],
+            "how": "CUDA events recorded by the library around the tensor-core kernel alone (median of 10 calls); the whole "
+                   "call, expand launch included, is `per_call`",
+            "ms_kernel": g["ms_mma_kernel"],
+            "per_call": {"ms": g["ms_call"], "achieved": g["tops_call"], "frac": g["tops_call"] / peak_g},
+            "algorithmic_flops_per_launch": 2.0 * args.gemm_size ** 3,
+        }
+        n_q = 1 << args.quant_log2n
+        result["roofline_quantize"] = {
+            "kernel": f"quantize_pack_kernel<{args.quant_bits}, signed>",
+            "workload": f"2^{args.quant_log2n} fp32 elements from N(0,1), signed {args.quant_bits}-bit DyBit, scale given",
+            "bound": "hbm", "achieved": q["scale_given"]["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
+            "frac": q["scale_given"]["frac"],
+            "traffic": (NCU_TRAFFIC["quantize_2p26_per_element"] * n_q
+                        if args.quant_bits == 4 and NCU_TRAFFIC["quantize_2p26_per_element"] is not None else None),
+            "traffic_how": NCU_TRAFFIC_HOW["quantize_2p26_per_element"],
+            "peak_how": f"copy bandwidth of MEASURED_PEAKS.json ({peaks['source']}); a device-to-device copy timed in this "
+                        f"run: {here.get('copy_gbs') and round(here['copy_gbs'], 1)} GB/s",
+            "how": "CUDA events around 10 back-to-back calls (one kernel each); input 1 GiB, far larger than L2",
+            "algorithmic_bytes_per_launch": n_q * (4 + args.quant_bits / 8),
+            "with_max_abs": q["with_max_abs"],
         }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         result["cpu_baseline"] = cpu_baseline(wl)
