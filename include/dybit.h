@@ -363,6 +363,15 @@ dybit_status dybit_gemm_static_ws(int64_t M, int64_t N, int64_t K,
  * otherwise.  detail: [host] optional, receives the raw status word. */
 dybit_status dybit_last_device_status(void *stream, uint32_t *detail);
 
+/* Self-test of the give-up path of the bounded device-side waits (no counterpart in the paper).  Launches one small
+ * kernel in which a single thread waits, with the same routine every kernel of the library waits with, on a barrier
+ * that nothing will ever signal, for at most limit_ns nanoseconds (1 .. 100,000,000).  The wait runs out, the
+ * kernel records it in the device status word and returns normally: afterwards dybit_last_device_status reports
+ * DYBIT_ERR_DEVICE_TIMEOUT once (detail = 0x5e01) and the device keeps working.  result: [device] two 32-bit words,
+ * [0] = 1 if the wait reported failure, [1] = the CTA's abort flag.  Errors: INVALID_ARG (null result, limit out of
+ * range), ALIGNMENT, CUDA. */
+dybit_status dybit_selftest_wait_timeout(uint64_t limit_ns, uint32_t *result, void *stream);
+
 /* ---------------------------------------------------------------- measurement hooks
  * (no counterpart in the paper: they exist so that a benchmark can attribute
  * time to the tensor-core kernel alone and count the library's launches) */

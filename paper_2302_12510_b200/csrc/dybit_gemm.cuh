@@ -904,10 +904,10 @@ struct GemmParams {
     int64_t c_bstride;        // batched GEMM: elements between consecutive entries of C / C_raw
 };
 
-// Waits for the phase with the given parity; gives up after kWaitLimitNs, records
-// the site in the device status word and raises the CTA-wide abort flag.
+// Waits for the phase with the given parity; gives up after `limit_ns` (kWaitLimitNs in every kernel of the
+// library), records the site in the device status word and raises the CTA-wide abort flag.
 __device__ __forceinline__ bool wait_bounded(uint64_t *bar, uint32_t parity, volatile uint32_t *abort_flag,
-                                             unsigned site) {
+                                             unsigned site, unsigned long long limit_ns = kWaitLimitNs) {
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = global_timer_ns();
     unsigned spins = 0;
@@ -915,7 +915,7 @@ __device__ __forceinline__ bool wait_bounded(uint64_t *bar, uint32_t parity, vol
         if (mbar_try_wait(bar, parity)) return true;
         if ((++spins & 63u) == 0u) {
             if (*abort_flag) return false;
-            if (global_timer_ns() - t0 > kWaitLimitNs) {
+            if (global_timer_ns() - t0 > limit_ns) {
                 atomicOr(&g_device_status, (site << 8) | 1u);
                 *abort_flag = 1u;
                 return false;
@@ -946,6 +946,24 @@ __device__ __forceinline__ bool wait_bounded_addr(uint32_t bar_addr, uint32_t pa
                                                   unsigned site) {
     if (mbar_try_wait_addr(bar_addr, parity)) return true;
     return wait_bounded_slow(bar_addr, parity, abort_flag, site);
+}
+
+// Self-test of the give-up path: one thread waits, with the library's own wait_bounded, on a barrier that nothing
+// ever arrives on.  The wait runs out after limit_ns, sets the status word (site kSelftestSite) and the abort flag
+// and returns; result[0] receives 1 if the wait reported failure, result[1] the abort flag.
+constexpr unsigned kSelftestSite = 0x5e;
+__global__ void wait_timeout_selftest_kernel(unsigned long long limit_ns, unsigned *result) {
+    __shared__ uint64_t bar;
+    __shared__ uint32_t abort_word;
+    pdl_enter();
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        abort_word = 0;
+        fence_mbar_init();
+        const bool got = wait_bounded(&bar, 0u, &abort_word, kSelftestSite, limit_ns);
+        result[0] = got ? 0u : 1u;
+        result[1] = abort_word;
+    }
 }
 
 // How the A tile reaches shared memory.
@@ -2230,6 +2248,14 @@ static dybit_status conv_impl(const dybit_conv_desc *d, const void *X, dybit_fmt
 }  // namespace dybit
 
 extern "C" {
+
+dybit_status dybit_selftest_wait_timeout(uint64_t limit_ns, uint32_t *result, void *stream) {
+    if (result == nullptr || limit_ns == 0 || limit_ns > 100000000ull) return DYBIT_ERR_INVALID_ARG;   // at most 0.1 s
+    if (!dybit::aligned(result, 4)) return DYBIT_ERR_ALIGNMENT;
+    dybit::launch_k(dybit::wait_timeout_selftest_kernel, dim3(1u), dim3(32u), (size_t)0, static_cast<cudaStream_t>(stream),
+                    (unsigned long long)limit_ns, result);
+    return dybit::launch_status();
+}
 
 dybit_status dybit_gemm(int64_t M, int64_t N, int64_t K, const void *A, dybit_fmt fa, const float *scale_a,
                         int64_t lda_bytes, const void *B, dybit_fmt fb, const float *scale_b, int64_t ldb_bytes,

@@ -114,18 +114,34 @@ def _square_gemm(size, fmt, rng, n_rows, n_cols, n_points):
     else:
         amax = float(spa[0]) * float(np.abs(orc.decode_table(fmt[0], bool(fmt[1]))).max())
         bmax = float(spb[0]) * float(np.abs(orc.decode_table(fmt[0], bool(fmt[1]))).max())
-        assert np.abs(got.astype(np.float64) - Cref.astype(np.float64)).max() <= 1e-5 * size * amax * bmax
+        tol = 1e-5 * size * amax * bmax
+        assert np.abs(got.astype(np.float64) - Cref.astype(np.float64)).max() <= tol
+        # the whole output through its row and column sums: the exact integer sums of the oracle's definition, scaled,
+        # against fp64 sums of the fp32 result; every entry may be off by tol, a sum of `size` entries by size * tol
+        m = fmt[0] - 1 if fmt[1] else fmt[0]
+        tab = np.round(orc.decode_table(fmt[0], bool(fmt[1])) * 2.0 ** (m - 1)).astype(np.int64)
+        IA, IB = tab[ca], tab[cb]
+        alpha = float(spa[0]) * float(spb[0]) * 2.0 ** (-2 * (m - 1))
+        row_ref = (IA @ IB.sum(axis=0)).astype(np.float64) * alpha
+        col_ref = (IA.sum(axis=0) @ IB.T).astype(np.float64) * alpha
+        row_got = C.sum(dim=1, dtype=torch.float64).cpu().numpy()
+        col_got = C.sum(dim=0, dtype=torch.float64).cpu().numpy()
+        assert np.abs(row_got - row_ref).max() <= size * tol
+        assert np.abs(col_got - col_ref).max() <= size * tol
+        # and far tighter in practice: products are exact in fp32, only the accumulation rounds
+        assert np.abs(row_got - row_ref).max() <= 1e-3 * np.abs(row_ref).max() + size * tol * 1e-3
     torch.cuda.empty_cache()
 
 
 def test_square_gemm_8192_4bit_bench_configuration():
-    _square_gemm(8192, (4, 1), np.random.default_rng(1), n_rows=16, n_cols=16, n_points=20000)
+    _square_gemm(8192, (4, 1), np.random.default_rng(1), n_rows=256, n_cols=256, n_points=20000)
 
 
-@pytest.mark.parametrize("size,fmt", [(1024, (4, 1)), (2048, (4, 1)), (4096, (4, 1)), (1024, (8, 1)), (4096, (8, 1)),
-                                      (8192, (8, 1))])
+@pytest.mark.parametrize("size,fmt", [(1024, (4, 1)), (2048, (4, 1)), (4096, (4, 1)), (1024, (8, 1)), (2048, (8, 1)),
+                                      (4096, (8, 1)), (8192, (8, 1))])
 def test_square_gemm_sweep(size, fmt):
-    _square_gemm(size, fmt, np.random.default_rng(size), n_rows=8, n_cols=8, n_points=5000)
+    # 256 whole rows + 256 whole columns (+ scattered points) against the oracle at every size, both containers
+    _square_gemm(size, fmt, np.random.default_rng(size), n_rows=256, n_cols=256, n_points=5000)
 
 
 def _conv_layer_sampled(L, fx, fw, seed, n_samples=1500, one_call_too=False):

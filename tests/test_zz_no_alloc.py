@@ -6,11 +6,13 @@ different operands, since every call reuses the same scratch bytes -- and that i
 larger than the built-in scratch.
 
 Collected last (file name) so that a run stopping at the first failure has finished all other tests."""
+import numpy as np
 import pytest
 import torch
 
 import paper_2302_12510_b200 as dy
 from paper_2302_12510_b200 import workloads as wl
+from oracle import dybit_oracle as orc
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -45,6 +47,31 @@ def test_static_scratch_gemm_matches_workspace_gemm_twice(fa, fb):
         assert torch.equal(got, want)
         if cont == 0:
             assert torch.equal(got_raw, want_raw)
+
+
+def test_static_scratch_gemm_matches_the_oracle_and_allocates_nothing():
+    # against the CPU oracle directly (not only against dybit_gemm), and with the allocator's books and the
+    # device's free memory read before and after a call: the entry point must leave both untouched
+    fa, fb = (4, 0), (4, 1)
+    M, N, K = 200, 136, 333
+    a = wl.half_normal((M, K), seed=31)
+    b = wl.normal((N, K), seed=32, std=0.05)
+    pa, sa = dy.dybit_quantize_pack_2d(a.to(DEV), fa)
+    pb, sb = dy.dybit_quantize_pack_2d(b.to(DEV), fb)
+    got = torch.empty((M, N), dtype=torch.float32, device=DEV)
+    got_raw = torch.empty((M, N), dtype=torch.int32, device=DEV)
+    dy.dybit_gemm_static_ws(M, N, K, pa, fa, sa, pb, fb, sb, got, got_raw)       # first call on this device: set-up
+    torch.cuda.synchronize()
+    allocated, reserved, free = torch.cuda.memory_allocated(), torch.cuda.memory_reserved(), torch.cuda.mem_get_info()[0]
+    dy.dybit_gemm_static_ws(M, N, K, pa, fa, sa, pb, fb, sb, got, got_raw)
+    torch.cuda.synchronize()
+    assert torch.cuda.memory_allocated() == allocated and torch.cuda.memory_reserved() == reserved
+    assert torch.cuda.mem_get_info()[0] == free
+    spa, spb = orc.absmax_scale(a.numpy(), 4, False), orc.absmax_scale(b.numpy(), 4, True)
+    S, C_ref = orc.gemm(orc.quantize(a.numpy(), 4, False, spa[1]), fa, spa[0],
+                        orc.quantize(b.numpy(), 4, True, spb[1]), fb, spb[0])
+    assert np.array_equal(got_raw.cpu().numpy().astype(np.int64), S)
+    assert np.array_equal(got.cpu().numpy(), C_ref)
 
 
 def test_static_scratch_gemm_refuses_oversized_problems():
