@@ -402,6 +402,31 @@ def target_gemm(dy, wl, device, peaks, size=8192, fmt=(4, 1)):
     return out
 
 
+def target_gemm_decode(dy, wl, device, shapes=((128, 28672, 8192), (128, 8192, 8192), (8192, 8192, 8192))):
+    """The two ways dybit_gemm can turn packed 4-bit weights into int8: a separate expand launch into the workspace, or
+    decode warps inside the GEMM kernel's main loop (dybit_set_gemm_decode).  Per-call time, L2 flushed before each call."""
+    fa, fb = (4, 0), (4, 1)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+    rows = []
+    for (M, N, K) in shapes:
+        pa, sa = dy.dybit_quantize_pack_2d(wl.half_normal((M, K), seed=1, device=device), fa)
+        pb, sb = dy.dybit_quantize_pack_2d(wl.normal((N, K), seed=2, device=device), fb)
+        C = torch.empty((M, N), dtype=torch.float32, device=device)
+        ws = torch.empty(dy.dybit_gemm_workspace_bytes(M, N, K, fa, fb) + 1024, dtype=torch.uint8, device=device)
+        us = {}
+        try:
+            for mode, name in ((0, "expand_launch"), (1, "decode_in_main_loop")):
+                dy.dybit_set_gemm_decode(mode)
+                us[name] = time_calls_flushed(lambda: dy.dybit_gemm(M, N, K, pa, fa, sa, pb, fb, sb, C_out=C, ws=ws), 7, flush) * 1e3
+        finally:
+            dy.dybit_set_gemm_decode(2)
+        rows.append({"M": M, "N": N, "K": K, "us_per_call": us,
+                     "packed_weight_gbs_decode_in_main_loop": N * K / 2 / us["decode_in_main_loop"] / 1e3})
+        del pa, pb, C, ws
+        torch.cuda.empty_cache()
+    return rows
+
+
 def target_quantize(dy, wl, device, peaks, log2n=28, bits=4):
     n = 1 << log2n
     x = wl.normal((n,), seed=21, device=device)
@@ -1050,7 +1075,7 @@ def main():
         result["peaks_measured_here"] = here
         g = target_gemm(dy, wl, device, peaks, size=args.gemm_size)
         q = target_quantize(dy, wl, device, peaks, log2n=args.quant_log2n, bits=args.quant_bits)
-        result["targets"] = {"gemm_w4a4": g, "quantize_pack": q}
+        result["targets"] = {"gemm_w4a4": g, "quantize_pack": q, "gemm_decode": target_gemm_decode(dy, wl, device)}
         # the metric's two figures as roofline objects: the tensor-core kernel of the square GEMM against the int8
         # tensor peak, the quantize/pack kernel (scale given) against the copy bandwidth
         lib_int8 = here.get("int8_matmul_tops")

@@ -380,7 +380,7 @@ dybit_status dybit_selftest_wait_timeout(uint64_t limit_ns, uint32_t *result, vo
  * format pair and per device (filled on first use, atomically, every thread computing the same values), kernels
  * launched are counted in one atomic counter, and the device status word lives in the loaded module.  The two
  * dybit_profile_next_gemm* hooks below arm state that is PER HOST THREAD (the arming thread's next GEMM / conv call
- * consumes it); dybit_set_conv_lowering is a process-wide atomic setting. */
+ * consumes it); dybit_set_conv_lowering and dybit_set_gemm_decode are process-wide atomic settings. */
 
 /* Which lowering dybit_conv2d and its variants take for stride-1 convolutions (Section III-C.4 maps conv layers onto
  * the GEMM array; the lowerings differ only in how the activation tile reaches shared memory, never in results):
@@ -391,6 +391,16 @@ dybit_status dybit_selftest_wait_timeout(uint64_t limit_ns, uint32_t *result, vo
  *   2            never halo tiles.
  * Returns DYBIT_ERR_INVALID_ARG for any other value.  Takes effect for calls that start afterwards. */
 dybit_status dybit_set_conv_lowering(int mode);
+
+/* Where dybit_gemm decodes its B operand (the weights) when B is a 4-bit format in the int8 container and the output
+ * is plain fp32 (Section III-B.1-2: decoders beside the array feed it directly):
+ *   0  both operands are expanded into the workspace by a separate launch, the GEMM kernel reads those copies;
+ *   1  B stays packed and is decoded in the GEMM kernel's main loop (table lookup in registers into the shared-memory
+ *      operand tile) wherever that kernel applies;
+ *   2 (default)  by shape: in the main loop when A has at most 128 rows and B at least 32 Mi codes (the GEMM is then
+ *      bound by the one pass over the weights, which shrinks from 2.5 to 0.5 bytes per weight), expanded otherwise.
+ * Results are identical bit for bit in every mode.  Returns DYBIT_ERR_INVALID_ARG for any other value. */
+dybit_status dybit_set_gemm_decode(int mode);
 
 /* Number of kernels this library has launched in the calling process so far. */
 uint64_t dybit_launch_count(void);

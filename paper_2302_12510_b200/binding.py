@@ -20,7 +20,7 @@ __all__ = [
     "dybit_choose_container", "dybit_gemm_workspace_bytes", "dybit_conv2d_workspace_bytes",
     "dybit_conv2d_out_hw", "dybit_absmax_scale", "dybit_quantize_pack", "dybit_quantize_pack_2d",
     "dybit_decode", "dybit_gemm", "dybit_conv2d", "dybit_last_device_status",
-    "dybit_launch_count", "dybit_set_conv_lowering", "dybit_selftest_wait_timeout", "dybit_profile_next_gemm", "dybit_profile_next_gemm_clock", "dybit_gemm_static_ws", "STATIC_WS_BYTES",
+    "dybit_launch_count", "dybit_set_conv_lowering", "dybit_set_gemm_decode", "dybit_selftest_wait_timeout", "dybit_profile_next_gemm", "dybit_profile_next_gemm_clock", "dybit_gemm_static_ws", "STATIC_WS_BYTES",
     "dybit_gemm_requant", "dybit_conv2d_requant", "dybit_depthwise_conv2d", "dybit_gemm_batched",
     "dybit_quantize_conv2d", "dybit_quantize_conv2d_requant",
     "dybit_gemm_batched_workspace_bytes", "dybit_rmse", "dybit_rmse_sweep", "dybit_fake_quant", "dybit_fake_quant_backward",
@@ -96,6 +96,7 @@ def _load() -> C.CDLL:
     lib.dybit_launch_count.restype = C.c_uint64
     lib.dybit_launch_count.argtypes = []
     lib.dybit_set_conv_lowering.argtypes = [i32]
+    lib.dybit_set_gemm_decode.argtypes = [i32]
     lib.dybit_selftest_wait_timeout.argtypes = [C.c_uint64, vp, vp]
     lib.dybit_profile_next_gemm.argtypes = [vp, vp]
     lib.dybit_profile_next_gemm_clock.argtypes = [vp]
@@ -313,6 +314,11 @@ def dybit_selftest_wait_timeout(limit_ns: int, device=None) -> torch.Tensor:
     result = torch.zeros(2, dtype=torch.int32, device=device or torch.device("cuda", torch.cuda.current_device()))
     _check(lib.dybit_selftest_wait_timeout(int(limit_ns), result.data_ptr(), _stream(None)), "dybit_selftest_wait_timeout")
     return result
+
+
+def dybit_set_gemm_decode(mode: int) -> None:
+    """0: expand pass for both operands; 1: decode B in the GEMM's main loop wherever possible; 2: by shape (default)."""
+    _check(lib.dybit_set_gemm_decode(int(mode)), "dybit_set_gemm_decode")
 
 
 def dybit_set_conv_lowering(mode: int) -> None:

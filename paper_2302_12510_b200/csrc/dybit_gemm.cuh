@@ -1843,6 +1843,16 @@ static dybit_status launch_conv_halo(dybit_container cont, const dybit_conv_desc
                                      const uint8_t *xe, const uint8_t *we, int64_t wrb, const GemmParams &p_in,
                                      cudaStream_t s);
 
+// The GEMM that decodes its B operand in the main loop (dybit_gemm_bdec.cuh).
+struct BdecTable {
+    unsigned tab[4];          // the 16 table bytes of the 4-bit format, as expand4_lookup wants them
+    int neg_high;
+};
+static std::atomic<int> &gemm_decode_mode();
+static bool gemm_bdec_applicable(dybit_container cont, dybit_fmt fb, const ElemTable &tb, const GemmParams &p, BdecTable *bt);
+static dybit_status launch_gemm_bdec(const uint8_t *ae, int64_t rb, const uint8_t *B, int64_t ldb_bytes, int64_t M, int64_t N,
+                                     int64_t K, const GemmParams &p_in, const BdecTable &bt, cudaStream_t s);
+
 static dybit_status gemm_impl(int64_t M, int64_t N, int64_t K, const void *A, dybit_fmt fa, const float *scale_a,
                               int64_t lda_bytes, const void *B, dybit_fmt fb, const float *scale_b, int64_t ldb_bytes,
                               float *C, int64_t ldc, int32_t *C_raw, const RequantSpec *rq, void *ws, size_t ws_bytes,
@@ -1880,15 +1890,7 @@ static dybit_status gemm_impl(int64_t M, int64_t N, int64_t K, const void *A, dy
     const ElemTable &tb = make_elem_table(fb, plan.container, plan.exp_b);
     const ExpandOperand opa = {static_cast<const uint8_t *>(A), fa.bits, M, lda_bytes, kp, ae, rb, &ta};
     const ExpandOperand opb = {static_cast<const uint8_t *>(B), fb.bits, N, ldb_bytes, kp, be, rb, &tb};
-    st = launch_expand_pair(opa, opb, elem, plan.container == DYBIT_CONTAINER_I8, s);
-    if (st != DYBIT_OK) return st;
-
     const int bn = choose_bn(M, N);
-    CUtensorMap map_a, map_b;
-    st = make_operand_map(&map_a, ae, M, rb, rb, kBM);
-    if (st != DYBIT_OK) return st;
-    st = make_operand_map(&map_b, be, N, rb, rb, bn);
-    if (st != DYBIT_OK) return st;
     GemmParams p = {};
     p.M = (int)M;
     p.N = (int)N;
@@ -1902,6 +1904,33 @@ static dybit_status gemm_impl(int64_t M, int64_t N, int64_t K, const void *A, dy
     p.scale_b = scale_b;
     p.pow2 = ldexp(1.0, -(plan.exp_a + plan.exp_b));
     apply_requant(p, rq);
+    {
+        // few rows of A against a long stream of 4-bit weights: leave the weights packed and decode them in the main
+        // loop (0.5 byte of global traffic per weight instead of 2.5); only A goes through the expand pass
+        const int mode = gemm_decode_mode().load(std::memory_order_relaxed);
+        BdecTable bt_val = {};
+        BdecTable *bt = &bt_val;
+        if ((mode == 1 || (mode == 2 && M <= 128 && N * kp >= ((int64_t)1 << 25))) &&
+            gemm_bdec_applicable(plan.container, fb, tb, p, bt)) {
+            const ExpandOperand none = {static_cast<const uint8_t *>(B), fb.bits, 0, ldb_bytes, kp, be, rb, &tb};
+            st = launch_expand_pair(opa, none, elem, true, s);
+            if (st != DYBIT_OK) return st;
+            st = launch_gemm_bdec(ae, rb, static_cast<const uint8_t *>(B), ldb_bytes, M, N, K, p, *bt, s);
+            if (st != DYBIT_ERR_UNSUPPORTED) return st;
+            // (the output cannot be described to the TMA: expand B as well and take the general kernel)
+            const ExpandOperand only_b = {static_cast<const uint8_t *>(A), fa.bits, 0, lda_bytes, kp, ae, rb, &ta};
+            st = launch_expand_pair(only_b, opb, elem, true, s);
+            if (st != DYBIT_OK) return st;
+        } else {
+            st = launch_expand_pair(opa, opb, elem, plan.container == DYBIT_CONTAINER_I8, s);
+            if (st != DYBIT_OK) return st;
+        }
+    }
+    CUtensorMap map_a, map_b;
+    st = make_operand_map(&map_a, ae, M, rb, rb, kBM);
+    if (st != DYBIT_OK) return st;
+    st = make_operand_map(&map_b, be, N, rb, rb, bn);
+    if (st != DYBIT_OK) return st;
     if (gemm_pair_eligible(M, N, p)) {
         // large plain products: 256 x 256 tiles on pairs of SMs (falls through when C cannot be described to the TMA)
         st = launch_gemm_pair(plan.container, ae, rb, be, rb, M, N, p, s);

@@ -5,5 +5,6 @@
 #include "dybit_gemm.cuh"
 #include "dybit_gemm_pair.cuh"
 #include "dybit_conv_halo.cuh"
+#include "dybit_gemm_bdec.cuh"
 #include "dybit_static_ws.cuh"
 #include "dybit_depthwise.cuh"

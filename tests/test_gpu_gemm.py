@@ -202,3 +202,43 @@ def test_cta_pair_kernel(M, N, K, fa, fb):
         bmax = float(spb[0]) * float(np.abs(orc.decode_table(fb[0], bool(fb[1]))).max())
         err = np.abs(C.cpu().numpy().astype(np.float64) - C_ref.astype(np.float64)).max()
         assert err <= 1e-5 * K * amax * bmax, err
+
+
+# The B operand decoded in the GEMM's main loop (packed 4-bit weights -> int8 through the register table, written into
+# the swizzled operand tile by decode warps) instead of expanded by a separate launch: forced on for every shape here
+# (by default only few-row products take it), and compared with the oracle AND with the expand path, bit for bit.
+@pytest.mark.parametrize("M,N,K", [(1, 1, 1), (32, 1000, 512), (128, 256, 128), (129, 257, 129), (300, 520, 400),
+                                   (7, 4100, 2000), (256, 64, 4096), (1000, 130, 77), (513, 768, 1153)])
+@pytest.mark.parametrize("fa,fb", [((4, 0), (4, 1)), ((4, 1), (4, 0)), ((2, 1), (4, 1)), ((5, 1), (4, 1))])
+def test_weights_decoded_in_the_main_loop(M, N, K, fa, fb):
+    a = wl.normal((M, K), seed=M + K)
+    if not fa[1]:
+        a = a.abs()
+    b = wl.normal((N, K), seed=N + K + 1, std=0.3)
+    if not fb[1]:
+        b = b.abs()
+    pa, sa, ca, spa = quantize_operand(a, fa)
+    pb, sb, cb, spb = quantize_operand(b, fb)
+    S, C_ref = orc.gemm(ca, fa, spa[0], cb, fb, spb[0])
+    outs = []
+    try:
+        for mode in (1, 0):
+            dy.dybit_set_gemm_decode(mode)
+            launches = dy.dybit_launch_count()
+            C, C_raw = dy.dybit_gemm(M, N, K, pa, fa, sa, pb, fb, sb, want_raw=True)
+            torch.cuda.synchronize()
+            assert dy.dybit_last_device_status() == (0, 0)
+            # the tensor-core kernel + one expand launch (two when A and B need different expand kernels)
+            assert dy.dybit_launch_count() - launches <= 3
+            assert np.array_equal(C_raw.cpu().numpy().astype(np.int64), S), mode
+            assert np.array_equal(C.cpu().numpy(), C_ref), mode
+            outs.append(C)
+    finally:
+        dy.dybit_set_gemm_decode(2)
+    assert torch.equal(outs[0], outs[1])
+
+
+def test_gemm_decode_mode_argument():
+    with pytest.raises(dy.DybitError):
+        dy.dybit_set_gemm_decode(5)
+    dy.dybit_set_gemm_decode(2)
