@@ -47,7 +47,8 @@ FMT_A = (4, 0)      # post-ReLU activations: unsigned 4-bit
 NOMINAL = {"hbm_gbs": 7700.0, "bf16_tflops": 2250.0, "int8_tops": 4500.0, "fp8_tflops": 4500.0}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, copied from the ncu summaries under profiles/ (bench.py cannot
 # read hardware counters itself); an entry is None while the kernel has changed since its counters were taken
-NCU_TRAFFIC = {"gemm_8192": None, "quantize_2p26_per_element": None, "conv_step": None}
+NCU_TRAFFIC = {"gemm_8192": 4 * (36588800 + 18511872), "quantize_2p26_per_element": (268467968 + 7936512) / float(1 << 26),
+               "conv_step": None}
 NCU_TRAFFIC_HOW = {
     "gemm_8192": "profiles/dybit_gemm_pair_kernel_i8_square4096.txt: one launch at M=N=K=4096 (a capture small enough to end "
                  "by itself), x 4 for 8192^3 (operand and output bytes both grow 4 x)",
@@ -842,6 +843,8 @@ def main():
     ap.add_argument("--step-only", action="store_true",
                     help="only the step itself (graph replays, direct launches, end to end): no device-clock pass, no "
                          "re-quantizing or two-call variants, no targets, no CPU baseline (for profiler captures)")
+    ap.add_argument("--conv-layer", default="",
+                    help="run only this ResNet-18 layer (e.g. layer1.0.conv1) at --batch, a few calls (for profiler captures)")
     ap.add_argument("--targets-only", action="store_true",
                     help="run only the single-kernel target measurements (small cases for profiler captures)")
     ap.add_argument("--gemm-size", type=int, default=8192, help="M=N=K of the square 4-bit GEMM target")
@@ -879,6 +882,16 @@ def main():
     if args.sweeps:
         only = [t for t in args.only.split(",") if t] if args.only else None
         print(json.dumps({"sweeps": run_sweeps(dy, wl, device, peaks, only=only, log2n=args.sweep_log2n)}))
+        return
+    if args.conv_layer:
+        # one layer of the step alone (a small case for a profiler capture): a few dybit_quantize_conv2d calls
+        layers = [L for L in wl.resnet18_layers(args.batch) if L.name == args.conv_layer]
+        if not layers:
+            raise SystemExit(f"no layer named {args.conv_layer}; names: {[L.name for L in wl.resnet18_layers(1)]}")
+        work = LayerwiseStep(dy, wl, device, layers, [(FMT_W[0], FMT_A[0])], host_copies=False)
+        ms = time_calls(work.step, max(1, args.steps), warmup=warmup)
+        print(json.dumps({"conv_layer": args.conv_layer, "batch": args.batch, "us_per_call": ms * 1e3,
+                          "device_status": dy.dybit_last_device_status()}))
         return
     if args.targets_only:
         out = {}

@@ -1193,30 +1193,49 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             constexpr uint32_t kCFormat = (KIND == Kind::I8) ? 2u : 1u;           // s32 : f32
             constexpr uint32_t kABFormat = (KIND == Kind::F8F6F4) ? 0u : 1u;      // e4m3 : (s8 | bf16)
             constexpr uint32_t idesc = umma_idesc(kCFormat, kABFormat, kBM, BN);
-            uint32_t it = 0, lt = 0;
-            bool ok = true;
+            // One thread runs at roughly six clocks per instruction and an MMA of a narrow tile takes under 100, so
+            // the loop is kept to 32-bit adds (descriptors = constant high word + stepped low word, barriers by
+            // shared-memory address).  A barrier probed right after a tcgen05.commit answers only once the MMAs in
+            // flight have drained (about 200 clocks; about 45 between two MMAs): the NEXT stage's barrier is probed
+            // right after the first MMA of the current stage.  A wait that runs out raises the abort flag and the
+            // loop simply runs on (later waits then give up at once; the epilogue stores nothing more).
+            constexpr uint32_t kHi = umma_desc_hi<SWB>();
+            constexpr uint32_t kA16 = L::kAStage >> 4, kB16 = L::kBStage >> 4;
+            const uint32_t a_lo0 = umma_desc_lo(smem_u32(a_stages)), b_lo0 = umma_desc_lo(smem_u32(b_stages));
+            const uint32_t full0 = smem_u32(full), empty0 = smem_u32(empty);
+            const uint32_t acc_full0 = smem_u32(acc_full), acc_empty0 = smem_u32(acc_empty);
             const bool b_res = !CONV && p.b_resident != 0;
-            if (b_res && (int)blockIdx.x < total_tiles) ok = wait_bounded(b_full, 0u, abort_flag, 6);
-            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++lt) {
-                const uint32_t as = lt & 1u, aph = (lt >> 1) & 1u;
-                if (!wait_bounded(&acc_empty[as], aph ^ 1u, abort_flag, 2)) { ok = false; break; }
+            const int k_blocks = p.k_blocks;
+            int s = 0;
+            uint32_t ph = 0, lt = 0;
+            bool ready = false, acc_ready = false;
+            if (b_res && (int)blockIdx.x < total_tiles) (void)wait_bounded(b_full, 0u, abort_flag, 6);
+            for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++lt) {
+                const uint32_t as = lt & 1u;
+                if (!acc_ready) (void)wait_bounded_addr(acc_empty0 + as * 8, ((lt >> 1) & 1u) ^ 1u, abort_flag, 2);
+                acc_ready = false;
                 tc_fence_after_sync();
                 const uint32_t d = tmem_base + as * BN;
-                for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
-                    const int s = it % kStages;
-                    const uint32_t ph = (it / kStages) & 1u;
-                    if (!wait_bounded(&full[s], ph, abort_flag, 3)) { ok = false; break; }
+                for (int kb = 0; kb < k_blocks; ++kb) {
+                    if (!ready) (void)wait_bounded_addr(full0 + s * 8, ph, abort_flag, 3);
                     tc_fence_after_sync();
-                    const uint64_t adesc = umma_desc_kmajor<SWB>(smem_u32(a_stages + s * L::kAStage));
-                    const uint64_t bdesc = umma_desc_kmajor<SWB>(smem_u32(b_stages + (b_res ? kb : s) * L::kBStage));
+                    int sn = s + 1;
+                    uint32_t phn = ph;
+                    if (sn == kStages) { sn = 0; phn ^= 1u; }
+                    const uint32_t a_lo = a_lo0 + s * kA16;
+                    const uint32_t b_lo = b_lo0 + (b_res ? kb : s) * kB16;
+                    umma_lo<KIND>(d, a_lo, b_lo, kHi, idesc, (uint32_t)(kb != 0));
+                    ready = mbar_try_wait_addr(full0 + sn * 8, phn);
+                    if (kb == k_blocks - 1)
+                        acc_ready = mbar_try_wait_addr(acc_empty0 + (as ^ 1u) * 8, (((lt + 1) >> 1) & 1u) ^ 1u);
 #pragma unroll
-                    for (int k = 0; k < SWB / kUmmaKBytes; ++k) {
-                        umma<KIND>(d, adesc + (uint64_t)(k * (kUmmaKBytes >> 4)), bdesc + (uint64_t)(k * (kUmmaKBytes >> 4)),
-                                   idesc, (uint32_t)((kb | k) != 0));
-                    }
-                    umma_commit(&empty[s]);
+                    for (int k = 1; k < SWB / kUmmaKBytes; ++k)
+                        umma_lo<KIND>(d, a_lo + k * (kUmmaKBytes >> 4), b_lo + k * (kUmmaKBytes >> 4), kHi, idesc, 1u);
+                    umma_commit_addr(empty0 + s * 8);
+                    s = sn;
+                    ph = phn;
                 }
-                if (ok) umma_commit(&acc_full[as]);
+                umma_commit_addr(acc_full0 + as * 8);
             }
         }
     } else if (warp < 2 + kEpilogueWarps) {
@@ -1237,7 +1256,8 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             const uint32_t as = lt & 1u, aph = (lt >> 1) & 1u;
             // The four warps of a group meet in named barriers below, so they must leave this loop together: the
             // outcome of the wait is AND-reduced over the group's 128 threads (every warp gets here in bounded time).
-            const bool ok = named_barrier_and(1 + group, 128, wait_bounded(&acc_full[as], aph, abort_flag, 4));
+            // (one thread per group polls; the others sleep in the hardware barrier that hands them the outcome)
+            const bool ok = named_barrier_and(1 + group, 128, issuer ? wait_bounded(&acc_full[as], aph, abort_flag, 4) : true);
             if (!ok) break;
             tc_fence_after_sync();
             // batched: the tile belongs to entry `bat`, rows count inside that entry
