@@ -26,7 +26,7 @@ namespace dybit {
 
 using namespace sm100;
 
-constexpr int kHaloMaxR = 3;                          // filter rows the A stage is sized for
+constexpr int kHaloMaxR = 4;                          // filter rows the A stage is sized for
 constexpr int kHaloRows = (16 + kHaloMaxR - 1) * 8;   // pixel rows x 8 columns = shared-memory rows of one A stage
 constexpr int kHaloMaxA = 8, kHaloMaxB = 18;          // ring depths the barrier block is sized for (B: slots)
 constexpr int kHaloMaxG = 8;                          // B slots are released in groups of R (one per A stage)
@@ -39,6 +39,8 @@ struct HaloParams {
     int th, hb, ni;          // output rows per image in a tile, th + R - 1, images per tile
     int trows, tcols;        // tiles per image column / row
     int cbs;                 // SWB-byte channel blocks per pixel
+    int pad_h, pad_w;        // window origin of output pixel (oh, ow): input row oh - pad_h, column ow - pad_w
+    int force;               // 1: the caller's workspace layout admits no other lowering (space-to-depth stem)
     int na, nb;              // ring depths: A stages; B slots = whole groups of R (one group per A stage)
     int b_res;               // 1: the whole weight panel (R*S*cbs blocks) is loaded once per CTA
     int m_tiles, n_tiles;
@@ -164,7 +166,7 @@ dybit_conv_halo_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
                     for (int fs = 0; fs < p.S && ok; ++fs) {
                         if (!wait_bounded(&a_empty[sa], pa, abort_flag, 1)) { ok = false; break; }
                         mbar_arrive_expect_tx(&a_full[sa], a_bytes);
-                        tma_load_4d(a_stages + sa * kAStage, &tmap_x, cb * SWB, t.ow0 - p.pad + fs, t.oh0 - p.pad, t.img0,
+                        tma_load_4d(a_stages + sa * kAStage, &tmap_x, cb * SWB, t.ow0 - hp.pad_w + fs, t.oh0 - hp.pad_h, t.img0,
                                     &a_full[sa]);
                         if (++sa == hp.na) { sa = 0; pa ^= 1u; }
                         if (hp.b_res) continue;
@@ -328,6 +330,23 @@ dybit_conv_halo_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
                             if (col0 + j < p.N) rrow[j] = (int)r[j];
                     }
                 }
+                if (!p.tma_store) {
+                    // the output cannot be described to the TMA (base or rows not 16-byte aligned): each thread writes
+                    // the 32 values of its own output pixel
+                    if (row >= 0) {
+                        float *dst = p.C + (int64_t)row * p.ldc + col0;
+                        if (col0 + 32 <= p.N && (reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
+#pragma unroll
+                            for (int j = 0; j < 8; ++j)
+                                __stcs(reinterpret_cast<float4 *>(dst) + j, make_float4(f[4 * j], f[4 * j + 1], f[4 * j + 2], f[4 * j + 3]));
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (col0 + j < p.N) dst[j] = f[j];
+                        }
+                    }
+                    continue;
+                }
                 // stage 128 rows x 32 columns in the TMA's 128-byte swizzle; one 4-D store per image of the tile writes
                 // the th x 8 pixels of that image and clips what lies outside the feature map
                 uint8_t *stage = c_stages + group * kHaloCStage;
@@ -377,6 +396,21 @@ static std::atomic<int> &conv_lowering_mode() {
     return mode;
 }
 
+// Tiles for a stride-1 window walk over `rows_r` filter rows: th output rows per image so that ni * (th + rows_r - 1)
+// pixel rows fit the A stage.
+static void halo_tiling(HaloPlan *h, int n, int oh, int ow, int rows_r) {
+    const int htiles = (oh + 15) / 16;
+    h->th = (oh + htiles - 1) / htiles;
+    h->hb = h->th + rows_r - 1;
+    h->ni = (16 + rows_r - 1) / h->hb;
+    if (h->ni < 1) h->ni = 1;
+    if (h->ni > n) h->ni = n;
+    h->trows = htiles;
+    h->tcols = (ow + 7) / 8;
+    const int64_t m_tiles = (int64_t)((n + h->ni - 1) / h->ni) * h->trows * h->tcols;
+    h->m_tiles = m_tiles > (1 << 24) ? 0 : (int)m_tiles;
+}
+
 static HaloPlan plan_halo(const dybit_conv_desc *d, int oh, int ow, int64_t cpb) {
     HaloPlan h = {};
     if (conv_lowering_mode().load(std::memory_order_relaxed) == 2) return h;
@@ -384,17 +418,8 @@ static HaloPlan plan_halo(const dybit_conv_desc *d, int oh, int ow, int64_t cpb)
     if (swb == 0 || d->stride != 1 || d->dilation != 1 || d->r > kHaloMaxR || d->s > 16) return h;
     if (d->r == 1 && d->s == 1) return h;                       // a plain GEMM on the activation: the tiled kernel
     if (cpb / swb > 64 || d->pad > 64) return h;
-    const int htiles = (oh + 15) / 16;
-    h.th = (oh + htiles - 1) / htiles;
-    h.hb = h.th + d->r - 1;
-    h.ni = (16 + d->r - 1) / h.hb;
-    if (h.ni < 1) h.ni = 1;
-    if (h.ni > d->n) h.ni = d->n;
-    h.trows = htiles;
-    h.tcols = (ow + 7) / 8;
-    const int64_t m_tiles = (int64_t)((d->n + h.ni - 1) / h.ni) * h.trows * h.tcols;
-    if (m_tiles > (1 << 24)) return h;
-    h.m_tiles = (int)m_tiles;
+    halo_tiling(&h, d->n, oh, ow, d->r);
+    if (h.m_tiles == 0) return h;
     h.swb = swb;
     h.cbs = (int)(cpb / swb);
     h.eligible = true;
@@ -465,7 +490,7 @@ static dybit_status launch_halo_inst(const CUtensorMap &tx, const CUtensorMap &t
     // the im2col lowering (12.2 against 17.0 us on the 64 -> 64 channel 3x3 layers); with one CTA per SM and a
     // weight ring they do not (10.5 against 9.0 us at 128 channels, 15.2 against 13.0 us at 512): there the single
     // MMA-issuing thread, not the operand traffic, sets the pace, and the plainer loop of dybit_gemm_kernel wins.
-    if (per_sm != 2 && conv_lowering_mode().load(std::memory_order_relaxed) != 1) return DYBIT_ERR_UNSUPPORTED;
+    if (per_sm != 2 && !hp.force && conv_lowering_mode().load(std::memory_order_relaxed) != 1) return DYBIT_ERR_UNSUPPORTED;
     const int smem = 1024 + 2 * kHaloCStage + (hp.b_res ? panel : hp.nb * kBStage) + hp.na * kAStage + 1024;
     auto kern = dybit_conv_halo_kernel<KIND, BN, SWB>;
     static std::atomic<bool> configured[64];
@@ -538,9 +563,64 @@ static dybit_status launch_conv_halo(dybit_container cont, const dybit_conv_desc
     hp.trows = h.trows;
     hp.tcols = h.tcols;
     hp.cbs = h.cbs;
+    hp.pad_h = d->pad;
+    hp.pad_w = d->pad;
     hp.m_tiles = h.m_tiles;
     hp.n_tiles = (d->k + bn - 1) / bn;
     return h.swb == 128 ? launch_halo_kind<128>(cont, bn, tx, tw, ty, hp, s) : launch_halo_kind<64>(cont, bn, tx, tw, ty, hp, s);
+}
+
+// Stride-2 convolution on at most four one-byte channels (the 3-channel 7 x 7 stem) after a 2 x 2 space-to-depth
+// rearrangement of the activation (plan_conv, kConvS2D): every 2 x 2 block of input pixels is one 16-byte pixel, the
+// filter becomes Rp x 4 taps walked with stride 1, and the four taps of one filter row are 64 CONTIGUOUS bytes of the
+// rearranged image.  The input map therefore has rows that overlap: row w of it is the 64-byte window that starts at
+// rearranged pixel w (16 bytes further on than row w - 1).  One TMA load brings the windows of th + Rp - 1 rows x 8
+// columns; filter row r' is a 64-byte K block of its own, read from pixel row g + r' of that tile.  The image carries
+// its horizontal padding physically (padL zero pixels in front of every row, three behind), since a window that
+// starts inside the image must not be zero-filled as a whole; rows above and below the image are the TMA's zero fill.
+static dybit_status launch_conv_s2d(dybit_container cont, const dybit_conv_desc *d, int oh, int ow, const S2dGeom &g,
+                                    const uint8_t *xs, const uint8_t *we, int64_t wrb, const GemmParams &p_in,
+                                    cudaStream_t s) {
+    HaloPlan h = {};
+    halo_tiling(&h, d->n, oh, ow, g.Rp);
+    if (h.m_tiles == 0) return DYBIT_ERR_UNSUPPORTED;
+    h.swb = 64;
+    h.cbs = 1;
+    HaloParams hp = {};
+    hp.g = p_in;
+    hp.g.R = g.Rp;
+    hp.g.S = 1;
+    CUtensorMap tx, tw, ty;
+    memset(&ty, 0, sizeof(ty));
+    hp.g.tma_store = (hp.g.Q == nullptr && make_halo_output_map(&ty, hp.g.C, d, oh, ow, h)) ? 1 : 0;
+    {
+        EncodeTiledFn fn = encode_tiled_fn();
+        if (fn == nullptr) return DYBIT_ERR_CUDA;
+        cuuint64_t dims[4] = {64, (cuuint64_t)(g.P - 3), (cuuint64_t)g.Hs, (cuuint64_t)d->n};
+        cuuint64_t strides[3] = {16, (cuuint64_t)g.P * 16, (cuuint64_t)g.P * 16 * g.Hs};
+        cuuint32_t box[4] = {64, 8, (cuuint32_t)h.hb, (cuuint32_t)h.ni};
+        cuuint32_t estr[4] = {1, 1, 1, 1};
+        if (fn(&tx, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<uint8_t *>(xs), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return DYBIT_ERR_CUDA;
+    }
+    const int bn = choose_bn_tiles(h.m_tiles, d->k);
+    dybit_status st = make_operand_map(&tw, we, d->k, wrb, wrb, bn, 64);
+    if (st != DYBIT_OK) return st;
+    hp.n_img = d->n;
+    hp.th = h.th;
+    hp.hb = h.hb;
+    hp.ni = h.ni;
+    hp.trows = h.trows;
+    hp.tcols = h.tcols;
+    hp.cbs = 1;
+    hp.pad_h = -g.lo_r;
+    hp.pad_w = 0;                       // the left padding is in the image: window of output column ow starts at pixel ow
+    hp.force = 1;
+    hp.m_tiles = h.m_tiles;
+    hp.n_tiles = (d->k + bn - 1) / bn;
+    return launch_halo_kind<64>(cont, bn, tx, tw, ty, hp, s);
 }
 
 }  // namespace dybit

@@ -245,7 +245,61 @@ struct FusedWeights {
     int use4;                 // 1: job4 describes the same rows for the 4-bit register-table expansion
     Expand4Job job4;
     int pix_c, pix_r, pix_s;  // pix_c > 0: filter rows of 8 taps x 4 bytes instead (see expand_weights_pix4)
+    int s2d;                  // 1 (with pix_c/r/s set): space-to-depth filter layout instead (see expand_weights_s2d)
+    int s2d_lo_r, s2d_lo_s, s2d_pad, s2d_rp;
 };
+
+// Geometry of the 2 x 2 space-to-depth rearrangement of a stride-2 convolution's input (ConvMode kConvS2D).
+// Rearranged pixel (hh, ww) holds input pixels (2hh + dy, 2ww + dx), dy, dx in {0, 1}, C bytes each at byte
+// (2dy + dx) * C; input row 2*oh - pad + r lies in rearranged row oh + lo_r + r' with r' = floor((r - pad) / 2) - lo_r.
+struct S2dGeom {
+    int Hs, Ws;               // rearranged image: H / 2 x W / 2 pixels of 16 bytes
+    int P;                    // pixels per stored row: padL zero pixels, Ws pixels, 3 zero pixels
+    int padL;                 // = -lo_s
+    int lo_r, lo_s;           // first rearranged row / column of a window, relative to the output pixel
+    int Rp, Sp;               // rearranged filter rows / columns (both <= 4)
+};
+
+// Where quantize_expand_kernel / expand_pix4_kernel put the container bytes of a pixel with <= 4 one-byte channels:
+// one 32-bit word per pixel in NHW order (s2d = 0), or the space-to-depth image (s2d = 1).
+struct PixLayout {
+    int c;                    // channels per pixel; 0: not a few-channel layout at all
+    int s2d;
+    int H, W, Hs, P, padL;
+};
+
+// Space-to-depth image: where the channel bytes of input pixel `px` (NHW index) go.
+__device__ __forceinline__ uint8_t *s2d_pixel_addr(uint8_t *xs, const PixLayout &pl, int64_t px) {
+    const int64_t img = px / ((int64_t)pl.H * pl.W);
+    const int rem = (int)(px - img * pl.H * pl.W);
+    const int h = rem / pl.W, w = rem - h * pl.W;
+    return xs + ((((img * pl.Hs + (h >> 1)) * pl.P + (w >> 1) + pl.padL) << 4) + ((h & 1) * 2 + (w & 1)) * pl.c);
+}
+
+// The zero bytes pixel `px` is responsible for: the unused tail of its 16-byte block (the block's last pixel writes
+// it) and the padding pixels of its stored row (the first and last pixel of every even input row write them).
+__device__ __forceinline__ void s2d_pixel_duties(uint8_t *xs, const PixLayout &pl, int64_t px) {
+    const int64_t img = px / ((int64_t)pl.H * pl.W);
+    const int rem = (int)(px - img * pl.H * pl.W);
+    const int h = rem / pl.W, w = rem - h * pl.W;
+    uint8_t *row = xs + (((img * pl.Hs + (h >> 1)) * pl.P) << 4);
+    if ((h & 1) && (w & 1)) {
+        uint8_t *blk = row + (((w >> 1) + pl.padL) << 4);
+        for (int b = 4 * pl.c; b < 16; ++b) blk[b] = 0;
+    }
+    if (!(h & 1)) {
+        if (w == 0)
+            for (int i = 0; i < pl.padL; ++i) reinterpret_cast<uint4 *>(row)[i] = make_uint4(0, 0, 0, 0);
+        if (w == pl.W - 1)
+            for (int i = 0; i < 3; ++i) reinterpret_cast<uint4 *>(row)[pl.padL + (pl.W >> 1) + i] = make_uint4(0, 0, 0, 0);
+    }
+}
+
+__device__ __forceinline__ void s2d_store_pixel(uint8_t *xs, const PixLayout &pl, int64_t px, unsigned word) {
+    uint8_t *dst = s2d_pixel_addr(xs, pl, px);
+    for (int b = 0; b < pl.c; ++b) dst[b] = (uint8_t)(word >> (8 * b));
+    s2d_pixel_duties(xs, pl, px);
+}
 
 // The activation's own 16-entry table for the register-table expansion of 4-bit codes (see expand4_lookup); use = 0
 // keeps the shared-memory table.
@@ -279,6 +333,37 @@ __device__ __forceinline__ void expand_weights_pix4(const FusedWeights &wj, cons
     *reinterpret_cast<uint4 *>(wj.out + row * wj.out_stride + g * 16) = make_uint4(o[0], o[1], o[2], o[3]);
 }
 
+// Weights for the space-to-depth lowering (ConvMode kConvS2D): row n of the output holds, for each rearranged filter
+// row r', four rearranged taps s' of 16 bytes; byte (2dy + dx) * C + c of tap (r', s') is the weight of the original
+// tap r = 2 (r' + lo_r) + dy + pad, s = 2 (s' + lo_s) + dx + pad, channel c, or zero when that tap does not exist.
+// Thread `idx` writes one 16-byte chunk (one rearranged tap); chunks past the last filter row are zero.
+__device__ __forceinline__ void expand_weights_s2d(const FusedWeights &wj, const uint16_t *s_lut, int64_t idx) {
+    const int64_t chunks_per_row = wj.out_stride / 16;
+    const int64_t row = idx / chunks_per_row;
+    const int g = (int)(idx - row * chunks_per_row);
+    const int rp = g >> 2, sp = g & 3;
+    const uint8_t *src = wj.packed + row * wj.in_stride;
+    const unsigned mask = (1u << wj.bits) - 1u;
+    unsigned o[4] = {0, 0, 0, 0};
+    if (rp < wj.s2d_rp) {
+        for (int dy = 0; dy < 2; ++dy) {
+            for (int dx = 0; dx < 2; ++dx) {
+                const int r = 2 * (rp + wj.s2d_lo_r) + dy + wj.s2d_pad, s = 2 * (sp + wj.s2d_lo_s) + dx + wj.s2d_pad;
+                if (r < 0 || r >= wj.pix_r || s < 0 || s >= wj.pix_s) continue;
+                for (int c = 0; c < wj.pix_c; ++c) {
+                    const int64_t bit = (int64_t)((r * wj.pix_s + s) * wj.pix_c + c) * wj.bits;
+                    const int sh = (int)(bit & 7);
+                    unsigned two = __ldg(src + (bit >> 3));
+                    if (sh + wj.bits > 8) two |= (unsigned)__ldg(src + (bit >> 3) + 1) << 8;
+                    const int byte = (dy * 2 + dx) * wj.pix_c + c;
+                    o[byte >> 2] |= (unsigned)(s_lut[(two >> sh) & mask] & 0xffu) << (8 * (byte & 3));
+                }
+            }
+        }
+    }
+    *reinterpret_cast<uint4 *>(wj.out + row * wj.out_stride + g * 16) = make_uint4(o[0], o[1], o[2], o[3]);
+}
+
 // fp32 activation -> packed codes AND their container elements, plus the layer's weights expanded by the
 // last blocks of the same grid: what dybit_quantize_pack followed by the expand launch of dybit_conv2d
 // compute, in one launch instead of two.  The activation is one flat run of n elements whose expanded
@@ -292,7 +377,8 @@ quantize_expand_kernel(const float *__restrict__ x, int64_t n, const float *__re
                        uint8_t *__restrict__ packed, int64_t packed_bytes, uint8_t *__restrict__ xe, int64_t xe_bytes,
                        const __grid_constant__ ElemTable tx, const FusedWeights wj, const __grid_constant__ ElemTable tw,
                        int x_blocks, const unsigned *__restrict__ partials, int n_partials, int m, float *__restrict__ scale_out,
-                       int pix_c, const XTab4 xt) {
+                       const PixLayout pl, const XTab4 xt) {
+    const int pix_c = pl.c;
     __shared__ __align__(16) unsigned s_codes[kWarpsPerBlock][kChunkCodes / 4];
     __shared__ __align__(16) unsigned s_words[kWarpsPerBlock][32 * BITS];
     __shared__ uint16_t s_lut[256];
@@ -335,8 +421,10 @@ quantize_expand_kernel(const float *__restrict__ x, int64_t n, const float *__re
         if (wj.pix_c > 0) {
             const int64_t total = wj.rows * (wj.out_stride / 16);
             for (int64_t idx = (int64_t)(blockIdx.x - x_blocks) * blockDim.x + threadIdx.x; idx < total;
-                 idx += (int64_t)(gridDim.x - x_blocks) * blockDim.x)
-                expand_weights_pix4(wj, s_lut, idx);
+                 idx += (int64_t)(gridDim.x - x_blocks) * blockDim.x) {
+                if (wj.s2d) expand_weights_s2d(wj, s_lut, idx);
+                else expand_weights_pix4(wj, s_lut, idx);
+            }
             return;
         }
         if (wj.use4) {
@@ -448,18 +536,31 @@ quantize_expand_kernel(const float *__restrict__ x, int64_t n, const float *__re
                         unsigned w = sb[o0];
                         if (pix_c > 1) w |= (unsigned)sb[o0 + 1] << 8;
                         if (pix_c > 2) w |= (unsigned)sb[o0 + 2] << 16;
-                        x4[px] = w;
+                        if (pix_c > 3) w |= (unsigned)sb[o0 + 3] << 24;
+                        if (pl.s2d) s2d_store_pixel(xe, pl, px, w);
+                        else x4[px] = w;
                     }
                     if (lane == 0 && p_lo * pix_c > c0 && c0 < e_end) {
                         // tail of the pixel that began in the previous chunk
                         const int64_t px = p_lo - 1;
-                        for (int64_t e = c0; e < min(p_lo * pix_c, e_end); ++e) xe[px * 4 + (e - px * pix_c)] = sb[e - c0];
+                        if (pl.s2d) {
+                            uint8_t *dst = s2d_pixel_addr(xe, pl, px);
+                            for (int64_t e = c0; e < min(p_lo * pix_c, e_end); ++e) dst[e - px * pix_c] = sb[e - c0];
+                            if (p_lo * pix_c <= e_end) s2d_pixel_duties(xe, pl, px);      // the pixel ends in this chunk
+                        } else {
+                            for (int64_t e = c0; e < min(p_lo * pix_c, e_end); ++e) xe[px * 4 + (e - px * pix_c)] = sb[e - c0];
+                        }
                     }
                     if (lane == 1 && p_hi * pix_c < e_end && p_hi >= p_lo) {
                         // head of the pixel that ends in the next chunk, and its padding bytes
                         const int64_t px = p_hi;
-                        for (int64_t e = px * pix_c; e < e_end; ++e) xe[px * 4 + (e - px * pix_c)] = sb[e - c0];
-                        for (int b = pix_c; b < 4; ++b) xe[px * 4 + b] = 0;
+                        if (pl.s2d) {
+                            uint8_t *dst = s2d_pixel_addr(xe, pl, px);
+                            for (int64_t e = px * pix_c; e < e_end; ++e) dst[e - px * pix_c] = sb[e - c0];
+                        } else {
+                            for (int64_t e = px * pix_c; e < e_end; ++e) xe[px * 4 + (e - px * pix_c)] = sb[e - c0];
+                            for (int b = pix_c; b < 4; ++b) xe[px * 4 + b] = 0;
+                        }
                     }
                 } else {
                 if (off + 16 <= xe_bytes) reinterpret_cast<uint4 *>(xe + off)[0] = make_uint4(o[0], o[1], o[2], o[3]);
@@ -503,7 +604,7 @@ template <int BITS, int ELEM>
 static dybit_status launch_quantize_expand_bits(const float *x, int64_t n, bool is_signed, const float *scale, uint8_t *packed,
                                                 int64_t packed_bytes, uint8_t *xe, int64_t xe_bytes, const ElemTable &tx,
                                                 const FusedWeights &wj, const ElemTable &tw, const unsigned *partials,
-                                                int n_partials, float *scale_out, int pix_c, const XTab4 &xt, cudaStream_t s) {
+                                                int n_partials, float *scale_out, const PixLayout &pl, const XTab4 &xt, cudaStream_t s) {
     const int m = is_signed ? BITS - 1 : BITS;
     constexpr int kChunkBytes = kChunkCodes * BITS / 8;
     // one wave: three blocks fit an SM, the weights' blocks (a few 16-byte chunks per thread) take their share of
@@ -520,10 +621,10 @@ static dybit_status launch_quantize_expand_bits(const float *x, int64_t n, bool 
     const unsigned grid = (unsigned)(x_blocks + w_blocks);
     if (is_signed)
         launch_k(quantize_expand_kernel<BITS, true, ELEM>, dim3(grid), dim3((unsigned)kStreamThreads), (size_t)0, s, x, n, scale, packed,
-                 packed_bytes, xe, xe_bytes, tx, wj, tw, x_blocks, partials, n_partials, m, scale_out, pix_c, xt);
+                 packed_bytes, xe, xe_bytes, tx, wj, tw, x_blocks, partials, n_partials, m, scale_out, pl, xt);
     else
         launch_k(quantize_expand_kernel<BITS, false, ELEM>, dim3(grid), dim3((unsigned)kStreamThreads), (size_t)0, s, x, n, scale, packed,
-                 packed_bytes, xe, xe_bytes, tx, wj, tw, x_blocks, partials, n_partials, m, scale_out, pix_c, xt);
+                 packed_bytes, xe, xe_bytes, tx, wj, tw, x_blocks, partials, n_partials, m, scale_out, pl, xt);
     return launch_status();
 }
 
@@ -531,16 +632,16 @@ template <int ELEM>
 static dybit_status launch_quantize_expand(const float *x, int64_t n, dybit_fmt fx, const float *scale, uint8_t *packed,
                                            int64_t packed_bytes, uint8_t *xe, int64_t xe_bytes, const ElemTable &tx,
                                            const FusedWeights &wj, const ElemTable &tw, const unsigned *partials,
-                                           int n_partials, float *scale_out, int pix_c, const XTab4 &xt, cudaStream_t s) {
+                                           int n_partials, float *scale_out, const PixLayout &pl, const XTab4 &xt, cudaStream_t s) {
     const bool sg = fx.is_signed != 0;
     switch (fx.bits) {
-        case 2: return launch_quantize_expand_bits<2, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pix_c, xt, s);
-        case 3: return launch_quantize_expand_bits<3, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pix_c, xt, s);
-        case 4: return launch_quantize_expand_bits<4, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pix_c, xt, s);
-        case 5: return launch_quantize_expand_bits<5, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pix_c, xt, s);
-        case 6: return launch_quantize_expand_bits<6, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pix_c, xt, s);
-        case 7: return launch_quantize_expand_bits<7, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pix_c, xt, s);
-        case 8: return launch_quantize_expand_bits<8, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pix_c, xt, s);
+        case 2: return launch_quantize_expand_bits<2, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pl, xt, s);
+        case 3: return launch_quantize_expand_bits<3, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pl, xt, s);
+        case 4: return launch_quantize_expand_bits<4, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pl, xt, s);
+        case 5: return launch_quantize_expand_bits<5, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pl, xt, s);
+        case 6: return launch_quantize_expand_bits<6, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pl, xt, s);
+        case 7: return launch_quantize_expand_bits<7, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pl, xt, s);
+        case 8: return launch_quantize_expand_bits<8, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pl, xt, s);
     }
     return DYBIT_ERR_INVALID_ARG;
 }
@@ -788,7 +889,7 @@ patch_gather_kernel(const PatchGatherParams p) {
 __global__ void __launch_bounds__(256)
 expand_pix4_kernel(const uint8_t *__restrict__ packed, int bits, int64_t pixels, int c, unsigned *__restrict__ x4,
                    const __grid_constant__ ElemTable tx, const FusedWeights wj, const __grid_constant__ ElemTable tw,
-                   int x_blocks) {
+                   int x_blocks, const PixLayout pl) {
     __shared__ uint16_t s_lut[256];
     const bool weights = (int)blockIdx.x >= x_blocks;
     for (int i = threadIdx.x; i < 256; i += blockDim.x) s_lut[i] = weights ? tw.v[i] : tx.v[i];
@@ -797,8 +898,10 @@ expand_pix4_kernel(const uint8_t *__restrict__ packed, int bits, int64_t pixels,
     if (weights) {
         const int64_t total = wj.rows * (wj.out_stride / 16);
         for (int64_t idx = (int64_t)(blockIdx.x - x_blocks) * blockDim.x + threadIdx.x; idx < total;
-             idx += (int64_t)(gridDim.x - x_blocks) * blockDim.x)
-            expand_weights_pix4(wj, s_lut, idx);
+             idx += (int64_t)(gridDim.x - x_blocks) * blockDim.x) {
+            if (wj.s2d) expand_weights_s2d(wj, s_lut, idx);
+            else expand_weights_pix4(wj, s_lut, idx);
+        }
         return;
     }
     const unsigned mask = (1u << bits) - 1u;
@@ -811,7 +914,8 @@ expand_pix4_kernel(const uint8_t *__restrict__ packed, int bits, int64_t pixels,
             if (sh + bits > 8) two |= (unsigned)__ldg(packed + (bit >> 3) + 1) << 8;
             w |= (unsigned)(s_lut[(two >> sh) & mask] & 0xffu) << (8 * ch);
         }
-        x4[px] = w;
+        if (pl.s2d) s2d_store_pixel(reinterpret_cast<uint8_t *>(x4), pl, px, w);
+        else x4[px] = w;
     }
 }
 
@@ -1762,7 +1866,7 @@ static void apply_requant(GemmParams &p, const RequantSpec *rq) {
 }
 
 // How a convolution is lowered, and what it needs in the workspace.
-enum ConvMode { kConvPointwise, kConvIm2col, kConvPix4, kConvPatch, kConvGather };
+enum ConvMode { kConvPointwise, kConvIm2col, kConvPix4, kConvPatch, kConvGather, kConvS2D };
 struct ConvPlan {
     ConvMode mode;
     int elem, swb;
@@ -1772,6 +1876,7 @@ struct ConvPlan {
     int64_t wrb;                   // bytes per expanded weight row
     bool pad_channels;             // expanded activation / weights carry zero channels c..cp-1
     int64_t xd_bytes;              // patch mode, dilation 1: dense container elements of the activation (third region)
+    S2dGeom s2d;                   // kConvS2D
 };
 
 static ConvPlan plan_conv(const dybit_conv_desc *d, int oh, int ow, int elem) {
@@ -1793,12 +1898,33 @@ static ConvPlan plan_conv(const dybit_conv_desc *d, int oh, int ow, int elem) {
     // at most four one-byte channels (the 3-channel stem): pixels become 32-bit words and the tensor-core kernel
     // gathers its A tile from them, four filter rows of eight taps per K block; no patch matrix is written
     const bool pix4_ok = elem == 1 && d->c <= 4 && d->dilation == 1 && d->s <= 8 && d->r <= 64;
+    // stride 2 on at most four one-byte channels, even image sides, filter no wider than four rearranged taps (the
+    // 3-channel 7 x 7 stem): 2 x 2 space-to-depth image + halo tiles (launch_conv_s2d)
+    auto floordiv2 = [](int v) { return v >= 0 ? v / 2 : -((-v + 1) / 2); };
+    S2dGeom g = {};
+    g.lo_r = floordiv2(-d->pad);
+    g.lo_s = g.lo_r;
+    g.Rp = floordiv2(d->r - 1 - d->pad) - g.lo_r + 1;
+    g.Sp = floordiv2(d->s - 1 - d->pad) - g.lo_s + 1;
+    g.Hs = d->h / 2;
+    g.Ws = d->w / 2;
+    g.padL = -g.lo_s;
+    g.P = g.padL + g.Ws + 3;
+    const bool s2d_ok = elem == 1 && d->c <= 4 && d->stride == 2 && d->dilation == 1 && d->h % 2 == 0 && d->w % 2 == 0 &&
+                        g.Rp >= 1 && g.Rp <= 4 && g.Sp >= 1 && g.Sp <= 4 && g.padL >= 0 && g.padL <= 2 && ow <= g.Ws + 1 &&
+                        (int64_t)d->n * g.Hs * g.P * 16 < ((int64_t)1 << 40);
     if (pointwise) c.mode = kConvPointwise;
     else if (im2col_ok) c.mode = kConvIm2col;
+    else if (s2d_ok) c.mode = kConvS2D;
     else if (pix4_ok) c.mode = kConvPix4;
     else if (krow <= 1024 && M * krow <= ((int64_t)1 << 32)) c.mode = kConvPatch;
     else c.mode = kConvGather;
-    if (c.mode == kConvPix4) {
+    if (c.mode == kConvS2D) {
+        c.s2d = g;
+        c.a_bytes = round_up((int64_t)d->n * g.Hs * g.P * 16, 1024) + 1024;
+        c.wrb = round_up((int64_t)g.Rp * 64, kBKBytes);
+        c.pad_channels = false;
+    } else if (c.mode == kConvPix4) {
         c.a_bytes = round_up(c.pixels * 4, 1024) + 1024;
         c.wrb = round_up((int64_t)d->r * 32, kBKBytes);
         c.pad_channels = false;
@@ -1872,6 +1998,10 @@ static std::atomic<int> &gemm_decode_mode();
 static bool gemm_bdec_applicable(dybit_container cont, dybit_fmt fb, const ElemTable &tb, const GemmParams &p, BdecTable *bt);
 static dybit_status launch_gemm_bdec(const uint8_t *ae, int64_t rb, const uint8_t *B, int64_t ldb_bytes, int64_t M, int64_t N,
                                      int64_t K, const GemmParams &p_in, const BdecTable &bt, cudaStream_t s);
+
+static dybit_status launch_conv_s2d(dybit_container cont, const dybit_conv_desc *d, int oh, int ow, const S2dGeom &g,
+                                    const uint8_t *xs, const uint8_t *we, int64_t wrb, const GemmParams &p_in,
+                                    cudaStream_t s);
 
 static dybit_status gemm_impl(int64_t M, int64_t N, int64_t K, const void *A, dybit_fmt fa, const float *scale_a,
                               int64_t lda_bytes, const void *B, dybit_fmt fb, const float *scale_b, int64_t ldb_bytes,
@@ -2084,8 +2214,13 @@ static dybit_status conv_impl(const dybit_conv_desc *d, const void *X, dybit_fmt
     uint8_t *we = xe + cv.a_bytes;
     uint8_t *xd = we + round_up(N * wrb, 1024);              // patch mode: dense container elements of the activation
     const bool patch_dense = cv.mode == kConvPatch && cv.xd_bytes > 0;
-    const bool pix4 = cv.mode == kConvPix4;
-    FusedWeights wpix = {static_cast<const uint8_t *>(W), fw.bits, N, ldw_bytes, wrb, we, wrb, 0, {}, d->c, d->r, d->s};
+    const bool s2d = cv.mode == kConvS2D;
+    const bool pix4 = cv.mode == kConvPix4 || s2d;           // pixels of <= 4 one-byte channels, written pixel by pixel
+    FusedWeights wpix = {static_cast<const uint8_t *>(W), fw.bits, N, ldw_bytes, wrb, we, wrb, 0, {}, d->c, d->r, d->s,
+                         s2d ? 1 : 0, cv.s2d.lo_r, cv.s2d.lo_s, d->pad, cv.s2d.Rp};
+    PixLayout pl = {};
+    if (s2d) pl = PixLayout{d->c, 1, d->h, d->w, cv.s2d.Hs, cv.s2d.P, cv.s2d.padL};
+    else if (pix4 && d->c < 4) pl.c = d->c;                  // four channels: the code order is the pixel-word layout already
     const ElemTable &tx = make_elem_table(fx, plan.container, plan.exp_a);
     const ElemTable &tw = make_elem_table(fw, plan.container, plan.exp_b);
     const bool i8 = plan.container == DYBIT_CONTAINER_I8;
@@ -2117,7 +2252,6 @@ static dybit_status conv_impl(const dybit_conv_desc *d, const void *X, dybit_fmt
             const ExpandOperand opw = {static_cast<const uint8_t *>(W), fw.bits, N, ldw_bytes, wrb / elem, we, wrb, &tw};
             wj.use4 = expand4_job(opw, elem, i8, &wj.job4) ? 1 : 0;
             if (pix4) wj = wpix;
-            const int pix_c = (pix4 && d->c < 4) ? d->c : 0;     // four channels: the code order is the pixel-word layout already
             XTab4 xt = {};
             {
                 Expand4Job xj;
@@ -2131,9 +2265,9 @@ static dybit_status conv_impl(const dybit_conv_desc *d, const void *X, dybit_fmt
             uint8_t *const dense = patch_dense ? xd : xe;         // code order either way
             const int64_t dense_bytes = patch_dense ? cv.xd_bytes : cv.a_bytes;
             st = elem == 1 ? launch_quantize_expand<1>(xq->x, n_x, fx, scale_x, packed, packed_bytes, dense, dense_bytes, tx, wj, tw,
-                                                       partials, n_partials, scale_dst, pix_c, xt, s)
+                                                       partials, n_partials, scale_dst, pl, xt, s)
                            : launch_quantize_expand<2>(xq->x, n_x, fx, scale_x, packed, packed_bytes, dense, dense_bytes, tx, wj, tw,
-                                                       partials, n_partials, scale_dst, 0, xt, s);
+                                                       partials, n_partials, scale_dst, PixLayout{}, xt, s);
             if (st != DYBIT_OK) return st;
             expanded = true;
         } else {
@@ -2149,7 +2283,7 @@ static dybit_status conv_impl(const dybit_conv_desc *d, const void *X, dybit_fmt
             if (w_blocks > sm_count()) w_blocks = sm_count();
             launch_k(expand_pix4_kernel, dim3((unsigned)(x_blocks + w_blocks)), dim3(256u), (size_t)0, s,
                      static_cast<const uint8_t *>(X), fx.bits, pixels, d->c, reinterpret_cast<unsigned *>(xe), tx, wpix, tw,
-                     (int)x_blocks);
+                     (int)x_blocks, pl);
             if (launch_status() != DYBIT_OK) return DYBIT_ERR_CUDA;
         }
     } else if (patch_dense) {
@@ -2287,6 +2421,7 @@ static dybit_status conv_impl(const dybit_conv_desc *d, const void *X, dybit_fmt
         return swb == 128 ? launch_gemm_kind<kAIm2col, 128>(plan.container, bn, map_a, map_b, p, s)
                           : launch_gemm_kind<kAIm2col, 64>(plan.container, bn, map_a, map_b, p, s);
     }
+    if (s2d) return launch_conv_s2d(plan.container, d, oh, ow, cv.s2d, xe, we, wrb, p, s);
     st = make_operand_map(&map_b, we, N, wrb, wrb, bn);
     if (st != DYBIT_OK) return st;
     p.k_blocks = (int)(wrb / kBKBytes);

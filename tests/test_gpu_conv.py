@@ -173,3 +173,21 @@ def test_conv_lowerings_agree_bit_for_bit():
         dy.dybit_set_conv_lowering(3)
     for Y, Y_raw in outs[1:]:
         assert torch.equal(Y, outs[0][0]) and torch.equal(Y_raw, outs[0][1])
+
+
+# Stride-2 convolutions on at most four one-byte channels with even image sides (the 7 x 7 stem) run on a 2 x 2
+# space-to-depth image with halo tiles: every filter size / padding that fits four rearranged taps, 1-4 channels,
+# output channel counts the TMA store cannot take (direct stores), several tile rows and columns, odd batch.
+@pytest.mark.parametrize("shape", [
+    wl.ConvLayer("stem_7x7_p3", 3, 64, 48, 3, 64, 7, 7, 2, 3),
+    wl.ConvLayer("stem_7x7_p3_c4", 2, 32, 32, 4, 64, 7, 7, 2, 3),
+    wl.ConvLayer("c1_5x5_p2", 2, 30, 28, 1, 24, 5, 5, 2, 2),
+    wl.ConvLayer("c2_3x3_p1", 5, 20, 36, 2, 40, 3, 3, 2, 1),
+    wl.ConvLayer("c3_4x4_p0", 2, 18, 22, 3, 128, 4, 4, 2, 0),
+    wl.ConvLayer("c3_2x2_p0", 2, 16, 16, 3, 16, 2, 2, 2, 0),
+    wl.ConvLayer("c3_6x6_p2_k70_direct_stores", 2, 24, 24, 3, 70, 6, 6, 2, 2),
+    wl.ConvLayer("c3_7x7_p3_k200_two_tile_columns", 1, 40, 40, 3, 200, 7, 7, 2, 3),
+], ids=lambda L: L.name)
+@pytest.mark.parametrize("fx,fw", [((4, 0), (4, 1)), ((5, 0), (4, 1)), ((2, 1), (3, 1))])
+def test_space_to_depth_stem_path(shape, fx, fw):
+    run_conv(shape, fx, fw, seed=len(shape.name) + fw[0])
