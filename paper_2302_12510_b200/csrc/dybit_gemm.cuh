@@ -531,7 +531,59 @@ quantize_expand_kernel(const float *__restrict__ x, int64_t n, const float *__re
                     const int64_t p_lo = (c0 + pix_c - 1) / pix_c;      // first pixel that starts in this chunk
                     const int64_t p_hi = e_end / pix_c;                 // one past the last pixel that ends in it
                     unsigned *x4 = reinterpret_cast<unsigned *>(xe);
-                    for (int64_t px = p_lo + lane; px < p_hi; px += 32) {
+                    int64_t p_first = p_lo, p_last = p_hi;       // pixels [p_first, p_last) go one by one below
+                    if (pl.s2d) {
+                        // Space-to-depth image: horizontally adjacent pixels (2q, 2q + 1) are 2c contiguous bytes of one
+                        // 16-byte block, so whole pairs go out as one or two aligned stores; the (at most two) single
+                        // pixels at the chunk's ends take the pixel-by-pixel route.  Pixel counts fit 32 bits (host check).
+                        const unsigned q_lo = (unsigned)((p_lo + 1) >> 1), q_hi = (unsigned)(p_hi >> 1);
+                        const unsigned hw = (unsigned)(pl.H * pl.W), half_w = (unsigned)(pl.W >> 1);
+                        for (unsigned q = q_lo + lane; q < q_hi; q += 32) {
+                            const unsigned px = 2u * q;
+                            const unsigned img = px / hw, rem = px - img * hw;
+                            const unsigned h = rem / (unsigned)pl.W, w = rem - h * (unsigned)pl.W;
+                            uint8_t *row = xe + (((int64_t)(img * (unsigned)pl.Hs + (h >> 1)) * pl.P) << 4);
+                            uint8_t *blk = row + (((w >> 1) + pl.padL) << 4);
+                            const int o0 = (int)((int64_t)px * pix_c - c0);
+                            unsigned long long v = 0;
+                            for (int b = 0; b < 2 * pix_c; ++b) v |= (unsigned long long)sb[o0 + b] << (8 * b);
+                            const unsigned dy = h & 1u;
+                            uint8_t *dst = blk + dy * 2 * pix_c;
+                            if (pix_c == 3) {
+                                if (dy == 0) {
+                                    *reinterpret_cast<unsigned *>(dst) = (unsigned)v;
+                                    *reinterpret_cast<unsigned short *>(dst + 4) = (unsigned short)(v >> 32);
+                                } else {
+                                    *reinterpret_cast<unsigned short *>(dst) = (unsigned short)v;
+                                    *reinterpret_cast<unsigned *>(dst + 2) = (unsigned)(v >> 16);
+                                    *reinterpret_cast<unsigned *>(blk + 12) = 0u;
+                                }
+                            } else if (pix_c == 4) {
+                                *reinterpret_cast<uint2 *>(dst) = make_uint2((unsigned)v, (unsigned)(v >> 32));
+                            } else if (pix_c == 2) {
+                                *reinterpret_cast<unsigned *>(dst) = (unsigned)v;
+                                if (dy) *reinterpret_cast<uint2 *>(blk + 8) = make_uint2(0u, 0u);
+                            } else {
+                                *reinterpret_cast<unsigned short *>(dst) = (unsigned short)v;
+                                if (dy) {
+                                    *reinterpret_cast<unsigned *>(blk + 4) = 0u;
+                                    *reinterpret_cast<uint2 *>(blk + 8) = make_uint2(0u, 0u);
+                                }
+                            }
+                            if (dy == 0) {
+                                if (w == 0)
+                                    for (int i = 0; i < pl.padL; ++i) reinterpret_cast<uint4 *>(row)[i] = make_uint4(0, 0, 0, 0);
+                                if (w + 2 == (unsigned)pl.W)
+                                    for (int i = 0; i < 3; ++i) reinterpret_cast<uint4 *>(row)[pl.padL + half_w + i] = make_uint4(0, 0, 0, 0);
+                            }
+                        }
+                        // the single pixels: an odd first pixel and / or an even last one
+                        p_first = p_hi;
+                        p_last = p_hi;
+                        if (lane == 2 && (p_lo & 1) && p_lo < p_hi) { p_first = p_lo; p_last = p_lo + 1; }
+                        if (lane == 3 && (p_hi & 1) && p_hi - 1 >= p_lo) { p_first = p_hi - 1; p_last = p_hi; }
+                    }
+                    for (int64_t px = p_first + (pl.s2d ? 0 : lane); px < p_last; px += 32) {
                         const int o0 = (int)(px * pix_c - c0);
                         unsigned w = sb[o0];
                         if (pix_c > 1) w |= (unsigned)sb[o0 + 1] << 8;
@@ -1912,7 +1964,7 @@ static ConvPlan plan_conv(const dybit_conv_desc *d, int oh, int ow, int elem) {
     g.P = g.padL + g.Ws + 3;
     const bool s2d_ok = elem == 1 && d->c <= 4 && d->stride == 2 && d->dilation == 1 && d->h % 2 == 0 && d->w % 2 == 0 &&
                         g.Rp >= 1 && g.Rp <= 4 && g.Sp >= 1 && g.Sp <= 4 && g.padL >= 0 && g.padL <= 2 && ow <= g.Ws + 1 &&
-                        (int64_t)d->n * g.Hs * g.P * 16 < ((int64_t)1 << 40);
+                        (int64_t)d->n * g.Hs * g.P * 16 < ((int64_t)1 << 40) && c.pixels < ((int64_t)1 << 31);
     if (pointwise) c.mode = kConvPointwise;
     else if (im2col_ok) c.mode = kConvIm2col;
     else if (s2d_ok) c.mode = kConvS2D;
