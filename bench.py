@@ -48,7 +48,7 @@ NOMINAL = {"hbm_gbs": 7700.0, "bf16_tflops": 2250.0, "int8_tops": 4500.0, "fp8_t
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, copied from the ncu summaries under profiles/ (bench.py cannot
 # read hardware counters itself); an entry is None while the kernel has changed since its counters were taken
 NCU_TRAFFIC = {"gemm_8192": 4 * (36588800 + 18511872), "quantize_2p26_per_element": (268467968 + 7936512) / float(1 << 26),
-               "conv_step": None}
+               "conv_step": (79310336 + 42336512) / 21.0}
 NCU_TRAFFIC_HOW = {
     "gemm_8192": "profiles/dybit_gemm_pair_kernel_i8_square4096.txt: one launch at M=N=K=4096 (a capture small enough to end "
                  "by itself), x 4 for 8192^3 (operand and output bytes both grow 4 x)",
