@@ -590,9 +590,24 @@ def sweep_quantize(dy, wl, device, flush):
                 so = torch.empty(2, dtype=torch.float32, device=device)
                 ms_g = time_calls_flushed(lambda: dy.dybit_quantize_pack(x, fmt, scale=scale, packed=packed), 7, flush)
                 ms_m = time_calls_flushed(lambda: dy.dybit_quantize_pack(x, fmt, packed=packed, scale_out=so), 7, flush)
-                rows.append({"log2n": log2n, "dist": dist, "bits": bits,
-                             "gbs_scale_given": n * (4 + bits / 8) / ms_g / 1e6,
-                             "gbs_with_max_abs": n * (8 + bits / 8) / ms_m / 1e6})
+                row = {"log2n": log2n, "dist": dist, "bits": bits,
+                       "gbs_scale_given": n * (4 + bits / 8) / ms_g / 1e6,
+                       "gbs_with_max_abs": n * (8 + bits / 8) / ms_m / 1e6}
+                if log2n <= 26 and dist == "normal":
+                    # the same launch back to back over buffers that rotate through more than the L2 holds (one CUDA
+                    # graph of nbuf launches): what a stream of such tensors sustains, without the per-launch gap of a
+                    # lone, event-bracketed call
+                    nbuf = min(64, max(4, (512 << 20) // (n * 4)))
+                    xs = [x] + [x.clone() for _ in range(nbuf - 1)]
+                    outs = [torch.empty_like(packed) for _ in range(nbuf)]
+
+                    def run():
+                        for xi, oi in zip(xs, outs):
+                            dy.dybit_quantize_pack(xi, fmt, scale=scale, packed=oi)
+                    ms_b = time_graph(run, 5) / nbuf
+                    row["gbs_scale_given_back_to_back"] = n * (4 + bits / 8) / ms_b / 1e6
+                    del xs, outs
+                rows.append(row)
             del x
             torch.cuda.empty_cache()
     return rows
@@ -693,15 +708,20 @@ def sweep_gemm_batched(dy, wl, device, peaks, flush):
 def sweep_resnet50(dy, wl, device):
     layers = wl.resnet50_layers(64)
     bits = wl.mixed_bitwidths(len(layers), seed=0)
-    work = LayerwiseStep(dy, wl, device, layers, bits, host_copies=False)
+    work = LayerwiseStep(dy, wl, device, layers, bits, host_copies=False, n_streams=3)
     for _ in range(3):
         work.step()
     graph = capture_step(work, device)
     for _ in range(3):
         graph.replay()
     ms = timed_region(graph.replay, 10, None, device) / 10
+    graph1 = capture_step(work, device, lambda: work.step(serial=True))
+    for _ in range(3):
+        graph1.replay()
+    ms1 = timed_region(graph1.replay, 10, None, device) / 10
     conts = [CONTAINERS[dy.dybit_choose_container(fa, fw)[0]] for fa, fw in zip(work.fa, work.fw)]
-    return {"ms_per_step": ms, "tops": 2.0 * work.macs / (ms * 1e-3) / 1e12, "layers": len(layers), "seed": 0,
+    return {"ms_per_step": ms, "ms_per_step_one_stream": ms1, "streams": 3,
+            "tops": 2.0 * work.macs / (ms * 1e-3) / 1e12, "layers": len(layers), "seed": 0,
             "containers": {c: conts.count(c) for c in sorted(set(conts))}, "bits_w_a": bits}
 
 
