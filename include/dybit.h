@@ -41,7 +41,8 @@ typedef enum {
     DYBIT_ERR_ALIGNMENT = 3,      /* a pointer or stride is not aligned as documented         */
     DYBIT_ERR_WORKSPACE = 4,      /* workspace missing or smaller than the *_workspace_bytes  */
     DYBIT_ERR_CUDA = 5,           /* a CUDA runtime / driver call failed                      */
-    DYBIT_ERR_DEVICE_TIMEOUT = 6  /* a bounded device-side wait expired (see dybit_last_device_status) */
+    DYBIT_ERR_DEVICE_TIMEOUT = 6, /* a bounded device-side wait expired (see dybit_last_device_status) */
+    DYBIT_ERR_DEVICE_BOUNDS = 7   /* debug build only (libdybit_debug.so): a range check skipped an access       */
 } dybit_status;
 
 /* One tensor's code format (Section III-A). */

@@ -64,7 +64,8 @@ CONTAINER_NAMES = {0: "int8", 1: "e4m3", 2: "bf16"}
 
 
 def _load() -> C.CDLL:
-    path = _build.LIB_PATH
+    # DYBIT_LIBRARY=debug selects the range-checked build (libdybit_debug.so); anything else is the product library
+    path = _build.DEBUG_LIB_PATH if os.environ.get("DYBIT_LIBRARY", "") == "debug" else _build.LIB_PATH
     if not os.path.exists(path):
         raise ImportError(
             f"{path} is missing: build it with `python -m paper_2302_12510_b200._build` "

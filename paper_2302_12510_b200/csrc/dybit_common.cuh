@@ -80,6 +80,20 @@ inline ProfileEvents &profile_events() {
 // wait that expired.  Kernels only ever OR a value in.
 __device__ unsigned int g_device_status = 0;
 
+// Range checks of the debug build (-DDYBIT_DEBUG_BOUNDS, libdybit_debug.so): global-memory stores whose extent the
+// kernel knows are wrapped in `if (DYBIT_CHECK(index condition, site))`.  A failing check skips the access and ORs
+// (site << 8) | 2 into the status word (dybit_last_device_status then reports DYBIT_ERR_DEVICE_BOUNDS); nothing
+// traps.  In the normal build the macro is the constant true and the condition is not evaluated.
+#ifdef DYBIT_DEBUG_BOUNDS
+__device__ __forceinline__ bool debug_range_ok(bool cond, unsigned site) {
+    if (!cond) atomicOr(&g_device_status, (site << 8) | 2u);
+    return cond;
+}
+#define DYBIT_CHECK(cond, site) ::dybit::debug_range_ok((cond), (site))
+#else
+#define DYBIT_CHECK(cond, site) true
+#endif
+
 // Number of SMs of the current device (cached per device id).
 int sm_count();
 

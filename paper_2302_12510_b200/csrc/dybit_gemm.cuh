@@ -192,6 +192,7 @@ __global__ void __launch_bounds__(256) expand4_kernel(const Expand4Job j0, const
         o1.x = expand4_lookup(w.z, t, ng); o1.y = expand4_lookup(w.z >> 16, t, ng);
         o1.z = expand4_lookup(w.w, t, ng); o1.w = expand4_lookup(w.w >> 16, t, ng);
         uint4 *dst = reinterpret_cast<uint4 *>(j.out + row * j.out_stride + col * 32);
+        if (!DYBIT_CHECK(row < j.rows && col * 32 + 32 <= (j.rows > 1 ? j.out_stride : j.vecs_per_row * 32), 0x23)) continue;
         dst[0] = o0;
         dst[1] = o1;
     }
@@ -634,6 +635,7 @@ quantize_expand_kernel(const float *__restrict__ x, int64_t n, const float *__re
         unsigned w[BITS];
         pack32<BITS>(cw, w);
         uint8_t *dst = packed + item * kChunkBytes;
+        if (!DYBIT_CHECK(item * kChunkBytes + (int64_t)nvec * 16 <= packed_bytes, 0x24)) continue;
         if constexpr (BITS == 4) {
             if (lane < nvec) reinterpret_cast<uint4 *>(dst)[lane] = make_uint4(w[0], w[1], w[2], w[3]);
         } else if constexpr (BITS == 8) {
@@ -1446,8 +1448,9 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
 #pragma unroll
                             for (int j = 0; j < 32; ++j) f[j] = fmaxf(f[j], 0.0f);
                         }
-                        requant_dispatch(p.q_bits, p.q_signed, f, inv_q,
-                                         p.Q + (int64_t)row * p.ldq + (int64_t)col0 * p.q_bits / 8, p.N - col0);
+                        if (DYBIT_CHECK((int64_t)col0 * p.q_bits / 8 + (int64_t)min(32, p.N - col0) * p.q_bits / 8 <= p.ldq, 0x25))
+                            requant_dispatch(p.q_bits, p.q_signed, f, inv_q,
+                                             p.Q + (int64_t)row * p.ldq + (int64_t)col0 * p.q_bits / 8, p.N - col0);
                     }
                     continue;
                 }

@@ -169,6 +169,7 @@ const char *dybit_status_string(dybit_status st) {
         case DYBIT_ERR_WORKSPACE: return "workspace missing or too small";
         case DYBIT_ERR_CUDA: return "CUDA call failed";
         case DYBIT_ERR_DEVICE_TIMEOUT: return "bounded device-side wait expired";
+        case DYBIT_ERR_DEVICE_BOUNDS: return "range check of the debug build failed (access skipped)";
     }
     return "unknown status";
 }
@@ -315,7 +316,8 @@ dybit_status dybit_last_device_status(void *stream, uint32_t *detail) {
         DYBIT_CUDA_TRY(cudaStreamSynchronize(s));
     }
     if (detail) *detail = word;
-    return word == 0 ? DYBIT_OK : DYBIT_ERR_DEVICE_TIMEOUT;
+    if (word == 0) return DYBIT_OK;
+    return (word & 1u) ? DYBIT_ERR_DEVICE_TIMEOUT : DYBIT_ERR_DEVICE_BOUNDS;
 }
 
 }  // extern "C"

@@ -15,6 +15,7 @@ namespace dybit {
 constexpr int kChunkCodes = 1024;
 constexpr int kWarpsPerBlock = 8;
 constexpr int kStreamThreads = kWarpsPerBlock * 32;
+constexpr int kMaxAbsmaxPartials = 1024;     // per-block maxima a max-abs launch may leave for its consumer
 
 // ------------------------------------------------------------------ encode
 
@@ -148,7 +149,7 @@ absmax_kernel(const float *__restrict__ x, int64_t rows, int64_t cols, int64_t l
         unsigned b = threadIdx.x < kWarpsPerBlock ? warp_best[threadIdx.x] : 0u;
         b = __reduce_max_sync(0xffffffffu, b);
         if (threadIdx.x == 0 && partials != nullptr) {
-            partials[blockIdx.x] = b;
+            if (DYBIT_CHECK(blockIdx.x < (unsigned)kMaxAbsmaxPartials, 0x20)) partials[blockIdx.x] = b;
         } else if (threadIdx.x == 0) {
             if (b != 0u) atomicMax(slot, b);                 // result unused: a fire-and-forget reduction
             __threadfence();
@@ -174,7 +175,6 @@ absmax_kernel(const float *__restrict__ x, int64_t rows, int64_t cols, int64_t l
 // previous kernel of the stream) into the tensor's maximum and derives the same {scale, 1/scale} pair with the
 // same two IEEE operations as the ticket path; block 0 also stores the pair for later kernels.  Returns 1/scale.
 // Must be called by all threads of the block, after pdl_enter().
-constexpr int kMaxAbsmaxPartials = 1024;
 __device__ __forceinline__ float scale_from_partials(const unsigned *__restrict__ partials, int n_partials, int m,
                                                      float *__restrict__ scale_out) {
     __shared__ unsigned s_part[kWarpsPerBlock];
@@ -315,6 +315,7 @@ quantize_pack_kernel(const float *__restrict__ x, int64_t rows, int64_t cols, in
         unsigned w[BITS];
         pack32<BITS>(cw, w);
         uint8_t *dst = out + row * row_stride_bytes + chunk * kChunkBytes;
+        if (!DYBIT_CHECK(row < rows && chunk * kChunkBytes + (int64_t)nvec * 16 <= row_stride_bytes, 0x21)) continue;
         if constexpr (BITS == 4) {
             if (lane < nvec) reinterpret_cast<uint4 *>(dst)[lane] = make_uint4(w[0], w[1], w[2], w[3]);
         } else if constexpr (BITS == 8) {
@@ -407,6 +408,7 @@ decode_kernel(const uint8_t *__restrict__ packed, int64_t n, const float *__rest
             r.z = s_lut[(c >> 16) & 0xffu];
             r.w = s_lut[c >> 24];
             const int64_t i0 = j * 128 + lane * 4;
+            if (!DYBIT_CHECK(c0 + i0 < n || i0 >= valid, 0x22)) continue;
             if (out_vec_ok && i0 + 3 < valid) {
                 __stcs(reinterpret_cast<float4 *>(dst + i0), r);
             } else {
