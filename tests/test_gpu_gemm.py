@@ -89,8 +89,8 @@ def test_bf16_container_within_tolerance(fa, fb):
     assert check_gemm(260, 300, 700, fa, fb, seed=fa[0] * 8 + fb[0]) == 2
 
 
-# Few output tiles and a long K: the contraction is cut into ranges that separate CTAs accumulate and the
-# last one to finish adds up (2 to 8 ranges, the last one shorter, every container, ragged M / N / K).
+# Few output tiles and a long K (many K blocks per tile, several trips round the stage ring, narrowed tiles):
+# every container, ragged M / N / K.  (The library does not split K: each tile's contraction runs in one CTA.)
 @pytest.mark.parametrize("M,N,K,fa,fb,cont", [
     (130, 70, 1100, (4, 1), (4, 1), 0),
     (64, 1000, 4096, (4, 0), (4, 1), 0),
@@ -101,11 +101,11 @@ def test_bf16_container_within_tolerance(fa, fb):
     (100, 520, 1500, (8, 1), (8, 1), 2),
     (500, 64, 2111, (6, 0), (7, 1), 2),
 ])
-def test_split_k_small_outputs_long_k(M, N, K, fa, fb, cont):
+def test_few_tiles_long_k(M, N, K, fa, fb, cont):
     assert check_gemm(M, N, K, fa, fb, seed=M + N + K) == cont
 
 
-def test_split_k_twice_in_a_row_reuses_the_tile_counters():
+def test_same_shape_three_times_in_a_row():
     for seed in (1, 2, 3):
         assert check_gemm(256, 256, 2048, (4, 1), (4, 1), seed=seed) == 0
 
