@@ -19,34 +19,50 @@ constexpr int kMaxAbsmaxPartials = 1024;     // per-block maxima a max-abs launc
 
 // ------------------------------------------------------------------ encode
 
-// Magnitude code of a = |x| (a >= 0, never NaN) for M magnitude bits: the
-// inverse of Eq. 1 with round-to-nearest, ties to the even code.  The result
-// is returned with a bias: its low byte is the code.
+// Magnitude code of a (|x| for a signed format, x itself for an unsigned one; may be negative or NaN) for M
+// magnitude bits: the inverse of Eq. 1 with round-to-nearest, ties to the even code.  The result is returned with
+// a bias: its low byte is the code.  `inv` is positive (or +inf when the scale underflowed).
 //
 // Codes grow with the value they stand for.  Below 1 they are linear, so the
 // code is round(t * 2^(M-1)).  In binade e (t in [2^e, 2^(e+1)): e+1 leading
 // ones, a zero, k = M-2-e fraction bits -- the encoder of Section III-B.2) the
 // code is first_code(e) + round(t * 2^(k-e) - 2^k); a carry out of the
 // fraction lands on the next binade's first code by itself.  Along the code
-// axis the sub-unit line lies above every binade's line for t >= 1 and below
-// the e = 0 line for t < 1, so taking the smaller of the two candidates picks
-// the right one without a branch.  Each candidate is ONE FMA: the product is
-// a power-of-two scaling (exact), and the addend is 1.5 * 2^23 plus the
-// integer constant of the line (first_code(e) - 2^k = 2^M - 3 * 2^k), so the
-// FMA's single rounding is round-to-nearest-even on the final code itself and
-// leaves 0x4B400000 + code in the result's bit pattern.  The binade's
-// constants come straight from the exponent field of t.
+// axis these M lines (slopes 2^(M-1), 2^(M-2), 2^(M-4), ...) join up into one
+// continuous concave function of t, which is therefore the smallest of them
+// at every t, and it ends at the all-ones code.  Each line is ONE FMA: the
+// product is a power-of-two scaling (exact), and the addend is 1.5 * 2^23 plus
+// the integer constant of the line (first_code(e) - 2^k = 2^M - 3 * 2^k), so
+// the FMA's single rounding is round-to-nearest-even on the final code itself
+// and leaves 0x4B400000 + code in the result's bit pattern; rounding is
+// monotonic, so the smallest rounded line is the rounded smallest line.
+//
+// Up to four magnitude bits every line is evaluated and the minimum taken
+// together with the all-ones code (which also catches t beyond the top value,
+// infinite included: positive floats order like their bit patterns).  Wider
+// formats evaluate two lines only: the sub-unit one and the line of t's own
+// binade, its constants taken straight from the exponent field of t.
 template <int M>
 __device__ __forceinline__ unsigned magnitude_code_biased(float a, float inv) {
     constexpr float kMagic = 12582912.0f;                                  // 1.5 * 2^23: ulp 1 on both sides
-    // largest float below the top value 2^(M-1): everything from 1.5 * 2^(M-2) up rounds to all-ones anyway
-    const float below_top = __uint_as_float(((unsigned)(127 + M - 1) << 23) - 1u);
-    // (0 * inf = NaN when the reciprocal scale overflowed: fmaxf folds it to 0, the code of a zero element)
-    const float t = fminf(fmaxf(__fmul_rn(a, inv), 0.0f), below_top);
-    const unsigned sub = __float_as_uint(__fmaf_rn(t, (float)(1u << (M - 1)), kMagic));
-    if constexpr (M == 1) {
-        return sub;
+    constexpr unsigned kMagicBits = 0x4B400000u;
+    // a negative product (unsigned format) and NaN (NaN input, or 0 * inf) both become 0, the code of a zero element
+    const float t0 = fmaxf(__fmul_rn(a, inv), 0.0f);
+    if constexpr (M <= 4) {
+        unsigned best = __float_as_uint(__fmaf_rn(t0, (float)(1u << (M - 1)), kMagic));
+#pragma unroll
+        for (int e = 0; e + 2 <= M; ++e) {
+            const int k = M - 2 - e;
+            const float slope = k >= e ? (float)(1u << (k - e)) : 1.0f / (float)(1u << (e - k));
+            const float addend = kMagic + (float)((1 << M) - 3 * (1 << k));
+            best = min(best, __float_as_uint(__fmaf_rn(t0, slope, addend)));
+        }
+        return min(best, kMagicBits + ((1u << M) - 1u));
     } else {
+        // largest float below the top value 2^(M-1): everything from 1.5 * 2^(M-2) up rounds to all-ones anyway
+        const float below_top = __uint_as_float(((unsigned)(127 + M - 1) << 23) - 1u);
+        const float t = fminf(t0, below_top);
+        const unsigned sub = __float_as_uint(__fmaf_rn(t, (float)(1u << (M - 1)), kMagic));
         // exponent field of max(t, 1): the sub-unit range is folded onto binade 0
         const unsigned eb = __float_as_uint(fmaxf(t, 1.0f)) & 0x7f800000u;
         const float scale_e = __uint_as_float(((unsigned)(379 + M) << 23) - 2u * eb);                 // 2^(k-e)
@@ -62,11 +78,10 @@ template <int BITS, bool SIGNED>
 __device__ __forceinline__ unsigned encode4(const float4 v, const float inv) {
     constexpr int M = SIGNED ? BITS - 1 : BITS;
     if constexpr (SIGNED) {
-        // fmaxf(|x|, 0) maps NaN to 0
-        const unsigned m0 = magnitude_code_biased<M>(fmaxf(fabsf(v.x), 0.0f), inv);
-        const unsigned m1 = magnitude_code_biased<M>(fmaxf(fabsf(v.y), 0.0f), inv);
-        const unsigned m2 = magnitude_code_biased<M>(fmaxf(fabsf(v.z), 0.0f), inv);
-        const unsigned m3 = magnitude_code_biased<M>(fmaxf(fabsf(v.w), 0.0f), inv);
+        const unsigned m0 = magnitude_code_biased<M>(fabsf(v.x), inv);
+        const unsigned m1 = magnitude_code_biased<M>(fabsf(v.y), inv);
+        const unsigned m2 = magnitude_code_biased<M>(fabsf(v.z), inv);
+        const unsigned m3 = magnitude_code_biased<M>(fabsf(v.w), inv);
         const unsigned mags = __byte_perm(__byte_perm(m0, m1, 0x0040), __byte_perm(m2, m3, 0x0040), 0x5410);
         // top byte of each float carries its sign in bit 7
         const unsigned tops = __byte_perm(__byte_perm(__float_as_uint(v.x), __float_as_uint(v.y), 0x0073),
@@ -76,10 +91,10 @@ __device__ __forceinline__ unsigned encode4(const float4 v, const float inv) {
         return mags | (((tops & nonzero) >> (7 - M)) & (0x01010101u << M));
     } else {
         // no sign bit: negative inputs (and NaN) take the nearest value the format has, 0
-        const unsigned m0 = magnitude_code_biased<M>(fmaxf(v.x, 0.0f), inv);
-        const unsigned m1 = magnitude_code_biased<M>(fmaxf(v.y, 0.0f), inv);
-        const unsigned m2 = magnitude_code_biased<M>(fmaxf(v.z, 0.0f), inv);
-        const unsigned m3 = magnitude_code_biased<M>(fmaxf(v.w, 0.0f), inv);
+        const unsigned m0 = magnitude_code_biased<M>(v.x, inv);
+        const unsigned m1 = magnitude_code_biased<M>(v.y, inv);
+        const unsigned m2 = magnitude_code_biased<M>(v.z, inv);
+        const unsigned m3 = magnitude_code_biased<M>(v.w, inv);
         return __byte_perm(__byte_perm(m0, m1, 0x0040), __byte_perm(m2, m3, 0x0040), 0x5410);
     }
 }
