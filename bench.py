@@ -136,9 +136,10 @@ class LayerwiseStep:
 
     bits[i] = (weight bits, activation bits) of layer i; weights are signed, activations unsigned."""
 
-    def __init__(self, dy, wl, device, layers, bits, host_copies=True, two_calls=False, n_streams=1):
+    def __init__(self, dy, wl, device, layers, bits, host_copies=True, two_calls=False, n_streams=1, fold=False):
         self.dy, self.device = dy, device
         self.two_calls = two_calls          # quantize_pack + conv2d as two library calls instead of one
+        self.fold = fold                    # max-abs and quantize + expand of ALL layers in two launches, then the convolutions
         self.n_streams = max(1, int(n_streams))
         self.layers = layers
         self.fw = [(wb, 1) for wb, _ in bits]
@@ -168,6 +169,11 @@ class LayerwiseStep:
         # one workspace per stream: layers on different streams run at the same time
         self.ws_pool = [self.ws] + [torch.empty_like(self.ws) for _ in range(self.n_streams - 1)]
         self.side = [torch.cuda.Stream(device) for _ in range(self.n_streams)] if self.n_streams > 1 else []
+        if fold:
+            # same buffers, every layer with a workspace of its own (all of them are in use at once)
+            self.folded = dy.ConvLayers([dict(desc=self.desc[i], X=self.x_dev[i], fx=self.fa[i], W=self.pw[i], fw=self.fw[i],
+                                              scale_w=self.sw[i], packed=self.px[i], scale_out=self.sx[i], Y=self.y[i])
+                                         for i in range(len(self.layers))])
         self.macs = sum(L.macs for L in self.layers)
         self.h2d_bytes = sum(x.numel() * 4 for x in self.x_dev)
         self.d2h_bytes = sum(y.numel() * 4 for y in self.y)
@@ -193,6 +199,18 @@ class LayerwiseStep:
         for whoever times or captures it.  `serial` keeps everything on the calling stream."""
         dy = self.dy
         profiling = events is not None or clocks is not None
+        if self.fold and not self.two_calls and only is None and not profiling and not serial:
+            # dybit_quantize_expand_layers: one max-abs launch and one quantize + expand launch for all layers, on
+            # the calling stream; then one tensor-core launch per layer, round-robin on the side streams
+            cur = torch.cuda.current_stream()
+            dy.dybit_quantize_expand_layers(self.folded)
+            for st in self.side:
+                st.wait_stream(cur)
+            for j in range(len(self.layers)):
+                dy.dybit_conv2d_prepared(self.folded, j, stream=self.side[j % self.n_streams] if self.side else None)
+            for st in self.side:
+                cur.wait_stream(st)
+            return
         if self.n_streams > 1 and only is None and not profiling and not serial:
             cur = torch.cuda.current_stream()
             for st in self.side:
@@ -858,6 +876,9 @@ def main():
     ap.add_argument("--batch", type=int, default=32, help="images per step (32 = the quoted configuration)")
     ap.add_argument("--streams", type=int, default=3,
                     help="streams the step's independent layers are issued on, round-robin (1 = one after the other)")
+    ap.add_argument("--per-layer-calls", action="store_true",
+                    help="time one dybit_quantize_conv2d call per layer as the step instead of the folded "
+                         "dybit_quantize_expand_layers + dybit_conv2d_prepared sequence")
     ap.add_argument("--no-targets", action="store_true", help="skip the single-kernel target measurements")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--step-only", action="store_true",
@@ -923,7 +944,8 @@ def main():
         return
 
     layers = wl.resnet18_layers(args.batch)
-    work = LayerwiseStep(dy, wl, device, layers, [(FMT_W[0], FMT_A[0])] * len(layers), n_streams=args.streams)
+    work = LayerwiseStep(dy, wl, device, layers, [(FMT_W[0], FMT_A[0])] * len(layers), n_streams=args.streams,
+                         fold=not args.per_layer_calls)
     for _ in range(warmup):
         work.step()
     torch.cuda.synchronize()
@@ -950,6 +972,16 @@ def main():
     ms_step = ms_total / args.steps
     value = whole_job_tops(work.macs, world, ms_step)
 
+    # ---- the same step as one dybit_quantize_conv2d call per layer on the same streams (three launches per layer)
+    ms_per_layer_calls = None
+    if work.fold:
+        work.fold = False
+        graph_pl = capture_step(work, device)
+        for _ in range(warmup):
+            graph_pl.replay()
+        ms_per_layer_calls = timed_region(graph_pl.replay, args.steps, dist, device) / args.steps
+        del graph_pl
+        work.fold = True
     # ---- the same step with every layer on one stream (what the per-kernel figures below are taken from)
     graph_serial = capture_step(work, device, lambda: work.step(serial=True))
     for _ in range(warmup):
@@ -1056,16 +1088,23 @@ def main():
         "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
         "config": {"workload": workload_name(args.batch),
                    "parallelism": "replicas only" if world > 1 else "single GPU",
-                   "launch": "one dybit_quantize_conv2d call per layer; one step captured once as a CUDA graph, timed "
-                             "region = K replays; the 21 independent layers "
-                             "are issued round-robin on %d streams (one workspace each) that fork from and join the "
-                             "step's stream" % work.n_streams,
+                   "launch": ("dybit_quantize_expand_layers for the 21 independent layers (one max-abs launch, one quantize + "
+                              "expand launch), then one dybit_conv2d_prepared call per layer round-robin on %d streams that "
+                              "fork from and join the step's stream; " if work.fold else
+                              "one dybit_quantize_conv2d call per layer; the 21 independent layers are issued round-robin on "
+                              "%d streams (one workspace each) that fork from and join the step's stream; ") % work.n_streams
+                             + "one step captured once as a CUDA graph, timed region = K replays",
                    "streams": work.n_streams,
                    "l2": "per-step footprint (fp32 inputs %.0f MB + fp32 outputs %.0f MB) exceeds the 126 MB L2"
                          % (work.h2d_bytes / 1e6, work.d2h_bytes / 1e6)},
         "gpu_launches": launches, "clocks": clocks, "e2e": e2e, "roofline_conv": roofline_conv,
         "quantize_elems_per_step": work.quant_elems,
     }
+    if ms_per_layer_calls is not None:
+        result["per_layer_call_step"] = {
+            "what": "the same step as one dybit_quantize_conv2d call per layer (max-abs, quantize + expand and the "
+                    "tensor-core kernel launched layer by layer) on the same streams",
+            "ms_per_step": ms_per_layer_calls, "value": whole_job_tops(work.macs, world, ms_per_layer_calls), "unit": "TOPS"}
     if args.step_only:
         result["roofline"] = roofline_conv
         if rank == 0:

@@ -222,6 +222,42 @@ dybit_status dybit_quantize_conv2d(const dybit_conv_desc *desc,
                                    const void *W, dybit_fmt fw, const float *scale_w, int64_t ldw_bytes,
                                    float *Y, int32_t *Y_raw, void *ws, size_t ws_bytes, void *stream);
 
+/* dybit_quantize_conv2d for SEVERAL layers whose inputs do not depend on one another (the branches of a block, the
+ * layers of a benchmark that feeds every layer its own activation; Section III-D treats the layers of a model one by
+ * one in the same way): the work in front of the tensor cores is folded into few launches, since for the short
+ * tensors of the later layers a launch costs more than the data.  One struct per layer, fields as the arguments of
+ * dybit_quantize_conv2d; every layer needs its OWN workspace, which stays in use from the first call below until its
+ * dybit_conv2d_prepared has run.
+ *
+ * dybit_quantize_expand_layers: ONE max-abs launch for all layers with scale_x == NULL (per 32 layers), then one
+ *   quantize + expand launch per group of layers with the same pair of formats: writes every layer's X_packed,
+ *   scale_x_out and, in its workspace, the operands of its tensor-core kernel.  Everything on `stream`.
+ * dybit_conv2d_prepared: the rest of one layer (its tensor-core kernel, and the patch gather where the lowering has
+ *   one), on any stream that is ordered after the call above.
+ * Together they give, bit for bit, what dybit_quantize_conv2d gives for each layer.
+ * DYBIT_ERR_UNSUPPORTED (nothing launched) when a layer's lowering is not one whose quantize launch also writes the
+ * expanded operands (channels neither a multiple of 16 nor at most 4 with one-byte elements): use
+ * dybit_quantize_conv2d for such a layer. */
+typedef struct {
+    dybit_conv_desc desc;
+    const float *X;              /* [dev] n*h*w*c floats */
+    dybit_fmt fx;
+    const float *scale_x;        /* [dev] pair to use, or NULL for the max-abs scale */
+    float *scale_x_out;          /* [dev] 2 floats, required */
+    void *X_packed;              /* [dev] dybit_packed_bytes(n*h*w*c, fx.bits) bytes, required */
+    const void *W;               /* [dev] packed weights, k rows */
+    dybit_fmt fw;
+    const float *scale_w;
+    int64_t ldw_bytes;
+    float *Y;                    /* [dev] n*oh*ow*k floats */
+    int32_t *Y_raw;              /* [dev] or NULL */
+    void *ws;                    /* [dev] dybit_conv2d_workspace_bytes(...) bytes of this layer's own */
+    size_t ws_bytes;
+} dybit_conv_layer;
+
+dybit_status dybit_quantize_expand_layers(const dybit_conv_layer *layers, int n_layers, void *stream);
+dybit_status dybit_conv2d_prepared(const dybit_conv_layer *layer, void *stream);
+
 /* Depth-wise convolution on coded operands (MobileNetV2, one of the models of Section IV-A, is built from 3x3
  * layers of this kind): channel ch of the output is channel ch of the input filtered by its own r x s kernel,
  *     Y[n][oh][ow][ch] = sX*sW * sum_{r,s} value(X[n][ih][iw][ch]) * value(W[ch][r][s])

@@ -23,6 +23,7 @@ __all__ = [
     "dybit_launch_count", "dybit_set_conv_lowering", "dybit_set_gemm_decode", "dybit_selftest_wait_timeout", "dybit_profile_next_gemm", "dybit_profile_next_gemm_clock", "dybit_gemm_static_ws", "STATIC_WS_BYTES",
     "dybit_gemm_requant", "dybit_conv2d_requant", "dybit_depthwise_conv2d", "dybit_gemm_batched",
     "dybit_quantize_conv2d", "dybit_quantize_conv2d_requant",
+    "ConvLayers", "dybit_quantize_expand_layers", "dybit_conv2d_prepared",
     "dybit_gemm_batched_workspace_bytes", "dybit_rmse", "dybit_rmse_sweep", "dybit_fake_quant", "dybit_fake_quant_backward",
     "dybit_search_bitwidths",
 ]
@@ -39,6 +40,13 @@ class _CFmt(C.Structure):
 
 class _CConvDesc(C.Structure):
     _fields_ = [(n, C.c_int) for n in ("n", "h", "w", "c", "k", "r", "s", "stride", "pad", "dilation")]
+
+
+class _CConvLayer(C.Structure):
+    _fields_ = [("desc", _CConvDesc), ("X", C.c_void_p), ("fx", _CFmt), ("scale_x", C.c_void_p),
+                ("scale_x_out", C.c_void_p), ("X_packed", C.c_void_p), ("W", C.c_void_p), ("fw", _CFmt),
+                ("scale_w", C.c_void_p), ("ldw_bytes", C.c_int64), ("Y", C.c_void_p), ("Y_raw", C.c_void_p),
+                ("ws", C.c_void_p), ("ws_bytes", C.c_size_t)]
 
 
 class ConvDesc(NamedTuple):
@@ -110,6 +118,8 @@ def _load() -> C.CDLL:
     lib.dybit_rmse.argtypes = [vp, i64, _CFmt, vp, vp, vp]
     lib.dybit_quantize_conv2d.argtypes = [C.POINTER(_CConvDesc), vp, _CFmt, vp, vp, vp, vp, _CFmt, vp, i64,
                                           vp, vp, vp, sz, vp]
+    lib.dybit_quantize_expand_layers.argtypes = [C.POINTER(_CConvLayer), i32, vp]
+    lib.dybit_conv2d_prepared.argtypes = [C.POINTER(_CConvLayer), vp]
     lib.dybit_gemm_batched_workspace_bytes.restype = sz
     lib.dybit_gemm_batched_workspace_bytes.argtypes = [i64, i64, i64, i64, _CFmt, _CFmt]
     lib.dybit_gemm_batched.argtypes = [i64, i64, i64, i64, vp, _CFmt, vp, i64, i64, vp, _CFmt, vp, i64, i64,
@@ -501,6 +511,60 @@ def dybit_quantize_conv2d(desc: ConvDesc, X: torch.Tensor, fx, W: torch.Tensor, 
                                      _ptr(W), _fmt(fw), _ptr(scale_w), W.stride(0), _ptr(Y), _ptr(raw), wp, wn,
                                      _stream(stream)), "dybit_quantize_conv2d")
     return Y, raw, packed, scale_out
+
+
+class ConvLayers:
+    """Arguments of dybit_quantize_conv2d for several independent layers, marshalled once into the C array that
+    dybit_quantize_expand_layers / dybit_conv2d_prepared take.  Each entry of `layers` is a dict with the keyword
+    arguments of dybit_quantize_conv2d (desc, X, fx, W, fw, scale_w and optionally scale_x, scale_out, packed, Y,
+    want_raw, ws); missing outputs and workspaces are allocated here, one workspace per layer."""
+
+    def __init__(self, layers):
+        self.n = len(layers)
+        self.array = (_CConvLayer * self.n)()
+        self.Y, self.raw, self.packed, self.scale, self._keep = [], [], [], [], []
+        for i, a in enumerate(layers):
+            desc, X, fx, W, fw = a["desc"], _dev_f32(a["X"], "X"), a["fx"], a["W"], a["fw"]
+            if X.numel() != desc.n * desc.h * desc.w * desc.c:
+                raise ValueError("X does not match the descriptor")
+            oh, ow = dybit_conv2d_out_hw(desc)
+            Y = a.get("Y")
+            if Y is None:
+                Y = torch.empty((desc.n, oh, ow, desc.k), dtype=torch.float32, device=X.device)
+            raw = torch.empty(Y.shape, dtype=torch.int32, device=X.device) if a.get("want_raw") else None
+            packed = a.get("packed")
+            if packed is None:
+                packed = torch.empty(dybit_packed_bytes(X.numel(), fx[0]), dtype=torch.uint8, device=X.device)
+            scale_out = a.get("scale_out")
+            if scale_out is None:
+                scale_out = torch.empty(2, dtype=torch.float32, device=X.device)
+            ws = a.get("ws")
+            if ws is None:
+                ws = torch.empty(dybit_conv2d_workspace_bytes(desc, fx, fw) + 1024, dtype=torch.uint8, device=X.device)
+            wp, wn = _ws_ptr(ws)
+            c = self.array[i]
+            c.desc = _cdesc(desc)
+            addr = lambda t: None if t is None else t.data_ptr()
+            c.X, c.fx, c.scale_x = addr(X), _fmt(fx), addr(a.get("scale_x"))
+            c.scale_x_out, c.X_packed = addr(scale_out), addr(packed)
+            c.W, c.fw, c.scale_w, c.ldw_bytes = addr(W), _fmt(fw), addr(a["scale_w"]), W.stride(0)
+            c.Y, c.Y_raw, c.ws, c.ws_bytes = addr(Y), addr(raw), wp.value, wn
+            self.Y.append(Y)
+            self.raw.append(raw)
+            self.packed.append(packed)
+            self.scale.append(scale_out)
+            self._keep.append((X, W, a["scale_w"], a.get("scale_x"), ws))
+
+
+def dybit_quantize_expand_layers(layers: ConvLayers, stream=None):
+    """Max-abs scales, codes and expanded operands of all the layers, in few launches on one stream."""
+    _check(lib.dybit_quantize_expand_layers(layers.array, layers.n, _stream(stream)), "dybit_quantize_expand_layers")
+
+
+def dybit_conv2d_prepared(layers: ConvLayers, i: int, stream=None):
+    """The tensor-core part of layer i, after dybit_quantize_expand_layers.  Returns (Y, Y_raw or None)."""
+    _check(lib.dybit_conv2d_prepared(C.byref(layers.array[i]), _stream(stream)), "dybit_conv2d_prepared")
+    return layers.Y[i], layers.raw[i]
 
 
 def dybit_depthwise_conv2d(desc: ConvDesc, X: torch.Tensor, fx, scale_x: torch.Tensor, W: torch.Tensor, fw,

@@ -372,18 +372,45 @@ __device__ __forceinline__ void expand_weights_s2d(const FusedWeights &wj, const
 // a warp 1024 elements at a time exactly as quantize_pack_kernel does; the others the weights, one
 // 16-byte output chunk per thread.  With `partials` the max-abs reduction is finished here as well (see
 // scale_from_partials) and block 0 stores the {scale, 1/scale} pair in scale_out.
+// What one activation, and the weights of its layer, need from quantize_expand_kernel.
+struct QeArgs {
+    const float *x;
+    int64_t n;
+    const float *scale;
+    uint8_t *packed;
+    int64_t packed_bytes;
+    uint8_t *xe;
+    int64_t xe_bytes;
+    FusedWeights wj;
+    int x_blocks;                    // blocks [0, x_blocks) of the layer's share take the activation, the rest the weights
+    const unsigned *partials;
+    int n_partials, m;
+    float *scale_out;
+    PixLayout pl;
+};
+
+// Block `bid` of the `nblk` blocks that work on the layer described by `a`.
 template <int BITS, bool SIGNED, int ELEM>
-__global__ void __launch_bounds__(kStreamThreads, 3)
-quantize_expand_kernel(const float *__restrict__ x, int64_t n, const float *__restrict__ scale,
-                       uint8_t *__restrict__ packed, int64_t packed_bytes, uint8_t *__restrict__ xe, int64_t xe_bytes,
-                       const __grid_constant__ ElemTable tx, const FusedWeights wj, const __grid_constant__ ElemTable tw,
-                       int x_blocks, const unsigned *__restrict__ partials, int n_partials, int m, float *__restrict__ scale_out,
-                       const PixLayout pl, const XTab4 xt) {
+__device__ __forceinline__ void quantize_expand_body(const QeArgs &a, const ElemTable &tx, const ElemTable &tw, const XTab4 &xt,
+                                                     const int bid, const int nblk) {
+    const float *__restrict__ x = a.x;
+    const int64_t n = a.n;
+    const float *__restrict__ scale = a.scale;
+    uint8_t *__restrict__ packed = a.packed;
+    const int64_t packed_bytes = a.packed_bytes;
+    uint8_t *__restrict__ xe = a.xe;
+    const int64_t xe_bytes = a.xe_bytes;
+    const FusedWeights &wj = a.wj;
+    const int x_blocks = a.x_blocks;
+    const unsigned *__restrict__ partials = a.partials;
+    const int n_partials = a.n_partials, m = a.m;
+    float *__restrict__ scale_out = a.scale_out;
+    const PixLayout &pl = a.pl;
     const int pix_c = pl.c;
     __shared__ __align__(16) unsigned s_codes[kWarpsPerBlock][kChunkCodes / 4];
     __shared__ __align__(16) unsigned s_words[kWarpsPerBlock][32 * BITS];
     __shared__ uint16_t s_lut[256];
-    const bool weights = (int)blockIdx.x >= x_blocks;
+    const bool weights = bid >= x_blocks;
     for (int i = threadIdx.x; i < 256; i += blockDim.x) s_lut[i] = weights ? tw.v[i] : tx.v[i];
     __syncthreads();
     const int lane = threadIdx.x & 31;
@@ -392,7 +419,7 @@ quantize_expand_kernel(const float *__restrict__ x, int64_t n, const float *__re
     constexpr int kChunkVecs = kChunkBytes / 16;
     const int64_t items = (packed_bytes + kChunkBytes - 1) / kChunkBytes;
     const bool vec_ok = (reinterpret_cast<uintptr_t>(x) & 15) == 0;
-    const int64_t first_item = (int64_t)blockIdx.x * kWarpsPerBlock + warp;
+    const int64_t first_item = (int64_t)bid * kWarpsPerBlock + warp;
     float4 v[8];
     auto load_item = [&](int64_t item) {
         const int64_t c0 = item * kChunkCodes;
@@ -421,8 +448,8 @@ quantize_expand_kernel(const float *__restrict__ x, int64_t n, const float *__re
     if (weights) {
         if (wj.pix_c > 0) {
             const int64_t total = wj.rows * (wj.out_stride / 16);
-            for (int64_t idx = (int64_t)(blockIdx.x - x_blocks) * blockDim.x + threadIdx.x; idx < total;
-                 idx += (int64_t)(gridDim.x - x_blocks) * blockDim.x) {
+            for (int64_t idx = (int64_t)(bid - x_blocks) * blockDim.x + threadIdx.x; idx < total;
+                 idx += (int64_t)(nblk - x_blocks) * blockDim.x) {
                 if (wj.s2d) expand_weights_s2d(wj, s_lut, idx);
                 else expand_weights_pix4(wj, s_lut, idx);
             }
@@ -434,8 +461,8 @@ quantize_expand_kernel(const float *__restrict__ x, int64_t n, const float *__re
             const int64_t total = j.rows * j.vecs_per_row;
             const unsigned t[4] = {j.tab[0], j.tab[1], j.tab[2], j.tab[3]};
             const bool ng = j.neg_high != 0;
-            for (int64_t i = (int64_t)(blockIdx.x - x_blocks) * blockDim.x + threadIdx.x; i < total;
-                 i += (int64_t)(gridDim.x - x_blocks) * blockDim.x) {
+            for (int64_t i = (int64_t)(bid - x_blocks) * blockDim.x + threadIdx.x; i < total;
+                 i += (int64_t)(nblk - x_blocks) * blockDim.x) {
                 const int64_t row = i / j.vecs_per_row, col = i - row * j.vecs_per_row;
                 const uint4 w = __ldg(reinterpret_cast<const uint4 *>(j.packed + row * j.in_stride) + col);
                 uint4 o0, o1;
@@ -453,8 +480,8 @@ quantize_expand_kernel(const float *__restrict__ x, int64_t n, const float *__re
         const int64_t chunks_per_row = wj.cols / per_chunk;
         const int64_t total = wj.rows * chunks_per_row;
         const unsigned mask = (1u << wj.bits) - 1u;
-        for (int64_t idx = (int64_t)(blockIdx.x - x_blocks) * blockDim.x + threadIdx.x; idx < total;
-             idx += (int64_t)(gridDim.x - x_blocks) * blockDim.x) {
+        for (int64_t idx = (int64_t)(bid - x_blocks) * blockDim.x + threadIdx.x; idx < total;
+             idx += (int64_t)(nblk - x_blocks) * blockDim.x) {
             const int64_t row = idx / chunks_per_row, g = idx - row * chunks_per_row;
             const uint8_t *src = wj.packed + row * wj.in_stride;
             unsigned o[4] = {0, 0, 0, 0};
@@ -473,7 +500,7 @@ quantize_expand_kernel(const float *__restrict__ x, int64_t n, const float *__re
         return;
     }
     // the scale is either there already, or made here from the per-block maxima the preceding absmax launch left
-    const float inv = partials ? scale_from_partials(partials, n_partials, m, scale_out) : __ldg(scale + 1);
+    const float inv = partials ? scale_from_partials(partials, n_partials, m, scale_out, bid == 0) : __ldg(scale + 1);
     for (int64_t item = first_item; item < items; item += (int64_t)x_blocks * kWarpsPerBlock) {
         const int64_t c0 = item * kChunkCodes;
         const int nvec = (int)min((int64_t)kChunkVecs, (packed_bytes - item * kChunkBytes) / 16);
@@ -654,51 +681,189 @@ quantize_expand_kernel(const float *__restrict__ x, int64_t n, const float *__re
     }
 }
 
-template <int BITS, int ELEM>
-static dybit_status launch_quantize_expand_bits(const float *x, int64_t n, bool is_signed, const float *scale, uint8_t *packed,
-                                                int64_t packed_bytes, uint8_t *xe, int64_t xe_bytes, const ElemTable &tx,
-                                                const FusedWeights &wj, const ElemTable &tw, const unsigned *partials,
-                                                int n_partials, float *scale_out, const PixLayout &pl, const XTab4 &xt, cudaStream_t s) {
-    const int m = is_signed ? BITS - 1 : BITS;
-    constexpr int kChunkBytes = kChunkCodes * BITS / 8;
-    // one wave: three blocks fit an SM, the weights' blocks (a few 16-byte chunks per thread) take their share of
-    // it and the activation's blocks loop over what is left of the chunks
+template <int BITS, bool SIGNED, int ELEM>
+__global__ void __launch_bounds__(kStreamThreads, 3)
+quantize_expand_kernel(const __grid_constant__ QeArgs a, const __grid_constant__ ElemTable tx, const __grid_constant__ ElemTable tw,
+                       const __grid_constant__ XTab4 xt) {
+    quantize_expand_body<BITS, SIGNED, ELEM>(a, tx, tw, xt, (int)blockIdx.x, (int)gridDim.x);
+}
+
+// The same for several layers of equal formats in ONE launch: blocks [first_block[l], first_block[l + 1]) work on
+// layer l.
+struct QeLayers {
+    int n_layers;
+    int first_block[kMaxGroupLayers + 1];
+    QeArgs L[kMaxGroupLayers];
+};
+
+template <int BITS, bool SIGNED, int ELEM>
+__global__ void __launch_bounds__(kStreamThreads, 3)
+quantize_expand_layers_kernel(const __grid_constant__ QeLayers g, const __grid_constant__ ElemTable tx,
+                              const __grid_constant__ ElemTable tw, const __grid_constant__ XTab4 xt) {
+    int l = 0;
+    while (l + 1 < g.n_layers && (int)blockIdx.x >= g.first_block[l + 1]) ++l;
+    quantize_expand_body<BITS, SIGNED, ELEM>(g.L[l], tx, tw, xt, (int)blockIdx.x - g.first_block[l],
+                                             g.first_block[l + 1] - g.first_block[l]);
+}
+
+// Arguments and grid share of one layer.  `one_wave`: the launch is this layer's alone, so its grid is what fits
+// the GPU at once (three blocks per SM) and the activation's blocks loop over the chunks; otherwise (several layers
+// in one launch, many waves) a warp takes about four chunks.
+static QeArgs make_qe_args(const float *x, int64_t n, dybit_fmt fx, int elem, const float *scale, uint8_t *packed,
+                           int64_t packed_bytes, uint8_t *xe, int64_t xe_bytes, const FusedWeights &wj,
+                           const unsigned *partials, int n_partials, float *scale_out, const PixLayout &pl, bool one_wave,
+                           int *blocks) {
+    const int64_t chunk_bytes = (int64_t)kChunkCodes * fx.bits / 8;
     const int64_t resident = (int64_t)sm_count() * 3;
-    const int64_t w_chunks = wj.pix_c > 0 ? wj.rows * (wj.out_stride / 16) : wj.rows * (wj.cols * ELEM / 16);
+    const int64_t w_chunks = wj.pix_c > 0 ? wj.rows * (wj.out_stride / 16) : wj.rows * (wj.cols * elem / 16);
     int64_t w_blocks = (w_chunks + kStreamThreads * 4 - 1) / (kStreamThreads * 4);
     if (w_blocks > sm_count()) w_blocks = sm_count();
     if (w_blocks < 1) w_blocks = 1;
-    int64_t x_blocks64 = ((packed_bytes + kChunkBytes - 1) / kChunkBytes + kWarpsPerBlock - 1) / kWarpsPerBlock;
-    if (x_blocks64 > resident - w_blocks) x_blocks64 = resident - w_blocks;
-    if (x_blocks64 < 1) x_blocks64 = 1;
-    const int x_blocks = (int)x_blocks64;
-    const unsigned grid = (unsigned)(x_blocks + w_blocks);
-    if (is_signed)
-        launch_k(quantize_expand_kernel<BITS, true, ELEM>, dim3(grid), dim3((unsigned)kStreamThreads), (size_t)0, s, x, n, scale, packed,
-                 packed_bytes, xe, xe_bytes, tx, wj, tw, x_blocks, partials, n_partials, m, scale_out, pl, xt);
-    else
-        launch_k(quantize_expand_kernel<BITS, false, ELEM>, dim3(grid), dim3((unsigned)kStreamThreads), (size_t)0, s, x, n, scale, packed,
-                 packed_bytes, xe, xe_bytes, tx, wj, tw, x_blocks, partials, n_partials, m, scale_out, pl, xt);
+    const int64_t chunks = (packed_bytes + chunk_bytes - 1) / chunk_bytes;
+    int64_t x_blocks = (chunks + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    if (one_wave) {
+        if (x_blocks > resident - w_blocks) x_blocks = resident - w_blocks;
+    } else {
+        // (the pixel-by-pixel layouts of few-channel images are a long chain per chunk: one chunk per warp there)
+        const int cpw = pl.c > 0 ? 1 : 4;
+        x_blocks = (x_blocks + cpw - 1) / cpw;
+        if (x_blocks > (1 << 20)) x_blocks = 1 << 20;
+    }
+    if (x_blocks < 1) x_blocks = 1;
+    QeArgs a = {};
+    a.x = x;
+    a.n = n;
+    a.scale = scale;
+    a.packed = packed;
+    a.packed_bytes = packed_bytes;
+    a.xe = xe;
+    a.xe_bytes = xe_bytes;
+    a.wj = wj;
+    a.x_blocks = (int)x_blocks;
+    a.partials = partials;
+    a.n_partials = n_partials;
+    a.m = mag_bits(fx);
+    a.scale_out = scale_out;
+    a.pl = pl;
+    *blocks = (int)(x_blocks + w_blocks);
+    return a;
+}
+
+template <int BITS, bool SIGNED, int ELEM>
+static dybit_status launch_qe_inst(const QeArgs &a, int blocks, const ElemTable &tx, const ElemTable &tw, const XTab4 &xt,
+                                   cudaStream_t s) {
+    launch_k(quantize_expand_kernel<BITS, SIGNED, ELEM>, dim3((unsigned)blocks), dim3((unsigned)kStreamThreads), (size_t)0, s, a, tx,
+             tw, xt);
     return launch_status();
 }
 
+template <int BITS, bool SIGNED, int ELEM>
+static dybit_status launch_qe_layers_inst(const QeLayers &g, int blocks, const ElemTable &tx, const ElemTable &tw,
+                                          const XTab4 &xt, cudaStream_t s) {
+    launch_k(quantize_expand_layers_kernel<BITS, SIGNED, ELEM>, dim3((unsigned)blocks), dim3((unsigned)kStreamThreads), (size_t)0, s,
+             g, tx, tw, xt);
+    return launch_status();
+}
+
+using QeLaunch = dybit_status (*)(const QeArgs &, int, const ElemTable &, const ElemTable &, const XTab4 &, cudaStream_t);
+using QeLayersLaunch = dybit_status (*)(const QeLayers &, int, const ElemTable &, const ElemTable &, const XTab4 &, cudaStream_t);
+
+template <int BITS, int ELEM>
+static void qe_launchers_bits(bool sg, QeLaunch *one, QeLayersLaunch *many) {
+    *one = sg ? launch_qe_inst<BITS, true, ELEM> : launch_qe_inst<BITS, false, ELEM>;
+    *many = sg ? launch_qe_layers_inst<BITS, true, ELEM> : launch_qe_layers_inst<BITS, false, ELEM>;
+}
+
 template <int ELEM>
-static dybit_status launch_quantize_expand(const float *x, int64_t n, dybit_fmt fx, const float *scale, uint8_t *packed,
-                                           int64_t packed_bytes, uint8_t *xe, int64_t xe_bytes, const ElemTable &tx,
-                                           const FusedWeights &wj, const ElemTable &tw, const unsigned *partials,
-                                           int n_partials, float *scale_out, const PixLayout &pl, const XTab4 &xt, cudaStream_t s) {
+static bool qe_launchers(dybit_fmt fx, QeLaunch *one, QeLayersLaunch *many) {
     const bool sg = fx.is_signed != 0;
     switch (fx.bits) {
-        case 2: return launch_quantize_expand_bits<2, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pl, xt, s);
-        case 3: return launch_quantize_expand_bits<3, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pl, xt, s);
-        case 4: return launch_quantize_expand_bits<4, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pl, xt, s);
-        case 5: return launch_quantize_expand_bits<5, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pl, xt, s);
-        case 6: return launch_quantize_expand_bits<6, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pl, xt, s);
-        case 7: return launch_quantize_expand_bits<7, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pl, xt, s);
-        case 8: return launch_quantize_expand_bits<8, ELEM>(x, n, sg, scale, packed, packed_bytes, xe, xe_bytes, tx, wj, tw, partials, n_partials, scale_out, pl, xt, s);
+        case 2: qe_launchers_bits<2, ELEM>(sg, one, many); return true;
+        case 3: qe_launchers_bits<3, ELEM>(sg, one, many); return true;
+        case 4: qe_launchers_bits<4, ELEM>(sg, one, many); return true;
+        case 5: qe_launchers_bits<5, ELEM>(sg, one, many); return true;
+        case 6: qe_launchers_bits<6, ELEM>(sg, one, many); return true;
+        case 7: qe_launchers_bits<7, ELEM>(sg, one, many); return true;
+        case 8: qe_launchers_bits<8, ELEM>(sg, one, many); return true;
     }
-    return DYBIT_ERR_INVALID_ARG;
+    return false;
 }
+
+// Layers gathered for dybit_quantize_expand_layers: their max-abs reductions go out as one launch per
+// kMaxGroupLayers tensors, their quantize + expand work as one launch per group of layers with equal formats.
+struct QeGroupHost {
+    dybit_fmt fx, fw;
+    int elem;
+    const ElemTable *tx, *tw;
+    XTab4 xt;
+    QeLayersLaunch launch;
+    QeLayers g;
+    int blocks;
+};
+
+struct LayerCollector {
+    std::vector<AbsmaxLayers> absmax;
+    std::vector<QeGroupHost> groups;
+
+    dybit_status add_absmax(const float *x, int64_t n, unsigned *partials, int *n_partials) {
+        int64_t blocks = (n / 4 + kStreamThreads * 16 - 1) / (kStreamThreads * 16);
+        if (blocks > kMaxAbsmaxPartials) blocks = kMaxAbsmaxPartials;
+        if (blocks < 1) blocks = 1;
+        if (absmax.empty() || absmax.back().n_layers == kMaxGroupLayers) {
+            absmax.emplace_back();
+            absmax.back().n_layers = 0;
+            absmax.back().first_block[0] = 0;
+        }
+        AbsmaxLayers &g = absmax.back();
+        const int l = g.n_layers++;
+        g.x[l] = x;
+        g.n[l] = n;
+        g.partials[l] = partials;
+        g.first_block[l + 1] = g.first_block[l] + (int)blocks;
+        *n_partials = (int)blocks;
+        return DYBIT_OK;
+    }
+
+    dybit_status add_qe(dybit_fmt fx, dybit_fmt fw, int elem, const ElemTable &tx, const ElemTable &tw, const XTab4 &xt,
+                        QeLayersLaunch launch, const QeArgs &a, int blocks) {
+        QeGroupHost *grp = nullptr;
+        for (QeGroupHost &c : groups)
+            if (c.fx.bits == fx.bits && c.fx.is_signed == fx.is_signed && c.fw.bits == fw.bits && c.fw.is_signed == fw.is_signed &&
+                c.elem == elem && c.tx == &tx && c.tw == &tw && c.g.n_layers < kMaxGroupLayers)
+                grp = &c;
+        if (grp == nullptr) {
+            groups.emplace_back();
+            grp = &groups.back();
+            grp->fx = fx;
+            grp->fw = fw;
+            grp->elem = elem;
+            grp->tx = &tx;
+            grp->tw = &tw;
+            grp->xt = xt;
+            grp->launch = launch;
+            grp->g.n_layers = 0;
+            grp->g.first_block[0] = 0;
+            grp->blocks = 0;
+        }
+        const int l = grp->g.n_layers++;
+        grp->g.L[l] = a;
+        grp->g.first_block[l + 1] = grp->g.first_block[l] + blocks;
+        grp->blocks += blocks;
+        return DYBIT_OK;
+    }
+
+    dybit_status launch_all(cudaStream_t s) {
+        for (const AbsmaxLayers &g : absmax) {
+            launch_k(absmax_layers_kernel, dim3((unsigned)g.first_block[g.n_layers]), dim3((unsigned)kStreamThreads), (size_t)0, s, g);
+            if (launch_status() != DYBIT_OK) return DYBIT_ERR_CUDA;
+        }
+        for (const QeGroupHost &c : groups) {
+            const dybit_status st = c.launch(c.g, c.blocks, *c.tx, *c.tw, c.xt, s);
+            if (st != DYBIT_OK) return st;
+        }
+        return DYBIT_OK;
+    }
+};
 
 // One operand's expand job: rows of `cols` codes -> rows of container elements.
 struct ExpandOperand {
@@ -2232,7 +2397,7 @@ struct QuantInput {
 static dybit_status conv_impl(const dybit_conv_desc *d, const void *X, dybit_fmt fx, const float *scale_x, const void *W,
                               dybit_fmt fw, const float *scale_w, int64_t ldw_bytes, float *Y, int32_t *Y_raw,
                               const RequantSpec *rq, void *ws, size_t ws_bytes, void *stream,
-                              const QuantInput *xq = nullptr) {
+                              const QuantInput *xq = nullptr, LayerCollector *col = nullptr, bool prepared = false) {
     int oh, ow;
     dybit_status st = dybit_conv2d_out_hw(d, &oh, &ow);
     if (st != DYBIT_OK) return st;
@@ -2280,19 +2445,27 @@ static dybit_status conv_impl(const dybit_conv_desc *d, const void *X, dybit_fmt
     const ElemTable &tw = make_elem_table(fw, plan.container, plan.exp_b);
     const bool i8 = plan.container == DYBIT_CONTAINER_I8;
     bool expanded = false;
-    if (xq) {
+    // `col`: the layer's max-abs and quantize + expand work is only gathered here (several layers then share a
+    // launch) and the call ends there; `prepared`: that work has been done, only what follows it is launched.
+    // Both need the lowering whose quantize launch also writes the expanded operands.
+    const bool fused_lowering = patch_dense || pix4 || (cv.mode != kConvPatch && !cv.pad_channels);
+    if ((col || prepared) && (!xq || !fused_lowering || pixels * d->c <= 0)) return DYBIT_ERR_UNSUPPORTED;
+    if (prepared) {
+        expanded = true;
+    } else if (xq) {
         // scale first (max-abs, or a copy of the given pair), then codes; where the expanded activation is the code
         // order itself, one launch writes the codes, their container elements and the expanded weights
         const int64_t n_x = pixels * d->c;
         float *scale_dst = const_cast<float *>(scale_x);
-        const bool fused = patch_dense || pix4 || (cv.mode != kConvPatch && !cv.pad_channels);
+        const bool fused = fused_lowering;
         // max-abs scale: in the fused case the absmax launch leaves one maximum per block in the workspace and the
         // quantize launch folds them (nothing to zero first, no atomics); otherwise the ticket version writes the pair
         unsigned *partials = nullptr;
         int n_partials = 0;
         if (xq->given == nullptr && fused && n_x > 0) {
             partials = reinterpret_cast<unsigned *>(static_cast<uint8_t *>(ws) + need - kMaxAbsmaxPartials * sizeof(unsigned));
-            st = launch_absmax(xq->x, 1, n_x, n_x, fx, scale_dst, s, partials, &n_partials);
+            st = col ? col->add_absmax(xq->x, n_x, partials, &n_partials)
+                     : launch_absmax(xq->x, 1, n_x, n_x, fx, scale_dst, s, partials, &n_partials);
             if (st != DYBIT_OK) return st;
         } else if (xq->given == nullptr) {
             st = launch_absmax(xq->x, 1, n_x, n_x, fx, scale_dst, s);
@@ -2319,10 +2492,14 @@ static dybit_status conv_impl(const dybit_conv_desc *d, const void *X, dybit_fmt
             }
             uint8_t *const dense = patch_dense ? xd : xe;         // code order either way
             const int64_t dense_bytes = patch_dense ? cv.xd_bytes : cv.a_bytes;
-            st = elem == 1 ? launch_quantize_expand<1>(xq->x, n_x, fx, scale_x, packed, packed_bytes, dense, dense_bytes, tx, wj, tw,
-                                                       partials, n_partials, scale_dst, pl, xt, s)
-                           : launch_quantize_expand<2>(xq->x, n_x, fx, scale_x, packed, packed_bytes, dense, dense_bytes, tx, wj, tw,
-                                                       partials, n_partials, scale_dst, PixLayout{}, xt, s);
+            QeLaunch one = nullptr;
+            QeLayersLaunch many = nullptr;
+            if (!(elem == 1 ? qe_launchers<1>(fx, &one, &many) : qe_launchers<2>(fx, &one, &many))) return DYBIT_ERR_INVALID_ARG;
+            int blocks = 0;
+            const QeArgs qa = make_qe_args(xq->x, n_x, fx, elem, scale_x, packed, packed_bytes, dense, dense_bytes, wj, partials,
+                                           n_partials, scale_dst, elem == 1 ? pl : PixLayout{}, col == nullptr, &blocks);
+            if (col) return col->add_qe(fx, fw, elem, tx, tw, xt, many, qa, blocks);
+            st = one(qa, blocks, tx, tw, xt, s);
             if (st != DYBIT_OK) return st;
             expanded = true;
         } else {
@@ -2523,6 +2700,28 @@ dybit_status dybit_quantize_conv2d(const dybit_conv_desc *d, const float *X, dyb
     if (scale_x_out == nullptr || X_packed == nullptr) return DYBIT_ERR_INVALID_ARG;
     const dybit::QuantInput xq = {X, scale_x};
     return dybit::conv_impl(d, X_packed, fx, scale_x_out, W, fw, scale_w, ldw_bytes, Y, Y_raw, nullptr, ws, ws_bytes, stream, &xq);
+}
+
+dybit_status dybit_quantize_expand_layers(const dybit_conv_layer *layers, int n_layers, void *stream) {
+    if (layers == nullptr || n_layers <= 0) return DYBIT_ERR_INVALID_ARG;
+    dybit::LayerCollector col;
+    for (int i = 0; i < n_layers; ++i) {
+        const dybit_conv_layer &l = layers[i];
+        if (l.scale_x_out == nullptr || l.X_packed == nullptr) return DYBIT_ERR_INVALID_ARG;
+        const dybit::QuantInput xq = {l.X, l.scale_x};
+        const dybit_status st = dybit::conv_impl(&l.desc, l.X_packed, l.fx, l.scale_x_out, l.W, l.fw, l.scale_w, l.ldw_bytes, l.Y,
+                                                 l.Y_raw, nullptr, l.ws, l.ws_bytes, stream, &xq, &col, false);
+        if (st != DYBIT_OK) return st;
+    }
+    return col.launch_all(static_cast<cudaStream_t>(stream));
+}
+
+dybit_status dybit_conv2d_prepared(const dybit_conv_layer *layer, void *stream) {
+    if (layer == nullptr || layer->scale_x_out == nullptr || layer->X_packed == nullptr) return DYBIT_ERR_INVALID_ARG;
+    const dybit_conv_layer &l = *layer;
+    const dybit::QuantInput xq = {l.X, l.scale_x};
+    return dybit::conv_impl(&l.desc, l.X_packed, l.fx, l.scale_x_out, l.W, l.fw, l.scale_w, l.ldw_bytes, l.Y, l.Y_raw, nullptr,
+                            l.ws, l.ws_bytes, stream, &xq, nullptr, true);
 }
 
 dybit_status dybit_gemm_requant(int64_t M, int64_t N, int64_t K, const void *A, dybit_fmt fa, const float *scale_a,

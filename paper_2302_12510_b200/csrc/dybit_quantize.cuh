@@ -106,6 +106,51 @@ __device__ __forceinline__ unsigned finite_abs_bits(float v) {
     return b < 0x7f800000u ? b : 0u;
 }
 
+// One thread's share of a flat run of n floats (thread tid of nthreads): scalar head up to the first 16-byte
+// boundary, vector body, scalar tail.  Returns the largest finite |x| it saw, as raw bits.
+template <bool STREAM>   // STREAM: evict-first loads (tensor larger than L2); otherwise leave it in L2 for the next pass
+__device__ __forceinline__ unsigned absmax_flat_share(const float *__restrict__ x, int64_t n, int64_t tid, int64_t nthreads) {
+    unsigned best = 0;
+    int64_t head = ((16 - (reinterpret_cast<uintptr_t>(x) & 15)) & 15) / 4;
+    if (head > n) head = n;
+    const int64_t nvec = (n - head) / 4;
+    const float4 *xv = reinterpret_cast<const float4 *>(x + head);
+    // sixteen independent 16-byte loads per thread and round trip (the ragged end reads zeros instead): with
+    // three blocks per SM one round covers 29 MB, so the activations of a ResNet layer take a single round
+    constexpr int kUnroll = 16;
+    for (int64_t i = tid; i < nvec; i += kUnroll * nthreads) {
+        float4 v[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            const int64_t iu = i + u * nthreads;
+            v[u] = iu < nvec ? (STREAM ? __ldcs(xv + iu) : __ldg(xv + iu)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            best = max(best, max(max(finite_abs_bits(v[u].x), finite_abs_bits(v[u].y)),
+                                 max(finite_abs_bits(v[u].z), finite_abs_bits(v[u].w))));
+        }
+    }
+    if (tid < head) best = max(best, finite_abs_bits(x[tid]));
+    const int64_t tail0 = head + nvec * 4;
+    if (tail0 + tid < n) best = max(best, finite_abs_bits(x[tail0 + tid]));   // tail < 4 elements
+    return best;
+}
+
+// Block-wide maximum; the result is valid in thread 0.
+__device__ __forceinline__ unsigned block_max_bits(unsigned best) {
+    best = __reduce_max_sync(0xffffffffu, best);
+    __shared__ unsigned warp_best[kWarpsPerBlock];
+    if ((threadIdx.x & 31) == 0) warp_best[threadIdx.x >> 5] = best;
+    __syncthreads();
+    unsigned b = 0;
+    if (threadIdx.x < 32) {
+        b = threadIdx.x < kWarpsPerBlock ? warp_best[threadIdx.x] : 0u;
+        b = __reduce_max_sync(0xffffffffu, b);
+    }
+    return b;
+}
+
 // Largest finite |x| as raw fp32 bits (non-negative floats order like their
 // bit patterns), max-reduced into slot[0]; slot[1] counts finished blocks.  The
 // host zeroes both words beforehand.  The block that finishes last turns the
@@ -115,7 +160,7 @@ __device__ __forceinline__ unsigned finite_abs_bits(float v) {
 // With `partials` set the kernel stops one step earlier: block b stores its own maximum in partials[b] (no
 // atomics, no ticket, nothing to zero beforehand) and the consumer folds the gridDim.x words itself
 // (scale_from_partials); `slot` is then unused.
-template <bool STREAM>   // STREAM: evict-first loads (tensor larger than L2); otherwise leave it in L2 for the next pass
+template <bool STREAM>
 __global__ void __launch_bounds__(kStreamThreads, 3)
 absmax_kernel(const float *__restrict__ x, int64_t rows, int64_t cols, int64_t ld,
               unsigned *__restrict__ slot, int m, unsigned *__restrict__ partials) {
@@ -124,31 +169,7 @@ absmax_kernel(const float *__restrict__ x, int64_t rows, int64_t cols, int64_t l
     const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int64_t nthreads = (int64_t)gridDim.x * blockDim.x;
     if (ld == cols) {
-        const int64_t n = rows * cols;
-        // scalar head up to the first 16-byte boundary, vector body, scalar tail
-        int64_t head = ((16 - (reinterpret_cast<uintptr_t>(x) & 15)) & 15) / 4;
-        if (head > n) head = n;
-        const int64_t nvec = (n - head) / 4;
-        const float4 *xv = reinterpret_cast<const float4 *>(x + head);
-        // sixteen independent 16-byte loads per thread and round trip (the ragged end reads zeros instead): with
-        // three blocks per SM one round covers 29 MB, so the activations of a ResNet layer take a single round
-        constexpr int kUnroll = 16;
-        for (int64_t i = tid; i < nvec; i += kUnroll * nthreads) {
-            float4 v[kUnroll];
-#pragma unroll
-            for (int u = 0; u < kUnroll; ++u) {
-                const int64_t iu = i + u * nthreads;
-                v[u] = iu < nvec ? (STREAM ? __ldcs(xv + iu) : __ldg(xv + iu)) : make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-#pragma unroll
-            for (int u = 0; u < kUnroll; ++u) {
-                best = max(best, max(max(finite_abs_bits(v[u].x), finite_abs_bits(v[u].y)),
-                                     max(finite_abs_bits(v[u].z), finite_abs_bits(v[u].w))));
-            }
-        }
-        if (tid < head) best = max(best, finite_abs_bits(x[tid]));
-        const int64_t tail0 = head + nvec * 4;
-        if (tail0 + tid < n) best = max(best, finite_abs_bits(x[tail0 + tid]));   // tail < 4 elements
+        best = absmax_flat_share<STREAM>(x, rows * cols, tid, nthreads);
     } else {
         const int64_t total = rows * cols;
         for (int64_t i = tid; i < total; i += nthreads) {
@@ -156,42 +177,57 @@ absmax_kernel(const float *__restrict__ x, int64_t rows, int64_t cols, int64_t l
             best = max(best, finite_abs_bits(x[r * ld + c]));
         }
     }
-    best = __reduce_max_sync(0xffffffffu, best);
-    __shared__ unsigned warp_best[kWarpsPerBlock];
-    if ((threadIdx.x & 31) == 0) warp_best[threadIdx.x >> 5] = best;
-    __syncthreads();
-    if (threadIdx.x < 32) {
-        unsigned b = threadIdx.x < kWarpsPerBlock ? warp_best[threadIdx.x] : 0u;
-        b = __reduce_max_sync(0xffffffffu, b);
-        if (threadIdx.x == 0 && partials != nullptr) {
-            if (DYBIT_CHECK(blockIdx.x < (unsigned)kMaxAbsmaxPartials, 0x20)) partials[blockIdx.x] = b;
-        } else if (threadIdx.x == 0) {
-            if (b != 0u) atomicMax(slot, b);                 // result unused: a fire-and-forget reduction
+    const unsigned b = block_max_bits(best);
+    if (threadIdx.x == 0 && partials != nullptr) {
+        if (DYBIT_CHECK(blockIdx.x < (unsigned)kMaxAbsmaxPartials, 0x20)) partials[blockIdx.x] = b;
+    } else if (threadIdx.x == 0) {
+        if (b != 0u) atomicMax(slot, b);                 // result unused: a fire-and-forget reduction
+        __threadfence();
+        const unsigned ticket = atomicAdd(slot + 1, 1u);
+        if (ticket == gridDim.x - 1) {
             __threadfence();
-            const unsigned ticket = atomicAdd(slot + 1, 1u);
-            if (ticket == gridDim.x - 1) {
-                __threadfence();
-                const float amax = __uint_as_float(atomicMax(slot, 0u));     // the final maximum, read at L2
-                float *scale = reinterpret_cast<float *>(slot);
-                if (amax == 0.0f) {
-                    scale[0] = 1.0f;
-                    scale[1] = 1.0f;
-                } else {
-                    const float vmax = (float)(1u << (m - 1));
-                    scale[0] = __fdiv_rn(amax, vmax);
-                    scale[1] = __fdiv_rn(vmax, amax);
-                }
+            const float amax = __uint_as_float(atomicMax(slot, 0u));     // the final maximum, read at L2
+            float *scale = reinterpret_cast<float *>(slot);
+            if (amax == 0.0f) {
+                scale[0] = 1.0f;
+                scale[1] = 1.0f;
+            } else {
+                const float vmax = (float)(1u << (m - 1));
+                scale[0] = __fdiv_rn(amax, vmax);
+                scale[1] = __fdiv_rn(vmax, amax);
             }
         }
     }
 }
 
+// The partials mode of absmax_kernel for several tensors in ONE launch: blocks [first_block[l], first_block[l + 1])
+// belong to tensor l and leave their maxima in partials[l][0 .. blocks of l).
+constexpr int kMaxGroupLayers = 32;
+struct AbsmaxLayers {
+    int n_layers;
+    int first_block[kMaxGroupLayers + 1];
+    const float *x[kMaxGroupLayers];
+    long long n[kMaxGroupLayers];
+    unsigned *partials[kMaxGroupLayers];
+};
+
+__global__ void __launch_bounds__(kStreamThreads, 3) absmax_layers_kernel(const __grid_constant__ AbsmaxLayers g) {
+    pdl_enter();
+    int l = 0;
+    while (l + 1 < g.n_layers && (int)blockIdx.x >= g.first_block[l + 1]) ++l;
+    const int bid = (int)blockIdx.x - g.first_block[l], nblk = g.first_block[l + 1] - g.first_block[l];
+    const unsigned best = absmax_flat_share<false>(g.x[l], (int64_t)g.n[l], (int64_t)bid * blockDim.x + threadIdx.x,
+                                                   (int64_t)nblk * blockDim.x);
+    const unsigned b = block_max_bits(best);
+    if (threadIdx.x == 0 && DYBIT_CHECK(bid < kMaxAbsmaxPartials, 0x26)) g.partials[l][bid] = b;
+}
+
 // Consumer side of the partials mode of absmax_kernel: every block folds the per-block maxima (written by the
 // previous kernel of the stream) into the tensor's maximum and derives the same {scale, 1/scale} pair with the
-// same two IEEE operations as the ticket path; block 0 also stores the pair for later kernels.  Returns 1/scale.
+// same two IEEE operations as the ticket path; the block called with `writer` also stores the pair for later kernels.  Returns 1/scale.
 // Must be called by all threads of the block, after pdl_enter().
 __device__ __forceinline__ float scale_from_partials(const unsigned *__restrict__ partials, int n_partials, int m,
-                                                     float *__restrict__ scale_out) {
+                                                     float *__restrict__ scale_out, bool writer) {
     __shared__ unsigned s_part[kWarpsPerBlock];
     __shared__ float s_inv;
     unsigned b = 0;
@@ -209,7 +245,7 @@ __device__ __forceinline__ float scale_from_partials(const unsigned *__restrict_
             inv = __fdiv_rn(vmax, amax);
         }
         s_inv = inv;
-        if (blockIdx.x == 0) {
+        if (writer) {
             scale_out[0] = sc;
             scale_out[1] = inv;
         }

@@ -132,3 +132,92 @@ def test_argument_errors():
                                          ((7, 0), (4, 1), False)])
 def test_few_channels_pixel_words(layer, fx, fw, given):
     run(layer, fx, fw, seed=len(layer.name) * 3 + fx[0], given_scale=given)
+
+
+def oracle_layer(layer, fx, fw, seed, given_scale):
+    """Inputs of one layer and what the oracle makes of them."""
+    x = wl.half_normal((layer.n, layer.h, layer.w, layer.c), seed=seed)
+    if fx[1]:
+        x = x - 0.5
+    w = wl.kaiming_normal(layer.k, layer.r, layer.s, layer.c, seed=seed + 1)
+    spw = orc.absmax_scale(w.numpy(), fw[0], bool(fw[1]))
+    cw = orc.quantize(w.numpy(), fw[0], bool(fw[1]), spw[1])
+    spx = orc.absmax_scale(x.numpy(), fx[0], bool(fx[1]))
+    if given_scale:
+        s0 = np.float32(spx[0]) * np.float32(0.7)
+        spx = (float(s0), float(np.float32(1.0) / s0))
+    cx = orc.quantize(x.numpy(), fx[0], bool(fx[1]), spx[1])
+    S, Y_ref = orc.conv2d(cx, fx, spx[0], cw, fw, spw[0], stride=layer.stride, pad=layer.pad)
+    return x, w, spx, orc.pack(cx, fx[0]), S, Y_ref
+
+
+# several independent layers through dybit_quantize_expand_layers + dybit_conv2d_prepared: one max-abs launch, one
+# quantize + expand launch per pair of formats, then one tensor-core launch per layer (the few-channel patch lowering
+# of the bf16 stem has a gather launch as well); results as the oracle's, layer by layer
+def test_layers_in_few_launches():
+    cases = [
+        (wl.ConvLayer("stem_s2d", 2, 64, 64, 3, 64, 7, 7, 2, 3), (4, 0), (4, 1), False),
+        (wl.ConvLayer("c64_3x3", 8, 28, 28, 64, 64, 3, 3, 1, 1), (4, 0), (4, 1), False),
+        (wl.ConvLayer("c128_3x3_s2", 6, 20, 20, 128, 96, 3, 3, 2, 1), (4, 0), (4, 1), True),
+        (wl.ConvLayer("c256_pointwise", 3, 13, 11, 256, 100, 1, 1, 1, 0), (4, 0), (4, 1), False),
+        (wl.ConvLayer("c48_gather", 2, 9, 9, 48, 64, 3, 3, 1, 1), (4, 0), (4, 1), False),
+        (wl.ConvLayer("fc_like", 5, 1, 1, 512, 1000, 1, 1, 1, 0), (4, 0), (4, 1), False),
+        (wl.ConvLayer("c64_e4m3", 2, 14, 14, 64, 96, 3, 3, 1, 1), (5, 0), (4, 1), False),
+        (wl.ConvLayer("c64_bf16", 6, 20, 20, 64, 96, 3, 3, 1, 1), (8, 0), (8, 1), True),
+        (wl.ConvLayer("c1_5x5_signed", 3, 30, 31, 1, 24, 5, 5, 1, 2), (4, 1), (3, 1), False),
+    ]
+    args, refs = [], []
+    for i, (L, fx, fw, given) in enumerate(cases):
+        x, w, spx, packed_ref, S, Y_ref = oracle_layer(L, fx, fw, 100 + 7 * i, given)
+        pw, sw = dy.dybit_quantize_pack_2d(w.reshape(L.k, -1).to(DEV), fw)
+        cont, _, _ = dy.dybit_choose_container(fx, fw)
+        a = dict(desc=dy.ConvDesc(L.n, L.h, L.w, L.c, L.k, L.r, L.s, L.stride, L.pad, 1), X=x.to(DEV), fx=fx, W=pw, fw=fw,
+                 scale_w=sw, want_raw=(cont == 0))
+        if given:
+            a["scale_x"] = torch.tensor(spx, dtype=torch.float32, device=DEV)
+        args.append(a)
+        refs.append((L, fx, fw, cont, spx, packed_ref, S, Y_ref, orc.absmax_scale(w.numpy(), fw[0], bool(fw[1]))))
+    layers = dy.ConvLayers(args)
+    torch.cuda.synchronize()
+    n0 = dy.dybit_launch_count()
+    dy.dybit_quantize_expand_layers(layers)
+    n1 = dy.dybit_launch_count()
+    assert n1 - n0 == 1 + 4                     # max-abs for all; (4,0)x(4,1), (5,0)x(4,1), (8,0)x(8,1), (4,1)x(3,1)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    for i in range(len(cases)):
+        dy.dybit_conv2d_prepared(layers, i, stream=side if i % 2 else None)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    assert dy.dybit_launch_count() - n1 <= len(cases) + 2
+    assert dy.dybit_last_device_status() == (0, 0)
+    for i, (L, fx, fw, cont, spx, packed_ref, S, Y_ref, spw) in enumerate(refs):
+        assert layers.scale[i].cpu().numpy().tolist() == [float(np.float32(spx[0])), float(np.float32(spx[1]))], L.name
+        assert np.array_equal(layers.packed[i].cpu().numpy(), packed_ref), L.name
+        Y = layers.Y[i].cpu().numpy()
+        if cont == 0:
+            assert np.array_equal(layers.raw[i].cpu().numpy().astype(np.int64), S), L.name
+            assert np.array_equal(Y, Y_ref), L.name
+        else:
+            amax = float(spx[0]) * float(np.abs(orc.decode_table(fx[0], bool(fx[1]))).max())
+            bmax = float(spw[0]) * float(np.abs(orc.decode_table(fw[0], bool(fw[1]))).max())
+            assert np.abs(Y.astype(np.float64) - Y_ref.astype(np.float64)).max() <= 1e-5 * L.gemm_k * amax * bmax, L.name
+        # and bit for bit what the one-layer call gives
+        a = args[i]
+        Y1, _, p1, s1 = dy.dybit_quantize_conv2d(a["desc"], a["X"], fx, a["W"], fw, a["scale_w"], scale_x=a.get("scale_x"))
+        assert np.array_equal(Y1.cpu().numpy().view(np.uint32), Y.view(np.uint32)), L.name
+        assert torch.equal(p1, layers.packed[i]) and torch.equal(s1, layers.scale[i]), L.name
+
+
+def test_layers_reject_a_lowering_without_fused_expand():
+    # 120 channels: padded to 128 per tap and too long a row for the patch matrix, so quantize and expand stay apart
+    L = wl.ConvLayer("c120_pad_channels", 2, 8, 8, 120, 24, 3, 3, 1, 1)
+    x = wl.half_normal((L.n, L.h, L.w, L.c), seed=1, device=DEV)
+    w = wl.kaiming_normal(L.k, L.r, L.s, L.c, seed=2)
+    pw, sw = dy.dybit_quantize_pack_2d(w.reshape(L.k, -1).to(DEV), (4, 1))
+    layers = dy.ConvLayers([dict(desc=dy.ConvDesc(L.n, L.h, L.w, L.c, L.k, L.r, L.s, L.stride, L.pad, 1), X=x, fx=(4, 0), W=pw,
+                                 fw=(4, 1), scale_w=sw)])
+    n0 = dy.dybit_launch_count()
+    with pytest.raises(dy.DybitError):
+        dy.dybit_quantize_expand_layers(layers)
+    assert dy.dybit_launch_count() == n0
