@@ -47,7 +47,7 @@ FMT_A = (4, 0)      # post-ReLU activations: unsigned 4-bit
 NOMINAL = {"hbm_gbs": 7700.0, "bf16_tflops": 2250.0, "int8_tops": 4500.0, "fp8_tflops": 4500.0}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, copied from the ncu summaries under profiles/ (bench.py cannot
 # read hardware counters itself); an entry is None while the kernel has changed since its counters were taken
-NCU_TRAFFIC = {"gemm_8192": 4 * (36588800 + 18511872), "quantize_2p26_per_element": (268467968 + 7936512) / float(1 << 26),
+NCU_TRAFFIC = {"gemm_8192": 4 * (36588800 + 18511872), "quantize_2p26_per_element": (268458496 + 8048640) / float(1 << 26),
                "conv_step": (79310336 + 42336512) / 21.0}
 NCU_TRAFFIC_HOW = {
     "gemm_8192": "profiles/dybit_gemm_pair_kernel_i8_square4096.txt: one launch at M=N=K=4096 (a capture small enough to end "
@@ -464,6 +464,28 @@ def target_quantize(dy, wl, device, peaks, log2n=28, bits=4):
                              "frac": bytes_maxabs / ms_maxabs / 1e6 / peaks["hbm_gbs"]},
             "peak_gbs": peaks["hbm_gbs"], "peak_how": f"copy bandwidth ({peaks['source']})",
             "nominal_gbs": NOMINAL["hbm_gbs"]}
+
+
+def target_quantize_expand(dy, wl, device, peaks, log2n=26):
+    """quantize_expand_kernel alone on an activation beyond the L2: fp32 in (4 B), packed 4-bit codes (0.5 B) and int8
+    tensor-core elements (1 B) out, scale given.  Reached through dybit_quantize_expand_layers on a single pointwise
+    layer (64 channels, 16 filters), whose only launch it then is."""
+    n_pix = (1 << log2n) // 64
+    desc = dy.ConvDesc(1, n_pix // 128, 128, 64, 16, 1, 1, 1, 0, 1)
+    fx, fw = (4, 0), (4, 1)
+    x = wl.half_normal((desc.n, desc.h, desc.w, desc.c), seed=23, device=device)
+    w = wl.kaiming_normal(16, 1, 1, 64, seed=24).reshape(16, -1).to(device)
+    pw, sw = dy.dybit_quantize_pack_2d(w, fw)
+    scale = dy.dybit_absmax_scale(x.reshape(-1), fx)
+    layer = dy.ConvLayers([dict(desc=desc, X=x, fx=fx, W=pw, fw=fw, scale_w=sw, scale_x=scale, scale_out=scale)])
+    n0 = dy.dybit_launch_count()
+    dy.dybit_quantize_expand_layers(layer)
+    launches = dy.dybit_launch_count() - n0
+    ms = time_calls(lambda: dy.dybit_quantize_expand_layers(layer), 10)
+    n = x.numel()
+    return {"elements": n, "bytes_per_element": 5.5, "launches_per_call": launches, "ms": ms, "gbs": n * 5.5 / ms / 1e6,
+            "frac": n * 5.5 / ms / 1e6 / peaks["hbm_gbs"], "peak_gbs": peaks["hbm_gbs"],
+            "peak_how": f"copy bandwidth ({peaks['source']})"}
 
 
 def measure_peaks_here(device, peaks, size=8192):
@@ -940,6 +962,7 @@ def main():
             out["gemm_w4a4"] = target_gemm(dy, wl, device, peaks, size=args.gemm_size)
         if args.quant_log2n > 0:
             out["quantize_pack"] = target_quantize(dy, wl, device, peaks, log2n=args.quant_log2n, bits=args.quant_bits)
+            out["quantize_expand"] = target_quantize_expand(dy, wl, device, peaks, log2n=min(args.quant_log2n, 26))
         print(json.dumps({"targets": out}))
         return
 
@@ -1147,7 +1170,8 @@ def main():
         result["peaks_measured_here"] = here
         g = target_gemm(dy, wl, device, peaks, size=args.gemm_size)
         q = target_quantize(dy, wl, device, peaks, log2n=args.quant_log2n, bits=args.quant_bits)
-        result["targets"] = {"gemm_w4a4": g, "quantize_pack": q, "gemm_decode": target_gemm_decode(dy, wl, device)}
+        result["targets"] = {"gemm_w4a4": g, "quantize_pack": q, "gemm_decode": target_gemm_decode(dy, wl, device),
+                             "quantize_expand": target_quantize_expand(dy, wl, device, peaks)}
         # the metric's two figures as roofline objects: the tensor-core kernel of the square GEMM against the int8
         # tensor peak, the quantize/pack kernel (scale given) against the copy bandwidth
         lib_int8 = here.get("int8_matmul_tops")
