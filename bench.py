@@ -759,8 +759,31 @@ def sweep_resnet50(dy, wl, device):
     for _ in range(3):
         graph1.replay()
     ms1 = timed_region(graph1.replay, 10, None, device) / 10
+    del graph, graph1
+    # the same step with the streaming launches folded over the layers (dybit_quantize_expand_layers: one max-abs
+    # launch per 32 layers, one quantize + expand launch per pair of formats), then the convolutions on three streams
+    ms_fold, fold_launches = None, None
+    try:
+        work.folded = dy.ConvLayers([dict(desc=work.desc[i], X=work.x_dev[i], fx=work.fa[i], W=work.pw[i], fw=work.fw[i],
+                                          scale_w=work.sw[i], packed=work.px[i], scale_out=work.sx[i], Y=work.y[i])
+                                     for i in range(len(layers))])
+        work.fold = True
+        for _ in range(3):
+            work.step()
+        n0 = dy.dybit_launch_count()
+        graph_f = capture_step(work, device)
+        fold_launches = dy.dybit_launch_count() - n0
+        for _ in range(3):
+            graph_f.replay()
+        ms_fold = timed_region(graph_f.replay, 10, None, device) / 10
+        del graph_f
+    except dy.DybitError as exc:        # a layer whose lowering has no fused expand
+        ms_fold = None
+        fold_note = str(exc)
+    work.fold = False
     conts = [CONTAINERS[dy.dybit_choose_container(fa, fw)[0]] for fa, fw in zip(work.fa, work.fw)]
     return {"ms_per_step": ms, "ms_per_step_one_stream": ms1, "streams": 3,
+            "ms_per_step_folded": ms_fold, "launches_per_folded_step": fold_launches,
             "tops": 2.0 * work.macs / (ms * 1e-3) / 1e12, "layers": len(layers), "seed": 0,
             "containers": {c: conts.count(c) for c in sorted(set(conts))}, "bits_w_a": bits}
 

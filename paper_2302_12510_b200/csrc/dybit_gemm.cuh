@@ -270,20 +270,21 @@ struct PixLayout {
 };
 
 // Space-to-depth image: where the channel bytes of input pixel `px` (NHW index) go.
+// (pixel counts fit 32 bits: the host checks it before it takes this lowering)
 __device__ __forceinline__ uint8_t *s2d_pixel_addr(uint8_t *xs, const PixLayout &pl, int64_t px) {
-    const int64_t img = px / ((int64_t)pl.H * pl.W);
-    const int rem = (int)(px - img * pl.H * pl.W);
-    const int h = rem / pl.W, w = rem - h * pl.W;
-    return xs + ((((img * pl.Hs + (h >> 1)) * pl.P + (w >> 1) + pl.padL) << 4) + ((h & 1) * 2 + (w & 1)) * pl.c);
+    const unsigned hw = (unsigned)(pl.H * pl.W);
+    const unsigned img = (unsigned)px / hw, rem = (unsigned)px - img * hw;
+    const unsigned h = rem / (unsigned)pl.W, w = rem - h * (unsigned)pl.W;
+    return xs + ((((int64_t)(img * (unsigned)pl.Hs + (h >> 1)) * pl.P + (w >> 1) + pl.padL) << 4) + ((h & 1) * 2 + (w & 1)) * pl.c);
 }
 
 // The zero bytes pixel `px` is responsible for: the unused tail of its 16-byte block (the block's last pixel writes
 // it) and the padding pixels of its stored row (the first and last pixel of every even input row write them).
 __device__ __forceinline__ void s2d_pixel_duties(uint8_t *xs, const PixLayout &pl, int64_t px) {
-    const int64_t img = px / ((int64_t)pl.H * pl.W);
-    const int rem = (int)(px - img * pl.H * pl.W);
-    const int h = rem / pl.W, w = rem - h * pl.W;
-    uint8_t *row = xs + (((img * pl.Hs + (h >> 1)) * pl.P) << 4);
+    const unsigned hw = (unsigned)(pl.H * pl.W);
+    const unsigned img = (unsigned)px / hw, rem = (unsigned)px - img * hw;
+    const int h = (int)(rem / (unsigned)pl.W), w = (int)(rem - (unsigned)h * (unsigned)pl.W);
+    uint8_t *row = xs + (((int64_t)(img * (unsigned)pl.Hs + ((unsigned)h >> 1)) * pl.P) << 4);
     if ((h & 1) && (w & 1)) {
         uint8_t *blk = row + (((w >> 1) + pl.padL) << 4);
         for (int b = 4 * pl.c; b < 16; ++b) blk[b] = 0;
