@@ -47,6 +47,20 @@ for L in (wl.ConvLayer("a", 2, 14, 14, 64, 64, 3, 3, 1, 1), wl.ConvLayer("b", 2,
     sa_, sb_ = orc.absmax_scale(xa.numpy(), 4, False), orc.absmax_scale(wa.numpy(), 4, True)
     Sc, Yc = orc.conv2d(orc.quantize(xa.numpy(), 4, False, sa_[1]), (4, 0), sa_[0], orc.quantize(wa.numpy(), 4, True, sb_[1]), (4, 1), sb_[0], stride=L.stride, pad=L.pad)
     assert np.array_equal(Y_raw.cpu().numpy().astype(np.int64), Sc) and np.array_equal(Y.cpu().numpy(), Yc)
+# the same three layers through the folded launches (absmax_layers_kernel, quantize_expand_layers_kernel)
+args, want = [], []
+for L in (wl.ConvLayer("a", 2, 14, 14, 64, 64, 3, 3, 1, 1), wl.ConvLayer("b", 2, 32, 32, 3, 64, 7, 7, 2, 3), wl.ConvLayer("c", 3, 9, 9, 128, 40, 3, 3, 2, 1)):
+    xa = wl.half_normal((L.n, L.h, L.w, L.c), seed=1); wa = wl.kaiming_normal(L.k, L.r, L.s, L.c, seed=2)
+    pw, sw = dy.dybit_quantize_pack_2d(wa.reshape(L.k, -1).to(dev), (4, 1))
+    d = dy.ConvDesc(L.n, L.h, L.w, L.c, L.k, L.r, L.s, L.stride, L.pad, 1)
+    args.append(dict(desc=d, X=xa.to(dev), fx=(4, 0), W=pw, fw=(4, 1), scale_w=sw, want_raw=True))
+    sa_, sb_ = orc.absmax_scale(xa.numpy(), 4, False), orc.absmax_scale(wa.numpy(), 4, True)
+    want.append(orc.conv2d(orc.quantize(xa.numpy(), 4, False, sa_[1]), (4, 0), sa_[0], orc.quantize(wa.numpy(), 4, True, sb_[1]), (4, 1), sb_[0], stride=L.stride, pad=L.pad))
+layers = dy.ConvLayers(args)
+dy.dybit_quantize_expand_layers(layers)
+for i in range(len(args)):
+    Y, Y_raw = dy.dybit_conv2d_prepared(layers, i)
+    assert np.array_equal(Y_raw.cpu().numpy().astype(np.int64), want[i][0]) and np.array_equal(Y.cpu().numpy(), want[i][1])
 torch.cuda.synchronize()
 assert dy.dybit_last_device_status() == (0, 0), dy.dybit_last_device_status()
 print("debug build ok")

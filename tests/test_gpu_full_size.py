@@ -198,6 +198,55 @@ def test_resnet18_batch32_uniform_4bit_sampled(i, L):
     assert _conv_layer_sampled(L, (4, 0), (4, 1), seed=1000 + i, one_call_too=True) == 0
 
 
+def test_resnet18_batch32_folded_step_in_the_bench_launch_configuration():
+    """The step as bench.py times it: dybit_quantize_expand_layers over all 21 layers, then dybit_conv2d_prepared per
+    layer round-robin on three streams.  Every layer's codes, scale and output must equal, bit for bit, what the
+    one-layer call gives (which the test above checks against the oracle), and sampled outputs of four layers are
+    checked against the oracle directly."""
+    layers = wl.resnet18_layers(32)
+    fx, fw = (4, 0), (4, 1)
+    args, ws = [], []
+    for i, L in enumerate(layers):
+        x = wl.half_normal((L.n, L.h, L.w, L.c), seed=1000 + i, device=DEV)
+        w = wl.kaiming_normal(L.k, L.r, L.s, L.c, seed=2000 + i)
+        pw, sw = dy.dybit_quantize_pack_2d(w.reshape(L.k, -1).to(DEV), fw)
+        args.append(dict(desc=dy.ConvDesc(L.n, L.h, L.w, L.c, L.k, L.r, L.s, L.stride, L.pad, 1), X=x, fx=fx, W=pw, fw=fw,
+                         scale_w=sw))
+        ws.append(w)
+    folded = dy.ConvLayers(args)
+    side = [torch.cuda.Stream(DEV) for _ in range(3)]
+    cur = torch.cuda.current_stream()
+    n0 = dy.dybit_launch_count()
+    dy.dybit_quantize_expand_layers(folded)
+    for st in side:
+        st.wait_stream(cur)
+    for j in range(len(layers)):
+        dy.dybit_conv2d_prepared(folded, j, stream=side[j % 3])
+    for st in side:
+        cur.wait_stream(st)
+    torch.cuda.synchronize()
+    assert dy.dybit_launch_count() - n0 == 2 + len(layers)
+    assert dy.dybit_last_device_status() == (0, 0)
+    for i, (L, a) in enumerate(zip(layers, args)):
+        Y1, _, p1, s1 = dy.dybit_quantize_conv2d(a["desc"], a["X"], fx, a["W"], fw, a["scale_w"])
+        assert torch.equal(p1, folded.packed[i]) and torch.equal(s1, folded.scale[i]), L.name
+        assert torch.equal(Y1, folded.Y[i]), L.name
+        del Y1, p1
+    for i in (0, 1, 11, 20):
+        L = layers[i]
+        xh = args[i]["X"].cpu().numpy()
+        spx = orc.absmax_scale(xh, 4, False)
+        spw = orc.absmax_scale(ws[i].numpy(), 4, True)
+        cw = orc.quantize(ws[i].numpy(), 4, True, spw[1])
+        total = folded.Y[i].numel()
+        idx = np.unique(np.concatenate([np.random.default_rng(i).integers(0, total, 400), [0, total - 1]]))
+        _, y_ref = orc.conv2d_sampled(xh, fx, spx, cw, fw, spw[0], idx, stride=L.stride, pad=L.pad)
+        got = folded.Y[i].reshape(-1)[torch.from_numpy(idx).to(DEV)].cpu().numpy()
+        assert np.array_equal(got, y_ref), L.name
+    del folded
+    torch.cuda.empty_cache()
+
+
 _R50 = wl.resnet50_layers(64)
 _R50_BITS = wl.mixed_bitwidths(len(_R50), seed=0)
 
