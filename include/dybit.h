@@ -234,7 +234,8 @@ dybit_status dybit_quantize_conv2d(const dybit_conv_desc *desc,
  *   scale_x_out and, in its workspace, the operands of its tensor-core kernel.  Everything on `stream`.
  * dybit_conv2d_prepared: the rest of one layer (its tensor-core kernel, and the patch gather where the lowering has
  *   one), on any stream that is ordered after the call above.
- * Together they give, bit for bit, what dybit_quantize_conv2d gives for each layer.
+ * Together they give, bit for bit, what dybit_quantize_conv2d (with Q set: dybit_quantize_conv2d_requant) gives for
+ * each layer.
  * DYBIT_ERR_UNSUPPORTED (nothing launched) when a layer's lowering is not one whose quantize launch also writes the
  * expanded operands (channels neither a multiple of 16 nor at most 4 with one-byte elements): use
  * dybit_quantize_conv2d for such a layer. */
@@ -249,10 +250,16 @@ typedef struct {
     dybit_fmt fw;
     const float *scale_w;
     int64_t ldw_bytes;
-    float *Y;                    /* [dev] n*oh*ow*k floats */
-    int32_t *Y_raw;              /* [dev] or NULL */
+    float *Y;                    /* [dev] n*oh*ow*k floats (unused when Q is set) */
+    int32_t *Y_raw;              /* [dev] or NULL (must be NULL when Q is set) */
     void *ws;                    /* [dev] dybit_conv2d_workspace_bytes(...) bytes of this layer's own */
     size_t ws_bytes;
+    /* Q != NULL: the layer leaves through the re-quantizing epilogue instead, as in dybit_conv2d_requant */
+    void *Q;                     /* [dev] packed output codes, or NULL for the fp32 output Y */
+    dybit_fmt fq;
+    const float *scale_q;        /* [dev] {scale, 1/scale} of the output tensor */
+    const float *bias;           /* [dev] k floats or NULL */
+    int relu;
 } dybit_conv_layer;
 
 dybit_status dybit_quantize_expand_layers(const dybit_conv_layer *layers, int n_layers, void *stream);

@@ -46,7 +46,8 @@ class _CConvLayer(C.Structure):
     _fields_ = [("desc", _CConvDesc), ("X", C.c_void_p), ("fx", _CFmt), ("scale_x", C.c_void_p),
                 ("scale_x_out", C.c_void_p), ("X_packed", C.c_void_p), ("W", C.c_void_p), ("fw", _CFmt),
                 ("scale_w", C.c_void_p), ("ldw_bytes", C.c_int64), ("Y", C.c_void_p), ("Y_raw", C.c_void_p),
-                ("ws", C.c_void_p), ("ws_bytes", C.c_size_t)]
+                ("ws", C.c_void_p), ("ws_bytes", C.c_size_t), ("Q", C.c_void_p), ("fq", _CFmt),
+                ("scale_q", C.c_void_p), ("bias", C.c_void_p), ("relu", C.c_int)]
 
 
 class ConvDesc(NamedTuple):
@@ -517,21 +518,30 @@ class ConvLayers:
     """Arguments of dybit_quantize_conv2d for several independent layers, marshalled once into the C array that
     dybit_quantize_expand_layers / dybit_conv2d_prepared take.  Each entry of `layers` is a dict with the keyword
     arguments of dybit_quantize_conv2d (desc, X, fx, W, fw, scale_w and optionally scale_x, scale_out, packed, Y,
-    want_raw, ws); missing outputs and workspaces are allocated here, one workspace per layer."""
+    want_raw, ws) or, with fq and scale_q given, of dybit_quantize_conv2d_requant (relu, bias, Q): that layer then
+    leaves as packed codes in self.Q[i] instead of fp32 in self.Y[i].  Missing outputs and workspaces are allocated
+    here, one workspace per layer."""
 
     def __init__(self, layers):
         self.n = len(layers)
         self.array = (_CConvLayer * self.n)()
-        self.Y, self.raw, self.packed, self.scale, self._keep = [], [], [], [], []
+        self.Y, self.raw, self.packed, self.scale, self.Q, self._keep = [], [], [], [], [], []
         for i, a in enumerate(layers):
             desc, X, fx, W, fw = a["desc"], _dev_f32(a["X"], "X"), a["fx"], a["W"], a["fw"]
             if X.numel() != desc.n * desc.h * desc.w * desc.c:
                 raise ValueError("X does not match the descriptor")
             oh, ow = dybit_conv2d_out_hw(desc)
-            Y = a.get("Y")
-            if Y is None:
-                Y = torch.empty((desc.n, oh, ow, desc.k), dtype=torch.float32, device=X.device)
-            raw = torch.empty(Y.shape, dtype=torch.int32, device=X.device) if a.get("want_raw") else None
+            requant = a.get("fq") is not None
+            Y, Q, raw = a.get("Y"), a.get("Q"), None
+            if requant:
+                if Q is None:
+                    Q = torch.zeros(dybit_packed_bytes(desc.n * oh * ow * desc.k, a["fq"][0]), dtype=torch.uint8, device=X.device)
+                Y = None
+            else:
+                if Y is None:
+                    Y = torch.empty((desc.n, oh, ow, desc.k), dtype=torch.float32, device=X.device)
+                if a.get("want_raw"):
+                    raw = torch.empty(Y.shape, dtype=torch.int32, device=X.device)
             packed = a.get("packed")
             if packed is None:
                 packed = torch.empty(dybit_packed_bytes(X.numel(), fx[0]), dtype=torch.uint8, device=X.device)
@@ -549,6 +559,12 @@ class ConvLayers:
             c.scale_x_out, c.X_packed = addr(scale_out), addr(packed)
             c.W, c.fw, c.scale_w, c.ldw_bytes = addr(W), _fmt(fw), addr(a["scale_w"]), W.stride(0)
             c.Y, c.Y_raw, c.ws, c.ws_bytes = addr(Y), addr(raw), wp.value, wn
+            if requant:
+                bias = a.get("bias")
+                c.Q, c.fq, c.scale_q, c.relu = addr(Q), _fmt(a["fq"]), addr(a["scale_q"]), int(bool(a.get("relu")))
+                c.bias = None if bias is None else _bias_ptr(bias, desc.k).value
+                self._keep.append((a["scale_q"], bias))
+            self.Q.append(Q)
             self.Y.append(Y)
             self.raw.append(raw)
             self.packed.append(packed)
@@ -562,9 +578,10 @@ def dybit_quantize_expand_layers(layers: ConvLayers, stream=None):
 
 
 def dybit_conv2d_prepared(layers: ConvLayers, i: int, stream=None):
-    """The tensor-core part of layer i, after dybit_quantize_expand_layers.  Returns (Y, Y_raw or None)."""
+    """The tensor-core part of layer i, after dybit_quantize_expand_layers.  Returns (Y, Y_raw or None), or (Q, None)
+    for a layer with the re-quantizing epilogue."""
     _check(lib.dybit_conv2d_prepared(C.byref(layers.array[i]), _stream(stream)), "dybit_conv2d_prepared")
-    return layers.Y[i], layers.raw[i]
+    return (layers.Y[i] if layers.Q[i] is None else layers.Q[i]), layers.raw[i]
 
 
 def dybit_depthwise_conv2d(desc: ConvDesc, X: torch.Tensor, fx, scale_x: torch.Tensor, W: torch.Tensor, fw,

@@ -2710,8 +2710,10 @@ dybit_status dybit_quantize_expand_layers(const dybit_conv_layer *layers, int n_
         const dybit_conv_layer &l = layers[i];
         if (l.scale_x_out == nullptr || l.X_packed == nullptr) return DYBIT_ERR_INVALID_ARG;
         const dybit::QuantInput xq = {l.X, l.scale_x};
-        const dybit_status st = dybit::conv_impl(&l.desc, l.X_packed, l.fx, l.scale_x_out, l.W, l.fw, l.scale_w, l.ldw_bytes, l.Y,
-                                                 l.Y_raw, nullptr, l.ws, l.ws_bytes, stream, &xq, &col, false);
+        const dybit::RequantSpec rq = {l.fq, l.scale_q, l.bias, l.relu ? 1 : 0, l.Q, (int64_t)l.desc.k * l.fq.bits / 8};
+        const dybit_status st = dybit::conv_impl(&l.desc, l.X_packed, l.fx, l.scale_x_out, l.W, l.fw, l.scale_w, l.ldw_bytes,
+                                                 l.Q ? nullptr : l.Y, l.Q ? nullptr : l.Y_raw, l.Q ? &rq : nullptr, l.ws,
+                                                 l.ws_bytes, stream, &xq, &col, false);
         if (st != DYBIT_OK) return st;
     }
     return col.launch_all(static_cast<cudaStream_t>(stream));
@@ -2721,8 +2723,10 @@ dybit_status dybit_conv2d_prepared(const dybit_conv_layer *layer, void *stream) 
     if (layer == nullptr || layer->scale_x_out == nullptr || layer->X_packed == nullptr) return DYBIT_ERR_INVALID_ARG;
     const dybit_conv_layer &l = *layer;
     const dybit::QuantInput xq = {l.X, l.scale_x};
-    return dybit::conv_impl(&l.desc, l.X_packed, l.fx, l.scale_x_out, l.W, l.fw, l.scale_w, l.ldw_bytes, l.Y, l.Y_raw, nullptr,
-                            l.ws, l.ws_bytes, stream, &xq, nullptr, true);
+    const dybit::RequantSpec rq = {l.fq, l.scale_q, l.bias, l.relu ? 1 : 0, l.Q, (int64_t)l.desc.k * l.fq.bits / 8};
+    if (l.Q != nullptr && l.Y_raw != nullptr) return DYBIT_ERR_INVALID_ARG;
+    return dybit::conv_impl(&l.desc, l.X_packed, l.fx, l.scale_x_out, l.W, l.fw, l.scale_w, l.ldw_bytes, l.Q ? nullptr : l.Y,
+                            l.Q ? nullptr : l.Y_raw, l.Q ? &rq : nullptr, l.ws, l.ws_bytes, stream, &xq, nullptr, true);
 }
 
 dybit_status dybit_gemm_requant(int64_t M, int64_t N, int64_t K, const void *A, dybit_fmt fa, const float *scale_a,

@@ -222,6 +222,48 @@ def test_quantize_conv_requant_one_call(layer):
     assert torch.equal(Q, Q2)
 
 
+# the same epilogue on layers that went through the folded launches (dybit_quantize_expand_layers, then
+# dybit_conv2d_prepared with Q set): one layer leaves as codes with bias + ReLU, one as codes without, one as fp32
+def test_layers_with_the_requant_epilogue():
+    fx, fw, fq = (4, 0), (4, 1), (4, 0)
+    shapes = [wl.ConvLayer("c64_3x3", 4, 28, 28, 64, 64, 3, 3, 1, 1), wl.ConvLayer("c128_1x1", 3, 14, 14, 128, 256, 1, 1, 1, 0),
+              wl.ConvLayer("c3_stem", 2, 32, 32, 3, 64, 7, 7, 2, 3)]
+    args, expect = [], []
+    for i, L in enumerate(shapes):
+        x = wl.half_normal((L.n, L.h, L.w, L.c), seed=41 + i)
+        w = wl.kaiming_normal(L.k, L.r, L.s, L.c, seed=51 + i)
+        pw, sw = dy.dybit_quantize_pack_2d(w.reshape(L.k, -1).to(DEV), fw)
+        spx = orc.absmax_scale(x.numpy(), 4, False)
+        spw = orc.absmax_scale(w.numpy(), 4, True)
+        _, y = orc.conv2d(orc.quantize(x.numpy(), 4, False, spx[1]), fx, spx[0], orc.quantize(w.numpy(), 4, True, spw[1]), fw,
+                          spw[0], stride=L.stride, pad=L.pad)
+        a = dict(desc=dy.ConvDesc(L.n, L.h, L.w, L.c, L.k, L.r, L.s, L.stride, L.pad, 1), X=x.to(DEV), fx=fx, W=pw, fw=fw,
+                 scale_w=sw)
+        if i == 0:
+            bias = wl.normal((L.k,), seed=61, std=float(np.abs(y).mean())).numpy().astype(np.float32)
+            y = np.maximum((y.astype(np.float32) + bias.reshape(1, 1, 1, -1)).astype(np.float32), 0)
+            a.update(bias=torch.from_numpy(bias).to(DEV), relu=True)
+        if i < 2:
+            sq = orc.absmax_scale(np.abs(y) * 0.9, 4, False)
+            a.update(fq=fq, scale_q=torch.tensor([float(sq[0]), float(sq[1])], dtype=torch.float32, device=DEV))
+            expect.append(orc.pack(orc.quantize(y if i == 0 else y.astype(np.float32), 4, False, sq[1]), 4))
+        else:
+            expect.append(y)
+        args.append(a)
+    layers = dy.ConvLayers(args)
+    dy.dybit_quantize_expand_layers(layers)
+    outs = [dy.dybit_conv2d_prepared(layers, i)[0] for i in range(len(shapes))]
+    torch.cuda.synchronize()
+    assert dy.dybit_last_device_status() == (0, 0)
+    for i, L in enumerate(shapes):
+        assert np.array_equal(outs[i].cpu().numpy(), expect[i]), L.name
+    # and bit for bit the one-layer call
+    a = args[0]
+    Q1, _, _ = dy.dybit_quantize_conv2d_requant(a["desc"], a["X"], fx, a["W"], fw, a["scale_w"], fq, a["scale_q"], relu=True,
+                                                bias=a["bias"])
+    assert torch.equal(Q1, outs[0])
+
+
 # products large enough for the CTA-pair kernel: its epilogue re-quantizes too (bias, ReLU, ragged last tiles)
 @pytest.mark.parametrize("M,N,K,fq,relu,with_bias", [(2304, 2304, 256, (4, 0), True, False),
                                                       (2400, 2344, 200, (8, 1), False, True),
