@@ -567,15 +567,35 @@ __device__ __forceinline__ void quantize_expand_body(const QeArgs &a, const Elem
                         // pixels at the chunk's ends take the pixel-by-pixel route.  Pixel counts fit 32 bits (host check).
                         const unsigned q_lo = (unsigned)((p_lo + 1) >> 1), q_hi = (unsigned)(p_hi >> 1);
                         const unsigned hw = (unsigned)(pl.H * pl.W), half_w = (unsigned)(pl.W >> 1);
-                        for (unsigned q = q_lo + lane; q < q_hi; q += 32) {
-                            const unsigned px = 2u * q;
-                            const unsigned img = px / hw, rem = px - img * hw;
-                            const unsigned h = rem / (unsigned)pl.W, w = rem - h * (unsigned)pl.W;
+                        // image coordinates of this lane's first pair by division, of its later pairs (64 pixels
+                        // further on each) by stepping; the pair's bytes come out of shared memory as three aligned
+                        // words and two funnel shifts
+                        unsigned img = 0, h = 0, w = 0;
+                        {
+                            const unsigned px0 = 2u * (q_lo + lane);
+                            img = px0 / hw;
+                            const unsigned rem = px0 - img * hw;
+                            h = rem / (unsigned)pl.W;
+                            w = rem - h * (unsigned)pl.W;
+                        }
+                        const unsigned *sw32 = reinterpret_cast<const unsigned *>(sb);
+                        int o0 = (int)((int64_t)(2u * (q_lo + lane)) * pix_c - c0);
+                        for (unsigned q = q_lo + lane; q < q_hi; q += 32, o0 += 64 * pix_c, w += 64) {
+                            while (w >= (unsigned)pl.W) {
+                                w -= (unsigned)pl.W;
+                                if (++h == (unsigned)pl.H) {
+                                    h = 0;
+                                    ++img;
+                                }
+                            }
                             uint8_t *row = xe + (((int64_t)(img * (unsigned)pl.Hs + (h >> 1)) * pl.P) << 4);
                             uint8_t *blk = row + (((w >> 1) + pl.padL) << 4);
-                            const int o0 = (int)((int64_t)px * pix_c - c0);
-                            unsigned long long v = 0;
-                            for (int b = 0; b < 2 * pix_c; ++b) v |= (unsigned long long)sb[o0 + b] << (8 * b);
+                            const int wi = o0 >> 2;
+                            const unsigned sh = (unsigned)(o0 & 3) * 8u;
+                            const unsigned w0 = sw32[wi], w1 = sw32[min(wi + 1, kChunkCodes / 4 - 1)],
+                                           w2 = sw32[min(wi + 2, kChunkCodes / 4 - 1)];
+                            const unsigned long long v = (unsigned long long)__funnelshift_r(w0, w1, sh) |
+                                                         ((unsigned long long)__funnelshift_r(w1, w2, sh) << 32);
                             const unsigned dy = h & 1u;
                             uint8_t *dst = blk + dy * 2 * pix_c;
                             if (pix_c == 3) {
