@@ -289,18 +289,22 @@ __device__ __forceinline__ void pack32(const unsigned (&cw)[8], unsigned (&out)[
         out[1] = __byte_perm(__byte_perm(b[4], b[5], 0x0040), __byte_perm(b[6], b[7], 0x0040), 0x5410);
         return;
     }
-    unsigned long long acc = 0;
-    int nb = 0, w = 0;
+    // other widths: the four codes of a word shrink to 4 * BITS bits in two steps (pairs inside each 16-bit half,
+    // then the halves), and the eight pieces are laid end to end; every shift is a compile-time constant
+    constexpr unsigned kPair = (1u << (2 * BITS)) - 1u;
+    unsigned q[8];
 #pragma unroll
-    for (int i = 0; i < 32; ++i) {
-        const unsigned code = (cw[i >> 2] >> ((i & 3) * 8)) & 0xffu;
-        acc |= (unsigned long long)code << nb;
-        nb += BITS;
-        if (nb >= 32) {
-            out[w++] = (unsigned)acc;
-            acc >>= 32;
-            nb -= 32;
-        }
+    for (int i = 0; i < 8; ++i) {
+        const unsigned u = (cw[i] & 0x00ff00ffu) | ((cw[i] >> (8 - BITS)) & ((((1u << BITS) - 1u) << BITS) * 0x00010001u));
+        q[i] = (u & kPair) | ((u >> (16 - 2 * BITS)) & (kPair << (2 * BITS)));
+    }
+#pragma unroll
+    for (int i = 0; i < BITS; ++i) out[i] = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int pos = i * 4 * BITS, word = pos >> 5, off = pos & 31;
+        out[word] |= q[i] << off;
+        if (off + 4 * BITS > 32) out[word + 1] |= q[i] >> (32 - off);
     }
 }
 
