@@ -178,23 +178,49 @@ __device__ __forceinline__ unsigned expand4_lookup(unsigned sel, const unsigned 
 __global__ void __launch_bounds__(256) expand4_kernel(const Expand4Job j0, const Expand4Job j1, int64_t vecs0) {
     pdl_enter();
     const int64_t total = vecs0 + j1.rows * j1.vecs_per_row;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
-        const bool first = i < vecs0;
-        const Expand4Job &j = first ? j0 : j1;
-        const int64_t v = first ? i : i - vecs0;
-        const int64_t row = v / j.vecs_per_row, col = v - row * j.vecs_per_row;
-        const uint4 w = __ldg(reinterpret_cast<const uint4 *>(j.packed + row * j.in_stride) + col);
-        const unsigned t[4] = {j.tab[0], j.tab[1], j.tab[2], j.tab[3]};
-        const bool ng = j.neg_high != 0;
-        uint4 o0, o1;
-        o0.x = expand4_lookup(w.x, t, ng); o0.y = expand4_lookup(w.x >> 16, t, ng);
-        o0.z = expand4_lookup(w.y, t, ng); o0.w = expand4_lookup(w.y >> 16, t, ng);
-        o1.x = expand4_lookup(w.z, t, ng); o1.y = expand4_lookup(w.z >> 16, t, ng);
-        o1.z = expand4_lookup(w.w, t, ng); o1.w = expand4_lookup(w.w >> 16, t, ng);
-        uint4 *dst = reinterpret_cast<uint4 *>(j.out + row * j.out_stride + col * 32);
-        if (!DYBIT_CHECK(row < j.rows && col * 32 + 32 <= (j.rows > 1 ? j.out_stride : j.vecs_per_row * 32), 0x23)) continue;
-        dst[0] = o0;
-        dst[1] = o1;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    // two 16-byte vectors of codes in flight per thread and round trip
+    for (int64_t i0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i0 < total; i0 += 2 * stride) {
+        uint4 w[2];
+        uint4 *dst[2];
+        bool ng[2];
+        unsigned t[2][4];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const int64_t i = i0 + u * stride;
+            dst[u] = nullptr;
+            if (i >= total) continue;
+            const bool first = i < vecs0;
+            const Expand4Job &j = first ? j0 : j1;
+            const int64_t v = first ? i : i - vecs0;
+            // (rows of up to 2^31 vectors: one 64-bit division only when the index does not fit 32 bits)
+            int64_t row, col;
+            if (v < ((int64_t)1 << 32) && j.vecs_per_row < ((int64_t)1 << 32)) {
+                const unsigned r32 = (unsigned)v / (unsigned)j.vecs_per_row;
+                row = r32;
+                col = (int64_t)((unsigned)v - r32 * (unsigned)j.vecs_per_row);
+            } else {
+                row = v / j.vecs_per_row;
+                col = v - row * j.vecs_per_row;
+            }
+            w[u] = __ldg(reinterpret_cast<const uint4 *>(j.packed + row * j.in_stride) + col);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) t[u][k] = j.tab[k];
+            ng[u] = j.neg_high != 0;
+            if (DYBIT_CHECK(row < j.rows && col * 32 + 32 <= (j.rows > 1 ? j.out_stride : j.vecs_per_row * 32), 0x23))
+                dst[u] = reinterpret_cast<uint4 *>(j.out + row * j.out_stride + col * 32);
+        }
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            if (dst[u] == nullptr) continue;
+            uint4 o0, o1;
+            o0.x = expand4_lookup(w[u].x, t[u], ng[u]); o0.y = expand4_lookup(w[u].x >> 16, t[u], ng[u]);
+            o0.z = expand4_lookup(w[u].y, t[u], ng[u]); o0.w = expand4_lookup(w[u].y >> 16, t[u], ng[u]);
+            o1.x = expand4_lookup(w[u].z, t[u], ng[u]); o1.y = expand4_lookup(w[u].z >> 16, t[u], ng[u]);
+            o1.z = expand4_lookup(w[u].w, t[u], ng[u]); o1.w = expand4_lookup(w[u].w >> 16, t[u], ng[u]);
+            dst[u][0] = o0;
+            dst[u][1] = o1;
+        }
     }
 }
 
