@@ -1271,6 +1271,7 @@ struct GemmParams {
     const float *bias;        // requant only: one fp32 per output column, or null
     unsigned long long *clock; // profiling: {min start after the dependency wait, max end} in %globaltimer ns, or null
     int bmt;                  // batched GEMM: M tiles per batch entry (0: not batched); M is then one entry's rows
+    int split_from;           // pair kernel: tiles from this index on are worked on as two 256 x 128 halves (see pair_item)
     int64_t c_bstride;        // batched GEMM: elements between consecutive entries of C / C_raw
 };
 

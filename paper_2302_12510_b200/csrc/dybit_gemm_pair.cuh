@@ -19,6 +19,21 @@ constexpr int kPairBStage = (kPairBN / 2) * kBKBytes;
 constexpr int kPairCStage = kBM * 128;
 constexpr int kPairSmemBytes = kPairStages * (kPairAStage + kPairBStage) + 2 * kPairCStage + 512 + 1024;
 
+// Work items of the pair kernel.  Tiles [0, split_from) are one item each; every later tile is two items, its left and
+// its right 256 x 128 half.  The host splits the tiles of a last, less than half-full wave: a half costs 0.61 of a
+// whole tile (an N = 128 instruction takes 78 clocks where an N = 256 one takes 128), so the wave ends sooner.
+__device__ __forceinline__ void pair_item(int item, const GemmParams &p, int &m_blk, int &n_blk, int &n_off, int &width) {
+    int tile = item, half = 0;
+    width = kPairBN;
+    if (item >= p.split_from) {
+        tile = p.split_from + ((item - p.split_from) >> 1);
+        half = (item - p.split_from) & 1;
+        width = kPairBN / 2;
+    }
+    tile_coords(tile, p.m_tiles, p.n_tiles, m_blk, n_blk);
+    n_off = half * (kPairBN / 2);
+}
+
 // p.m_tiles counts 256-row blocks here; p.n_tiles counts 256-column blocks.
 template <Kind KIND>
 __global__ void __launch_bounds__(320, 1)
@@ -44,7 +59,8 @@ dybit_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
     const uint32_t rank = cluster_ctarank();     // 0 = leader
     const int pair = blockIdx.x >> 1;
     const int num_pairs = gridDim.x >> 1;
-    const int total_tiles = p.m_tiles * p.n_tiles;
+    const int whole_tiles = p.m_tiles * p.n_tiles;
+    const int total_tiles = whole_tiles + (whole_tiles - p.split_from);      // work items: a split tile counts twice
     constexpr uint32_t kTmemCols = 2 * BN;       // two accumulators of 256 columns: all of TMEM
 
     if (threadIdx.x == 0) {
@@ -80,10 +96,11 @@ dybit_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
             uint32_t it = 0;
             bool ok = true;
             for (int tile = pair; tile < total_tiles && ok; tile += num_pairs) {
-                int m_blk, n_blk;
-                tile_coords(tile, p.m_tiles, p.n_tiles, m_blk, n_blk);
+                int m_blk, n_blk, n_off, width;
+                pair_item(tile, p, m_blk, n_blk, n_off, width);
                 const int a_row = m_blk * 2 * kBM + (int)rank * kBM;
-                const int b_row = n_blk * BN + (int)rank * (BN / 2);
+                // (a half item still loads 128 rows of B per CTA; the instruction reads the first 64 of each)
+                const int b_row = n_blk * BN + n_off + (int)rank * (width / 2);
                 for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
                     const int s = it % kStages;
                     const uint32_t ph = (it / kStages) & 1u;
@@ -104,10 +121,12 @@ dybit_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
         if (lane == 0 && rank == 0) {
             constexpr uint32_t kCFormat = (KIND == Kind::I8) ? 2u : 1u;
             constexpr uint32_t kABFormat = (KIND == Kind::F8F6F4) ? 0u : 1u;
-            constexpr uint32_t idesc = umma_idesc(kCFormat, kABFormat, 2 * kBM, BN);
+            constexpr uint32_t idesc_whole = umma_idesc(kCFormat, kABFormat, 2 * kBM, BN);
+            constexpr uint32_t idesc_half = umma_idesc(kCFormat, kABFormat, 2 * kBM, BN / 2);
             uint32_t it = 0, lt = 0;
             bool ok = true;
             for (int tile = pair; tile < total_tiles && ok; tile += num_pairs, ++lt) {
+                const uint32_t idesc = tile >= p.split_from ? idesc_half : idesc_whole;
                 const uint32_t as = lt & 1u, aph = (lt >> 1) & 1u;
                 if (!wait_bounded(&acc_empty[as], aph ^ 1u, abort_flag, 2)) { ok = false; break; }
                 tc_fence_after_sync();
@@ -139,8 +158,8 @@ dybit_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
         const float inv_q = p.Q ? __ldg(p.scale_q + 1) : 1.0f;
         uint32_t lt = 0;
         for (int tile = pair; tile < total_tiles; tile += num_pairs, ++lt) {
-            int m_blk, n_blk;
-            tile_coords(tile, p.m_tiles, p.n_tiles, m_blk, n_blk);
+            int m_blk, n_blk, n_off, width;
+            pair_item(tile, p, m_blk, n_blk, n_off, width);
             const uint32_t as = lt & 1u, aph = (lt >> 1) & 1u;
             // one outcome for the group's 128 threads, which meet in named barriers below
             const bool ok = named_barrier_and(1 + group, 128, wait_bounded(&acc_full[as], aph, abort_flag, 4));
@@ -150,8 +169,8 @@ dybit_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
             const uint32_t taddr = tmem_base + as * BN + ((uint32_t)(q * 32) << 16);
             const bool last_tile = tile + num_pairs >= total_tiles;
 #pragma unroll 1
-            for (int cc = group; cc < BN / 32; cc += kEpilogueWarps / 4) {
-                const int col0 = n_blk * BN + cc * 32;
+            for (int cc = group; cc < width / 32; cc += kEpilogueWarps / 4) {
+                const int col0 = n_blk * BN + n_off + cc * 32;
                 if (col0 >= p.N || row0 >= p.M) break;
                 uint32_t r[32];
                 tmem_ld_32x32(taddr + cc * 32, r);
@@ -260,6 +279,9 @@ static dybit_status launch_gemm_pair_kind(const CUtensorMap &ta, const CUtensorM
     const int tiles = p.m_tiles * p.n_tiles;
     const int resident = max_clusters[dev];
     const int pairs = tiles < resident ? tiles : resident;
+    // a last wave that fills at most half of the pairs is worked on as halves (see pair_item)
+    const int rest = tiles % pairs;
+    p.split_from = (rest > 0 && 2 * rest <= pairs) ? tiles - rest : tiles;
     cfg.gridDim = dim3((unsigned)(2 * pairs));
     cfg.numAttrs = 2;
     ProfileEvents ev = profile_events();
