@@ -47,11 +47,12 @@ FMT_A = (4, 0)      # post-ReLU activations: unsigned 4-bit
 NOMINAL = {"hbm_gbs": 7700.0, "bf16_tflops": 2250.0, "int8_tops": 4500.0, "fp8_tflops": 4500.0}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, copied from the ncu summaries under profiles/ (bench.py cannot
 # read hardware counters itself); an entry is None while the kernel has changed since its counters were taken
-NCU_TRAFFIC = {"gemm_8192": 4 * (36588800 + 18511872), "quantize_2p26_per_element": (268458496 + 8048640) / float(1 << 26),
+NCU_TRAFFIC = {"gemm_8192": (147033344 + 111412480) * (8192.0 / 6144.0) ** 2, "quantize_2p26_per_element": (268458496 + 8048640) / float(1 << 26),
                "conv_step": (79310336 + 42336512) / 21.0}
 NCU_TRAFFIC_HOW = {
-    "gemm_8192": "profiles/dybit_gemm_pair_kernel_i8_square4096.txt: one launch at M=N=K=4096 (a capture small enough to end "
-                 "by itself), x 4 for 8192^3 (operand and output bytes both grow 4 x)",
+    "gemm_8192": "profiles/dybit_gemm_pair_kernel_i8_square6144_and_4096.txt: one launch at M=N=K=6144 (a capture small "
+                 "enough to end by itself, whole tiles only as at 8192^3), x (8192 / 6144)^2 for 8192^3 (operand and output "
+                 "bytes both grow with the square of the size)",
     "quantize_2p26_per_element": "profiles/quantize_pack_kernel_4bit_signed_2p26.txt: bytes per element of one launch at "
                                  "2^26 elements x the elements of this launch (streaming kernel: traffic is proportional)",
     "conv_step": "profiles/dybit_gemm_kernel_conv_resnet18_b32_dram_traffic.txt: mean over the 21 conv launches of one step",
