@@ -201,16 +201,10 @@ class LayerwiseStep:
         dy = self.dy
         profiling = events is not None or clocks is not None
         if self.fold and not self.two_calls and only is None and not profiling and not serial:
-            # dybit_quantize_expand_layers: one max-abs launch and one quantize + expand launch for all layers, on
-            # the calling stream; then one tensor-core launch per layer, round-robin on the side streams
-            cur = torch.cuda.current_stream()
+            # dybit_quantize_expand_layers: one max-abs launch and one quantize + expand launch for all layers; then
+            # dybit_conv2d_prepared_layers: the tensor-core work, layers of one kernel configuration sharing launches
             dy.dybit_quantize_expand_layers(self.folded)
-            for st in self.side:
-                st.wait_stream(cur)
-            for j in range(len(self.layers)):
-                dy.dybit_conv2d_prepared(self.folded, j, stream=self.side[j % self.n_streams] if self.side else None)
-            for st in self.side:
-                cur.wait_stream(st)
+            dy.dybit_conv2d_prepared_layers(self.folded)
             return
         if self.n_streams > 1 and only is None and not profiling and not serial:
             cur = torch.cuda.current_stream()
@@ -251,14 +245,8 @@ class LayerwiseStep:
                                                     fw=self.fw[i], scale_w=self.sw[i], packed=self.px[i], scale_out=self.sx[i],
                                                     fq=self.fq, scale_q=self.sq[i], relu=True, Q=self.q[i])
                                                for i in range(len(self.layers))])
-            cur = torch.cuda.current_stream()
             dy.dybit_quantize_expand_layers(self.folded_q)
-            for st in self.side:
-                st.wait_stream(cur)
-            for j in range(len(self.layers)):
-                dy.dybit_conv2d_prepared(self.folded_q, j, stream=self.side[j % self.n_streams] if self.side else None)
-            for st in self.side:
-                cur.wait_stream(st)
+            dy.dybit_conv2d_prepared_layers(self.folded_q)
             return
 
         def layer(i, ws):
@@ -1151,10 +1139,10 @@ def main():
         "config": {"workload": workload_name(args.batch),
                    "parallelism": "replicas only" if world > 1 else "single GPU",
                    "launch": ("dybit_quantize_expand_layers for the 21 independent layers (one max-abs launch, one quantize + "
-                              "expand launch), then one dybit_conv2d_prepared call per layer round-robin on %d streams that "
-                              "fork from and join the step's stream; " if work.fold else
+                              "expand launch), then dybit_conv2d_prepared_layers (the 21 tensor-core problems in shared "
+                              "launches, one per kernel configuration), all on one stream; " if work.fold else
                               "one dybit_quantize_conv2d call per layer; the 21 independent layers are issued round-robin on "
-                              "%d streams (one workspace each) that fork from and join the step's stream; ") % work.n_streams
+                              "%d streams (one workspace each) that fork from and join the step's stream; " % work.n_streams)
                              + "one step captured once as a CUDA graph, timed region = K replays",
                    "streams": work.n_streams,
                    "l2": "per-step footprint (fp32 inputs %.0f MB + fp32 outputs %.0f MB) exceeds the 126 MB L2"
@@ -1165,7 +1153,7 @@ def main():
     if ms_per_layer_calls is not None:
         result["per_layer_call_step"] = {
             "what": "the same step as one dybit_quantize_conv2d call per layer (max-abs, quantize + expand and the "
-                    "tensor-core kernel launched layer by layer) on the same streams",
+                    "tensor-core kernel launched layer by layer), round-robin on %d streams" % work.n_streams,
             "ms_per_step": ms_per_layer_calls, "value": whole_job_tops(work.macs, world, ms_per_layer_calls), "unit": "TOPS"}
     if args.step_only:
         result["roofline"] = roofline_conv

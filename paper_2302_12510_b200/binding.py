@@ -23,7 +23,7 @@ __all__ = [
     "dybit_launch_count", "dybit_set_conv_lowering", "dybit_set_gemm_decode", "dybit_selftest_wait_timeout", "dybit_profile_next_gemm", "dybit_profile_next_gemm_clock", "dybit_gemm_static_ws", "STATIC_WS_BYTES",
     "dybit_gemm_requant", "dybit_conv2d_requant", "dybit_depthwise_conv2d", "dybit_gemm_batched",
     "dybit_quantize_conv2d", "dybit_quantize_conv2d_requant",
-    "ConvLayers", "dybit_quantize_expand_layers", "dybit_conv2d_prepared",
+    "ConvLayers", "dybit_quantize_expand_layers", "dybit_conv2d_prepared", "dybit_conv2d_prepared_layers",
     "dybit_gemm_batched_workspace_bytes", "dybit_rmse", "dybit_rmse_sweep", "dybit_fake_quant", "dybit_fake_quant_backward",
     "dybit_search_bitwidths",
 ]
@@ -121,6 +121,7 @@ def _load() -> C.CDLL:
                                           vp, vp, vp, sz, vp]
     lib.dybit_quantize_expand_layers.argtypes = [C.POINTER(_CConvLayer), i32, vp]
     lib.dybit_conv2d_prepared.argtypes = [C.POINTER(_CConvLayer), vp]
+    lib.dybit_conv2d_prepared_layers.argtypes = [C.POINTER(_CConvLayer), i32, vp]
     lib.dybit_gemm_batched_workspace_bytes.restype = sz
     lib.dybit_gemm_batched_workspace_bytes.argtypes = [i64, i64, i64, i64, _CFmt, _CFmt]
     lib.dybit_gemm_batched.argtypes = [i64, i64, i64, i64, vp, _CFmt, vp, i64, i64, vp, _CFmt, vp, i64, i64,
@@ -582,6 +583,11 @@ def dybit_conv2d_prepared(layers: ConvLayers, i: int, stream=None):
     for a layer with the re-quantizing epilogue."""
     _check(lib.dybit_conv2d_prepared(C.byref(layers.array[i]), _stream(stream)), "dybit_conv2d_prepared")
     return (layers.Y[i] if layers.Q[i] is None else layers.Q[i]), layers.raw[i]
+
+
+def dybit_conv2d_prepared_layers(layers: ConvLayers, stream=None):
+    """The tensor-core part of all layers on one stream, layers of one kernel configuration sharing launches."""
+    _check(lib.dybit_conv2d_prepared_layers(layers.array, layers.n, _stream(stream)), "dybit_conv2d_prepared_layers")
 
 
 def dybit_depthwise_conv2d(desc: ConvDesc, X: torch.Tensor, fx, scale_x: torch.Tensor, W: torch.Tensor, fw,

@@ -90,10 +90,11 @@ __device__ __forceinline__ int halo_row(const HaloParams &hp, const HaloTile &t,
 template <int BN, int SWB>
 constexpr int halo_ctas_per_sm() { return (BN == 64 && SWB == 64) ? 2 : 1; }
 
+// CTA `bid` of the `nblk` CTAs that work on the layer (tensor maps and parameters live in the kernel's parameter
+// space, whichever kernel below passes them).
 template <Kind KIND, int BN, int SWB>
-__global__ void __launch_bounds__(320, halo_ctas_per_sm<BN, SWB>())
-dybit_conv_halo_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
-                       const __grid_constant__ CUtensorMap tmap_y, const HaloParams hp) {
+__device__ __forceinline__ void conv_halo_body(const CUtensorMap &tmap_x, const CUtensorMap &tmap_w, const CUtensorMap &tmap_y,
+                                               const HaloParams &hp, const int bid, const int nblk) {
     constexpr int kAStage = kHaloRows * SWB;
     constexpr int kBStage = BN * SWB;
     const GemmParams &p = hp.g;
@@ -155,12 +156,12 @@ dybit_conv_halo_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
             const int ngroups = hp.b_res ? 1 : hp.nb / p.R;
             bool ok = true;
             const uint32_t a_bytes = (uint32_t)(hp.ni * hp.hb * 8 * SWB);
-            if (hp.b_res && (int)blockIdx.x < total_tiles) {
+            if (hp.b_res && bid < total_tiles) {
                 const int blocks = p.R * p.S * hp.cbs;
                 mbar_arrive_expect_tx(panel_full, (uint32_t)blocks * kBStage);
                 for (int j = 0; j < blocks; ++j) tma_load_2d(b_stages + j * kBStage, &tmap_w, j * SWB, 0, panel_full);
             }
-            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+            for (int tile = bid; tile < total_tiles && ok; tile += nblk) {
                 const HaloTile t = halo_tile(hp, tile);
                 for (int cb = 0; cb < hp.cbs && ok; ++cb) {
                     for (int fs = 0; fs < p.S && ok; ++fs) {
@@ -214,8 +215,8 @@ dybit_conv_halo_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
             uint32_t pa = 0, pb = 0, lt = 0;
             uint32_t a_bar = a_full0, a_lo_s = a_lo0, b_bar = b_full0, b_lo_s = b_lo0, g_bar = b_gempty0;
             bool a_ready = false, b_ready = false, acc_ready = false;
-            if (b_res && (int)blockIdx.x < total_tiles) (void)wait_bounded(panel_full, 0u, abort_flag, 6);
-            for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++lt) {
+            if (b_res && bid < total_tiles) (void)wait_bounded(panel_full, 0u, abort_flag, 6);
+            for (int tile = bid; tile < total_tiles; tile += nblk, ++lt) {
                 const uint32_t as = lt & 1u;
                 if (!acc_ready) (void)wait_bounded_addr(acc_empty0 + as * 8, ((lt >> 1) & 1u) ^ 1u, abort_flag, 2);
                 acc_ready = false;
@@ -279,7 +280,7 @@ dybit_conv_halo_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
         const float alpha = (float)((double)__ldg(p.scale_a) * (double)__ldg(p.scale_b) * p.pow2);
         const float inv_q = p.Q ? __ldg(p.scale_q + 1) : 1.0f;
         uint32_t lt = 0;
-        for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++lt) {
+        for (int tile = bid; tile < total_tiles; tile += nblk, ++lt) {
             const HaloTile t = halo_tile(hp, tile);
             const uint32_t as = lt & 1u, aph = (lt >> 1) & 1u;
             // one thread per group polls the accumulator's barrier; the other 127 sleep in the hardware barrier that
@@ -380,6 +381,56 @@ dybit_conv_halo_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, kTmemCols);
     }
+}
+
+template <Kind KIND, int BN, int SWB>
+__global__ void __launch_bounds__(320, halo_ctas_per_sm<BN, SWB>())
+dybit_conv_halo_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
+                       const __grid_constant__ CUtensorMap tmap_y, const HaloParams hp) {
+    conv_halo_body<KIND, BN, SWB>(tmap_x, tmap_w, tmap_y, hp, (int)blockIdx.x, (int)gridDim.x);
+}
+
+// Several layers of one kernel configuration (and one shared-memory size) in ONE launch, as GemmMulti.
+struct HaloMulti {
+    int n;
+    int first_block[kMaxMulti + 1];
+    CUtensorMap tx[kMaxMulti], tw[kMaxMulti], ty[kMaxMulti];
+    HaloParams hp[kMaxMulti];
+};
+static_assert(sizeof(HaloParams) <= sizeof(MultiEntry::extra), "MultiEntry::extra holds a HaloParams");
+
+template <Kind KIND, int BN, int SWB>
+__global__ void __launch_bounds__(320, halo_ctas_per_sm<BN, SWB>()) dybit_conv_halo_multi_kernel(const __grid_constant__ HaloMulti m) {
+    int g = 0;
+    while (g + 1 < m.n && (int)blockIdx.x >= m.first_block[g + 1]) ++g;
+    conv_halo_body<KIND, BN, SWB>(m.tx[g], m.tw[g], m.ty[g], m.hp[g], (int)blockIdx.x - m.first_block[g],
+                                  m.first_block[g + 1] - m.first_block[g]);
+}
+
+template <Kind KIND, int BN, int SWB>
+static dybit_status launch_halo_multi(const MultiEntry *e, int n, cudaStream_t s) {
+    auto kern = dybit_conv_halo_multi_kernel<KIND, BN, SWB>;
+    static std::atomic<bool> configured[64];
+    int dev = 0;
+    DYBIT_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return DYBIT_ERR_CUDA;
+    if (!configured[dev]) {
+        DYBIT_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kHaloSmemBudget));
+        configured[dev] = true;
+    }
+    HaloMulti m;
+    memset(&m, 0, sizeof(m));
+    m.n = n;
+    // (the entries of one launch share per_sm and the shared-memory size: the collector groups by both)
+    multi_shares(e, n, e[0].per_sm * sm_count(), m.first_block);
+    for (int i = 0; i < n; ++i) {
+        m.tx[i] = e[i].ta;
+        m.tw[i] = e[i].tb;
+        m.ty[i] = e[i].tc;
+        memcpy(&m.hp[i], e[i].extra, sizeof(HaloParams));
+    }
+    launch_k(kern, dim3((unsigned)m.first_block[n]), dim3(320u), (size_t)e[0].smem, s, m);
+    return launch_status();
 }
 
 // ------------------------------------------------------------------ host side
@@ -503,6 +554,24 @@ static dybit_status launch_halo_inst(const CUtensorMap &tx, const CUtensorMap &t
     }
     const int grid = tiles < per_sm * sm_count() ? tiles : per_sm * sm_count();
     ProfileEvents ev = profile_events();
+    if constexpr (KIND == Kind::I8) {
+        // inside dybit_conv2d_prepared_layers: gathered, launched together with its like at the end of that call
+        // (a resident weight panel presumes CTAs that take several tiles, which a share of a launch still does)
+        if (gemm_collector() != nullptr && !ev.start && !ev.stop && !ev.clock) {
+            MultiEntry e;
+            memset(&e, 0, sizeof(e));
+            e.ta = tx;
+            e.tb = tw;
+            e.tc = ty;
+            memcpy(e.extra, &hp, sizeof(hp));
+            e.tiles = tiles;
+            e.per_sm = per_sm;
+            e.smem = smem;
+            e.work = (double)tiles * (double)(hp.g.R * hp.g.S * hp.cbs + 8);
+            gemm_collector()->add(launch_halo_multi<KIND, BN, SWB>, e);
+            return DYBIT_OK;
+        }
+    }
     profile_events() = ProfileEvents();
     hp.g.clock = ev.clock;
     if (ev.start) DYBIT_CUDA_TRY(cudaEventRecord(ev.start, s));

@@ -1438,10 +1438,11 @@ __device__ __forceinline__ void tile_coords(int tile, int m_tiles, int n_tiles, 
     n_blk = in_group / gsz;
 }
 
+// CTA `bid` of the `nblk` CTAs that work on the problem (tensor maps and parameters live in the kernel's
+// parameter space, whichever kernel below passes them).
 template <Kind KIND, int BN, int AMODE, int SWB>
-__global__ void __launch_bounds__(AMODE == kAGather4 ? 576 : (AMODE == kAGather ? 448 : 320), 1)
-dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-                  const __grid_constant__ CUtensorMap tmap_c, const GemmParams p) {
+__device__ __forceinline__ void gemm_body(const CUtensorMap &tmap_a, const CUtensorMap &tmap_b, const CUtensorMap &tmap_c,
+                                          const GemmParams &p, const int bid, const int nblk) {
     static_assert((AMODE != kAGather && AMODE != kAGather4) || SWB == 128, "the cp.async gather writes 128-byte rows");
     constexpr bool CONV = AMODE == kAGather || AMODE == kAGather4;          // extra gather warps present
     using L = GemmSmem<BN, SWB>;
@@ -1508,8 +1509,8 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         return o;
     };
     TileOrigin first = {0, 0, 0, 0, 0};
-    if (threadIdx.x == 0 && (int)blockIdx.x < total_tiles) {
-        first = tile_origin(blockIdx.x);
+    if (threadIdx.x == 0 && bid < total_tiles) {
+        first = tile_origin(bid);
         asm volatile("" : "+r"(first.m_blk), "+r"(first.n_blk), "+r"(first.iw), "+r"(first.ih), "+r"(first.img));
     }
     // everything above touched only this CTA's own resources; operands, scales and outputs come next
@@ -1522,14 +1523,14 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             uint32_t it = 0;
             bool ok = true;
             const bool b_res = !CONV && p.b_resident != 0;
-            if (b_res && (int)blockIdx.x < total_tiles) {
+            if (b_res && bid < total_tiles) {
                 // every tile of this CTA multiplies by the same B panel: fetch it once, K block kb into slot kb
                 mbar_arrive_expect_tx(b_full, (uint32_t)p.k_blocks * L::kBStage);
                 for (int kb = 0; kb < p.k_blocks; ++kb)
                     tma_load_2d(b_stages + kb * L::kBStage, &tmap_b, kb * SWB, 0, b_full);
             }
-            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-                const TileOrigin o = tile == (int)blockIdx.x ? first : tile_origin(tile);
+            for (int tile = bid; tile < total_tiles && ok; tile += nblk) {
+                const TileOrigin o = tile == bid ? first : tile_origin(tile);
                 const int m_blk = o.m_blk, n_blk = o.n_blk, iw = o.iw, ih = o.ih, img = o.img;
                 int fr = 0, fs = 0, cb = 0;                     // im2col mode: the running filter tap
                 for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
@@ -1580,8 +1581,8 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             int s = 0;
             uint32_t ph = 0, lt = 0;
             bool ready = false, acc_ready = false;
-            if (b_res && (int)blockIdx.x < total_tiles) (void)wait_bounded(b_full, 0u, abort_flag, 6);
-            for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++lt) {
+            if (b_res && bid < total_tiles) (void)wait_bounded(b_full, 0u, abort_flag, 6);
+            for (int tile = bid; tile < total_tiles; tile += nblk, ++lt) {
                 const uint32_t as = lt & 1u;
                 if (!acc_ready) (void)wait_bounded_addr(acc_empty0 + as * 8, ((lt >> 1) & 1u) ^ 1u, abort_flag, 2);
                 acc_ready = false;
@@ -1621,7 +1622,7 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         const bool vec_ok = ((reinterpret_cast<uintptr_t>(p.C) & 15) == 0) && (p.ldc % 4 == 0) &&
                             (p.C_raw == nullptr || (reinterpret_cast<uintptr_t>(p.C_raw) & 15) == 0);
         uint32_t lt = 0;
-        for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++lt) {
+        for (int tile = bid; tile < total_tiles; tile += nblk, ++lt) {
             int m_blk, n_blk;
             tile_coords(tile, p.m_tiles, p.n_tiles, m_blk, n_blk);
             const uint32_t as = lt & 1u, aph = (lt >> 1) & 1u;
@@ -1672,7 +1673,7 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     // rows / columns beyond C are clipped by the tensor map.  In the CTA's last tile the operand
                     // stages are idle (the commit that published this accumulator followed the last MMA), so every
                     // chunk takes a buffer of its own there and no store waits for the one before it.
-                    const bool last_tile = tile + (int)gridDim.x >= total_tiles;
+                    const bool last_tile = tile + nblk >= total_tiles;
                     uint8_t *stage = last_tile ? a_stages + cc * L::kCStage : c_stages + group * L::kCStage;
                     if (issuer && !last_tile) bulk_wait_group_read<0>();   // the store that last read this buffer is done with it
                     named_barrier(1 + group, 128);
@@ -1787,7 +1788,7 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     for (int w = 0; w < 8; ++w) v[j2][w] = ((mask >> w) & 1u) ? __ldg(src_row + w) : 0u;
                 }
             };
-            int tile = blockIdx.x, kb = 0;
+            int tile = bid, kb = 0;
             if (tile < total_tiles) {
                 RowState cur = row_state(tile);
                 unsigned v[2][8], vn[2][8];
@@ -1796,7 +1797,7 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     int ntile = tile, nkb = kb + 1;
                     if (nkb == p.k_blocks) {
                         nkb = 0;
-                        ntile = tile + gridDim.x;
+                        ntile = tile + nblk;
                     }
                     const bool has_next = ntile < total_tiles;
                     if (has_next) {
@@ -1833,7 +1834,7 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 }
             }
         }
-        for (int tile = blockIdx.x; AMODE != kAGather4 && tile < total_tiles && ok; tile += gridDim.x) {
+        for (int tile = bid; AMODE != kAGather4 && tile < total_tiles && ok; tile += nblk) {
             int m_blk, n_blk;
             tile_coords(tile, p.m_tiles, p.n_tiles, m_blk, n_blk);
             const int m = m_blk * kBM + t;
@@ -1904,6 +1905,31 @@ dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, kTmemCols);
     }
+}
+
+template <Kind KIND, int BN, int AMODE, int SWB>
+__global__ void __launch_bounds__(AMODE == kAGather4 ? 576 : (AMODE == kAGather ? 448 : 320), 1)
+dybit_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                  const __grid_constant__ CUtensorMap tmap_c, const GemmParams p) {
+    gemm_body<KIND, BN, AMODE, SWB>(tmap_a, tmap_b, tmap_c, p, (int)blockIdx.x, (int)gridDim.x);
+}
+
+// Several problems of one kernel configuration in ONE launch: CTAs [first_block[g], first_block[g + 1]) work on
+// problem g exactly as the CTAs of a launch of its own would (same persistent tile loop over its own tiles).
+constexpr int kMaxMulti = 8;
+struct GemmMulti {
+    int n;
+    int first_block[kMaxMulti + 1];
+    CUtensorMap ta[kMaxMulti], tb[kMaxMulti], tc[kMaxMulti];
+    GemmParams p[kMaxMulti];
+};
+
+template <Kind KIND, int BN, int AMODE, int SWB>
+__global__ void __launch_bounds__(320, 1) dybit_gemm_multi_kernel(const __grid_constant__ GemmMulti m) {
+    int g = 0;
+    while (g + 1 < m.n && (int)blockIdx.x >= m.first_block[g + 1]) ++g;
+    gemm_body<KIND, BN, AMODE, SWB>(m.ta[g], m.tb[g], m.tc[g], m.p[g], (int)blockIdx.x - m.first_block[g],
+                                    m.first_block[g + 1] - m.first_block[g]);
 }
 
 // ------------------------------------------------------------------ host side
@@ -2016,6 +2042,95 @@ static bool make_output_map(CUtensorMap *map, float *C, int64_t M, int64_t N, in
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Tensor-core launches gathered instead of issued (dybit_conv2d_prepared_layers): problems that run on the same kernel
+// configuration then share launches, up to kMaxMulti each.  One collector per host thread, active only inside that call.
+struct MultiEntry {
+    CUtensorMap ta, tb, tc;
+    GemmParams p;
+    unsigned char extra[512];      // the halo kernel's own parameter block (HaloParams) when fn launches that kernel
+    int tiles, per_sm, smem;
+    double work;                   // tiles x (K blocks + epilogue): what the CTA shares are proportional to
+};
+using MultiLaunchFn = dybit_status (*)(const MultiEntry *, int, cudaStream_t);
+struct MultiGroup {
+    MultiLaunchFn fn;
+    int per_sm, smem;
+    std::vector<MultiEntry> entries;
+};
+struct GemmCollector {
+    std::vector<MultiGroup> groups;
+    void add(MultiLaunchFn fn, const MultiEntry &e) {
+        for (MultiGroup &g : groups)
+            if (g.fn == fn && g.per_sm == e.per_sm && g.smem == e.smem) {
+                g.entries.push_back(e);
+                return;
+            }
+        groups.push_back(MultiGroup{fn, e.per_sm, e.smem, {e}});
+    }
+    dybit_status launch_all(cudaStream_t s) {
+        for (const MultiGroup &g : groups)
+            for (size_t i = 0; i < g.entries.size(); i += kMaxMulti) {
+                const size_t n = g.entries.size() - i < (size_t)kMaxMulti ? g.entries.size() - i : (size_t)kMaxMulti;
+                const dybit_status st = g.fn(g.entries.data() + i, (int)n, s);
+                if (st != DYBIT_OK) return st;
+            }
+        return DYBIT_OK;
+    }
+};
+inline GemmCollector *&gemm_collector() {
+    static thread_local GemmCollector *c = nullptr;
+    return c;
+}
+
+// CTAs of a shared launch: every problem gets a share of the `budget` CTAs the device holds at once in proportion
+// to its work (so that the problems end together), at least one, at most one per tile; if all fit, one per tile.
+static void multi_shares(const MultiEntry *e, int n, int budget, int *first_block) {
+    long long all_tiles = 0;
+    double all_work = 0.0;
+    for (int i = 0; i < n; ++i) {
+        all_tiles += e[i].tiles;
+        all_work += e[i].work;
+    }
+    first_block[0] = 0;
+    for (int i = 0; i < n; ++i) {
+        int share = e[i].tiles;
+        if (all_tiles > budget) {
+            share = (int)((double)budget * e[i].work / all_work);
+            if (share < 1) share = 1;
+            if (share > e[i].tiles) share = e[i].tiles;
+        }
+        first_block[i + 1] = first_block[i] + share;
+    }
+}
+
+template <Kind KIND, int BN, int AMODE, int SWB>
+static dybit_status launch_gemm_multi(const MultiEntry *e, int n, cudaStream_t s) {
+    using L = GemmSmem<BN, SWB>;
+    auto kern = dybit_gemm_multi_kernel<KIND, BN, AMODE, SWB>;
+    static std::atomic<bool> configured[64];
+    int dev = 0;
+    DYBIT_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return DYBIT_ERR_CUDA;
+    if (!configured[dev]) {
+        DYBIT_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kBytes));
+        configured[dev] = true;
+    }
+    GemmMulti m;
+    memset(&m, 0, sizeof(m));
+    m.n = n;
+    multi_shares(e, n, sm_count(), m.first_block);
+    for (int i = 0; i < n; ++i) {
+        m.ta[i] = e[i].ta;
+        m.tb[i] = e[i].tb;
+        m.tc[i] = e[i].tc;
+        m.p[i] = e[i].p;
+        const int share = m.first_block[i + 1] - m.first_block[i];
+        m.p[i].b_resident = (m.p[i].bmt == 0 && m.p[i].n_tiles == 1 && m.p[i].k_blocks <= L::kStages && e[i].tiles > share) ? 1 : 0;
+    }
+    launch_k(kern, dim3((unsigned)m.first_block[n]), dim3(320u), (size_t)L::kBytes, s, m);
+    return launch_status();
+}
+
 template <Kind KIND, int BN, int AMODE, int SWB>
 static dybit_status launch_gemm_inst(const CUtensorMap &ta, const CUtensorMap &tb, const GemmParams &p_in, cudaStream_t s) {
     GemmParams p = p_in;
@@ -2036,6 +2151,23 @@ static dybit_status launch_gemm_inst(const CUtensorMap &ta, const CUtensorMap &t
     const int tiles = p.m_tiles * p.n_tiles;
     const int grid = tiles < sm_count() ? tiles : sm_count();
     ProfileEvents ev = profile_events();
+    if constexpr (KIND == Kind::I8 && (AMODE == kAIm2col || AMODE == kATiled)) {
+        // inside dybit_conv2d_prepared_layers: gathered, launched together with its like at the end of that call
+        if (gemm_collector() != nullptr && !ev.start && !ev.stop && !ev.clock) {
+            MultiEntry e;
+            memset(&e, 0, sizeof(e));
+            e.ta = ta;
+            e.tb = tb;
+            e.tc = tc;
+            e.p = p;
+            e.tiles = tiles;
+            e.per_sm = 1;
+            e.smem = L::kBytes;
+            e.work = (double)tiles * (double)(p.k_blocks + 8);      // + a tile's epilogue, about eight K blocks' worth
+            gemm_collector()->add(launch_gemm_multi<KIND, BN, AMODE, SWB>, e);
+            return DYBIT_OK;
+        }
+    }
     profile_events() = ProfileEvents();
     p.clock = ev.clock;
     // a B panel that fits the B stage slots is fetched once per CTA when every tile shares it and CTAs take several tiles
@@ -2774,6 +2906,17 @@ dybit_status dybit_conv2d_prepared(const dybit_conv_layer *layer, void *stream) 
     if (l.Q != nullptr && l.Y_raw != nullptr) return DYBIT_ERR_INVALID_ARG;
     return dybit::conv_impl(&l.desc, l.X_packed, l.fx, l.scale_x_out, l.W, l.fw, l.scale_w, l.ldw_bytes, l.Q ? nullptr : l.Y,
                             l.Q ? nullptr : l.Y_raw, l.Q ? &rq : nullptr, l.ws, l.ws_bytes, stream, &xq, nullptr, true);
+}
+
+dybit_status dybit_conv2d_prepared_layers(const dybit_conv_layer *layers, int n_layers, void *stream) {
+    if (layers == nullptr || n_layers <= 0) return DYBIT_ERR_INVALID_ARG;
+    dybit::GemmCollector col;
+    dybit::gemm_collector() = &col;
+    dybit_status st = DYBIT_OK;
+    for (int i = 0; i < n_layers && st == DYBIT_OK; ++i) st = dybit_conv2d_prepared(&layers[i], stream);
+    dybit::gemm_collector() = nullptr;
+    if (st != DYBIT_OK) return st;
+    return col.launch_all(static_cast<cudaStream_t>(stream));
 }
 
 dybit_status dybit_gemm_requant(int64_t M, int64_t N, int64_t K, const void *A, dybit_fmt fa, const float *scale_a,

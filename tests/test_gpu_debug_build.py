@@ -61,6 +61,9 @@ dy.dybit_quantize_expand_layers(layers)
 for i in range(len(args)):
     Y, Y_raw = dy.dybit_conv2d_prepared(layers, i)
     assert np.array_equal(Y_raw.cpu().numpy().astype(np.int64), want[i][0]) and np.array_equal(Y.cpu().numpy(), want[i][1])
+dy.dybit_conv2d_prepared_layers(layers)
+for i in range(len(args)):
+    assert np.array_equal(layers.raw[i].cpu().numpy().astype(np.int64), want[i][0]) and np.array_equal(layers.Y[i].cpu().numpy(), want[i][1])
 torch.cuda.synchronize()
 assert dy.dybit_last_device_status() == (0, 0), dy.dybit_last_device_status()
 print("debug build ok")

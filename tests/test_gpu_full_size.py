@@ -199,8 +199,9 @@ def test_resnet18_batch32_uniform_4bit_sampled(i, L):
 
 
 def test_resnet18_batch32_folded_step_in_the_bench_launch_configuration():
-    """The step as bench.py times it: dybit_quantize_expand_layers over all 21 layers, then dybit_conv2d_prepared per
-    layer round-robin on three streams.  Every layer's codes, scale and output must equal, bit for bit, what the
+    """The step as bench.py times it: dybit_quantize_expand_layers over all 21 layers, then the tensor-core work, first as
+    dybit_conv2d_prepared per layer round-robin on three streams, then as dybit_conv2d_prepared_layers (shared
+    launches; the form the bench uses).  Every layer's codes, scale and output must equal, bit for bit, what the
     one-layer call gives (which the test above checks against the oracle), and sampled outputs of four layers are
     checked against the oracle directly."""
     layers = wl.resnet18_layers(32)
@@ -227,6 +228,17 @@ def test_resnet18_batch32_folded_step_in_the_bench_launch_configuration():
     torch.cuda.synchronize()
     assert dy.dybit_launch_count() - n0 == 2 + len(layers)
     assert dy.dybit_last_device_status() == (0, 0)
+    per_layer = [y.clone() for y in folded.Y]
+    for y in folded.Y:
+        y.zero_()
+    n1 = dy.dybit_launch_count()
+    dy.dybit_conv2d_prepared_layers(folded)
+    torch.cuda.synchronize()
+    assert dy.dybit_launch_count() - n1 <= 8
+    assert dy.dybit_last_device_status() == (0, 0)
+    for i, L in enumerate(layers):
+        assert torch.equal(per_layer[i], folded.Y[i]), L.name
+    del per_layer
     for i, (L, a) in enumerate(zip(layers, args)):
         Y1, _, p1, s1 = dy.dybit_quantize_conv2d(a["desc"], a["X"], fx, a["W"], fw, a["scale_w"])
         assert torch.equal(p1, folded.packed[i]) and torch.equal(s1, folded.scale[i]), L.name

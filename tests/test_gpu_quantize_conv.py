@@ -165,6 +165,7 @@ def test_layers_in_few_launches():
         (wl.ConvLayer("c64_e4m3", 2, 14, 14, 64, 96, 3, 3, 1, 1), (5, 0), (4, 1), False),
         (wl.ConvLayer("c64_bf16", 6, 20, 20, 64, 96, 3, 3, 1, 1), (8, 0), (8, 1), True),
         (wl.ConvLayer("c1_5x5_signed", 3, 30, 31, 1, 24, 5, 5, 1, 2), (4, 1), (3, 1), False),
+        (wl.ConvLayer("c64_3x3_again", 8, 28, 28, 64, 64, 3, 3, 1, 1), (4, 0), (4, 1), False),     # shares a launch with c64_3x3
     ]
     args, refs = [], []
     for i, (L, fx, fw, given) in enumerate(cases):
@@ -191,6 +192,19 @@ def test_layers_in_few_launches():
     torch.cuda.synchronize()
     assert dy.dybit_launch_count() - n1 <= len(cases) + 2
     assert dy.dybit_last_device_status() == (0, 0)
+    # the same tensor-core work through dybit_conv2d_prepared_layers (problems of one kernel configuration share a
+    # launch): fewer launches, the same bits
+    one_by_one = [(y.clone(), None if r is None else r.clone()) for y, r in zip(layers.Y, layers.raw)]
+    for y in layers.Y:
+        y.zero_()
+    n2 = dy.dybit_launch_count()
+    dy.dybit_conv2d_prepared_layers(layers)
+    torch.cuda.synchronize()
+    assert dy.dybit_launch_count() - n2 < len(cases)
+    assert dy.dybit_last_device_status() == (0, 0)
+    for i, (y, r) in enumerate(one_by_one):
+        assert torch.equal(y, layers.Y[i]), cases[i][0].name
+        assert r is None or torch.equal(r, layers.raw[i]), cases[i][0].name
     for i, (L, fx, fw, cont, spx, packed_ref, S, Y_ref, spw) in enumerate(refs):
         assert layers.scale[i].cpu().numpy().tolist() == [float(np.float32(spx[0])), float(np.float32(spx[1]))], L.name
         assert np.array_equal(layers.packed[i].cpu().numpy(), packed_ref), L.name

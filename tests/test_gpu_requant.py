@@ -257,6 +257,14 @@ def test_layers_with_the_requant_epilogue():
     assert dy.dybit_last_device_status() == (0, 0)
     for i, L in enumerate(shapes):
         assert np.array_equal(outs[i].cpu().numpy(), expect[i]), L.name
+    # shared launches give the same codes and outputs
+    for o in outs:
+        o.zero_()
+    dy.dybit_conv2d_prepared_layers(layers)
+    torch.cuda.synchronize()
+    assert dy.dybit_last_device_status() == (0, 0)
+    for i, L in enumerate(shapes):
+        assert np.array_equal((layers.Q[i] if layers.Q[i] is not None else layers.Y[i]).cpu().numpy(), expect[i]), L.name
     # and bit for bit the one-layer call
     a = args[0]
     Q1, _, _ = dy.dybit_quantize_conv2d_requant(a["desc"], a["X"], fx, a["W"], fw, a["scale_w"], fq, a["scale_q"], relu=True,
