@@ -1105,6 +1105,28 @@ def main():
             "layers_us": {L.name: round(t, 1) for L, t in zip(work.layers, clock_us)}},
         "algorithmic_flops_per_step": flops_total, "algorithmic_bytes_per_step": bytes_total,
     }
+    if work.fold:
+        # the two halves of the timed step on their own (graph replays): the folded streaming launches, and the 21
+        # tensor-core problems in shared launches against the same layer-wise bound
+        g_a = capture_step(work, device, lambda: dy.dybit_quantize_expand_layers(work.folded))
+        g_b = capture_step(work, device, lambda: dy.dybit_conv2d_prepared_layers(work.folded))
+        for _ in range(3):
+            g_a.replay()
+            g_b.replay()
+        ms_a = timed_region(g_a.replay, args.steps, dist, device) / args.steps
+        n0 = dy.dybit_launch_count()
+        dy.dybit_conv2d_prepared_layers(work.folded)
+        conv_launches = dy.dybit_launch_count() - n0
+        ms_b = timed_region(g_b.replay, args.steps, dist, device) / args.steps
+        del g_a, g_b
+        roofline_conv["shared_launches"] = {
+            "what": "dybit_conv2d_prepared_layers alone (the tensor-core part of the timed step: problems of one kernel "
+                    "configuration share a launch), CUDA-graph replays",
+            "launches": conv_launches, "ms_per_step": ms_b,
+            "achieved": (flops_total / 1e12 if tensor_bound else bytes_total / 1e9) / (ms_b * 1e-3),
+            "frac": (flops_total / 1e12 if tensor_bound else bytes_total / 1e9) / (ms_b * 1e-3) / peak,
+            "frac_of_layerwise_bound": ideal_s / (ms_b * 1e-3),
+            "streaming_launches_ms_per_step": ms_a}
     # whole step against its memory roofline: fp32 activation read twice (max-abs, quantize), codes written, conv traffic
     step_bytes = work.quant_elems * (8.0 + FMT_A[0] / 8.0) + bytes_total
     roofline_conv["whole_step"] = {"algorithmic_bytes": step_bytes, "gbs": step_bytes / (ms_step * 1e-3) / 1e9,
