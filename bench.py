@@ -141,6 +141,7 @@ class LayerwiseStep:
         self.dy, self.device = dy, device
         self.two_calls = two_calls          # quantize_pack + conv2d as two library calls instead of one
         self.fold = fold                    # max-abs and quantize + expand of ALL layers in two launches, then the convolutions
+        self.shared_launches = True         # ... as dybit_conv2d_prepared_layers (False: one launch per layer on the side streams)
         self.n_streams = max(1, int(n_streams))
         self.layers = layers
         self.fw = [(wb, 1) for wb, _ in bits]
@@ -204,7 +205,17 @@ class LayerwiseStep:
             # dybit_quantize_expand_layers: one max-abs launch and one quantize + expand launch for all layers; then
             # dybit_conv2d_prepared_layers: the tensor-core work, layers of one kernel configuration sharing launches
             dy.dybit_quantize_expand_layers(self.folded)
-            dy.dybit_conv2d_prepared_layers(self.folded)
+            if self.shared_launches:
+                dy.dybit_conv2d_prepared_layers(self.folded)
+                return
+            # one tensor-core launch per layer, round-robin on the side streams
+            cur = torch.cuda.current_stream()
+            for st in self.side:
+                st.wait_stream(cur)
+            for j in range(len(self.layers)):
+                dy.dybit_conv2d_prepared(self.folded, j, stream=self.side[j % self.n_streams] if self.side else None)
+            for st in self.side:
+                cur.wait_stream(st)
             return
         if self.n_streams > 1 and only is None and not profiling and not serial:
             cur = torch.cuda.current_stream()
@@ -766,28 +777,36 @@ def sweep_resnet50(dy, wl, device):
     del graph, graph1
     # the same step with the streaming launches folded over the layers (dybit_quantize_expand_layers: one max-abs
     # launch per 32 layers, one quantize + expand launch per pair of formats), then the convolutions on three streams
-    ms_fold, fold_launches = None, None
+    ms_fold, fold_launches, fold_variants = None, None, {}
     try:
         work.folded = dy.ConvLayers([dict(desc=work.desc[i], X=work.x_dev[i], fx=work.fa[i], W=work.pw[i], fw=work.fw[i],
                                           scale_w=work.sw[i], packed=work.px[i], scale_out=work.sx[i], Y=work.y[i])
                                      for i in range(len(layers))])
         work.fold = True
-        for _ in range(3):
-            work.step()
-        n0 = dy.dybit_launch_count()
-        graph_f = capture_step(work, device)
-        fold_launches = dy.dybit_launch_count() - n0
-        for _ in range(3):
-            graph_f.replay()
-        ms_fold = timed_region(graph_f.replay, 10, None, device) / 10
-        del graph_f
+        best = None
+        for shared in (False, True):      # tensor-core launches per layer on three streams / shared, on one stream
+            work.shared_launches = shared
+            for _ in range(3):
+                work.step()
+            n0 = dy.dybit_launch_count()
+            graph_f = capture_step(work, device)
+            launches = dy.dybit_launch_count() - n0
+            for _ in range(3):
+                graph_f.replay()
+            t = timed_region(graph_f.replay, 10, None, device) / 10
+            del graph_f
+            fold_variants = dict(fold_variants, **{("shared_launches" if shared else "per_layer_launches_3_streams"):
+                                                   {"ms_per_step": t, "launches": launches}})
+            if best is None or t < best:
+                best, fold_launches = t, launches
+        ms_fold = best
     except dy.DybitError as exc:        # a layer whose lowering has no fused expand
         ms_fold = None
         fold_note = str(exc)
     work.fold = False
     conts = [CONTAINERS[dy.dybit_choose_container(fa, fw)[0]] for fa, fw in zip(work.fa, work.fw)]
     return {"ms_per_step": ms, "ms_per_step_one_stream": ms1, "streams": 3,
-            "ms_per_step_folded": ms_fold, "launches_per_folded_step": fold_launches,
+            "ms_per_step_folded": ms_fold, "launches_per_folded_step": fold_launches, "folded_variants": fold_variants,
             "tops": 2.0 * work.macs / (ms * 1e-3) / 1e12, "layers": len(layers), "seed": 0,
             "containers": {c: conts.count(c) for c in sorted(set(conts))}, "bits_w_a": bits}
 
