@@ -266,7 +266,7 @@ dybit_status dybit_quantize_expand_layers(const dybit_conv_layer *layers, int n_
 dybit_status dybit_conv2d_prepared(const dybit_conv_layer *layer, void *stream);
 /* dybit_conv2d_prepared for all the layers on one stream, with the tensor-core work of layers that run on the same
  * kernel configuration (4-bit-class formats on the int8 path: halo-tile, im2col and row-major lowerings) folded into
- * shared launches of up to 8 layers: every layer gets a share of the SMs in proportion to its work and its CTAs walk
+ * shared launches of up to 16 layers: every layer gets a share of the SMs in proportion to its work and its CTAs walk
  * its own tiles as they would in a launch of their own, so results are the same bits.  Layers that do not fit this
  * (other element types, gather lowerings) are launched one by one, in order. */
 dybit_status dybit_conv2d_prepared_layers(const dybit_conv_layer *layers, int n_layers, void *stream);
