@@ -587,7 +587,7 @@ def time_graph(run, replays):
     return e0.elapsed_time(e1) / replays
 
 
-SWEEP_SECTIONS = ("quantize_sweep", "rmse", "rmse_sweep", "fake_quant", "depthwise", "gemm_batched", "gemm_sweep",
+SWEEP_SECTIONS = ("quantize_sweep", "rmse", "rmse_sweep", "fake_quant", "decode", "depthwise", "gemm_batched", "gemm_sweep",
                   "bitwidth_search", "resnet50_b64_mixed")
 
 
@@ -603,7 +603,7 @@ def run_sweeps(dy, wl, device, peaks, only=None, log2n=28):
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
     if "quantize_sweep" in want:
         out["quantize_sweep"] = sweep_quantize(dy, wl, device, flush)
-    if want & {"rmse", "rmse_sweep", "fake_quant"}:
+    if want & {"rmse", "rmse_sweep", "fake_quant", "decode"}:
         x = wl.normal((1 << log2n,), seed=5, device=device)
         if "rmse" in want:
             out["rmse"] = sweep_rmse(dy, x, log2n, flush)
@@ -611,6 +611,8 @@ def run_sweeps(dy, wl, device, peaks, only=None, log2n=28):
             out["rmse_sweep"] = sweep_rmse_candidates(dy, x, log2n, flush)
         if "fake_quant" in want:
             out["fake_quant"] = sweep_fake_quant(dy, x, log2n, flush)
+        if "decode" in want:
+            out["decode"] = sweep_decode(dy, x, log2n, flush)
         del x
         torch.cuda.empty_cache()
     if "depthwise" in want:
@@ -711,6 +713,18 @@ def sweep_fake_quant(dy, x, log2n, flush):
     g = torch.empty_like(x).normal_()
     ms = time_calls_flushed(lambda: dy.dybit_fake_quant_backward(x, g, (4, 1), scale, out=y), 5, flush)
     rows.append({"log2n": log2n, "fmt": [4, 1], "direction": "backward", "ms": ms, "gbs": x.numel() * 12 / ms / 1e6})
+    return rows
+
+
+def sweep_decode(dy, x, log2n, flush):
+    """dybit_decode: packed codes back to fp32 (bits/8 B read + 4 B written per element)."""
+    rows = []
+    out = torch.empty_like(x)
+    for fmt in ((2, 1), (4, 1), (6, 1), (8, 1)):
+        packed, scale = dy.dybit_quantize_pack(x, fmt)
+        ms = time_calls_flushed(lambda: dy.dybit_decode(packed, x.numel(), fmt, scale, out=out), 5, flush)
+        rows.append({"log2n": log2n, "fmt": list(fmt), "ms": ms, "gbs": x.numel() * (4 + fmt[0] / 8) / ms / 1e6})
+        del packed
     return rows
 
 
