@@ -86,13 +86,14 @@ static const ElemTable &make_elem_table(dybit_fmt f, dybit_container cont, int i
     return e.table;
 }
 
-// Rows of packed codes -> rows of container elements.  A warp expands 1024 codes at a time.
+// Rows of packed codes -> rows of container elements.  A warp expands 1024 codes at a time and keeps the packed
+// vectors of two such chunks in flight.
 template <int BITS, int ELEM>
 __global__ void __launch_bounds__(kStreamThreads)
 expand_rows_kernel(const uint8_t *__restrict__ packed, int64_t rows, int64_t in_stride, int64_t cols,
                    uint8_t *__restrict__ out, int64_t out_stride, const __grid_constant__ ElemTable table) {
     __shared__ uint16_t s_lut[256];
-    __shared__ __align__(16) unsigned s_words[kWarpsPerBlock][32 * BITS];
+    __shared__ __align__(16) unsigned s_words[kWarpsPerBlock][2][32 * BITS];
     for (int i = threadIdx.x; i < 256; i += blockDim.x) s_lut[i] = table.v[i];
     __syncthreads();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -102,42 +103,53 @@ expand_rows_kernel(const uint8_t *__restrict__ packed, int64_t rows, int64_t in_
     const int64_t chunks_per_row = (cols + kChunkCodes - 1) / kChunkCodes;
     const int64_t items = rows * chunks_per_row;
     const int64_t in_row_bytes = ((cols * BITS + 7) / 8 + 15) / 16 * 16;
-    for (int64_t item = (int64_t)blockIdx.x * kWarpsPerBlock + warp; item < items;
-         item += (int64_t)gridDim.x * kWarpsPerBlock) {
-        const int64_t row = item / chunks_per_row, chunk = item - row * chunks_per_row;
-        const int64_t c0 = chunk * kChunkCodes;
-        const int valid = (int)min((int64_t)kChunkCodes, cols - c0);
-        const int nvec = (int)min((int64_t)kChunkVecs, (in_row_bytes - chunk * kChunkBytes) / 16);
-        const uint4 *src = reinterpret_cast<const uint4 *>(packed + row * in_stride + chunk * kChunkBytes);
-        uint4 *s4 = reinterpret_cast<uint4 *>(&s_words[warp][0]);
-        for (int i = lane; i < kChunkVecs; i += 32) s4[i] = (i < nvec) ? __ldg(src + i) : make_uint4(0, 0, 0, 0);
+    const int64_t stride = (int64_t)gridDim.x * kWarpsPerBlock;
+    for (int64_t item0 = (int64_t)blockIdx.x * kWarpsPerBlock + warp; item0 < items; item0 += 2 * stride) {
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const int64_t item = item0 + u * stride;
+            if (item >= items) continue;
+            const int64_t row = item / chunks_per_row, chunk = item - row * chunks_per_row;
+            const int nvec = (int)min((int64_t)kChunkVecs, (in_row_bytes - chunk * kChunkBytes) / 16);
+            const uint4 *src = reinterpret_cast<const uint4 *>(packed + row * in_stride + chunk * kChunkBytes);
+            uint4 *s4 = reinterpret_cast<uint4 *>(&s_words[warp][u][0]);
+            for (int i = lane; i < kChunkVecs; i += 32) s4[i] = (i < nvec) ? __ldg(src + i) : make_uint4(0, 0, 0, 0);
+        }
         __syncwarp();
-        unsigned w[BITS], cw[8];
 #pragma unroll
-        for (int i = 0; i < BITS; ++i) w[i] = s_words[warp][lane * BITS + i];
-        unpack32<BITS>(w, cw);
-        uint8_t *dst = out + row * out_stride + (c0 + lane * 32) * ELEM;
-        if constexpr (ELEM == 1) {
-            unsigned o[8];
+        for (int u = 0; u < 2; ++u) {
+            const int64_t item = item0 + u * stride;
+            if (item >= items) continue;
+            const int64_t row = item / chunks_per_row, chunk = item - row * chunks_per_row;
+            const int64_t c0 = chunk * kChunkCodes;
+            const int valid = (int)min((int64_t)kChunkCodes, cols - c0);
+            unsigned w[BITS], cw[8];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                o[i] = (unsigned)(s_lut[cw[i] & 0xffu] & 0xffu) | ((unsigned)(s_lut[(cw[i] >> 8) & 0xffu] & 0xffu) << 8) |
-                       ((unsigned)(s_lut[(cw[i] >> 16) & 0xffu] & 0xffu) << 16) |
-                       ((unsigned)(s_lut[cw[i] >> 24] & 0xffu) << 24);
+            for (int i = 0; i < BITS; ++i) w[i] = s_words[warp][u][lane * BITS + i];
+            unpack32<BITS>(w, cw);
+            uint8_t *dst = out + row * out_stride + (c0 + lane * 32) * ELEM;
+            if constexpr (ELEM == 1) {
+                unsigned o[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    o[i] = (unsigned)(s_lut[cw[i] & 0xffu] & 0xffu) | ((unsigned)(s_lut[(cw[i] >> 8) & 0xffu] & 0xffu) << 8) |
+                           ((unsigned)(s_lut[(cw[i] >> 16) & 0xffu] & 0xffu) << 16) |
+                           ((unsigned)(s_lut[cw[i] >> 24] & 0xffu) << 24);
+                }
+                if (lane * 32 < valid) reinterpret_cast<uint4 *>(dst)[0] = make_uint4(o[0], o[1], o[2], o[3]);
+                if (lane * 32 + 16 < valid) reinterpret_cast<uint4 *>(dst)[1] = make_uint4(o[4], o[5], o[6], o[7]);
+            } else {
+                unsigned o[16];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    o[2 * i] = (unsigned)s_lut[cw[i] & 0xffu] | ((unsigned)s_lut[(cw[i] >> 8) & 0xffu] << 16);
+                    o[2 * i + 1] = (unsigned)s_lut[(cw[i] >> 16) & 0xffu] | ((unsigned)s_lut[cw[i] >> 24] << 16);
+                }
+#pragma unroll
+                for (int v = 0; v < 4; ++v)
+                    if (lane * 32 + v * 8 < valid)
+                        reinterpret_cast<uint4 *>(dst)[v] = make_uint4(o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
             }
-            if (lane * 32 < valid) reinterpret_cast<uint4 *>(dst)[0] = make_uint4(o[0], o[1], o[2], o[3]);
-            if (lane * 32 + 16 < valid) reinterpret_cast<uint4 *>(dst)[1] = make_uint4(o[4], o[5], o[6], o[7]);
-        } else {
-            unsigned o[16];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                o[2 * i] = (unsigned)s_lut[cw[i] & 0xffu] | ((unsigned)s_lut[(cw[i] >> 8) & 0xffu] << 16);
-                o[2 * i + 1] = (unsigned)s_lut[(cw[i] >> 16) & 0xffu] | ((unsigned)s_lut[cw[i] >> 24] << 16);
-            }
-#pragma unroll
-            for (int v = 0; v < 4; ++v)
-                if (lane * 32 + v * 8 < valid)
-                    reinterpret_cast<uint4 *>(dst)[v] = make_uint4(o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
         }
         __syncwarp();
     }
@@ -1188,9 +1200,15 @@ expand_pix4_kernel(const uint8_t *__restrict__ packed, int bits, int64_t pixels,
 template <int ELEM>
 static dybit_status launch_expand_rows(const uint8_t *packed, int bits, int64_t rows, int64_t in_stride, int64_t cols,
                                        uint8_t *out, int64_t out_stride, const ElemTable &t, cudaStream_t s) {
+    // rows that follow one another without gaps on both sides are one flat run of codes: short rows (a K of 64 is
+    // 128 codes) then fill whole 1024-code chunks instead of an eighth of one
+    if (rows > 1 && in_stride * 8 == cols * bits && out_stride == cols * ELEM) {
+        cols *= rows;
+        rows = 1;
+    }
     const int64_t items = rows * ((cols + kChunkCodes - 1) / kChunkCodes);
     if (items == 0) return DYBIT_OK;
-    const int grid = stream_grid(items);
+    const int grid = stream_grid((items + 1) / 2);
     switch (bits) {
         case 2: launch_k(expand_rows_kernel<2, ELEM>, dim3((unsigned)(grid)), dim3((unsigned)(kStreamThreads)), (size_t)(0), s, packed, rows, in_stride, cols, out, out_stride, t); break;
         case 3: launch_k(expand_rows_kernel<3, ELEM>, dim3((unsigned)(grid)), dim3((unsigned)(kStreamThreads)), (size_t)(0), s, packed, rows, in_stride, cols, out, out_stride, t); break;

@@ -393,23 +393,35 @@ quantize_pack_kernel(const float *__restrict__ x, int64_t rows, int64_t cols, in
 
 struct FloatTable { float v[256]; };
 
-// Inverse of pack32: BITS words -> this lane's 32 codes as bytes in 8 words.
+// Inverse of pack32: BITS words -> this lane's 32 codes as bytes in 8 words.  Every shift is a compile-time
+// constant: the eight 4 * BITS-bit pieces are cut out of the words, each is spread over two 16-bit halves and each
+// half over two bytes.
 template <int BITS>
 __device__ __forceinline__ void unpack32(const unsigned (&in)[BITS], unsigned (&cw)[8]) {
-    unsigned long long acc = 0;
-    int nb = 0, w = 0;
+    if constexpr (BITS == 8) {
 #pragma unroll
-    for (int i = 0; i < 8; ++i) cw[i] = 0;
+        for (int i = 0; i < 8; ++i) cw[i] = in[i];
+        return;
+    } else if constexpr (BITS == 4) {
 #pragma unroll
-    for (int i = 0; i < 32; ++i) {
-        if (nb < BITS) {
-            acc |= (unsigned long long)in[w++] << nb;
-            nb += 32;
+        for (int i = 0; i < 4; ++i) {
+            const unsigned lo = in[i] & 0x0f0f0f0fu, hi = (in[i] >> 4) & 0x0f0f0f0fu;      // even / odd codes
+            cw[2 * i] = __byte_perm(lo, hi, 0x5140);
+            cw[2 * i + 1] = __byte_perm(lo, hi, 0x7362);
         }
-        const unsigned code = (unsigned)acc & ((1u << BITS) - 1u);
-        acc >>= BITS;
-        nb -= BITS;
-        cw[i >> 2] |= code << ((i & 3) * 8);
+        return;
+    }
+    constexpr unsigned kPiece = (BITS == 8) ? 0xffffffffu : ((1u << (4 * BITS % 32)) - 1u);
+    constexpr unsigned kPair = (1u << (2 * BITS)) - 1u;
+    constexpr unsigned kCode = (1u << BITS) - 1u;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int pos = i * 4 * BITS, word = pos >> 5, off = pos & 31;
+        unsigned q = in[word] >> off;
+        if (off + 4 * BITS > 32) q |= in[word + 1] << (32 - off);
+        q &= kPiece;
+        const unsigned u = (q & kPair) | ((q << (16 - 2 * BITS)) & (kPair << 16));
+        cw[i] = (u & (kCode * 0x00010001u)) | ((u << (8 - BITS)) & ((kCode << 8) * 0x00010001u));
     }
 }
 
