@@ -1116,7 +1116,7 @@ def main():
         achieved, peak, unit = bytes_total / (mma_total_ms * 1e-3) / 1e9, peaks["hbm_gbs"], "GB/s"
     roofline_conv = {
         "kernel": "dybit_conv_halo_kernel<I8> / dybit_gemm_kernel<I8, conv> (21 launches per step, one per layer)",
-        "workload": f"resnet18_b{args.batch}_w4a4, layers on one stream",
+        "workload": f"resnet18_b{args.batch}_w4a4, the 21 layers of one step",
         "bound": "tensor" if tensor_bound else "hbm", "achieved": achieved, "peak": peak, "unit": unit,
         "frac": achieved / peak,
         "traffic": NCU_TRAFFIC["conv_step"] if args.batch == 32 else None,
@@ -1160,6 +1160,16 @@ def main():
             "frac": (flops_total / 1e12 if tensor_bound else bytes_total / 1e9) / (ms_b * 1e-3) / peak,
             "frac_of_layerwise_bound": ideal_s / (ms_b * 1e-3),
             "streaming_launches_ms_per_step": ms_a}
+        # the figures at the top of this object are those of the configuration the step is timed in (shared launches);
+        # the launch-by-launch ones (events and device clock per layer) move one level down
+        sl = roofline_conv["shared_launches"]
+        roofline_conv["per_layer_launches"] = {k: roofline_conv[k] for k in ("achieved", "frac", "frac_of_layerwise_bound", "how",
+                                                                             "ms_per_step_in_kernel")}
+        roofline_conv.update({"achieved": sl["achieved"], "frac": sl["frac"], "frac_of_layerwise_bound": sl["frac_of_layerwise_bound"],
+                              "ms_per_step_in_kernel": ms_b,
+                              "kernel": "dybit_conv_halo_multi_kernel<I8> / dybit_gemm_multi_kernel<I8, conv> (%d launches per step "
+                                        "for the 21 layers)" % conv_launches,
+                              "how": "CUDA-graph replays of dybit_conv2d_prepared_layers alone, CUDA events around K replays"})
     # whole step against its memory roofline: fp32 activation read twice (max-abs, quantize), codes written, conv traffic
     step_bytes = work.quant_elems * (8.0 + FMT_A[0] / 8.0) + bytes_total
     roofline_conv["whole_step"] = {"algorithmic_bytes": step_bytes, "gbs": step_bytes / (ms_step * 1e-3) / 1e9,
